@@ -1,0 +1,173 @@
+/*
+ * sna.h — C ABI of the spherical neighborhood attention library for NVIDIA B200 (sm_100a).
+ *
+ * The operator (paper: "Attention on the Sphere", arXiv 2505.11157):
+ *
+ *   out[n,h,w,:] = sum_j alpha_j v_j / sum_j alpha_j ,   alpha_j = exp(q[n,h,w,:] . k_j / sqrt(C)) * omega_j
+ *
+ * where j runs over the input grid points inside the geodesic disc of radius theta_cutoff around the
+ * output point (h, w) (Eq. s2_neighborhood_attention), omega_j is the quadrature weight of the input
+ * point (Eq. quadrature), and the discrete form is Eq. s2_attention_discrete_detailed of App. B.3.
+ * The backward pass returns the gradients of App. B.4 with respect to q, k and v.
+ *
+ * Conventions that hold for every call:
+ *   - No exception crosses this boundary; every call returns an sna_status_t (0 = success).
+ *   - "host" pointers are ordinary CPU memory owned by the caller; "device" pointers are CUDA global
+ *     memory on the device that was current when the plan was created, owned by the caller.
+ *   - Tensors are contiguous fp32, channels last, batch and heads leading:
+ *         q, out, dout, dq : [B][H][nlat_out][nlon_out][C]
+ *         k, v, dk, dv     : [B][H][nlat_in ][nlon_in ][C]
+ *         lse, and each half of the workspace : [B][H][nlat_out][nlon_out]
+ *     Device pointers must be 16-byte aligned.  B*H heads are independent problems.
+ *   - C must be one of 4, 8, 16, 32, 64, 128 (SNA_ERR_UNSUPPORTED otherwise).
+ *   - Compute calls enqueue work on the given CUDA stream (a cudaStream_t passed as void*; NULL is the
+ *     default stream) and return without synchronising.  They validate arguments on the host first and
+ *     launch nothing if validation fails.  Outputs are overwritten, never accumulated into.
+ *   - A plan is immutable after creation and may be used from several streams at once, as long as
+ *     calls that run concurrently do not share a workspace (see sna_backward).
+ */
+#ifndef SNA_H
+#define SNA_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct sna_plan sna_plan_t; /* opaque; created and destroyed by the library */
+
+typedef enum {
+    SNA_OK = 0,
+    SNA_ERR_INVALID_ARG = 1,        /* null pointer, non-positive size, NaN or non-positive cutoff, misaligned pointer */
+    SNA_ERR_UNSUPPORTED = 2,        /* nlon_in not a multiple of nlon_out; unsupported C; unknown grid */
+    SNA_ERR_EMPTY_NEIGHBORHOOD = 3, /* some output latitude has no input point inside its disc */
+    SNA_ERR_ALLOC = 4,              /* host or device allocation failed */
+    SNA_ERR_CUDA = 5,               /* a CUDA call or launch failed; see sna_last_error_message */
+    SNA_ERR_AMBIGUOUS_TIE = 6,      /* a point lies within 1e-8 rad of the disc boundary without being on it */
+    SNA_ERR_WORKSPACE = 7           /* caller-supplied workspace or static scratch too small */
+} sna_status_t;
+
+typedef enum {
+    /* theta_h = pi*h/(nlat-1), h = 0..nlat-1: both poles are grid rings; Clenshaw-Curtis latitude weights.
+     * (The equiangular grid of App. A.1, Eq. latlon_grid, with the pole-including variant of the rule.) */
+    SNA_GRID_EQUIANGULAR = 0,
+    /* "Gaussian grid" (Sec. 3.3): theta_h = arccos(x_h), x_h the roots of the Legendre polynomial P_nlat in
+     * descending order (north to south), Gauss-Legendre weights. */
+    SNA_GRID_LEGENDRE_GAUSS = 1
+} sna_grid_t;
+
+/*
+ * Build a plan: colatitudes of both grids, fp64 quadrature weights omega[h'] = w_lat[h'] * 2*pi/nlon_in of the
+ * input grid (Eq. quadrature; they sum to 4*pi over all points), and the neighborhood table of App. B.3: for
+ * every output latitude h the set of (lat_in, lon_off) with geodesic distance between the output point
+ * (h, longitude 0) and the input point (lat_in, lon_off) at most theta_cutoff.  Because the grids are invariant
+ * under rotation about the pole the same row serves every output longitude w: the input column is
+ * (lon_off + w*ps) mod nlon_in with ps = nlon_in / nlon_out.
+ *
+ * Points exactly on the disc boundary are members: the test is d <= theta_cutoff + 1e-10, and a point with
+ * 1e-12 < |d - theta_cutoff| < 1e-8 makes creation fail with SNA_ERR_AMBIGUOUS_TIE rather than letting rounding
+ * decide.  theta_cutoff >= pi selects every input point.
+ *
+ * The plan's tables are copied to the current CUDA device; the plan must be used and destroyed with that
+ * device.  *plan_out is written only on success.  nlat_* >= 2, nlon_* >= 1, nlon_in % nlon_out == 0.
+ */
+sna_status_t sna_plan_create(int nlat_in, int nlon_in, int nlat_out, int nlon_out,
+                             sna_grid_t grid_in, sna_grid_t grid_out, double theta_cutoff,
+                             sna_plan_t** plan_out);
+
+/* Same construction, but nothing is copied to a GPU and no CUDA call is made: the plan serves the
+ * introspection calls below only (compute calls on it return SNA_ERR_INVALID_ARG).  For inspecting or
+ * validating tables on a machine without a GPU. */
+sna_status_t sna_plan_create_host_only(int nlat_in, int nlon_in, int nlat_out, int nlon_out,
+                                       sna_grid_t grid_in, sna_grid_t grid_out, double theta_cutoff,
+                                       sna_plan_t** plan_out);
+
+/* Free the plan's host and device memory (including a workspace it may have grown).  NULL is accepted. */
+sna_status_t sna_plan_destroy(sna_plan_t* plan);
+
+/* ---- introspection into caller-owned HOST buffers ------------------------------------------------------ */
+
+/* Number of (lat_in, lon_off) entries in the table. */
+sna_status_t sna_plan_get_nnz(const sna_plan_t* plan, int64_t* nnz);
+/* theta_in[nlat_in], theta_out[nlat_out] in radians; either pointer may be NULL. */
+sna_status_t sna_plan_get_colatitudes(const sna_plan_t* plan, double* theta_in, double* theta_out);
+/* omega_in[nlat_in]: per-point quadrature weight of each input ring. */
+sna_status_t sna_plan_get_quad_weights(const sna_plan_t* plan, double* omega_in);
+/* CSR table in canonical order: rows = output latitudes, entries sorted by lat_in, then lon_off in [0, nlon_in).
+ * row_ptr[nlat_out+1], lat_in[nnz], lon_off[nnz]. */
+sna_status_t sna_plan_get_table(const sna_plan_t* plan, int64_t* row_ptr, int32_t* lat_in, int32_t* lon_off);
+/* Transposed table used by the backward pass: row (lat_in*ps + r) lists, for input columns congruent to r
+ * modulo ps, the pairs (lat_out, lon_off) of the forward table with lat_in in them and lon_off % ps == r,
+ * sorted by lat_out, then lon_off.  The output longitude is w = ((column - lon_off) mod nlon_in) / ps.
+ * row_ptr[nlat_in*ps+1], lat_out[nnz], lon_off[nnz]. */
+sna_status_t sna_plan_get_table_transposed(const sna_plan_t* plan, int64_t* row_ptr, int32_t* lat_out,
+                                           int32_t* lon_off);
+
+/* ---- compute -------------------------------------------------------------------------------------------- */
+
+/* Bytes of device workspace sna_backward_ex needs for this problem size (two fp32 values per output point,
+ * rounded up to 256 bytes).  Returns 0 for invalid arguments. */
+size_t sna_workspace_bytes(const sna_plan_t* plan, int B, int H, int C);
+
+/* Forward pass (Eq. s2_attention_discrete_detailed).  q, k, v, out: device. */
+sna_status_t sna_forward(const sna_plan_t* plan, const float* q, const float* k, const float* v, float* out,
+                         int B, int H, int C, void* cuda_stream);
+
+/* Forward pass that also stores lse[n,h,w] = log(sum_j exp(s_j) omega_j) (device, may be NULL), which the
+ * backward pass can reuse. */
+sna_status_t sna_forward_ex(const sna_plan_t* plan, const float* q, const float* k, const float* v, float* out,
+                            float* lse, int B, int H, int C, void* cuda_stream);
+
+/*
+ * Backward pass (App. B.4): given dout = dL/dout, writes dq, dk, dv (device, all three required).
+ * With p_j = alpha_j / sum_l alpha_l, t_j = dout_i . v_j, D_i = sum_j p_j t_j:
+ *     dq_i = (1/sqrt(C)) sum_j p_j (t_j - D_i) k_j
+ *     dk_j = (1/sqrt(C)) sum_{i: j in disc(i)} p_ij (t_ij - D_i) q_i        dv_j = sum_{i: j in disc(i)} p_ij dout_i
+ * dk and dv are gathered per input point over the transposed table; no atomics are used, so results are
+ * reproducible bit for bit.  This form recomputes the softmax statistics and keeps them in a workspace owned
+ * by the plan, which is (re)allocated with cudaMalloc when a call needs a larger one than any call before —
+ * such a call synchronises the device.  Two sna_backward calls on the same plan must not overlap on the GPU.
+ */
+sna_status_t sna_backward(const sna_plan_t* plan, const float* q, const float* k, const float* v,
+                          const float* dout, float* dq, float* dk, float* dv,
+                          int B, int H, int C, void* cuda_stream);
+
+/*
+ * Backward pass with caller-supplied state.  out and lse (device) are the results of sna_forward_ex on the same
+ * q, k, v; either may be NULL, in which case the statistics it would provide are recomputed.  workspace is
+ * device memory of at least sna_workspace_bytes(plan, B, H, C) bytes, 256-byte aligned, private to this call
+ * until the call's work on the stream has finished.  Never allocates.
+ */
+sna_status_t sna_backward_ex(const sna_plan_t* plan, const float* q, const float* k, const float* v,
+                             const float* dout, const float* out, const float* lse,
+                             float* dq, float* dk, float* dv,
+                             void* workspace, size_t workspace_bytes,
+                             int B, int H, int C, void* cuda_stream);
+
+/*
+ * The two stages of sna_backward_ex as separate calls, for callers that want to overlap or time them.
+ *
+ * sna_backward_dq: dq of App. B.4 (quotient-rule form) for every output point, plus D[n,h,w] = sum_j p_j t_j,
+ * which the second stage needs.  lse (device, required) is the forward pass's lse; out (device) may be NULL.
+ * D is device memory of B*H*nlat_out*nlon_out floats, written by this call.
+ *
+ * sna_backward_dkdv: dk and dv gathered per input point over the transposed table, from lse and D.
+ */
+sna_status_t sna_backward_dq(const sna_plan_t* plan, const float* q, const float* k, const float* v,
+                             const float* dout, const float* out, const float* lse, float* dq, float* D,
+                             int B, int H, int C, void* cuda_stream);
+sna_status_t sna_backward_dkdv(const sna_plan_t* plan, const float* q, const float* k, const float* v,
+                               const float* dout, const float* lse, const float* D, float* dk, float* dv,
+                               int B, int H, int C, void* cuda_stream);
+
+/* Human-readable name of a status code (static string). */
+const char* sna_status_string(sna_status_t status);
+/* Detail of the most recent failure on the calling thread (static thread-local buffer; "" if none). */
+const char* sna_last_error_message(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SNA_H */

@@ -1,0 +1,331 @@
+// C ABI of the library (declared in include/sna.h): plan life cycle, introspection and the compute entry
+// points.  Host-side validation happens here; kernels live in the other translation units.
+#include "../../include/sna.h"
+
+#include <cuda_runtime.h>
+
+#include <algorithm>
+#include <cmath>
+#include <cstdarg>
+#include <cstdio>
+#include <cstring>
+#include <mutex>
+#include <new>
+#include <numeric>
+#include <string>
+#include <vector>
+
+#include "sna_kernels.cuh"
+#include "sna_plan.hpp"
+
+namespace {
+
+thread_local char g_last_error[512] = "";
+
+void set_error(const char* fmt, ...) __attribute__((format(printf, 1, 2)));
+void set_error(const char* fmt, ...) {
+    va_list ap;
+    va_start(ap, fmt);
+    vsnprintf(g_last_error, sizeof(g_last_error), fmt, ap);
+    va_end(ap);
+}
+
+sna_status_t cuda_fail(cudaError_t e, const char* what) {
+    set_error("%s: %s", what, cudaGetErrorString(e));
+    return SNA_ERR_CUDA;
+}
+
+bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+}  // namespace
+
+struct sna_plan {
+    sna::HostPlan host;
+    sna::DevPlan dev{};
+    int device = 0;
+    void* dev_blob = nullptr;          // one allocation holding every device table
+    mutable std::mutex ws_mutex;
+    mutable void* ws = nullptr;        // workspace grown on demand by sna_backward
+    mutable size_t ws_bytes = 0;
+};
+
+namespace {
+
+bool supported_C(int C) { return C == 4 || C == 8 || C == 16 || C == 32 || C == 64 || C == 128; }
+
+sna_status_t check_problem(const sna_plan_t* plan, int B, int H, int C) {
+    if (plan == nullptr) { set_error("plan is NULL"); return SNA_ERR_INVALID_ARG; }
+    if (plan->dev_blob == nullptr) { set_error("plan was created host-only; it cannot compute"); return SNA_ERR_INVALID_ARG; }
+    if (B <= 0 || H <= 0 || C <= 0) { set_error("B, H and C must be positive"); return SNA_ERR_INVALID_ARG; }
+    if (!supported_C(C)) { set_error("C=%d unsupported (4, 8, 16, 32, 64 or 128)", C); return SNA_ERR_UNSUPPORTED; }
+    const long long N = (long long)B * H;
+    const long long big = std::max((long long)plan->host.nlat_in * plan->host.nlon_in,
+                                   (long long)plan->host.nlat_out * plan->host.nlon_out);
+    if (N > 0x7fffffffLL || N * big > 0x7fffffffLL) { set_error("problem too large: B*H*nlat*nlon must fit in 31 bits"); return SNA_ERR_UNSUPPORTED; }
+    return SNA_OK;
+}
+
+template <typename... P>
+bool all_aligned(P... ptrs) { return (aligned16(ptrs) && ...); }
+
+size_t stats_elems(const sna_plan_t* plan, int B, int H) {
+    return (size_t)B * H * plan->host.nlat_out * plan->host.nlon_out;
+}
+size_t round256(size_t x) { return (x + 255) / 256 * 256; }
+
+}  // namespace
+
+extern "C" {
+
+const char* sna_status_string(sna_status_t s) {
+    switch (s) {
+        case SNA_OK: return "SNA_OK";
+        case SNA_ERR_INVALID_ARG: return "SNA_ERR_INVALID_ARG";
+        case SNA_ERR_UNSUPPORTED: return "SNA_ERR_UNSUPPORTED";
+        case SNA_ERR_EMPTY_NEIGHBORHOOD: return "SNA_ERR_EMPTY_NEIGHBORHOOD";
+        case SNA_ERR_ALLOC: return "SNA_ERR_ALLOC";
+        case SNA_ERR_CUDA: return "SNA_ERR_CUDA";
+        case SNA_ERR_AMBIGUOUS_TIE: return "SNA_ERR_AMBIGUOUS_TIE";
+        case SNA_ERR_WORKSPACE: return "SNA_ERR_WORKSPACE";
+    }
+    return "SNA_ERR_UNKNOWN";
+}
+
+const char* sna_last_error_message(void) { return g_last_error; }
+
+static sna_status_t plan_create(int nlat_in, int nlon_in, int nlat_out, int nlon_out, sna_grid_t grid_in,
+                                sna_grid_t grid_out, double theta_cutoff, bool upload, sna_plan_t** plan_out) {
+    if (plan_out == nullptr) { set_error("plan_out is NULL"); return SNA_ERR_INVALID_ARG; }
+    sna_plan* plan = new (std::nothrow) sna_plan();
+    if (plan == nullptr) { set_error("out of host memory"); return SNA_ERR_ALLOC; }
+    std::string why;
+    sna::PlanStatus ps;
+    try {
+        ps = sna::build_plan(nlat_in, nlon_in, nlat_out, nlon_out, (int)grid_in, (int)grid_out, theta_cutoff, plan->host, why);
+    } catch (const std::bad_alloc&) {
+        delete plan;
+        set_error("out of host memory while building the table");
+        return SNA_ERR_ALLOC;
+    }
+    if (ps != sna::PLAN_OK) {
+        delete plan;
+        set_error("%s", why.c_str());
+        return ps == sna::PLAN_INVALID ? SNA_ERR_INVALID_ARG : ps == sna::PLAN_UNSUPPORTED ? SNA_ERR_UNSUPPORTED
+             : ps == sna::PLAN_EMPTY ? SNA_ERR_EMPTY_NEIGHBORHOOD : SNA_ERR_AMBIGUOUS_TIE;
+    }
+    const sna::HostPlan& hp = plan->host;
+    if (!upload) { *plan_out = plan; return SNA_OK; }
+    // heavy-first orders
+    std::vector<int32_t> row_order(hp.nlat_out), t_row_order(hp.nlat_in);
+    std::iota(row_order.begin(), row_order.end(), 0);
+    std::iota(t_row_order.begin(), t_row_order.end(), 0);
+    std::stable_sort(row_order.begin(), row_order.end(), [&](int a, int b) { return hp.row_nnz[a] > hp.row_nnz[b]; });
+    std::stable_sort(t_row_order.begin(), t_row_order.end(), [&](int a, int b) { return hp.t_row_nnz[a] > hp.t_row_nnz[b]; });
+    std::vector<int32_t> win_lat(hp.windows.size()), win_m(hp.windows.size()), t_lat(hp.t_windows.size()), t_m(hp.t_windows.size());
+    for (size_t i = 0; i < hp.windows.size(); ++i) { win_lat[i] = hp.windows[i].lat; win_m[i] = hp.windows[i].m; }
+    for (size_t i = 0; i < hp.t_windows.size(); ++i) { t_lat[i] = hp.t_windows[i].lat; t_m[i] = hp.t_windows[i].m; }
+    std::vector<float> log2_omega(hp.nlat_in);
+    for (int h = 0; h < hp.nlat_in; ++h) log2_omega[h] = (float)std::log2(hp.omega[h]);
+
+    // pack everything into one device allocation (each array 256-byte aligned)
+    struct Piece { const void* src; size_t bytes; size_t offset; };
+    std::vector<Piece> pieces = {
+        {hp.row_ptr.data(), hp.row_ptr.size() * 4, 0}, {win_lat.data(), win_lat.size() * 4, 0}, {win_m.data(), win_m.size() * 4, 0},
+        {row_order.data(), row_order.size() * 4, 0}, {hp.t_row_ptr.data(), hp.t_row_ptr.size() * 4, 0}, {t_lat.data(), t_lat.size() * 4, 0},
+        {t_m.data(), t_m.size() * 4, 0}, {t_row_order.data(), t_row_order.size() * 4, 0}, {log2_omega.data(), log2_omega.size() * 4, 0}};
+    size_t total = 0;
+    for (Piece& p : pieces) { p.offset = total; total += round256(p.bytes); }
+    cudaError_t e = cudaGetDevice(&plan->device);
+    if (e != cudaSuccess) { delete plan; return cuda_fail(e, "cudaGetDevice"); }
+    e = cudaMalloc(&plan->dev_blob, total);
+    if (e != cudaSuccess) { delete plan; set_error("cudaMalloc of %zu bytes: %s", total, cudaGetErrorString(e)); return SNA_ERR_ALLOC; }
+    for (const Piece& p : pieces) {
+        e = cudaMemcpy((char*)plan->dev_blob + p.offset, p.src, p.bytes, cudaMemcpyHostToDevice);
+        if (e != cudaSuccess) { cudaFree(plan->dev_blob); delete plan; return cuda_fail(e, "cudaMemcpy of plan tables"); }
+    }
+    auto at = [&](int i) { return (const int32_t*)((char*)plan->dev_blob + pieces[i].offset); };
+    sna::DevPlan& d = plan->dev;
+    d.nlat_in = hp.nlat_in; d.nlon_in = hp.nlon_in; d.nlat_out = hp.nlat_out; d.nlon_out = hp.nlon_out; d.ps = hp.ps;
+    d.row_ptr = at(0); d.win_lat = at(1); d.win_m = at(2); d.row_order = at(3);
+    d.t_row_ptr = at(4); d.t_win_lat = at(5); d.t_win_m = at(6); d.t_row_order = at(7);
+    d.log2_omega = (const float*)at(8);
+    *plan_out = plan;
+    return SNA_OK;
+}
+
+sna_status_t sna_plan_create(int nlat_in, int nlon_in, int nlat_out, int nlon_out, sna_grid_t grid_in,
+                             sna_grid_t grid_out, double theta_cutoff, sna_plan_t** plan_out) {
+    return plan_create(nlat_in, nlon_in, nlat_out, nlon_out, grid_in, grid_out, theta_cutoff, true, plan_out);
+}
+
+sna_status_t sna_plan_create_host_only(int nlat_in, int nlon_in, int nlat_out, int nlon_out, sna_grid_t grid_in,
+                                       sna_grid_t grid_out, double theta_cutoff, sna_plan_t** plan_out) {
+    return plan_create(nlat_in, nlon_in, nlat_out, nlon_out, grid_in, grid_out, theta_cutoff, false, plan_out);
+}
+
+sna_status_t sna_plan_destroy(sna_plan_t* plan) {
+    if (plan == nullptr) return SNA_OK;
+    cudaError_t e1 = plan->dev_blob ? cudaFree(plan->dev_blob) : cudaSuccess;
+    cudaError_t e2 = plan->ws ? cudaFree(plan->ws) : cudaSuccess;
+    delete plan;
+    if (e1 != cudaSuccess) return cuda_fail(e1, "cudaFree");
+    if (e2 != cudaSuccess) return cuda_fail(e2, "cudaFree");
+    return SNA_OK;
+}
+
+sna_status_t sna_plan_get_nnz(const sna_plan_t* plan, int64_t* nnz) {
+    if (!plan || !nnz) { set_error("NULL argument"); return SNA_ERR_INVALID_ARG; }
+    *nnz = plan->host.nnz;
+    return SNA_OK;
+}
+
+sna_status_t sna_plan_get_colatitudes(const sna_plan_t* plan, double* theta_in, double* theta_out) {
+    if (!plan) { set_error("plan is NULL"); return SNA_ERR_INVALID_ARG; }
+    if (theta_in) std::memcpy(theta_in, plan->host.theta_in.data(), sizeof(double) * plan->host.nlat_in);
+    if (theta_out) std::memcpy(theta_out, plan->host.theta_out.data(), sizeof(double) * plan->host.nlat_out);
+    return SNA_OK;
+}
+
+sna_status_t sna_plan_get_quad_weights(const sna_plan_t* plan, double* omega_in) {
+    if (!plan || !omega_in) { set_error("NULL argument"); return SNA_ERR_INVALID_ARG; }
+    std::memcpy(omega_in, plan->host.omega.data(), sizeof(double) * plan->host.nlat_in);
+    return SNA_OK;
+}
+
+sna_status_t sna_plan_get_table(const sna_plan_t* plan, int64_t* row_ptr, int32_t* lat_in, int32_t* lon_off) {
+    if (!plan || !row_ptr || !lat_in || !lon_off) { set_error("NULL argument"); return SNA_ERR_INVALID_ARG; }
+    const sna::HostPlan& hp = plan->host;
+    int64_t n = 0;
+    for (int h = 0; h < hp.nlat_out; ++h) {
+        row_ptr[h] = n;
+        for (int e = hp.row_ptr[h]; e < hp.row_ptr[h + 1]; ++e) {
+            const sna::RingWindow& w = hp.windows[e];
+            // canonical order: offsets ascending in [0, nlon_in): 0..m first, then nlon_in-m..nlon_in-1
+            if (w.m < 0) {
+                for (int o = 0; o < hp.nlon_in; ++o) { lat_in[n] = w.lat; lon_off[n++] = o; }
+            } else {
+                for (int o = 0; o <= w.m; ++o) { lat_in[n] = w.lat; lon_off[n++] = o; }
+                for (int o = hp.nlon_in - w.m; o < hp.nlon_in; ++o) { lat_in[n] = w.lat; lon_off[n++] = o; }
+            }
+        }
+    }
+    row_ptr[hp.nlat_out] = n;
+    return SNA_OK;
+}
+
+sna_status_t sna_plan_get_table_transposed(const sna_plan_t* plan, int64_t* row_ptr, int32_t* lat_out, int32_t* lon_off) {
+    if (!plan || !row_ptr || !lat_out || !lon_off) { set_error("NULL argument"); return SNA_ERR_INVALID_ARG; }
+    const sna::HostPlan& hp = plan->host;
+    int64_t n = 0;
+    for (int hin = 0; hin < hp.nlat_in; ++hin) {
+        for (int r = 0; r < hp.ps; ++r) {
+            row_ptr[(int64_t)hin * hp.ps + r] = n;
+            for (int e = hp.t_row_ptr[hin]; e < hp.t_row_ptr[hin + 1]; ++e) {
+                const sna::RingWindow& w = hp.t_windows[e];
+                auto emit = [&](int lo, int hi) {
+                    for (int o = lo; o <= hi; ++o)
+                        if (o % hp.ps == r) { lat_out[n] = w.lat; lon_off[n++] = o; }
+                };
+                if (w.m < 0) emit(0, hp.nlon_in - 1);
+                else { emit(0, w.m); emit(hp.nlon_in - w.m, hp.nlon_in - 1); }
+            }
+        }
+    }
+    row_ptr[(int64_t)hp.nlat_in * hp.ps] = n;
+    return SNA_OK;
+}
+
+size_t sna_workspace_bytes(const sna_plan_t* plan, int B, int H, int C) {
+    if (plan == nullptr || B <= 0 || H <= 0 || C <= 0) return 0;
+    return round256(2 * stats_elems(plan, B, H) * sizeof(float));
+}
+
+sna_status_t sna_forward_ex(const sna_plan_t* plan, const float* q, const float* k, const float* v, float* out,
+                            float* lse, int B, int H, int C, void* cuda_stream) {
+    sna_status_t st = check_problem(plan, B, H, C);
+    if (st != SNA_OK) return st;
+    if (!q || !k || !v || !out) { set_error("q, k, v and out must not be NULL"); return SNA_ERR_INVALID_ARG; }
+    if (!all_aligned(q, k, v, out) || (reinterpret_cast<uintptr_t>(lse) & 3u)) { set_error("device pointers must be 16-byte aligned"); return SNA_ERR_INVALID_ARG; }
+    cudaError_t e = sna::launch_forward_generic(plan->dev, q, k, v, out, lse, B * H, C, (cudaStream_t)cuda_stream);
+    if (e != cudaSuccess) return cuda_fail(e, "forward launch");
+    return SNA_OK;
+}
+
+sna_status_t sna_forward(const sna_plan_t* plan, const float* q, const float* k, const float* v, float* out,
+                         int B, int H, int C, void* cuda_stream) {
+    return sna_forward_ex(plan, q, k, v, out, nullptr, B, H, C, cuda_stream);
+}
+
+sna_status_t sna_backward_dq(const sna_plan_t* plan, const float* q, const float* k, const float* v,
+                             const float* dout, const float* out, const float* lse, float* dq, float* D,
+                             int B, int H, int C, void* cuda_stream) {
+    sna_status_t st = check_problem(plan, B, H, C);
+    if (st != SNA_OK) return st;
+    if (!q || !k || !v || !dout || !lse || !dq || !D) { set_error("q, k, v, dout, lse, dq and D must not be NULL"); return SNA_ERR_INVALID_ARG; }
+    if (!all_aligned(q, k, v, dout, dq, out) || ((reinterpret_cast<uintptr_t>(lse) | reinterpret_cast<uintptr_t>(D)) & 3u)) { set_error("device pointers must be 16-byte aligned"); return SNA_ERR_INVALID_ARG; }
+    cudaError_t e = sna::launch_backward_dq_generic(plan->dev, q, k, v, dout, out, lse, dq, D, B * H, C, (cudaStream_t)cuda_stream);
+    if (e != cudaSuccess) return cuda_fail(e, "backward dq launch");
+    return SNA_OK;
+}
+
+sna_status_t sna_backward_dkdv(const sna_plan_t* plan, const float* q, const float* k, const float* v,
+                               const float* dout, const float* lse, const float* D, float* dk, float* dv,
+                               int B, int H, int C, void* cuda_stream) {
+    sna_status_t st = check_problem(plan, B, H, C);
+    if (st != SNA_OK) return st;
+    if (!q || !k || !v || !dout || !lse || !D || !dk || !dv) { set_error("q, k, v, dout, lse, D, dk and dv must not be NULL"); return SNA_ERR_INVALID_ARG; }
+    if (!all_aligned(q, k, v, dout, dk, dv) || ((reinterpret_cast<uintptr_t>(lse) | reinterpret_cast<uintptr_t>(D)) & 3u)) { set_error("device pointers must be 16-byte aligned"); return SNA_ERR_INVALID_ARG; }
+    cudaError_t e = sna::launch_backward_dkdv_generic(plan->dev, q, k, v, dout, lse, D, dk, dv, B * H, C, (cudaStream_t)cuda_stream);
+    if (e != cudaSuccess) return cuda_fail(e, "backward dk/dv launch");
+    return SNA_OK;
+}
+
+sna_status_t sna_backward_ex(const sna_plan_t* plan, const float* q, const float* k, const float* v,
+                             const float* dout, const float* out, const float* lse, float* dq, float* dk, float* dv,
+                             void* workspace, size_t workspace_bytes, int B, int H, int C, void* cuda_stream) {
+    sna_status_t st = check_problem(plan, B, H, C);
+    if (st != SNA_OK) return st;
+    if (!q || !k || !v || !dout || !dq || !dk || !dv) { set_error("q, k, v, dout, dq, dk and dv must not be NULL"); return SNA_ERR_INVALID_ARG; }
+    if (!all_aligned(q, k, v, dout, dq, dk, dv, out) || (reinterpret_cast<uintptr_t>(lse) & 3u)) { set_error("device pointers must be 16-byte aligned"); return SNA_ERR_INVALID_ARG; }
+    if (workspace == nullptr || (reinterpret_cast<uintptr_t>(workspace) & 255u)) { set_error("workspace must be non-NULL and 256-byte aligned"); return SNA_ERR_INVALID_ARG; }
+    if (workspace_bytes < sna_workspace_bytes(plan, B, H, C)) { set_error("workspace too small: %zu < %zu bytes", workspace_bytes, sna_workspace_bytes(plan, B, H, C)); return SNA_ERR_WORKSPACE; }
+    cudaStream_t stream = (cudaStream_t)cuda_stream;
+    const int N = B * H;
+    float* ws_lse = (float*)workspace;
+    float* ws_D = ws_lse + stats_elems(plan, B, H);
+    cudaError_t e;
+    if (lse == nullptr) {   // recompute the softmax statistics
+        e = sna::launch_forward_generic(plan->dev, q, k, v, nullptr, ws_lse, N, C, stream);
+        if (e != cudaSuccess) return cuda_fail(e, "statistics launch");
+        lse = ws_lse;
+    }
+    st = sna_backward_dq(plan, q, k, v, dout, out, lse, dq, ws_D, B, H, C, cuda_stream);
+    if (st != SNA_OK) return st;
+    return sna_backward_dkdv(plan, q, k, v, dout, lse, ws_D, dk, dv, B, H, C, cuda_stream);
+}
+
+sna_status_t sna_backward(const sna_plan_t* plan, const float* q, const float* k, const float* v, const float* dout,
+                          float* dq, float* dk, float* dv, int B, int H, int C, void* cuda_stream) {
+    sna_status_t st = check_problem(plan, B, H, C);
+    if (st != SNA_OK) return st;
+    const size_t need = sna_workspace_bytes(plan, B, H, C);
+    void* ws;
+    {
+        std::lock_guard<std::mutex> lock(plan->ws_mutex);
+        if (plan->ws_bytes < need) {
+            // a larger workspace than ever before: wait for work that may still use the old one, then replace it
+            cudaError_t e = cudaDeviceSynchronize();
+            if (e != cudaSuccess) return cuda_fail(e, "cudaDeviceSynchronize");
+            if (plan->ws) cudaFree(plan->ws);
+            plan->ws = nullptr;
+            plan->ws_bytes = 0;
+            e = cudaMalloc(&plan->ws, need);
+            if (e != cudaSuccess) { set_error("cudaMalloc of %zu workspace bytes: %s", need, cudaGetErrorString(e)); return SNA_ERR_ALLOC; }
+            plan->ws_bytes = need;
+        }
+        ws = plan->ws;
+    }
+    return sna_backward_ex(plan, q, k, v, dout, nullptr, nullptr, dq, dk, dv, ws, need, B, H, C, cuda_stream);
+}
+
+}  // extern "C"

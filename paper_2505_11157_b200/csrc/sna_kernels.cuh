@@ -1,0 +1,38 @@
+// Device-side view of a plan and the launchers of the CUDA kernels.
+#pragma once
+#include <cuda_runtime.h>
+#include <cstdint>
+
+namespace sna {
+
+// All pointers are device memory owned by the plan.
+struct DevPlan {
+    int nlat_in, nlon_in, nlat_out, nlon_out, ps;
+    // forward table, run-length form: windows [row_ptr[h], row_ptr[h+1]) of output latitude h
+    const int32_t* row_ptr;
+    const int32_t* win_lat;     // input ring
+    const int32_t* win_m;       // half width in input columns, -1 = whole ring
+    const int32_t* row_order;   // output latitudes, most table entries first
+    // transposed table: windows [t_row_ptr[h'], t_row_ptr[h'+1]) of input latitude h'
+    const int32_t* t_row_ptr;
+    const int32_t* t_win_lat;   // output ring
+    const int32_t* t_win_m;
+    const int32_t* t_row_order; // input latitudes, most work first
+    const float* log2_omega;    // [nlat_in] log2 of the per-point quadrature weight
+};
+
+// Generic kernels (any supported C): C/4 lanes cooperate on one grid point.
+// forward: out and/or lse may be null (lse-only pass = softmax statistics).
+cudaError_t launch_forward_generic(const DevPlan& p, const float* q, const float* k, const float* v, float* out,
+                                   float* lse, int N, int C, cudaStream_t stream);
+// dq pass.  lse is required.  If out != null, D_i = dout_i . out_i is used; otherwise D_i is accumulated.
+// Writes dq and Dws[i] = D_i.
+cudaError_t launch_backward_dq_generic(const DevPlan& p, const float* q, const float* k, const float* v,
+                                       const float* dout, const float* out, const float* lse, float* dq, float* Dws,
+                                       int N, int C, cudaStream_t stream);
+// dk, dv gather pass over the transposed table; needs lse and D of every output point.
+cudaError_t launch_backward_dkdv_generic(const DevPlan& p, const float* q, const float* k, const float* v,
+                                         const float* dout, const float* lse, const float* Dws, float* dk, float* dv,
+                                         int N, int C, cudaStream_t stream);
+
+}  // namespace sna

@@ -1,0 +1,188 @@
+// Host planner.  Grids and quadrature: App. A.1 and Eq. (quadrature); neighborhood indicator: App. B.3,
+// disc of Eq. (s2_neighborhood_attention).
+//
+// Construction (deliberately not a brute-force scan): on a fixed input ring the geodesic distance to the
+// output point grows monotonically with the longitude difference, so each ring contributes one window
+// symmetric about offset 0.  The half width follows from the spherical law of cosines,
+//     cos(dphi_max) = (cos(theta_c) - cos(t_o) cos(t_i)) / (sin(t_o) sin(t_i)),
+// and the columns around that estimate are then tested exactly with a cross/dot (atan2) distance, which is
+// accurate for small and large angles alike.  Boundary ties are members (d <= theta_c + 1e-10); a candidate in
+// the band 1e-12 < |d - theta_c| < 1e-8 aborts the build as ambiguous.
+#include "sna_plan.hpp"
+
+#include <algorithm>
+#include <cmath>
+
+namespace sna {
+namespace {
+
+const long double PI_L = 3.14159265358979323846264338327950288L;
+const double TIE_SLACK = 1e-10, BAND_LO = 1e-12, BAND_HI = 1e-8;
+
+// Gauss-Legendre nodes (descending) and weights by Newton iteration in extended precision, started from
+// Tricomi's asymptotic estimate of the roots.
+void legendre_gauss(int n, std::vector<double>& x, std::vector<double>& w) {
+    x.resize(n);
+    w.resize(n);
+    for (int i = 1; i <= (n + 1) / 2; ++i) {
+        long double z = (1.0L - (n - 1.0L) / (8.0L * n * n * n)) * cosl(PI_L * (4.0L * i - 1.0L) / (4.0L * n + 2.0L));
+        long double pn = 0, pn1 = 0;
+        for (int it = 0; it < 64; ++it) {
+            long double a = 1.0L, b = z;   // P_0, P_1
+            for (int l = 1; l < n; ++l) {
+                long double c = ((2 * l + 1) * z * b - l * a) / (l + 1);
+                a = b;
+                b = c;
+            }
+            pn = b;
+            pn1 = a;
+            long double deriv = n * (pn1 - z * pn) / (1.0L - z * z);
+            long double step = pn / deriv;
+            z -= step;
+            if (fabsl(step) < 1e-19L) break;
+        }
+        // re-evaluate at the converged node for the weight
+        long double a = 1.0L, b = z;
+        for (int l = 1; l < n; ++l) {
+            long double c = ((2 * l + 1) * z * b - l * a) / (l + 1);
+            a = b;
+            b = c;
+        }
+        long double deriv = n * (a - z * b) / (1.0L - z * z);
+        long double wt = 2.0L / ((1.0L - z * z) * deriv * deriv);
+        x[i - 1] = (double)z;
+        w[i - 1] = (double)wt;
+        x[n - i] = (double)(-z);
+        w[n - i] = (double)wt;
+    }
+    if (n % 2 == 1) x[n / 2] = 0.0;
+}
+
+// Clenshaw-Curtis weights on nlat equally spaced colatitudes including both poles.
+void clenshaw_curtis(int nlat, std::vector<double>& w) {
+    const int n = nlat - 1;
+    w.resize(nlat);
+    for (int h = 0; h <= n; ++h) {
+        long double acc = 1.0L;
+        for (int k = 1; k <= n / 2; ++k) {
+            long long arg = (2LL * k * h) % (2LL * n);           // cos(2 k pi h / n) with an exactly reduced argument
+            long double bk = (2 * k == n) ? 1.0L : 2.0L;
+            acc -= bk * cosl(PI_L * (long double)arg / (long double)n) / (4.0L * k * k - 1.0L);
+        }
+        long double ch = (h == 0 || h == n) ? 1.0L : 2.0L;
+        w[h] = (double)(ch * acc / n);
+    }
+}
+
+bool make_grid(int grid, int nlat, std::vector<double>& theta, std::vector<double>& wlat) {
+    if (grid == 0) {
+        theta.resize(nlat);
+        for (int h = 0; h < nlat; ++h) theta[h] = (double)(PI_L * h / (nlat - 1));
+        clenshaw_curtis(nlat, wlat);
+        return true;
+    }
+    if (grid == 1) {
+        std::vector<double> x;
+        legendre_gauss(nlat, x, wlat);
+        theta.resize(nlat);
+        for (int h = 0; h < nlat; ++h) theta[h] = std::acos(x[h]);
+        return true;
+    }
+    return false;
+}
+
+// Geodesic distance between (t_o, 0) and (t_i, phi) from cross and dot products of the unit vectors.
+double geodesic(double so, double co, double si, double ci, double phi) {
+    const double cp = std::cos(phi), sp = std::sin(phi);
+    const double ox = so, oz = co;
+    const double ix = si * cp, iy = si * sp, iz = ci;
+    const double cx = -oz * iy, cy = oz * ix - ox * iz, cz = ox * iy;
+    return std::atan2(std::sqrt(cx * cx + cy * cy + cz * cz), ox * ix + oz * iz);
+}
+
+}  // namespace
+
+PlanStatus build_plan(int nlat_in, int nlon_in, int nlat_out, int nlon_out, int grid_in, int grid_out,
+                      double theta_cutoff, HostPlan& P, std::string& why) {
+    if (nlat_in < 2 || nlat_out < 2 || nlon_in < 1 || nlon_out < 1) { why = "nlat must be >= 2 and nlon >= 1"; return PLAN_INVALID; }
+    if (!(theta_cutoff > 0.0) || std::isnan(theta_cutoff)) { why = "theta_cutoff must be positive"; return PLAN_INVALID; }
+    if (nlon_in % nlon_out != 0) { why = "nlon_in must be a multiple of nlon_out"; return PLAN_UNSUPPORTED; }
+    P = HostPlan();
+    P.nlat_in = nlat_in; P.nlon_in = nlon_in; P.nlat_out = nlat_out; P.nlon_out = nlon_out;
+    P.ps = nlon_in / nlon_out; P.grid_in = grid_in; P.grid_out = grid_out; P.theta_cutoff = theta_cutoff;
+    std::vector<double> wlat_in, wlat_out;
+    if (!make_grid(grid_in, nlat_in, P.theta_in, wlat_in) || !make_grid(grid_out, nlat_out, P.theta_out, wlat_out)) {
+        why = "unknown grid type";
+        return PLAN_UNSUPPORTED;
+    }
+    P.omega.resize(nlat_in);
+    for (int h = 0; h < nlat_in; ++h) P.omega[h] = wlat_in[h] * (double)(2.0L * PI_L / nlon_in);
+
+    const bool everything = theta_cutoff >= (double)PI_L;
+    const int half = nlon_in / 2;                        // largest |column offset| on a ring
+    const double dphi = (double)(2.0L * PI_L / nlon_in);
+    const double cos_tc = std::cos(theta_cutoff);
+    bool ambiguous = false;
+    auto member = [&](double d) {
+        const double gap = std::fabs(d - theta_cutoff);
+        if (gap > BAND_LO && gap < BAND_HI) ambiguous = true;
+        return d <= theta_cutoff + TIE_SLACK;
+    };
+
+    P.row_ptr.assign(nlat_out + 1, 0);
+    P.row_nnz.assign(nlat_out, 0);
+    std::vector<std::vector<RingWindow>> by_input(nlat_in);
+    for (int h = 0; h < nlat_out; ++h) {
+        const double so = std::sin(P.theta_out[h]), co = std::cos(P.theta_out[h]);
+        for (int hp = 0; hp < nlat_in; ++hp) {
+            int m = -2;   // -2: ring not in the disc, -1: whole ring, >= 0: half width
+            if (everything) {
+                m = -1;
+            } else {
+                const double si = std::sin(P.theta_in[hp]), ci = std::cos(P.theta_in[hp]);
+                if (!member(geodesic(so, co, si, ci, 0.0))) continue;   // nearest point of the ring is outside
+                const double denom = so * si;
+                int guess;
+                if (denom < 1e-300) {
+                    guess = half;   // a pole is involved: every column is equally far
+                } else {
+                    const double r = (cos_tc - co * ci) / denom;
+                    guess = r <= -1.0 ? half : (r >= 1.0 ? 0 : (int)std::floor(std::acos(r) / dphi));
+                }
+                // exact test around the estimate; membership is monotone in the offset
+                int lo = std::max(0, guess - 2), hi = std::min(half, guess + 2);
+                while (lo > 0 && !member(geodesic(so, co, si, ci, lo * dphi))) lo = std::max(0, lo - 4);
+                m = lo;
+                for (int j = lo + 1; j <= hi; ++j) {
+                    if (member(geodesic(so, co, si, ci, j * dphi))) m = j; else break;
+                }
+                if (m == hi && hi < half) {   // estimate was too small (never seen, but stay correct)
+                    int j = hi + 1;
+                    while (j <= half && member(geodesic(so, co, si, ci, j * dphi))) m = j++;
+                }
+                if (2 * m + 1 >= nlon_in) m = -1;
+            }
+            RingWindow w{hp, m};
+            P.windows.push_back(w);
+            P.row_nnz[h] += P.window_count(w);
+            by_input[hp].push_back(RingWindow{h, m});
+        }
+        P.row_ptr[h + 1] = (int32_t)P.windows.size();
+        if (P.row_ptr[h + 1] == P.row_ptr[h] && !ambiguous) { why = "an output latitude has no input point within theta_cutoff"; return PLAN_EMPTY; }
+        P.nnz += P.row_nnz[h];
+    }
+    if (ambiguous) { why = "a grid point lies within 1e-8 rad of the disc boundary without being on it"; return PLAN_AMBIGUOUS; }
+
+    P.t_row_ptr.assign(nlat_in + 1, 0);
+    P.t_row_nnz.assign(nlat_in, 0);
+    for (int hp = 0; hp < nlat_in; ++hp) {
+        for (const RingWindow& w : by_input[hp]) {
+            P.t_windows.push_back(w);
+            P.t_row_nnz[hp] += P.window_count(w);
+        }
+        P.t_row_ptr[hp + 1] = (int32_t)P.t_windows.size();
+    }
+    return PLAN_OK;
+}
+
+}  // namespace sna

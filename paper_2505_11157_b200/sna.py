@@ -1,0 +1,255 @@
+"""Thin Python binding of the C ABI in ``include/sna.h`` (ctypes).
+
+Only argument marshalling happens here: tensors are handed over as raw device pointers, the stream as a
+``cudaStream_t``.  Every step of the computation runs in the library's CUDA kernels.  PyTorch provides device
+memory and streams, nothing else.  There is no CPU fallback: if the shared library is missing, importing this
+module raises.
+
+The module-level functions carry the names of the C entry points; :class:`Plan` is a convenience wrapper
+around them.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import Optional
+
+import numpy as np
+
+_PKG = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_PKG, "libsna.so")
+
+SNA_GRID_EQUIANGULAR = 0
+SNA_GRID_LEGENDRE_GAUSS = 1
+
+SNA_OK = 0
+SNA_ERR_INVALID_ARG = 1
+SNA_ERR_UNSUPPORTED = 2
+SNA_ERR_EMPTY_NEIGHBORHOOD = 3
+SNA_ERR_ALLOC = 4
+SNA_ERR_CUDA = 5
+SNA_ERR_AMBIGUOUS_TIE = 6
+SNA_ERR_WORKSPACE = 7
+
+if not os.path.exists(LIB_PATH):
+    raise ImportError(
+        f"{LIB_PATH} is missing: build it first (python -m paper_2505_11157_b200.build). "
+        "There is no fallback implementation.")
+
+_lib = ctypes.CDLL(LIB_PATH)
+
+_vp, _i, _d, _sz = ctypes.c_void_p, ctypes.c_int, ctypes.c_double, ctypes.c_size_t
+_SIGNATURES = {
+    "sna_plan_create": (_i, [_i, _i, _i, _i, _i, _i, _d, ctypes.POINTER(_vp)]),
+    "sna_plan_create_host_only": (_i, [_i, _i, _i, _i, _i, _i, _d, ctypes.POINTER(_vp)]),
+    "sna_plan_destroy": (_i, [_vp]),
+    "sna_plan_get_nnz": (_i, [_vp, ctypes.POINTER(ctypes.c_int64)]),
+    "sna_plan_get_colatitudes": (_i, [_vp, _vp, _vp]),
+    "sna_plan_get_quad_weights": (_i, [_vp, _vp]),
+    "sna_plan_get_table": (_i, [_vp, _vp, _vp, _vp]),
+    "sna_plan_get_table_transposed": (_i, [_vp, _vp, _vp, _vp]),
+    "sna_workspace_bytes": (_sz, [_vp, _i, _i, _i]),
+    "sna_forward": (_i, [_vp, _vp, _vp, _vp, _vp, _i, _i, _i, _vp]),
+    "sna_forward_ex": (_i, [_vp, _vp, _vp, _vp, _vp, _vp, _i, _i, _i, _vp]),
+    "sna_backward": (_i, [_vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _i, _i, _i, _vp]),
+    "sna_backward_ex": (_i, [_vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _sz, _i, _i, _i, _vp]),
+    "sna_backward_dq": (_i, [_vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _i, _i, _i, _vp]),
+    "sna_backward_dkdv": (_i, [_vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _i, _i, _i, _vp]),
+    "sna_status_string": (ctypes.c_char_p, [_i]),
+    "sna_last_error_message": (ctypes.c_char_p, []),
+}
+for _name, (_res, _args) in _SIGNATURES.items():
+    _fn = getattr(_lib, _name)
+    _fn.restype = _res
+    _fn.argtypes = _args
+
+
+class SnaError(RuntimeError):
+    def __init__(self, status: int):
+        self.status = status
+        name = _lib.sna_status_string(status).decode()
+        detail = _lib.sna_last_error_message().decode()
+        super().__init__(f"{name}: {detail}" if detail else name)
+
+
+def _check(status: int):
+    if status != SNA_OK:
+        raise SnaError(status)
+
+
+def _ptr(t) -> Optional[int]:
+    """Device pointer of a CUDA tensor (or pass through an int / None)."""
+    if t is None:
+        return None
+    if isinstance(t, int):
+        return t
+    if not t.is_cuda:
+        raise ValueError("expected a CUDA tensor")
+    if not t.is_contiguous():
+        raise ValueError("tensor must be contiguous")
+    return t.data_ptr()
+
+
+def _stream(stream) -> Optional[int]:
+    if stream is None:
+        import torch
+        return torch.cuda.current_stream().cuda_stream or None
+    if isinstance(stream, int):
+        return stream or None
+    return stream.cuda_stream or None
+
+
+# ---- functions with the names of the C entry points --------------------------------------------------------
+
+def sna_plan_create(nlat_in, nlon_in, nlat_out, nlon_out, grid_in, grid_out, theta_cutoff, host_only=False) -> int:
+    handle = _vp()
+    fn = _lib.sna_plan_create_host_only if host_only else _lib.sna_plan_create
+    _check(fn(nlat_in, nlon_in, nlat_out, nlon_out, grid_in, grid_out, float(theta_cutoff), ctypes.byref(handle)))
+    return handle.value
+
+
+def sna_plan_create_host_only(nlat_in, nlon_in, nlat_out, nlon_out, grid_in, grid_out, theta_cutoff) -> int:
+    return sna_plan_create(nlat_in, nlon_in, nlat_out, nlon_out, grid_in, grid_out, theta_cutoff, host_only=True)
+
+
+def sna_plan_destroy(plan: int):
+    _check(_lib.sna_plan_destroy(plan))
+
+
+def sna_plan_get_nnz(plan: int) -> int:
+    n = ctypes.c_int64()
+    _check(_lib.sna_plan_get_nnz(plan, ctypes.byref(n)))
+    return n.value
+
+
+def sna_workspace_bytes(plan: int, B: int, H: int, C: int) -> int:
+    return int(_lib.sna_workspace_bytes(plan, B, H, C))
+
+
+def sna_forward(plan, q, k, v, out, B, H, C, stream=None):
+    _check(_lib.sna_forward(plan, _ptr(q), _ptr(k), _ptr(v), _ptr(out), B, H, C, _stream(stream)))
+
+
+def sna_forward_ex(plan, q, k, v, out, lse, B, H, C, stream=None):
+    _check(_lib.sna_forward_ex(plan, _ptr(q), _ptr(k), _ptr(v), _ptr(out), _ptr(lse), B, H, C, _stream(stream)))
+
+
+def sna_backward(plan, q, k, v, dout, dq, dk, dv, B, H, C, stream=None):
+    _check(_lib.sna_backward(plan, _ptr(q), _ptr(k), _ptr(v), _ptr(dout), _ptr(dq), _ptr(dk), _ptr(dv), B, H, C,
+                             _stream(stream)))
+
+
+def sna_backward_ex(plan, q, k, v, dout, out, lse, dq, dk, dv, workspace, workspace_bytes, B, H, C, stream=None):
+    _check(_lib.sna_backward_ex(plan, _ptr(q), _ptr(k), _ptr(v), _ptr(dout), _ptr(out), _ptr(lse), _ptr(dq), _ptr(dk),
+                                _ptr(dv), _ptr(workspace), workspace_bytes, B, H, C, _stream(stream)))
+
+
+def sna_backward_dq(plan, q, k, v, dout, out, lse, dq, D, B, H, C, stream=None):
+    _check(_lib.sna_backward_dq(plan, _ptr(q), _ptr(k), _ptr(v), _ptr(dout), _ptr(out), _ptr(lse), _ptr(dq), _ptr(D),
+                                B, H, C, _stream(stream)))
+
+
+def sna_backward_dkdv(plan, q, k, v, dout, lse, D, dk, dv, B, H, C, stream=None):
+    _check(_lib.sna_backward_dkdv(plan, _ptr(q), _ptr(k), _ptr(v), _ptr(dout), _ptr(lse), _ptr(D), _ptr(dk), _ptr(dv),
+                                  B, H, C, _stream(stream)))
+
+
+# ---- convenience wrapper -----------------------------------------------------------------------------------
+
+class Plan:
+    """Owns one ``sna_plan_t``.  Shapes follow the header: q/out [B,H,nlat_out,nlon_out,C], k/v [B,H,nlat_in,nlon_in,C]."""
+
+    def __init__(self, nlat_in, nlon_in, nlat_out, nlon_out, grid_in=SNA_GRID_EQUIANGULAR,
+                 grid_out=SNA_GRID_EQUIANGULAR, theta_cutoff=0.1, host_only=False):
+        self.nlat_in, self.nlon_in, self.nlat_out, self.nlon_out = nlat_in, nlon_in, nlat_out, nlon_out
+        self.grid_in, self.grid_out, self.theta_cutoff = grid_in, grid_out, float(theta_cutoff)
+        self.host_only = host_only
+        self.handle = None
+        self.handle = sna_plan_create(nlat_in, nlon_in, nlat_out, nlon_out, grid_in, grid_out, theta_cutoff, host_only)
+        self.ps = nlon_in // nlon_out
+
+    def close(self):
+        if self.handle is not None:
+            handle, self.handle = self.handle, None
+            sna_plan_destroy(handle)
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    def __enter__(self):
+        return self
+
+    def __exit__(self, *exc):
+        self.close()
+
+    # introspection (host)
+    @property
+    def nnz(self) -> int:
+        return sna_plan_get_nnz(self.handle)
+
+    def colatitudes(self):
+        ti = np.empty(self.nlat_in, dtype=np.float64)
+        to = np.empty(self.nlat_out, dtype=np.float64)
+        _check(_lib.sna_plan_get_colatitudes(self.handle, ti.ctypes.data, to.ctypes.data))
+        return ti, to
+
+    def quad_weights(self):
+        w = np.empty(self.nlat_in, dtype=np.float64)
+        _check(_lib.sna_plan_get_quad_weights(self.handle, w.ctypes.data))
+        return w
+
+    def table(self):
+        nnz = self.nnz
+        row_ptr = np.empty(self.nlat_out + 1, dtype=np.int64)
+        lat = np.empty(nnz, dtype=np.int32)
+        off = np.empty(nnz, dtype=np.int32)
+        _check(_lib.sna_plan_get_table(self.handle, row_ptr.ctypes.data, lat.ctypes.data, off.ctypes.data))
+        return row_ptr, lat, off
+
+    def table_transposed(self):
+        nnz = self.nnz
+        row_ptr = np.empty(self.nlat_in * self.ps + 1, dtype=np.int64)
+        lat = np.empty(nnz, dtype=np.int32)
+        off = np.empty(nnz, dtype=np.int32)
+        _check(_lib.sna_plan_get_table_transposed(self.handle, row_ptr.ctypes.data, lat.ctypes.data, off.ctypes.data))
+        return row_ptr, lat, off
+
+    # compute (device tensors)
+    def _bhc(self, q, k):
+        if q.dim() != 5 or k.dim() != 5:
+            raise ValueError("q and k must be [B, H, nlat, nlon, C]")
+        B, H, C = q.shape[0], q.shape[1], q.shape[4]
+        if tuple(q.shape[2:4]) != (self.nlat_out, self.nlon_out) or tuple(k.shape) != (B, H, self.nlat_in, self.nlon_in, C):
+            raise ValueError("tensor shapes do not match the plan")
+        return B, H, C
+
+    def workspace_bytes(self, B, H, C) -> int:
+        return sna_workspace_bytes(self.handle, B, H, C)
+
+    def forward(self, q, k, v, out=None, lse=None, return_lse=False, stream=None):
+        import torch
+        B, H, C = self._bhc(q, k)
+        if out is None:
+            out = torch.empty_like(q)
+        if return_lse and lse is None:
+            lse = torch.empty(q.shape[:-1], dtype=torch.float32, device=q.device)
+        sna_forward_ex(self.handle, q, k, v, out, lse, B, H, C, stream)
+        return (out, lse) if return_lse else out
+
+    def backward(self, q, k, v, dout, out=None, lse=None, dq=None, dk=None, dv=None, workspace=None, stream=None):
+        import torch
+        B, H, C = self._bhc(q, k)
+        dq = torch.empty_like(q) if dq is None else dq
+        dk = torch.empty_like(k) if dk is None else dk
+        dv = torch.empty_like(k) if dv is None else dv
+        if workspace is None and out is None and lse is None:
+            sna_backward(self.handle, q, k, v, dout, dq, dk, dv, B, H, C, stream)
+        else:
+            need = self.workspace_bytes(B, H, C)
+            if workspace is None:
+                workspace = torch.empty(need, dtype=torch.uint8, device=q.device)
+            sna_backward_ex(self.handle, q, k, v, dout, out, lse, dq, dk, dv, workspace, workspace.numel(), B, H, C, stream)
+        return dq, dk, dv

@@ -1,0 +1,114 @@
+"""CPU tests of the C-ABI library: it loads, exports what the header declares, and its host planner
+reproduces the oracle's grids, weights and tables bit for bit (no GPU, no compute calls)."""
+import ctypes
+import math
+import os
+import re
+
+import numpy as np
+import pytest
+
+from oracle import sna_oracle as orc
+from paper_2505_11157_b200 import sna
+from paper_2505_11157_b200.synthetic import WORKLOADS
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+EQ, GL = 0, 1
+
+
+def _declared_functions():
+    text = open(os.path.join(ROOT, "include", "sna.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(sna_[a-z_0-9]+)\s*\(", text)))
+
+
+def test_library_exports_every_declared_symbol():
+    names = _declared_functions()
+    assert "sna_plan_create" in names and "sna_forward" in names and "sna_backward" in names and len(names) >= 14
+    lib = ctypes.CDLL(sna.LIB_PATH)
+    for name in names:
+        assert hasattr(lib, name), f"{name} is declared in sna.h but not exported"
+    # and the binding names every one of them
+    for name in names:
+        assert name in sna._SIGNATURES, f"binding lacks {name}"
+
+
+def test_status_strings():
+    assert sna._lib.sna_status_string(0) == b"SNA_OK"
+    assert sna._lib.sna_status_string(6) == b"SNA_ERR_AMBIGUOUS_TIE"
+
+
+CASES = {
+    "c1": (32, 64, 32, 64, EQ, EQ, 0.3),
+    "c2": (128, 256, 128, 256, EQ, EQ, 4 * math.pi / 127),
+    "c5": (64, 128, 64, 128, EQ, EQ, math.pi),
+    "down2": (33, 64, 17, 32, EQ, EQ, 2 * math.pi / 16),
+    "down4_mixed": (24, 48, 9, 12, GL, EQ, 0.6),
+    "gl": (24, 48, 24, 48, GL, GL, 0.37),
+    "gl_c4_like": (61, 120, 61, 120, GL, GL, 5 * math.pi / 60),
+    "odd_nlon": (10, 15, 10, 15, EQ, EQ, 0.8),
+    "tiny": (4, 8, 4, 8, EQ, EQ, 1.1),
+    "wide": (16, 32, 16, 32, EQ, EQ, 2.5),
+}
+
+
+@pytest.mark.parametrize("name", list(CASES))
+def test_planner_matches_oracle_bit_for_bit(name):
+    args = CASES[name]
+    g = orc.geometry(*args)
+    with sna.Plan(*args, host_only=True) as p:
+        assert p.nnz == g.nnz
+        row_ptr, lat, off = p.table()
+        assert np.array_equal(row_ptr, g.row_ptr)
+        assert np.array_equal(lat, g.lat_in)
+        assert np.array_equal(off, g.lon_off)
+        ti, to = p.colatitudes()
+        assert np.allclose(ti, orc.colatitudes(args[4], args[0]), rtol=0, atol=2e-15)
+        assert np.allclose(to, orc.colatitudes(args[5], args[2]), rtol=0, atol=2e-15)
+        assert np.allclose(p.quad_weights(), g.omega, rtol=1e-13, atol=0)
+        assert abs(p.quad_weights().sum() * args[1] - 4 * math.pi) < 1e-12
+        # transposed table, rebuilt here from the oracle's table
+        ps = args[1] // args[3]
+        t_ptr, t_lat, t_off = p.table_transposed()
+        h_of_entry = np.repeat(np.arange(args[2]), np.diff(g.row_ptr))
+        expect = []
+        for hin in range(args[0]):
+            for r in range(ps):
+                sel = (g.lat_in == hin) & (g.lon_off % ps == r)
+                expect.append(sorted(zip(h_of_entry[sel].tolist(), g.lon_off[sel].tolist())))
+        assert t_ptr[-1] == g.nnz
+        for row, exp in enumerate(expect):
+            got = list(zip(t_lat[t_ptr[row]:t_ptr[row + 1]].tolist(), t_off[t_ptr[row]:t_ptr[row + 1]].tolist()))
+            assert got == exp, row
+
+
+def test_headline_table_sizes():
+    for name, nnz in (("c3", 53800), ("c4", 98995)):
+        wl = WORKLOADS[name]
+        with sna.Plan(wl.nlat_in, wl.nlon_in, wl.nlat_out, wl.nlon_out, wl.grid_in, wl.grid_out, wl.theta_cutoff,
+                      host_only=True) as p:
+            assert p.nnz == nnz
+
+
+@pytest.mark.parametrize("args, status", [
+    ((8, 16, 8, 5, EQ, EQ, 0.5), sna.SNA_ERR_UNSUPPORTED),
+    ((8, 16, 8, 16, EQ, 5, 0.5), sna.SNA_ERR_UNSUPPORTED),
+    ((1, 16, 8, 16, EQ, EQ, 0.5), sna.SNA_ERR_INVALID_ARG),
+    ((8, 16, 8, 16, EQ, EQ, 0.0), sna.SNA_ERR_INVALID_ARG),
+    ((8, 16, 8, 16, EQ, EQ, float("nan")), sna.SNA_ERR_INVALID_ARG),
+    ((5, 8, 16, 8, EQ, GL, 0.02), sna.SNA_ERR_EMPTY_NEIGHBORHOOD),
+    ((17, 32, 17, 32, EQ, EQ, 2 * math.pi / 16 + 1e-10), sna.SNA_ERR_AMBIGUOUS_TIE),
+])
+def test_plan_errors(args, status):
+    with pytest.raises(sna.SnaError) as e:
+        sna.Plan(*args, host_only=True)
+    assert e.value.status == status
+    assert str(e.value)
+
+
+def test_host_only_plan_refuses_to_compute():
+    with sna.Plan(8, 16, 8, 16, EQ, EQ, 0.5, host_only=True) as p:
+        assert sna._lib.sna_forward(p.handle, 16, 16, 16, 16, 1, 1, 4, None) == sna.SNA_ERR_INVALID_ARG
+        assert sna._lib.sna_forward(None, 16, 16, 16, 16, 1, 1, 4, None) == sna.SNA_ERR_INVALID_ARG
+        assert sna.sna_workspace_bytes(p.handle, 2, 3, 4) == 2 * 3 * 8 * 16 * 2 * 4
+        assert sna.sna_workspace_bytes(p.handle, 0, 3, 4) == 0

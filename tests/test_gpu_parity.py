@@ -1,0 +1,203 @@
+"""GPU parity: the CUDA path (through the C ABI) against the fp64 CPU oracle on the same seeded inputs.
+
+Gate (stated by the benchmark definition): neighborhood tables bit-exact; normalised max error
+max|x - o| / max|o| per tensor <= 1e-5 for the forward output and <= 1e-4 for each of dq, dk, dv.
+"""
+import math
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import sna_oracle as orc
+from paper_2505_11157_b200 import sna
+from paper_2505_11157_b200.synthetic import WORKLOADS, make_inputs, sample_points, small_workload
+
+pytestmark = pytest.mark.gpu
+
+EQ, GL = 0, 1
+FWD_TOL, BWD_TOL = 1e-5, 1e-4
+
+
+def nerr(x, ref):
+    """Normalised max error of a tensor against the oracle's."""
+    x = np.asarray(x, dtype=np.float64)
+    return float(np.max(np.abs(x - ref)) / np.max(np.abs(ref)))
+
+
+def _geometry(wl):
+    return orc.geometry(wl.nlat_in, wl.nlon_in, wl.nlat_out, wl.nlon_out, wl.grid_in, wl.grid_out, wl.theta_cutoff)
+
+
+def _plan(wl):
+    return sna.Plan(wl.nlat_in, wl.nlon_in, wl.nlat_out, wl.nlon_out, wl.grid_in, wl.grid_out, wl.theta_cutoff)
+
+
+def _dev(*arrays):
+    return [torch.from_numpy(a).cuda() for a in arrays]
+
+
+def _run_gpu(plan, q, k, v, dout, reuse_forward_state=True):
+    qd, kd, vd, dd = _dev(q, k, v, dout)
+    out, lse = plan.forward(qd, kd, vd, return_lse=True)
+    if reuse_forward_state:
+        dq, dk, dv = plan.backward(qd, kd, vd, dd, out=out, lse=lse)
+    else:
+        dq, dk, dv = plan.backward(qd, kd, vd, dd)
+    torch.cuda.synchronize()
+    return [t.cpu().numpy() for t in (out, lse, dq, dk, dv)]
+
+
+SMALL = [
+    # name, nlat_in, nlon_in, nlat_out, nlon_out, grid_in, grid_out, theta, B, H, C, seed
+    small_workload("eq_c32", 24, 48, 24, 48, EQ, EQ, 0.45, 1, 3, 32, 10),
+    small_workload("eq_c32_ragged", 19, 90, 19, 90, EQ, EQ, 0.3, 2, 1, 32, 11),           # 90 is not a tile multiple
+    small_workload("eq_down2_c32", 33, 64, 17, 32, EQ, EQ, 2 * math.pi / 16, 1, 2, 32, 12),
+    small_workload("gl_c32", 20, 40, 20, 40, GL, GL, 0.5, 2, 2, 32, 13),
+    small_workload("gl_to_eq_down4_c16", 24, 48, 9, 12, GL, EQ, 0.6, 1, 2, 16, 14),
+    small_workload("eq_c4", 12, 24, 12, 24, EQ, EQ, 0.6, 1, 2, 4, 15),
+    small_workload("eq_c8_oddlon", 10, 15, 10, 15, EQ, EQ, 0.8, 1, 1, 8, 16),
+    small_workload("eq_c64", 16, 32, 16, 32, EQ, EQ, 0.5, 1, 1, 64, 17),
+    small_workload("eq_c128", 12, 24, 12, 24, EQ, EQ, 0.7, 1, 1, 128, 18),
+    small_workload("global_c32", 12, 24, 12, 24, EQ, EQ, math.pi, 1, 2, 32, 19),
+    small_workload("eq_wide_c32", 40, 160, 40, 160, EQ, EQ, 0.5, 1, 1, 32, 20),           # several tiles per ring
+    small_workload("eq_single_neighbor", 9, 16, 9, 16, EQ, EQ, 0.05, 1, 1, 32, 21),       # degenerate: disc = the point itself
+    small_workload("eq_down2_wide_c32", 41, 320, 21, 160, EQ, EQ, 0.25, 1, 1, 32, 22),
+]
+
+
+@pytest.mark.parametrize("wl", SMALL + [WORKLOADS["c1"]], ids=lambda w: w.name)
+@pytest.mark.parametrize("reuse", [True, False], ids=["reuse_lse_out", "recompute_stats"])
+def test_small_cases_full_comparison(wl, reuse):
+    g = _geometry(wl)
+    q, k, v, dout = make_inputs(wl)
+    with _plan(wl) as plan:
+        row_ptr, lat, off = plan.table()
+        assert np.array_equal(row_ptr, g.row_ptr) and np.array_equal(lat, g.lat_in) and np.array_equal(off, g.lon_off)
+        out, lse, dq, dk, dv = _run_gpu(plan, q, k, v, dout, reuse)
+    N = wl.N
+    ref_out, ref_lse = orc.forward(g, q, k, v, return_lse=True)
+    rdq, rdk, rdv = orc.backward(g, q, k, v, dout)
+    assert nerr(out.reshape(ref_out.shape), ref_out) <= FWD_TOL
+    assert np.max(np.abs(lse.reshape(ref_lse.shape) - ref_lse)) <= 1e-5 * max(1.0, np.max(np.abs(ref_lse)))
+    assert nerr(dq.reshape(rdq.shape), rdq) <= BWD_TOL
+    assert nerr(dk.reshape(rdk.shape), rdk) <= BWD_TOL
+    assert nerr(dv.reshape(rdv.shape), rdv) <= BWD_TOL
+
+
+@pytest.mark.parametrize("name", ["c2", "c3"])
+def test_benchmark_configurations_full_comparison(name):
+    wl = WORKLOADS[name]
+    g = _geometry(wl)
+    q, k, v, dout = make_inputs(wl)
+    with _plan(wl) as plan:
+        row_ptr, lat, off = plan.table()
+        assert np.array_equal(row_ptr, g.row_ptr) and np.array_equal(lat, g.lat_in) and np.array_equal(off, g.lon_off)
+        out, lse, dq, dk, dv = _run_gpu(plan, q, k, v, dout, True)
+    ref_out = orc.forward(g, q, k, v)
+    assert nerr(out.reshape(ref_out.shape), ref_out) <= FWD_TOL
+    del ref_out
+    rdq, rdk, rdv = orc.backward(g, q, k, v, dout)
+    assert nerr(dq.reshape(rdq.shape), rdq) <= BWD_TOL
+    assert nerr(dk.reshape(rdk.shape), rdk) <= BWD_TOL
+    assert nerr(dv.reshape(rdv.shape), rdv) <= BWD_TOL
+
+
+@pytest.mark.parametrize("name, n_out, n_in", [("c3", 192, 96), ("c4", 160, 64), ("c5", 48, 12)])
+def test_benchmark_configurations_sampled(name, n_out, n_in):
+    """Full-size runs in the launch configuration the benchmark times; the oracle evaluates sampled points one
+    by one.  The normalisation max|o| is taken over the sampled oracle values of each tensor."""
+    wl = WORKLOADS[name]
+    g = _geometry(wl)
+    q, k, v, dout = make_inputs(wl)
+    with _plan(wl) as plan:
+        assert plan.nnz == g.nnz
+        out, lse, dq, dk, dv = _run_gpu(plan, q, k, v, dout, True)
+    rng = np.random.default_rng(100 + wl.seed)
+    po = sample_points(rng, wl.N, wl.nlat_out, wl.nlon_out, n_out)
+    pi = sample_points(rng, wl.N, wl.nlat_in, wl.nlon_in, n_in)
+    shape_o = (wl.N, wl.nlat_out, wl.nlon_out, wl.C)
+    shape_i = (wl.N, wl.nlat_in, wl.nlon_in, wl.C)
+    pick = lambda a, shape, p: a.reshape(shape)[p[:, 0], p[:, 1], p[:, 2]]
+    assert nerr(pick(out, shape_o, po), orc.forward_points(g, q, k, v, po)) <= FWD_TOL
+    assert nerr(pick(dq, shape_o, po), orc.dq_points(g, q, k, v, dout, po)) <= BWD_TOL
+    rdk, rdv = orc.dkdv_points(g, q, k, v, dout, pi)
+    assert nerr(pick(dk, shape_i, pi), rdk) <= BWD_TOL
+    assert nerr(pick(dv, shape_i, pi), rdv) <= BWD_TOL
+    # properties that hold at any size, over the whole tensors
+    assert np.isfinite(out).all() and np.isfinite(dq).all() and np.isfinite(dk).all() and np.isfinite(dv).all()
+    dv64, do64 = dv.reshape(shape_i).astype(np.float64), dout.reshape(shape_o).astype(np.float64)
+    assert np.max(np.abs(dv64.sum((1, 2)) - do64.sum((1, 2)))) <= 1e-4 * np.max(np.abs(do64).sum((1, 2)))
+    dk64 = dk.reshape(shape_i).astype(np.float64)
+    assert np.max(np.abs(dk64.sum((1, 2)))) <= 1e-4 * np.max(np.abs(dk64).sum((1, 2)))
+
+
+def test_global_limit_against_dense_oracle():
+    wl = small_workload("global", 16, 32, 16, 32, EQ, EQ, math.pi, 1, 2, 32, 30)
+    g = _geometry(wl)
+    q, k, v, dout = make_inputs(wl)
+    with _plan(wl) as plan:
+        out = plan.forward(*_dev(q, k, v)).cpu().numpy()
+    ref = orc.dense_forward(np.repeat(g.omega, wl.nlon_in), q.reshape(wl.N, -1, wl.C), k.reshape(wl.N, -1, wl.C),
+                            v.reshape(wl.N, -1, wl.C))
+    assert nerr(out.reshape(ref.shape), ref) <= FWD_TOL
+
+
+def test_results_are_reproducible_bit_for_bit():
+    wl = SMALL[2]
+    q, k, v, dout = make_inputs(wl)
+    with _plan(wl) as plan:
+        a = _run_gpu(plan, q, k, v, dout, True)
+        b = _run_gpu(plan, q, k, v, dout, True)
+    for x, y in zip(a, b):
+        assert np.array_equal(x, y)
+
+
+def test_longitude_roll_equivariance_on_gpu():
+    wl = SMALL[2]
+    q, k, v, dout = make_inputs(wl)
+    ps, s = wl.nlon_in // wl.nlon_out, 5
+    with _plan(wl) as plan:
+        out, _, dq, dk, dv = _run_gpu(plan, q, k, v, dout)
+        r_o = lambda a: np.ascontiguousarray(np.roll(a, s, axis=3))
+        r_i = lambda a: np.ascontiguousarray(np.roll(a, s * ps, axis=3))
+        out2, _, dq2, dk2, dv2 = _run_gpu(plan, r_o(q), r_i(k), r_i(v), r_o(dout))
+    for a, b, roll in ((out, out2, r_o), (dq, dq2, r_o), (dk, dk2, r_i), (dv, dv2, r_i)):
+        assert np.max(np.abs(roll(a) - b)) <= 2e-5 * np.max(np.abs(a))
+
+
+def test_argument_errors_launch_nothing():
+    wl = SMALL[0]
+    q, k, v, dout = make_inputs(wl)
+    with _plan(wl) as plan:
+        qd, kd, vd, dd = _dev(q, k, v, dout)
+        out = torch.empty_like(qd)
+        with pytest.raises(sna.SnaError) as e:
+            sna.sna_forward(plan.handle, qd, kd, vd, out, wl.B, wl.H, 12)
+        assert e.value.status == sna.SNA_ERR_UNSUPPORTED
+        with pytest.raises(sna.SnaError) as e:
+            sna.sna_forward(plan.handle, qd.data_ptr() + 4, kd, vd, out, wl.B, wl.H, wl.C)
+        assert e.value.status == sna.SNA_ERR_INVALID_ARG
+        with pytest.raises(sna.SnaError) as e:
+            sna.sna_forward(plan.handle, None, kd, vd, out, wl.B, wl.H, wl.C)
+        assert e.value.status == sna.SNA_ERR_INVALID_ARG
+        ws = torch.empty(256, dtype=torch.uint8, device="cuda")
+        with pytest.raises(sna.SnaError) as e:
+            sna.sna_backward_ex(plan.handle, qd, kd, vd, dd, None, None, torch.empty_like(qd), torch.empty_like(kd),
+                                torch.empty_like(kd), ws, ws.numel(), wl.B, wl.H, wl.C)
+        assert e.value.status == sna.SNA_ERR_WORKSPACE
+        torch.cuda.synchronize()
+
+
+def test_runs_on_a_side_stream():
+    wl = SMALL[0]
+    g = _geometry(wl)
+    q, k, v, dout = make_inputs(wl)
+    ref = orc.forward(g, q, k, v)
+    stream = torch.cuda.Stream()
+    with _plan(wl) as plan:
+        with torch.cuda.stream(stream):
+            qd, kd, vd = _dev(q, k, v)
+            out = plan.forward(qd, kd, vd, stream=stream)
+        stream.synchronize()
+    assert nerr(out.cpu().numpy().reshape(ref.shape), ref) <= FWD_TOL
