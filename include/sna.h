@@ -162,6 +162,33 @@ sna_status_t sna_backward_dkdv(const sna_plan_t* plan, const float* q, const flo
                                const float* dout, const float* lse, const float* D, float* dk, float* dv,
                                int B, int H, int C, void* cuda_stream);
 
+/*
+ * Backward pass for callers that must not allocate device memory.  (The paper has no counterpart; this is a
+ * packaging variant of sna_backward.)
+ *
+ * Some hosts of this library cannot call cudaMalloc at the point where they need gradients: code running
+ * inside a memory-pool or arena that owns the whole device, real-time loops where an allocation (and the
+ * device synchronisation it implies) is not acceptable, or plug-ins that are only handed input and output
+ * buffers.  sna_backward needs scratch memory for the per-output-point softmax statistics (lse and D);
+ * here that scratch is a fixed array that is part of the library image itself, so neither this call nor
+ * anything it uses calls cudaMalloc, cudaFree or any allocating routine.
+ *
+ * Limit: the array holds the statistics of at most SNA_STATIC_SCRATCH_MAX_POINTS output points
+ * (B*H*nlat_out*nlon_out); it occupies 8 MiB on every GPU that loads the library, until the process exits.
+ * A larger problem is rejected with SNA_ERR_WORKSPACE and nothing is launched.
+ *
+ * Arguments, layouts and results are those of sna_backward.  Things to know:
+ *   - The first call on each device looks up the array's device address (once per device, with that device
+ *     current).  Make that first call outside any CUDA stream capture.
+ *   - Every call on a device uses the same array.  Nothing in it has to start at zero (both halves are fully
+ *     rewritten before they are read), and it keeps the last call's values afterwards.  Two calls whose GPU
+ *     work overlaps (different streams, or several host threads) race on it: serialise them.
+ */
+#define SNA_STATIC_SCRATCH_MAX_POINTS (1 << 20)
+sna_status_t sna_backward_static(const sna_plan_t* plan, const float* q, const float* k, const float* v,
+                                 const float* dout, float* dq, float* dk, float* dv,
+                                 int B, int H, int C, void* cuda_stream);
+
 /* Human-readable name of a status code (static string). */
 const char* sna_status_string(sna_status_t status);
 /* Detail of the most recent failure on the calling thread (static thread-local buffer; "" if none). */

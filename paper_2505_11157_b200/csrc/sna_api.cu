@@ -329,3 +329,54 @@ sna_status_t sna_backward(const sna_plan_t* plan, const float* q, const float* k
 }
 
 }  // extern "C"
+
+// ---------------------------------------------------------------------------------------------------------
+// Allocation-free backward pass: the scratch for the softmax statistics lives in the library image.
+// ---------------------------------------------------------------------------------------------------------
+
+// lse and D of up to SNA_STATIC_SCRATCH_MAX_POINTS output points.  In host code this name is only a handle for
+// the runtime, not a device address: the address is looked up per device below and passed to the kernels.
+static __device__ __align__(256) float g_static_scratch[2 * SNA_STATIC_SCRATCH_MAX_POINTS];
+
+namespace {
+constexpr int MAX_DEVICES = 64;
+std::mutex g_static_scratch_mutex;
+float* g_static_scratch_ptr[MAX_DEVICES] = {};
+
+// Device address of g_static_scratch on the current device; resolved on the first call per device.
+sna_status_t static_scratch_for_current_device(float** ptr_out) {
+    int dev = -1;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return cuda_fail(e, "cudaGetDevice");
+    if (dev < 0 || dev >= MAX_DEVICES) { set_error("device ordinal %d out of range", dev); return SNA_ERR_UNSUPPORTED; }
+    std::lock_guard<std::mutex> lock(g_static_scratch_mutex);
+    if (g_static_scratch_ptr[dev] == nullptr) {
+        void* p = nullptr;
+        e = cudaGetSymbolAddress(&p, g_static_scratch);
+        if (e != cudaSuccess) return cuda_fail(e, "cudaGetSymbolAddress(static scratch)");
+        if (p == nullptr) { set_error("cudaGetSymbolAddress returned a null address"); return SNA_ERR_CUDA; }
+        g_static_scratch_ptr[dev] = static_cast<float*>(p);
+    }
+    *ptr_out = g_static_scratch_ptr[dev];
+    return SNA_OK;
+}
+}  // namespace
+
+extern "C" sna_status_t sna_backward_static(const sna_plan_t* plan, const float* q, const float* k, const float* v,
+                                            const float* dout, float* dq, float* dk, float* dv,
+                                            int B, int H, int C, void* cuda_stream) {
+    sna_status_t st = check_problem(plan, B, H, C);
+    if (st != SNA_OK) return st;
+    const size_t points = stats_elems(plan, B, H);
+    if (points > (size_t)SNA_STATIC_SCRATCH_MAX_POINTS) {
+        set_error("problem has %zu output points; the static scratch of sna_backward_static holds at most %d "
+                  "(use sna_backward or sna_backward_ex)", points, SNA_STATIC_SCRATCH_MAX_POINTS);
+        return SNA_ERR_WORKSPACE;
+    }
+    float* scratch = nullptr;
+    st = static_scratch_for_current_device(&scratch);
+    if (st != SNA_OK) return st;
+    // statistics are recomputed into the scratch (lse half, then D half); nothing needs clearing
+    return sna_backward_ex(plan, q, k, v, dout, nullptr, nullptr, dq, dk, dv, scratch,
+                           sizeof(float) * 2 * (size_t)SNA_STATIC_SCRATCH_MAX_POINTS, B, H, C, cuda_stream);
+}

@@ -55,6 +55,7 @@ _SIGNATURES = {
     "sna_backward_ex": (_i, [_vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _sz, _i, _i, _i, _vp]),
     "sna_backward_dq": (_i, [_vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _i, _i, _i, _vp]),
     "sna_backward_dkdv": (_i, [_vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _i, _i, _i, _vp]),
+    "sna_backward_static": (_i, [_vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _i, _i, _i, _vp]),
     "sna_status_string": (ctypes.c_char_p, [_i]),
     "sna_last_error_message": (ctypes.c_char_p, []),
 }
@@ -152,6 +153,17 @@ def sna_backward_dq(plan, q, k, v, dout, out, lse, dq, D, B, H, C, stream=None):
 def sna_backward_dkdv(plan, q, k, v, dout, lse, D, dk, dv, B, H, C, stream=None):
     _check(_lib.sna_backward_dkdv(plan, _ptr(q), _ptr(k), _ptr(v), _ptr(dout), _ptr(lse), _ptr(D), _ptr(dk), _ptr(dv),
                                   B, H, C, _stream(stream)))
+
+
+SNA_STATIC_SCRATCH_MAX_POINTS = 1 << 20
+
+
+def sna_backward_static(plan, q, k, v, dout, dq, dk, dv, B, H, C, stream=None):
+    """Backward pass that allocates nothing: its scratch is a fixed array inside the library (at most
+    SNA_STATIC_SCRATCH_MAX_POINTS output points).  For callers that cannot call cudaMalloc; calls whose GPU work
+    overlaps share that array and must be serialised."""
+    _check(_lib.sna_backward_static(plan, _ptr(q), _ptr(k), _ptr(v), _ptr(dout), _ptr(dq), _ptr(dk), _ptr(dv),
+                                    B, H, C, _stream(stream)))
 
 
 # ---- convenience wrapper -----------------------------------------------------------------------------------
