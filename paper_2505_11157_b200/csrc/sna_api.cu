@@ -127,12 +127,25 @@ static sna_status_t plan_create(int nlat_in, int nlon_in, int nlat_out, int nlon
     std::vector<float> log2_omega(hp.nlat_in);
     for (int h = 0; h < hp.nlat_in; ++h) log2_omega[h] = (float)std::log2(hp.omega[h]);
 
+    sna::Stream fwd_stream, t_stream;
+    try {
+        sna::build_forward_stream(hp, fwd_stream);
+        sna::build_transposed_stream(hp, t_stream);
+    } catch (const std::bad_alloc&) {
+        delete plan;
+        set_error("out of host memory while building the column streams");
+        return SNA_ERR_ALLOC;
+    }
+    static_assert(sizeof(sna::StreamEntry) == 16, "stream entries are read as int4");
+
     // pack everything into one device allocation (each array 256-byte aligned)
     struct Piece { const void* src; size_t bytes; size_t offset; };
     std::vector<Piece> pieces = {
         {hp.row_ptr.data(), hp.row_ptr.size() * 4, 0}, {win_lat.data(), win_lat.size() * 4, 0}, {win_m.data(), win_m.size() * 4, 0},
         {row_order.data(), row_order.size() * 4, 0}, {hp.t_row_ptr.data(), hp.t_row_ptr.size() * 4, 0}, {t_lat.data(), t_lat.size() * 4, 0},
-        {t_m.data(), t_m.size() * 4, 0}, {t_row_order.data(), t_row_order.size() * 4, 0}, {log2_omega.data(), log2_omega.size() * 4, 0}};
+        {t_m.data(), t_m.size() * 4, 0}, {t_row_order.data(), t_row_order.size() * 4, 0}, {log2_omega.data(), log2_omega.size() * 4, 0},
+        {fwd_stream.entries.data(), fwd_stream.entries.size() * 16, 0}, {fwd_stream.chunk_ptr.data(), fwd_stream.chunk_ptr.size() * 4, 0},
+        {t_stream.entries.data(), t_stream.entries.size() * 16, 0}, {t_stream.chunk_ptr.data(), t_stream.chunk_ptr.size() * 4, 0}};
     size_t total = 0;
     for (Piece& p : pieces) { p.offset = total; total += round256(p.bytes); }
     cudaError_t e = cudaGetDevice(&plan->device);
@@ -149,6 +162,8 @@ static sna_status_t plan_create(int nlat_in, int nlon_in, int nlat_out, int nlon
     d.row_ptr = at(0); d.win_lat = at(1); d.win_m = at(2); d.row_order = at(3);
     d.t_row_ptr = at(4); d.t_win_lat = at(5); d.t_win_m = at(6); d.t_row_order = at(7);
     d.log2_omega = (const float*)at(8);
+    d.fwd_stream = (const int4*)at(9); d.fwd_chunk_ptr = at(10);
+    d.t_stream = (const int4*)at(11); d.t_chunk_ptr = at(12);
     *plan_out = plan;
     return SNA_OK;
 }
@@ -246,7 +261,9 @@ sna_status_t sna_forward_ex(const sna_plan_t* plan, const float* q, const float*
     if (st != SNA_OK) return st;
     if (!q || !k || !v || !out) { set_error("q, k, v and out must not be NULL"); return SNA_ERR_INVALID_ARG; }
     if (!all_aligned(q, k, v, out) || (reinterpret_cast<uintptr_t>(lse) & 3u)) { set_error("device pointers must be 16-byte aligned"); return SNA_ERR_INVALID_ARG; }
-    cudaError_t e = sna::launch_forward_generic(plan->dev, q, k, v, out, lse, B * H, C, (cudaStream_t)cuda_stream);
+    cudaError_t e = sna::mma_path_supported(plan->dev, C)
+                        ? sna::launch_forward_mma(plan->dev, q, k, v, out, lse, B * H, C, (cudaStream_t)cuda_stream)
+                        : sna::launch_forward_generic(plan->dev, q, k, v, out, lse, B * H, C, (cudaStream_t)cuda_stream);
     if (e != cudaSuccess) return cuda_fail(e, "forward launch");
     return SNA_OK;
 }

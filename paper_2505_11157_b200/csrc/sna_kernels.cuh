@@ -19,7 +19,17 @@ struct DevPlan {
     const int32_t* t_win_m;
     const int32_t* t_row_order; // input latitudes, most work first
     const float* log2_omega;    // [nlat_in] log2 of the per-point quadrature weight
+    // column streams of the tensor-core kernels (see sna_plan.hpp); null if not built
+    const int4* fwd_stream;         // 16 entries per chunk: {base|abs flag, e | mask<<16, bias, aux}
+    const int32_t* fwd_chunk_ptr;   // [nlat_out+1]
+    const int4* t_stream;
+    const int32_t* t_chunk_ptr;     // [nlat_in*ps+1]
 };
+
+// Tensor-core kernels (C = 16, 32 or 64, nlon_out >= 32); same contracts as the generic launchers.
+bool mma_path_supported(const DevPlan& p, int C);
+cudaError_t launch_forward_mma(const DevPlan& p, const float* q, const float* k, const float* v, float* out, float* lse,
+                               int N, int C, cudaStream_t stream);
 
 // Generic kernels (any supported C): C/4 lanes cooperate on one grid point.
 // forward: out and/or lse may be null (lse-only pass = softmax statistics).

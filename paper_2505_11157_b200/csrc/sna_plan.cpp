@@ -185,4 +185,76 @@ PlanStatus build_plan(int nlat_in, int nlon_in, int nlat_out, int nlon_out, int 
     return PLAN_OK;
 }
 
+namespace {
+
+inline int floor_div(int a, int b) { int q = a / b; return ((a % b != 0) && ((a < 0) != (b < 0))) ? q - 1 : q; }
+inline int ceil_div(int a, int b) { return -floor_div(-a, b); }
+
+// Appends the columns of one window (offsets e_lo..e_hi) or of a whole ring (count partners, absolute index).
+void append_window(std::vector<StreamEntry>& v, int32_t base, float bias, int32_t aux, bool whole, int e_lo, int e_hi, int count) {
+    if (whole) {
+        for (int u = 0; u < count; ++u)
+            v.push_back(StreamEntry{(int32_t)(base | (int32_t)0x80000000), (int32_t)((u & 0xffff) | (0xffff << 16)), bias, aux});
+        return;
+    }
+    const int E = e_hi - e_lo + 1;
+    if (E <= 0) return;
+    for (int x = 0; x < 15 + E; ++x) {
+        uint32_t mask = 0;
+        for (int i = 0; i < 16; ++i)
+            if (x - i >= 0 && x - i <= E - 1) mask |= 1u << i;
+        const int e_rel = e_lo + x;
+        v.push_back(StreamEntry{base, (int32_t)(((uint32_t)e_rel & 0xffffu) | (mask << 16)), bias, aux});
+    }
+}
+
+void pad_row(std::vector<StreamEntry>& v, size_t row_start) {
+    while ((v.size() - row_start) % 16 != 0) {
+        StreamEntry pad = v.size() > row_start ? v.back() : StreamEntry{0, 0, 0.f, 0};
+        pad.e_mask &= 0xffff;   // row mask 0: the column is ignored
+        v.push_back(pad);
+    }
+}
+
+}  // namespace
+
+void build_forward_stream(const HostPlan& P, Stream& S) {
+    S.chunk_ptr.assign(P.nlat_out + 1, 0);
+    S.entries.clear();
+    for (int h = 0; h < P.nlat_out; ++h) {
+        const size_t start = S.entries.size();
+        for (int e = P.row_ptr[h]; e < P.row_ptr[h + 1]; ++e) {
+            const RingWindow& w = P.windows[e];
+            const float bias = (float)std::log2(P.omega[w.lat]);
+            for (int r = 0; r < P.ps; ++r) {
+                const int32_t base = w.lat * P.nlon_in + r;
+                if (w.m < 0) append_window(S.entries, base, bias, 0, true, 0, 0, P.nlon_out);
+                else append_window(S.entries, base, bias, 0, false, ceil_div(-w.m - r, P.ps), floor_div(w.m - r, P.ps), 0);
+            }
+        }
+        pad_row(S.entries, start);
+        S.chunk_ptr[h + 1] = (int32_t)(S.entries.size() / 16);
+    }
+}
+
+void build_transposed_stream(const HostPlan& P, Stream& S) {
+    // Row (h', r): tile rows are input columns c = ps*u + r, u = u0 + i.  Output point (h, w) is a partner iff
+    // c - w*ps in [-m, m]  <=>  w - u in [ceil((r - m)/ps), floor((r + m)/ps)].
+    S.chunk_ptr.assign((size_t)P.nlat_in * P.ps + 1, 0);
+    S.entries.clear();
+    for (int hp = 0; hp < P.nlat_in; ++hp) {
+        for (int r = 0; r < P.ps; ++r) {
+            const size_t start = S.entries.size();
+            for (int e = P.t_row_ptr[hp]; e < P.t_row_ptr[hp + 1]; ++e) {
+                const RingWindow& w = P.t_windows[e];
+                const int32_t base = w.lat * P.nlon_out;
+                if (w.m < 0) append_window(S.entries, base, 0.f, w.lat, true, 0, 0, P.nlon_out);
+                else append_window(S.entries, base, 0.f, w.lat, false, ceil_div(r - w.m, P.ps), floor_div(r + w.m, P.ps), 0);
+            }
+            pad_row(S.entries, start);
+            S.chunk_ptr[(size_t)hp * P.ps + r + 1] = (int32_t)(S.entries.size() / 16);
+        }
+    }
+}
+
 }  // namespace sna

@@ -33,6 +33,31 @@ struct HostPlan {
     int window_count(const RingWindow& w) const { return w.m < 0 ? nlon_in : 2 * w.m + 1; }
 };
 
+// Column streams for the tensor-core kernels.  A warp owns a tile of 16 consecutive points of one ring
+// ("tile rows" i = 0..15, first point w0) and walks a stream of partner points ("columns"), 16 per step.
+// For a window with offsets e in [e_lo, e_hi] (in units of ps input columns for the forward table, of output
+// columns for the transposed one) the tile needs partners u = w0 + e_rel, e_rel = e_lo .. e_hi + 15, and tile
+// row i uses the column iff e_lo <= e_rel - i <= e_hi: that is the 16-bit row mask.  The stream of a ring row
+// is the concatenation of its windows' columns, padded to a multiple of 16 with mask-0 columns, and is the
+// same for every tile of the row, so it is built once on the host.
+struct StreamEntry {
+    int32_t base;      // flat row index of the partner ring plus the residue r; bit 31 set = e is absolute
+    int32_t e_mask;    // low 16 bits: e_rel (signed) or the absolute partner index; high 16 bits: row mask
+    float bias;        // forward: log2 of the partner ring's quadrature weight; transposed: unused (0)
+    int32_t aux;       // forward: unused; transposed: output ring index h (for lse / D lookups)
+};
+
+struct Stream {
+    std::vector<int32_t> chunk_ptr;     // [rows+1] first 16-column chunk of each row
+    std::vector<StreamEntry> entries;   // 16 * chunk_ptr.back()
+};
+
+// Forward stream: rows = output latitudes, partners = input points; partner flat index = base + u*ps.
+void build_forward_stream(const HostPlan& plan, Stream& out);
+// Transposed stream for dk/dv: rows = (input latitude, residue r of the input column mod ps), tile rows are
+// input columns c = ps*(u0+i)+r, partners are output points (h, w).
+void build_transposed_stream(const HostPlan& plan, Stream& out);
+
 // Builds the plan.  On failure returns a status and fills `why`.
 PlanStatus build_plan(int nlat_in, int nlon_in, int nlat_out, int nlon_out, int grid_in, int grid_out,
                       double theta_cutoff, HostPlan& plan, std::string& why);
