@@ -280,7 +280,9 @@ sna_status_t sna_backward_dq(const sna_plan_t* plan, const float* q, const float
     if (st != SNA_OK) return st;
     if (!q || !k || !v || !dout || !lse || !dq || !D) { set_error("q, k, v, dout, lse, dq and D must not be NULL"); return SNA_ERR_INVALID_ARG; }
     if (!all_aligned(q, k, v, dout, dq, out) || ((reinterpret_cast<uintptr_t>(lse) | reinterpret_cast<uintptr_t>(D)) & 3u)) { set_error("device pointers must be 16-byte aligned"); return SNA_ERR_INVALID_ARG; }
-    cudaError_t e = sna::launch_backward_dq_generic(plan->dev, q, k, v, dout, out, lse, dq, D, B * H, C, (cudaStream_t)cuda_stream);
+    cudaError_t e = (out != nullptr && sna::mma_path_supported(plan->dev, C))
+                        ? sna::launch_backward_dq_mma(plan->dev, q, k, v, dout, out, lse, dq, D, B * H, C, (cudaStream_t)cuda_stream)
+                        : sna::launch_backward_dq_generic(plan->dev, q, k, v, dout, out, lse, dq, D, B * H, C, (cudaStream_t)cuda_stream);
     if (e != cudaSuccess) return cuda_fail(e, "backward dq launch");
     return SNA_OK;
 }
@@ -292,7 +294,9 @@ sna_status_t sna_backward_dkdv(const sna_plan_t* plan, const float* q, const flo
     if (st != SNA_OK) return st;
     if (!q || !k || !v || !dout || !lse || !D || !dk || !dv) { set_error("q, k, v, dout, lse, D, dk and dv must not be NULL"); return SNA_ERR_INVALID_ARG; }
     if (!all_aligned(q, k, v, dout, dk, dv) || ((reinterpret_cast<uintptr_t>(lse) | reinterpret_cast<uintptr_t>(D)) & 3u)) { set_error("device pointers must be 16-byte aligned"); return SNA_ERR_INVALID_ARG; }
-    cudaError_t e = sna::launch_backward_dkdv_generic(plan->dev, q, k, v, dout, lse, D, dk, dv, B * H, C, (cudaStream_t)cuda_stream);
+    cudaError_t e = sna::mma_path_supported(plan->dev, C)
+                        ? sna::launch_backward_dkdv_mma(plan->dev, q, k, v, dout, lse, D, dk, dv, B * H, C, (cudaStream_t)cuda_stream)
+                        : sna::launch_backward_dkdv_generic(plan->dev, q, k, v, dout, lse, D, dk, dv, B * H, C, (cudaStream_t)cuda_stream);
     if (e != cudaSuccess) return cuda_fail(e, "backward dk/dv launch");
     return SNA_OK;
 }
@@ -311,7 +315,16 @@ sna_status_t sna_backward_ex(const sna_plan_t* plan, const float* q, const float
     float* ws_lse = (float*)workspace;
     float* ws_D = ws_lse + stats_elems(plan, B, H);
     cudaError_t e;
-    if (lse == nullptr) {   // recompute the softmax statistics
+    if (sna::mma_path_supported(plan->dev, C)) {
+        if (lse == nullptr || out == nullptr) {
+            // recompute the forward pass: lse into the workspace, out into the dq buffer, which the dq stage
+            // reads row by row before it overwrites the same rows with dq
+            e = sna::launch_forward_mma(plan->dev, q, k, v, dq, ws_lse, N, C, stream);
+            if (e != cudaSuccess) return cuda_fail(e, "statistics launch");
+            lse = ws_lse;
+            out = dq;
+        }
+    } else if (lse == nullptr) {   // recompute the softmax statistics
         e = sna::launch_forward_generic(plan->dev, q, k, v, nullptr, ws_lse, N, C, stream);
         if (e != cudaSuccess) return cuda_fail(e, "statistics launch");
         lse = ws_lse;

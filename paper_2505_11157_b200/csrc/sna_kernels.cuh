@@ -30,6 +30,11 @@ struct DevPlan {
 bool mma_path_supported(const DevPlan& p, int C);
 cudaError_t launch_forward_mma(const DevPlan& p, const float* q, const float* k, const float* v, float* out, float* lse,
                                int N, int C, cudaStream_t stream);
+// out is required (D_i = dout_i . out_i); out and dq may be the same buffer.
+cudaError_t launch_backward_dq_mma(const DevPlan& p, const float* q, const float* k, const float* v, const float* dout,
+                                   const float* out, const float* lse, float* dq, float* Dws, int N, int C, cudaStream_t stream);
+cudaError_t launch_backward_dkdv_mma(const DevPlan& p, const float* q, const float* k, const float* v, const float* dout,
+                                     const float* lse, const float* Dws, float* dk, float* dv, int N, int C, cudaStream_t stream);
 
 // Generic kernels (any supported C): C/4 lanes cooperate on one grid point.
 // forward: out and/or lse may be null (lse-only pass = softmax statistics).

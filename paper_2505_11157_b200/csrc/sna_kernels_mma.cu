@@ -1,17 +1,27 @@
 // Tensor-core kernels (sm_100a): every contraction of the path runs on mma.sync m16n8k8 TF32 with a three-term
-// split (x = hi + lo; hi*hi + lo*hi + hi*lo, fp32 accumulate), which keeps fp32-level accuracy
-// (measured ~1e-6 normalised error) at four times the FP32 FMA rate for dense tiles.
+// split (x = hi + lo; lo*hi + hi*lo + hi*hi, fp32 accumulate), which keeps fp32-level accuracy
+// (measured < 1e-6 normalised error) at four times the FP32 FMA rate for dense tiles.
 //
-// Work decomposition: one warp owns 16 consecutive points of one ring (the M dimension of the MMA) and walks
-// the host-built column stream of that ring row, 16 partner points per step.  Band structure and ragged edges
-// are expressed by the 16-bit row mask carried by every stream column; masked scores become -inf.
+// Work decomposition: one warp owns 16 consecutive points of one ring (the M dimension of the MMA: "tile rows")
+// and walks the host-built column stream of that ring row, 16 partner points ("columns") per step.  Band
+// structure and ragged edges are expressed by the 16-bit row mask carried by every stream column.
 // Operands are loaded straight from global memory (L1/L2) in fragment order; warps never synchronise with
 // each other, and there is no shared memory.
+//
+// Fragment conventions (g = lane / 4, t = lane % 4, CPT = C/4, KS = C/8):
+//   "row fragment" of a point: the CPT channels [t*CPT, (t+1)*CPT) of that point.  As an A operand it belongs to
+//   tile rows g and g+8; as a B operand to tile column g.  MMA k index t of k-step ks is channel t*CPT + 2*ks,
+//   k index t+4 is channel t*CPT + 2*ks + 1 (the same permutation on both operands, so the contraction is exact).
+//   "column fragment" of a point: the KS channels [g*KS, (g+1)*KS) of the point in tile column 2t (and 2t+1).
+//   With the accumulator's column n <-> channel n*KS + nt for n-tile nt, a thread ends up owning channels
+//   [t*CPT, (t+1)*CPT) of tile rows g and g+8 again.  A score fragment (rows g, g+8; columns 2t, 2t+1) is
+//   reused as the A operand of the second contraction with k index t <-> column 2t and t+4 <-> column 2t+1.
 //
 // Forward: Eq. (s2_attention_discrete_detailed).  Backward: App. B.4.
 #include "sna_kernels.cuh"
 
 #include <cstdint>
+#include <type_traits>
 
 namespace sna {
 namespace {
@@ -20,6 +30,7 @@ constexpr int WARPS = 8;
 constexpr int THREADS = WARPS * 32;
 constexpr float LOG2E = 1.4426950408889634f;
 constexpr float LN2 = 0.6931471805599453f;
+constexpr unsigned FULL = 0xffffffffu;
 
 __device__ __forceinline__ float ex2(float x) {
     float y;
@@ -27,44 +38,164 @@ __device__ __forceinline__ float ex2(float x) {
     return y;
 }
 
-// x ~ hi + lo, both rounded to nearest to 11 significand bits by integer add (a truncated lo would bias long sums).
-__device__ __forceinline__ void split_tf32(float x, uint32_t& hi, uint32_t& lo) {
+// Split for operands that are used once: the MMA reads only the top 19 bits of a TF32 operand, so the raw fp32
+// word serves as hi, and lo is the exact remainder after that truncation (itself truncated by the MMA: the
+// representation error is below 2^-20 relative).
+__device__ __forceinline__ void split_fast(float x, uint32_t& hi, uint32_t& lo) {
+    hi = __float_as_uint(x);
+    lo = __float_as_uint(x - __uint_as_float(hi & 0xffffe000u));
+}
+// Split for operands that are reused over the whole stream: both parts rounded to nearest.
+__device__ __forceinline__ void split_rn(float x, uint32_t& hi, uint32_t& lo) {
     const uint32_t h = (__float_as_uint(x) + 0x1000u) & 0xffffe000u;
     hi = h;
     lo = (__float_as_uint(x - __uint_as_float(h)) + 0x1000u) & 0xffffe000u;
-}
-
-__device__ __forceinline__ void mma_tf32(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0, uint32_t b1) {
-    asm volatile("mma.sync.aligned.m16n8k8.row.col.f32.tf32.tf32.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
-                 : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
-                 : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
 }
 
 // The tensor core adds into its fp32 accumulator with truncation, so a long chain of MMAs into one fragment
 // drifts towards zero (measured: 3e-5 relative after ~1000 steps).  Every chain here is therefore short: the
 // small correction terms lo*hi + hi*lo go first, the main terms hi*hi last, into a fragment that starts at
 // zero, and long sums are carried in fp32 FMAs outside the tensor core.
-__device__ __forceinline__ void mma_corr(float (&d)[4], const uint32_t (&ah)[4], const uint32_t (&al)[4],
-                                         uint32_t bh0, uint32_t bh1, uint32_t bl0, uint32_t bl1) {
-    mma_tf32(d, al[0], al[1], al[2], al[3], bh0, bh1);
-    mma_tf32(d, ah[0], ah[1], ah[2], ah[3], bl0, bl1);
+__device__ __forceinline__ void mma_acc(float (&d)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
+    asm volatile("mma.sync.aligned.m16n8k8.row.col.f32.tf32.tf32.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+                 : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+                 : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
 }
-__device__ __forceinline__ void mma_main(float (&d)[4], const uint32_t (&ah)[4], uint32_t bh0, uint32_t bh1) {
-    mma_tf32(d, ah[0], ah[1], ah[2], ah[3], bh0, bh1);
+__device__ __forceinline__ void mma_zero(float (&d)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
+    asm volatile("mma.sync.aligned.m16n8k8.row.col.f32.tf32.tf32.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%10,%10,%10,%10};"
+                 : "=f"(d[0]), "=f"(d[1]), "=f"(d[2]), "=f"(d[3])
+                 : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1), "f"(0.f));
 }
 
 __device__ __forceinline__ float4 ldg4(const float* p) { return __ldg(reinterpret_cast<const float4*>(p)); }
 
-// Flat index (within one batch*head slice) of the partner point of a stream column for a tile starting at w0.
-__device__ __forceinline__ int partner_index(const int4& e, int w0, int nlon_tile, int stride) {
-    int u = (int)(short)(e.y & 0xffff);
-    if (e.x >= 0) {            // relative to the tile
-        u += w0;
-        if (u < 0) u += nlon_tile;
-        if (u >= nlon_tile) u -= nlon_tile;
-        if (u >= nlon_tile) u -= nlon_tile;
+// Row fragment (CPT contiguous channels) of the point at `p`, raw.
+template <int CPT>
+__device__ __forceinline__ void load_row(const float* p, float (&x)[CPT]) {
+#pragma unroll
+    for (int j = 0; j < CPT / 4; ++j) {
+        const float4 a = ldg4(p + 4 * j);
+        x[4 * j] = a.x; x[4 * j + 1] = a.y; x[4 * j + 2] = a.z; x[4 * j + 3] = a.w;
     }
-    return (e.x & 0x7fffffff) + u * stride;
+}
+// Column fragment (KS contiguous channels).
+template <int KS>
+__device__ __forceinline__ void load_col(const float* p, float (&x)[KS]) {
+    if constexpr (KS % 4 == 0) {
+#pragma unroll
+        for (int j = 0; j < KS / 4; ++j) {
+            const float4 a = ldg4(p + 4 * j);
+            x[4 * j] = a.x; x[4 * j + 1] = a.y; x[4 * j + 2] = a.z; x[4 * j + 3] = a.w;
+        }
+    } else {
+        const float2 a = __ldg(reinterpret_cast<const float2*>(p));
+        x[0] = a.x; x[1] = a.y;
+    }
+}
+
+// A operand (tile rows g and g+8) from the row fragments of the two points, pre-multiplied by `mul`.
+template <int CPT>
+__device__ __forceinline__ void make_a_operand(const float* p0, const float* p1, float mul, uint32_t (&hi)[CPT / 2][4], uint32_t (&lo)[CPT / 2][4]) {
+    float a[CPT], b[CPT];
+    load_row<CPT>(p0, a);
+    load_row<CPT>(p1, b);
+#pragma unroll
+    for (int ks = 0; ks < CPT / 2; ++ks) {
+        split_rn(a[2 * ks] * mul, hi[ks][0], lo[ks][0]);       // (row g,   k = t)
+        split_rn(b[2 * ks] * mul, hi[ks][1], lo[ks][1]);       // (row g+8, k = t)
+        split_rn(a[2 * ks + 1] * mul, hi[ks][2], lo[ks][2]);   // (row g,   k = t+4)
+        split_rn(b[2 * ks + 1] * mul, hi[ks][3], lo[ks][3]);   // (row g+8, k = t+4)
+    }
+}
+
+// d[16x8] = A (tile rows x channels) . B^T, B = row fragment `x` of the point in tile column g.
+template <int CPT>
+__device__ __forceinline__ void rows_dot_point(float (&d)[4], const uint32_t (&ah)[CPT / 2][4], const uint32_t (&al)[CPT / 2][4], const float (&x)[CPT]) {
+    uint32_t bh[CPT], bl[CPT];
+#pragma unroll
+    for (int j = 0; j < CPT; ++j) split_fast(x[j], bh[j], bl[j]);
+    mma_zero(d, al[0], bh[0], bh[1]);
+    mma_acc(d, ah[0], bl[0], bl[1]);
+#pragma unroll
+    for (int ks = 1; ks < CPT / 2; ++ks) {
+        mma_acc(d, al[ks], bh[2 * ks], bh[2 * ks + 1]);
+        mma_acc(d, ah[ks], bl[2 * ks], bl[2 * ks + 1]);
+    }
+#pragma unroll
+    for (int ks = 0; ks < CPT / 2; ++ks) mma_acc(d, ah[ks], bh[2 * ks], bh[2 * ks + 1]);
+}
+
+// A operand from two score-layout fragments w[tl] (rows g, g+8; columns 2t, 2t+1 of 8-column tile tl).
+__device__ __forceinline__ void scores_as_a(const float (&w)[2][4], uint32_t (&hi)[2][4], uint32_t (&lo)[2][4]) {
+#pragma unroll
+    for (int tl = 0; tl < 2; ++tl) {
+        split_fast(w[tl][0], hi[tl][0], lo[tl][0]);
+        split_fast(w[tl][2], hi[tl][1], lo[tl][1]);
+        split_fast(w[tl][1], hi[tl][2], lo[tl][2]);
+        split_fast(w[tl][3], hi[tl][3], lo[tl][3]);
+    }
+}
+
+// d[nt] (16 rows x 8 channels of n-tile nt) = W (16 x 16 columns, as A operand) times the column fragments
+// x[tl][j] of the 16 partner points, in a zero-started fragment per n-tile.
+template <int KS>
+__device__ __forceinline__ void scores_times_points(float (&d)[KS][4], const uint32_t (&wh)[2][4], const uint32_t (&wl)[2][4], const float (&x)[2][2][KS]) {
+    uint32_t xh[2][2][KS], xl[2][2][KS];
+#pragma unroll
+    for (int tl = 0; tl < 2; ++tl)
+#pragma unroll
+        for (int j = 0; j < 2; ++j)
+#pragma unroll
+            for (int nt = 0; nt < KS; ++nt) split_fast(x[tl][j][nt], xh[tl][j][nt], xl[tl][j][nt]);
+#pragma unroll
+    for (int nt = 0; nt < KS; ++nt) {
+        mma_zero(d[nt], wl[0], xh[0][0][nt], xh[0][1][nt]);
+        mma_acc(d[nt], wh[0], xl[0][0][nt], xl[0][1][nt]);
+        mma_acc(d[nt], wl[1], xh[1][0][nt], xh[1][1][nt]);
+        mma_acc(d[nt], wh[1], xl[1][0][nt], xl[1][1][nt]);
+        mma_acc(d[nt], wh[0], xh[0][0][nt], xh[0][1][nt]);
+        mma_acc(d[nt], wh[1], xh[1][0][nt], xh[1][1][nt]);
+    }
+}
+
+// One 16-column chunk of a stream as seen by a warp: lane l holds column l % 16.
+struct ChunkColumn {
+    int idx;        // flat index of the partner point inside one batch*head slice
+    uint32_t mask;  // tile rows that use this column
+    float bias;     // forward stream: log2 of the partner's quadrature weight
+};
+
+__device__ __forceinline__ ChunkColumn load_chunk_column(const int4* chunk, int lane, int first, int ring_len, int stride) {
+    const int4 e = __ldg(chunk + (lane & 15));
+    int u = (int)(short)(e.y & 0xffff);
+    if (e.x >= 0) {   // offset relative to the tile's first point, wrapped around the ring
+        u += first;
+        if (u < 0) u += ring_len;
+        if (u >= ring_len) u -= ring_len;
+        if (u >= ring_len) u -= ring_len;
+    }
+    ChunkColumn c;
+    c.idx = (e.x & 0x7fffffff) + u * stride;
+    c.mask = (uint32_t)e.y >> 16;
+    c.bias = __int_as_float(e.z);
+    return c;
+}
+
+// Decode a warp task into (slice n, rank of the ring row in heavy-first order, tile).
+__device__ __forceinline__ bool decode_task(int N, int tiles_per_row, long long total, int& n, int& row_rank, int& tile) {
+    const long long task = (long long)blockIdx.x * WARPS + (threadIdx.x >> 5);
+    if (task >= total) return false;
+    tile = (int)(task % tiles_per_row);
+    const long long rest = task / tiles_per_row;
+    n = (int)(rest % N);
+    row_rank = (int)(rest / N);
+    return true;
+}
+
+template <int CPT>
+__device__ __forceinline__ void store_row(float* p, const float (&x)[CPT]) {
+#pragma unroll
+    for (int j = 0; j < CPT / 4; ++j) *reinterpret_cast<float4*>(p + 4 * j) = make_float4(x[4 * j], x[4 * j + 1], x[4 * j + 2], x[4 * j + 3]);
 }
 
 // ---------------------------------------------------------------------------------------------------------
@@ -74,91 +205,55 @@ template <int C>
 __global__ void __launch_bounds__(THREADS)
 forward_mma_kernel(DevPlan p, const float* __restrict__ q, const float* __restrict__ k, const float* __restrict__ v,
                    float* __restrict__ out, float* __restrict__ lse, int N, float scale_log2, int tiles_per_row, long long total_tasks) {
-    constexpr int CPT = C / 4;    // channels per thread in A/C fragments (thread t owns [t*CPT, (t+1)*CPT))
-    constexpr int KS = C / 8;     // k-steps of q.k, and n-tiles of p.v
+    constexpr int CPT = C / 4, KS = C / 8;
     const int lane = threadIdx.x & 31, g = lane >> 2, t = lane & 3;
-    const long long task = (long long)blockIdx.x * WARPS + (threadIdx.x >> 5);
-    if (task >= total_tasks) return;
-    const int tile = (int)(task % tiles_per_row);
-    const long long rest = task / tiles_per_row;
-    const int n = (int)(rest % N);
-    const int h = p.row_order[rest / N];
+    int n, rank, tile;
+    if (!decode_task(N, tiles_per_row, total_tasks, n, rank, tile)) return;
+    const int h = p.row_order[rank];
     const int w0 = tile * 16;
     const int r0 = min(w0 + g, p.nlon_out - 1), r1 = min(w0 + g + 8, p.nlon_out - 1);   // clamped tile rows
     const size_t orow = (size_t)(n * p.nlat_out + h) * p.nlon_out;
 
-    // A fragments of q (pre-scaled into the log2 domain), split once
-    uint32_t qh[KS][4], ql[KS][4];
-    {
-        const float* q0 = q + (orow + r0) * C + t * CPT;
-        const float* q1 = q + (orow + r1) * C + t * CPT;
-#pragma unroll
-        for (int j = 0; j < CPT / 4; ++j) {
-            const float4 a = ldg4(q0 + 4 * j), b = ldg4(q1 + 4 * j);
-            const float av[4] = {a.x, a.y, a.z, a.w}, bv[4] = {b.x, b.y, b.z, b.w};
-#pragma unroll
-            for (int i = 0; i < 4; i += 2) {
-                const int ks = (4 * j + i) / 2;
-                split_tf32(av[i] * scale_log2, qh[ks][0], ql[ks][0]);       // (row g,   k = t)
-                split_tf32(bv[i] * scale_log2, qh[ks][1], ql[ks][1]);       // (row g+8, k = t)
-                split_tf32(av[i + 1] * scale_log2, qh[ks][2], ql[ks][2]);   // (row g,   k = t+4)
-                split_tf32(bv[i + 1] * scale_log2, qh[ks][3], ql[ks][3]);   // (row g+8, k = t+4)
-            }
-        }
-    }
+    uint32_t qh[KS][4], ql[KS][4];   // q in the log2 domain
+    make_a_operand<CPT>(q + (orow + r0) * C + t * CPT, q + (orow + r1) * C + t * CPT, scale_log2, qh, ql);
     float o[KS][4];
 #pragma unroll
     for (int nt = 0; nt < KS; ++nt) o[nt][0] = o[nt][1] = o[nt][2] = o[nt][3] = 0.f;
     float m0 = -INFINITY, m1 = -INFINITY, l0 = 0.f, l1 = 0.f;
 
-    const float* kb = k + (size_t)n * p.nlat_in * p.nlon_in * C;
-    const float* vb = v + (size_t)n * p.nlat_in * p.nlon_in * C;
+    const float* kb = k + (size_t)n * p.nlat_in * p.nlon_in * C + t * CPT;
+    const float* vb = v + (size_t)n * p.nlat_in * p.nlon_in * C + g * KS;
     const int4* stream = p.fwd_stream + (size_t)p.fwd_chunk_ptr[h] * 16;
     const int nchunks = p.fwd_chunk_ptr[h + 1] - p.fwd_chunk_ptr[h];
 
     for (int c = 0; c < nchunks; ++c) {
-        const int4* ce = stream + c * 16;
-        // two 8-column tiles: columns g (K operand) and 2t, 2t+1 (scores / V operand) of each
+        const ChunkColumn col = load_chunk_column(stream + c * 16, lane, w0, p.nlon_out, p.ps);
         float s[2][4];
 #pragma unroll
         for (int tl = 0; tl < 2; ++tl) {
-            const int4 ek = __ldg(ce + tl * 8 + g);
-            const float* kp = kb + (size_t)partner_index(ek, w0, p.nlon_out, p.ps) * C + t * CPT;
             float kr[CPT];
-#pragma unroll
-            for (int j = 0; j < CPT / 4; ++j) {
-                const float4 a = ldg4(kp + 4 * j);
-                kr[4 * j] = a.x; kr[4 * j + 1] = a.y; kr[4 * j + 2] = a.z; kr[4 * j + 3] = a.w;
-            }
-            s[tl][0] = s[tl][1] = s[tl][2] = s[tl][3] = 0.f;
-            uint32_t kh[CPT], kl[CPT];
-#pragma unroll
-            for (int j = 0; j < CPT; ++j) split_tf32(kr[j], kh[j], kl[j]);
-#pragma unroll
-            for (int ks = 0; ks < KS; ++ks) mma_corr(s[tl], qh[ks], ql[ks], kh[2 * ks], kh[2 * ks + 1], kl[2 * ks], kl[2 * ks + 1]);
-#pragma unroll
-            for (int ks = 0; ks < KS; ++ks) mma_main(s[tl], qh[ks], kh[2 * ks], kh[2 * ks + 1]);
+            load_row<CPT>(kb + (size_t)__shfl_sync(FULL, col.idx, tl * 8 + g) * C, kr);
+            rows_dot_point<CPT>(s[tl], qh, ql, kr);
         }
-        // bias (log2 omega), mask, online softmax
-        int4 ev[2][2];
+        float vr[2][2][KS];
 #pragma unroll
-        for (int tl = 0; tl < 2; ++tl) {
-            ev[tl][0] = __ldg(ce + tl * 8 + 2 * t);
-            ev[tl][1] = __ldg(ce + tl * 8 + 2 * t + 1);
+        for (int tl = 0; tl < 2; ++tl)
 #pragma unroll
             for (int j = 0; j < 2; ++j) {
-                const float bias = __int_as_float(ev[tl][j].z);
-                const uint32_t mask = (uint32_t)ev[tl][j].y >> 16;
-                s[tl][j] = (mask >> g) & 1u ? s[tl][j] + bias : -INFINITY;
-                s[tl][2 + j] = (mask >> (g + 8)) & 1u ? s[tl][2 + j] + bias : -INFINITY;
+                const int src = tl * 8 + 2 * t + j;
+                load_col<KS>(vb + (size_t)__shfl_sync(FULL, col.idx, src) * C, vr[tl][j]);
+                const float bias = __shfl_sync(FULL, col.bias, src);
+                const uint32_t mask = __shfl_sync(FULL, col.mask, src) >> g;
+                s[tl][j] = (mask & 1u) ? s[tl][j] + bias : -INFINITY;
+                s[tl][2 + j] = (mask & 0x100u) ? s[tl][2 + j] + bias : -INFINITY;
             }
-        }
+        // online softmax over the chunk (row maxima across the four threads of a group)
         float mx0 = fmaxf(fmaxf(s[0][0], s[0][1]), fmaxf(s[1][0], s[1][1]));
         float mx1 = fmaxf(fmaxf(s[0][2], s[0][3]), fmaxf(s[1][2], s[1][3]));
-        mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, 1));
-        mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, 1));
-        mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, 2));
-        mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, 2));
+        mx0 = fmaxf(mx0, __shfl_xor_sync(FULL, mx0, 1));
+        mx1 = fmaxf(mx1, __shfl_xor_sync(FULL, mx1, 1));
+        mx0 = fmaxf(mx0, __shfl_xor_sync(FULL, mx0, 2));
+        mx1 = fmaxf(mx1, __shfl_xor_sync(FULL, mx1, 2));
         const float mn0 = fmaxf(m0, mx0), mn1 = fmaxf(m1, mx1);
         const float ms0 = mn0 == -INFINITY ? 0.f : mn0, ms1 = mn1 == -INFINITY ? 0.f : mn1;
         const float corr0 = ex2(m0 - ms0), corr1 = ex2(m1 - ms1);
@@ -173,72 +268,242 @@ forward_mma_kernel(DevPlan p, const float* __restrict__ q, const float* __restri
         }
         l0 = fmaf(l0, corr0, ps0);
         l1 = fmaf(l1, corr1, ps1);
-        // this chunk's P V goes into a zeroed fragment; P (A operand) comes from the score fragments with
-        // k index t <-> tile column 2t and t+4 <-> 2t+1
+        uint32_t ph[2][4], pl[2][4];
+        scores_as_a(s, ph, pl);
         float pv[KS][4];
-#pragma unroll
-        for (int nt = 0; nt < KS; ++nt) pv[nt][0] = pv[nt][1] = pv[nt][2] = pv[nt][3] = 0.f;
-        uint32_t ph[2][4], pl[2][4], vh[2][2][KS], vl[2][2][KS];
-#pragma unroll
-        for (int tl = 0; tl < 2; ++tl) {
-            split_tf32(s[tl][0], ph[tl][0], pl[tl][0]);
-            split_tf32(s[tl][2], ph[tl][1], pl[tl][1]);
-            split_tf32(s[tl][1], ph[tl][2], pl[tl][2]);
-            split_tf32(s[tl][3], ph[tl][3], pl[tl][3]);
-#pragma unroll
-            for (int j = 0; j < 2; ++j) {
-                const float* vp = vb + (size_t)partner_index(ev[tl][j], w0, p.nlon_out, p.ps) * C + g * KS;
-                float vr[KS];
-                if constexpr (KS % 4 == 0) {
-#pragma unroll
-                    for (int i = 0; i < KS / 4; ++i) {
-                        const float4 a = ldg4(vp + 4 * i);
-                        vr[4 * i] = a.x; vr[4 * i + 1] = a.y; vr[4 * i + 2] = a.z; vr[4 * i + 3] = a.w;
-                    }
-                } else {
-                    const float2 a = __ldg(reinterpret_cast<const float2*>(vp));
-                    vr[0] = a.x; vr[1] = a.y;
-                }
-#pragma unroll
-                for (int nt = 0; nt < KS; ++nt) split_tf32(vr[nt], vh[tl][j][nt], vl[tl][j][nt]);
-            }
-        }
+        scores_times_points<KS>(pv, ph, pl, vr);
 #pragma unroll
         for (int nt = 0; nt < KS; ++nt) {
-#pragma unroll
-            for (int tl = 0; tl < 2; ++tl) mma_corr(pv[nt], ph[tl], pl[tl], vh[tl][0][nt], vh[tl][1][nt], vl[tl][0][nt], vl[tl][1][nt]);
-#pragma unroll
-            for (int tl = 0; tl < 2; ++tl) mma_main(pv[nt], ph[tl], vh[tl][0][nt], vh[tl][1][nt]);
             o[nt][0] = fmaf(o[nt][0], corr0, pv[nt][0]); o[nt][1] = fmaf(o[nt][1], corr0, pv[nt][1]);
             o[nt][2] = fmaf(o[nt][2], corr1, pv[nt][2]); o[nt][3] = fmaf(o[nt][3], corr1, pv[nt][3]);
         }
     }
     // row sums across the four threads of a group, normalise, store
-    l0 += __shfl_xor_sync(0xffffffffu, l0, 1); l1 += __shfl_xor_sync(0xffffffffu, l1, 1);
-    l0 += __shfl_xor_sync(0xffffffffu, l0, 2); l1 += __shfl_xor_sync(0xffffffffu, l1, 2);
-    const float inv0 = 1.f / l0, inv1 = 1.f / l1;
-    // thread owns channels t*CPT + {2t'-style interleave}: o[nt][0] -> channel 2t*KS + nt, o[nt][1] -> (2t+1)*KS + nt
+    l0 += __shfl_xor_sync(FULL, l0, 1); l1 += __shfl_xor_sync(FULL, l1, 1);
+    l0 += __shfl_xor_sync(FULL, l0, 2); l1 += __shfl_xor_sync(FULL, l1, 2);
     if (out != nullptr) {
-        float* o0 = out + (orow + w0 + g) * C + t * CPT;
-        float* o1 = out + (orow + w0 + g + 8) * C + t * CPT;
-        float r0v[CPT], r1v[CPT];
+        const float inv0 = 1.f / l0, inv1 = 1.f / l1;
+        float r0v[CPT], r1v[CPT];   // o[nt][0] is channel t*CPT + nt, o[nt][1] is channel t*CPT + KS + nt
 #pragma unroll
         for (int nt = 0; nt < KS; ++nt) {
             r0v[nt] = o[nt][0] * inv0; r0v[KS + nt] = o[nt][1] * inv0;
             r1v[nt] = o[nt][2] * inv1; r1v[KS + nt] = o[nt][3] * inv1;
         }
-        if (w0 + g < p.nlon_out) {
-#pragma unroll
-            for (int j = 0; j < CPT / 4; ++j) *reinterpret_cast<float4*>(o0 + 4 * j) = make_float4(r0v[4 * j], r0v[4 * j + 1], r0v[4 * j + 2], r0v[4 * j + 3]);
-        }
-        if (w0 + g + 8 < p.nlon_out) {
-#pragma unroll
-            for (int j = 0; j < CPT / 4; ++j) *reinterpret_cast<float4*>(o1 + 4 * j) = make_float4(r1v[4 * j], r1v[4 * j + 1], r1v[4 * j + 2], r1v[4 * j + 3]);
-        }
+        if (w0 + g < p.nlon_out) store_row<CPT>(out + (orow + w0 + g) * C + t * CPT, r0v);
+        if (w0 + g + 8 < p.nlon_out) store_row<CPT>(out + (orow + w0 + g + 8) * C + t * CPT, r1v);
     }
     if (lse != nullptr && t == 0) {
         if (w0 + g < p.nlon_out) lse[orow + w0 + g] = (m0 + log2f(l0)) * LN2;
         if (w0 + g + 8 < p.nlon_out) lse[orow + w0 + g + 8] = (m1 + log2f(l1)) * LN2;
+    }
+}
+
+// ---------------------------------------------------------------------------------------------------------
+// backward, dq:  dq_i = scale * sum_j p_ij (t_ij - D_i) k_j,  D_i = dout_i . out_i  (App. B.4)
+// `out` and `dq` may be the same buffer: a warp reads its own 16 rows of `out` before it writes them as dq.
+// ---------------------------------------------------------------------------------------------------------
+template <int C>
+__global__ void __launch_bounds__(THREADS, 1)
+backward_dq_mma_kernel(DevPlan p, const float* __restrict__ q, const float* __restrict__ k, const float* __restrict__ v,
+                       const float* __restrict__ dout, const float* out, const float* __restrict__ lse,
+                       float* dq, float* __restrict__ Dws, int N, float scale, int tiles_per_row, long long total_tasks) {
+    constexpr int CPT = C / 4, KS = C / 8;
+    const int lane = threadIdx.x & 31, g = lane >> 2, t = lane & 3;
+    int n, rank, tile;
+    if (!decode_task(N, tiles_per_row, total_tasks, n, rank, tile)) return;
+    const int h = p.row_order[rank];
+    const int w0 = tile * 16;
+    const int r0 = min(w0 + g, p.nlon_out - 1), r1 = min(w0 + g + 8, p.nlon_out - 1);
+    const size_t orow = (size_t)(n * p.nlat_out + h) * p.nlon_out;
+    const float scale_log2 = scale * LOG2E;
+
+    uint32_t qh[KS][4], ql[KS][4], yh[KS][4], yl[KS][4];
+    make_a_operand<CPT>(q + (orow + r0) * C + t * CPT, q + (orow + r1) * C + t * CPT, scale_log2, qh, ql);
+    make_a_operand<CPT>(dout + (orow + r0) * C + t * CPT, dout + (orow + r1) * C + t * CPT, 1.f, yh, yl);
+    // D of the two tile rows
+    float D0 = 0.f, D1 = 0.f;
+    {
+        float a[CPT], b[CPT], ya[CPT], yb[CPT];
+        load_row<CPT>(out + (orow + r0) * C + t * CPT, a);
+        load_row<CPT>(out + (orow + r1) * C + t * CPT, b);
+        load_row<CPT>(dout + (orow + r0) * C + t * CPT, ya);
+        load_row<CPT>(dout + (orow + r1) * C + t * CPT, yb);
+#pragma unroll
+        for (int j = 0; j < CPT; ++j) { D0 = fmaf(a[j], ya[j], D0); D1 = fmaf(b[j], yb[j], D1); }
+        D0 += __shfl_xor_sync(FULL, D0, 1); D1 += __shfl_xor_sync(FULL, D1, 1);
+        D0 += __shfl_xor_sync(FULL, D0, 2); D1 += __shfl_xor_sync(FULL, D1, 2);
+        if (t == 0) {
+            if (w0 + g < p.nlon_out) Dws[orow + w0 + g] = D0;
+            if (w0 + g + 8 < p.nlon_out) Dws[orow + w0 + g + 8] = D1;
+        }
+    }
+    const float nl0 = -lse[orow + r0] * LOG2E, nl1 = -lse[orow + r1] * LOG2E;
+    float acc[KS][4];
+#pragma unroll
+    for (int nt = 0; nt < KS; ++nt) acc[nt][0] = acc[nt][1] = acc[nt][2] = acc[nt][3] = 0.f;
+
+    const size_t slice = (size_t)n * p.nlat_in * p.nlon_in * C;
+    const float* kb = k + slice + t * CPT;
+    const float* vb = v + slice + t * CPT;
+    const float* kc = k + slice + g * KS;
+    const int4* stream = p.fwd_stream + (size_t)p.fwd_chunk_ptr[h] * 16;
+    const int nchunks = p.fwd_chunk_ptr[h + 1] - p.fwd_chunk_ptr[h];
+
+    for (int c = 0; c < nchunks; ++c) {
+        const ChunkColumn col = load_chunk_column(stream + c * 16, lane, w0, p.nlon_out, p.ps);
+        float s[2][4], tt[2][4];
+#pragma unroll
+        for (int tl = 0; tl < 2; ++tl) {
+            const size_t off = (size_t)__shfl_sync(FULL, col.idx, tl * 8 + g) * C;
+            float xr[CPT];
+            load_row<CPT>(kb + off, xr);
+            rows_dot_point<CPT>(s[tl], qh, ql, xr);
+            load_row<CPT>(vb + off, xr);
+            rows_dot_point<CPT>(tt[tl], yh, yl, xr);
+        }
+        float kr[2][2][KS];
+#pragma unroll
+        for (int tl = 0; tl < 2; ++tl)
+#pragma unroll
+            for (int j = 0; j < 2; ++j) {
+                const int src = tl * 8 + 2 * t + j;
+                load_col<KS>(kc + (size_t)__shfl_sync(FULL, col.idx, src) * C, kr[tl][j]);
+                const float bias = __shfl_sync(FULL, col.bias, src);
+                const uint32_t mask = __shfl_sync(FULL, col.mask, src) >> g;
+                const float p0 = (mask & 1u) ? ex2(s[tl][j] + bias + nl0) : 0.f;
+                const float p1 = (mask & 0x100u) ? ex2(s[tl][2 + j] + bias + nl1) : 0.f;
+                s[tl][j] = p0 * (tt[tl][j] - D0);          // ds
+                s[tl][2 + j] = p1 * (tt[tl][2 + j] - D1);
+            }
+        uint32_t dh[2][4], dl[2][4];
+        scores_as_a(s, dh, dl);
+        float part[KS][4];
+        scores_times_points<KS>(part, dh, dl, kr);
+#pragma unroll
+        for (int nt = 0; nt < KS; ++nt) {
+            acc[nt][0] += part[nt][0]; acc[nt][1] += part[nt][1]; acc[nt][2] += part[nt][2]; acc[nt][3] += part[nt][3];
+        }
+    }
+    float r0v[CPT], r1v[CPT];
+#pragma unroll
+    for (int nt = 0; nt < KS; ++nt) {
+        r0v[nt] = acc[nt][0] * scale; r0v[KS + nt] = acc[nt][1] * scale;
+        r1v[nt] = acc[nt][2] * scale; r1v[KS + nt] = acc[nt][3] * scale;
+    }
+    if (w0 + g < p.nlon_out) store_row<CPT>(dq + (orow + w0 + g) * C + t * CPT, r0v);
+    if (w0 + g + 8 < p.nlon_out) store_row<CPT>(dq + (orow + w0 + g + 8) * C + t * CPT, r1v);
+}
+
+// ---------------------------------------------------------------------------------------------------------
+// backward, dk and dv, gathered per input point over the transposed stream (no atomics):
+//   dk_j = scale * sum_i p_ij (t_ij - D_i) q_i,   dv_j = sum_i p_ij dout_i          (App. B.4)
+// Tile rows are 16 input columns c = ps*(u0+i) + r of one input ring; stream columns are output points.
+// ---------------------------------------------------------------------------------------------------------
+template <int C>
+__global__ void __launch_bounds__(THREADS, 1)
+backward_dkdv_mma_kernel(DevPlan p, const float* __restrict__ q, const float* __restrict__ k, const float* __restrict__ v,
+                         const float* __restrict__ dout, const float* __restrict__ lse, const float* __restrict__ Dws,
+                         float* __restrict__ dk, float* __restrict__ dv, int N, float scale, int tiles_per_row, long long total_tasks) {
+    constexpr int CPT = C / 4, KS = C / 8;
+    const int lane = threadIdx.x & 31, g = lane >> 2, t = lane & 3;
+    int n, rank, tile;
+    if (!decode_task(N, tiles_per_row * p.ps, total_tasks, n, rank, tile)) return;
+    const int hp = p.t_row_order[rank];
+    const int r = tile % p.ps;
+    const int u0 = (tile / p.ps) * 16;
+    const int i0 = min(u0 + g, p.nlon_out - 1), i1 = min(u0 + g + 8, p.nlon_out - 1);   // clamped tile rows (units of ps columns)
+    const size_t irow = (size_t)(n * p.nlat_in + hp) * p.nlon_in + r;
+    const float scale_log2 = scale * LOG2E;
+
+    uint32_t kh[KS][4], kl[KS][4], vh[KS][4], vl[KS][4];
+    make_a_operand<CPT>(k + (irow + (size_t)i0 * p.ps) * C + t * CPT, k + (irow + (size_t)i1 * p.ps) * C + t * CPT, scale_log2, kh, kl);
+    make_a_operand<CPT>(v + (irow + (size_t)i0 * p.ps) * C + t * CPT, v + (irow + (size_t)i1 * p.ps) * C + t * CPT, 1.f, vh, vl);
+    const float bias = p.log2_omega[hp];
+    float gk[KS][4], gv[KS][4];
+#pragma unroll
+    for (int nt = 0; nt < KS; ++nt) {
+        gk[nt][0] = gk[nt][1] = gk[nt][2] = gk[nt][3] = 0.f;
+        gv[nt][0] = gv[nt][1] = gv[nt][2] = gv[nt][3] = 0.f;
+    }
+    const size_t oslice = (size_t)n * p.nlat_out * p.nlon_out;
+    const float* qb = q + oslice * C + t * CPT;
+    const float* yb = dout + oslice * C + t * CPT;
+    const float* qc = q + oslice * C + g * KS;
+    const float* yc = dout + oslice * C + g * KS;
+    const float* lse_n = lse + oslice;
+    const float* D_n = Dws + oslice;
+    const int srow = hp * p.ps + r;
+    const int4* stream = p.t_stream + (size_t)p.t_chunk_ptr[srow] * 16;
+    const int nchunks = p.t_chunk_ptr[srow + 1] - p.t_chunk_ptr[srow];
+
+    for (int c = 0; c < nchunks; ++c) {
+        const ChunkColumn col = load_chunk_column(stream + c * 16, lane, u0, p.nlon_out, 1);
+        const float col_nl = fmaf(-__ldg(lse_n + col.idx), LOG2E, bias);   // -lse_i (log2) + log2 omega_j
+        const float col_D = __ldg(D_n + col.idx);
+        float s[2][4], tt[2][4];
+#pragma unroll
+        for (int tl = 0; tl < 2; ++tl) {
+            const size_t off = (size_t)__shfl_sync(FULL, col.idx, tl * 8 + g) * C;
+            float xr[CPT];
+            load_row<CPT>(qb + off, xr);
+            rows_dot_point<CPT>(s[tl], kh, kl, xr);
+            load_row<CPT>(yb + off, xr);
+            rows_dot_point<CPT>(tt[tl], vh, vl, xr);
+        }
+        float qr[2][2][KS], yr[2][2][KS];
+        float pr[2][4];
+#pragma unroll
+        for (int tl = 0; tl < 2; ++tl)
+#pragma unroll
+            for (int j = 0; j < 2; ++j) {
+                const int src = tl * 8 + 2 * t + j;
+                const size_t off = (size_t)__shfl_sync(FULL, col.idx, src) * C;
+                load_col<KS>(qc + off, qr[tl][j]);
+                load_col<KS>(yc + off, yr[tl][j]);
+                const float nl = __shfl_sync(FULL, col_nl, src);
+                const float Di = __shfl_sync(FULL, col_D, src);
+                const uint32_t mask = __shfl_sync(FULL, col.mask, src) >> g;
+                const float p0 = (mask & 1u) ? ex2(s[tl][j] + nl) : 0.f;
+                const float p1 = (mask & 0x100u) ? ex2(s[tl][2 + j] + nl) : 0.f;
+                pr[tl][j] = p0; pr[tl][2 + j] = p1;
+                s[tl][j] = p0 * (tt[tl][j] - Di);          // ds
+                s[tl][2 + j] = p1 * (tt[tl][2 + j] - Di);
+            }
+        uint32_t wh[2][4], wl[2][4];
+        float part[KS][4];
+        scores_as_a(pr, wh, wl);
+        scores_times_points<KS>(part, wh, wl, yr);
+#pragma unroll
+        for (int nt = 0; nt < KS; ++nt) { gv[nt][0] += part[nt][0]; gv[nt][1] += part[nt][1]; gv[nt][2] += part[nt][2]; gv[nt][3] += part[nt][3]; }
+        scores_as_a(s, wh, wl);
+        scores_times_points<KS>(part, wh, wl, qr);
+#pragma unroll
+        for (int nt = 0; nt < KS; ++nt) { gk[nt][0] += part[nt][0]; gk[nt][1] += part[nt][1]; gk[nt][2] += part[nt][2]; gk[nt][3] += part[nt][3]; }
+    }
+    // k was pre-multiplied by scale*log2e for the scores only; dk carries the plain scale
+    float a0[CPT], a1[CPT], b0[CPT], b1[CPT];
+#pragma unroll
+    for (int nt = 0; nt < KS; ++nt) {
+        a0[nt] = gk[nt][0] * scale; a0[KS + nt] = gk[nt][1] * scale; a1[nt] = gk[nt][2] * scale; a1[KS + nt] = gk[nt][3] * scale;
+        b0[nt] = gv[nt][0]; b0[KS + nt] = gv[nt][1]; b1[nt] = gv[nt][2]; b1[KS + nt] = gv[nt][3];
+    }
+    if (u0 + g < p.nlon_out) {
+        store_row<CPT>(dk + (irow + (size_t)(u0 + g) * p.ps) * C + t * CPT, a0);
+        store_row<CPT>(dv + (irow + (size_t)(u0 + g) * p.ps) * C + t * CPT, b0);
+    }
+    if (u0 + g + 8 < p.nlon_out) {
+        store_row<CPT>(dk + (irow + (size_t)(u0 + g + 8) * p.ps) * C + t * CPT, a1);
+        store_row<CPT>(dv + (irow + (size_t)(u0 + g + 8) * p.ps) * C + t * CPT, b1);
+    }
+}
+
+template <typename F>
+cudaError_t dispatch_c(int C, F&& f) {
+    switch (C) {
+        case 16: return f(std::integral_constant<int, 16>());
+        case 32: return f(std::integral_constant<int, 32>());
+        case 64: return f(std::integral_constant<int, 64>());
+        default: return cudaErrorInvalidValue;
     }
 }
 
@@ -255,13 +520,36 @@ cudaError_t launch_forward_mma(const DevPlan& p, const float* q, const float* k,
     const long long tasks = (long long)tiles * p.nlat_out * N;
     const long long blocks = (tasks + WARPS - 1) / WARPS;
     if (blocks > 0x7fffffffLL) return cudaErrorInvalidValue;
-    switch (C) {
-        case 16: forward_mma_kernel<16><<<(unsigned)blocks, THREADS, 0, stream>>>(p, q, k, v, out, lse, N, scale_log2, tiles, tasks); break;
-        case 32: forward_mma_kernel<32><<<(unsigned)blocks, THREADS, 0, stream>>>(p, q, k, v, out, lse, N, scale_log2, tiles, tasks); break;
-        case 64: forward_mma_kernel<64><<<(unsigned)blocks, THREADS, 0, stream>>>(p, q, k, v, out, lse, N, scale_log2, tiles, tasks); break;
-        default: return cudaErrorInvalidValue;
-    }
-    return cudaGetLastError();
+    return dispatch_c(C, [&](auto c) {
+        forward_mma_kernel<decltype(c)::value><<<(unsigned)blocks, THREADS, 0, stream>>>(p, q, k, v, out, lse, N, scale_log2, tiles, tasks);
+        return cudaGetLastError();
+    });
+}
+
+cudaError_t launch_backward_dq_mma(const DevPlan& p, const float* q, const float* k, const float* v, const float* dout,
+                                   const float* out, const float* lse, float* dq, float* Dws, int N, int C, cudaStream_t stream) {
+    const float scale = 1.0f / sqrtf((float)C);
+    const int tiles = (p.nlon_out + 15) / 16;
+    const long long tasks = (long long)tiles * p.nlat_out * N;
+    const long long blocks = (tasks + WARPS - 1) / WARPS;
+    if (blocks > 0x7fffffffLL) return cudaErrorInvalidValue;
+    return dispatch_c(C, [&](auto c) {
+        backward_dq_mma_kernel<decltype(c)::value><<<(unsigned)blocks, THREADS, 0, stream>>>(p, q, k, v, dout, out, lse, dq, Dws, N, scale, tiles, tasks);
+        return cudaGetLastError();
+    });
+}
+
+cudaError_t launch_backward_dkdv_mma(const DevPlan& p, const float* q, const float* k, const float* v, const float* dout,
+                                     const float* lse, const float* Dws, float* dk, float* dv, int N, int C, cudaStream_t stream) {
+    const float scale = 1.0f / sqrtf((float)C);
+    const int tiles = (p.nlon_out + 15) / 16;
+    const long long tasks = (long long)tiles * p.ps * p.nlat_in * N;
+    const long long blocks = (tasks + WARPS - 1) / WARPS;
+    if (blocks > 0x7fffffffLL) return cudaErrorInvalidValue;
+    return dispatch_c(C, [&](auto c) {
+        backward_dkdv_mma_kernel<decltype(c)::value><<<(unsigned)blocks, THREADS, 0, stream>>>(p, q, k, v, dout, lse, Dws, dk, dv, N, scale, tiles, tasks);
+        return cudaGetLastError();
+    });
 }
 
 }  // namespace sna
