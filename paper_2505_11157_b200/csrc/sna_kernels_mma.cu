@@ -5,8 +5,8 @@
 // Work decomposition: one warp owns 16 consecutive points of one ring (the M dimension of the MMA: "tile rows")
 // and walks the host-built column stream of that ring row, 16 partner points ("columns") per step.  Band
 // structure and ragged edges are expressed by the 16-bit row mask carried by every stream column.
-// Operands are loaded straight from global memory (L1/L2) in fragment order; warps never synchronise with
-// each other, and there is no shared memory.
+// The 16 partner points of a chunk are staged by cp.async into a warp-private, two-stage shared-memory ring
+// while the previous chunk is consumed; warps never synchronise with each other (no block-level barrier).
 //
 // Fragment conventions (g = lane / 4, t = lane % 4, CPT = C/4, KS = C/8):
 //   "row fragment" of a point: the CPT channels [t*CPT, (t+1)*CPT) of that point.  As an A operand it belongs to
@@ -26,7 +26,7 @@
 namespace sna {
 namespace {
 
-constexpr int WARPS = 8;
+constexpr int WARPS = 4;
 constexpr int THREADS = WARPS * 32;
 constexpr float LOG2E = 1.4426950408889634f;
 constexpr float LN2 = 0.6931471805599453f;
@@ -158,15 +158,37 @@ __device__ __forceinline__ void scores_times_points(float (&d)[KS][4], const uin
     }
 }
 
-// One 16-column chunk of a stream as seen by a warp: lane l holds column l % 16.
-struct ChunkColumn {
-    int idx;        // flat index of the partner point inside one batch*head slice
-    uint32_t mask;  // tile rows that use this column
-    float bias;     // forward stream: log2 of the partner's quadrature weight
+// ---------------------------------------------------------------------------------------------------------
+// Warp-private staging of a chunk's 16 partner points in shared memory (cp.async, two stages).
+// Two point arrays are staged per chunk (forward / dq: k and v rows; dk/dv: q and dout rows), each row padded
+// to C+4 floats so that both fragment layouts read without bank conflicts, plus per-column metadata.
+// ---------------------------------------------------------------------------------------------------------
+template <int C>
+struct Stage {
+    static constexpr int PITCH = C + 4;
+    float a[16][PITCH];
+    float b[16][PITCH];
+    uint32_t mask[16];   // tile rows that use the column
+    float m0[16];        // forward stream: log2 omega of the partner ring; transposed stream: lse of the partner
+    float m1[16];        // transposed stream: D of the partner
+    float pad[16];
 };
 
-__device__ __forceinline__ ChunkColumn load_chunk_column(const int4* chunk, int lane, int first, int ring_len, int stride) {
-    const int4 e = __ldg(chunk + (lane & 15));
+__device__ __forceinline__ void cp_async16(void* smem_dst, const void* gmem_src) {
+    const uint32_t d = (uint32_t)__cvta_generic_to_shared(smem_dst);
+    asm volatile("cp.async.ca.shared.global [%0], [%1], 16;" ::"r"(d), "l"(gmem_src) : "memory");
+}
+__device__ __forceinline__ void cp_async4(void* smem_dst, const void* gmem_src) {
+    const uint32_t d = (uint32_t)__cvta_generic_to_shared(smem_dst);
+    asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(d), "l"(gmem_src) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
+
+// Flat index (inside one batch*head slice) of the partner point of stream entry e for a tile whose first point
+// is `first` on a ring of `ring_len` points; consecutive partners are `stride` apart in memory.
+__device__ __forceinline__ int partner_index(const int4& e, int first, int ring_len, int stride) {
     int u = (int)(short)(e.y & 0xffff);
     if (e.x >= 0) {   // offset relative to the tile's first point, wrapped around the ring
         u += first;
@@ -174,11 +196,55 @@ __device__ __forceinline__ ChunkColumn load_chunk_column(const int4* chunk, int 
         if (u >= ring_len) u -= ring_len;
         if (u >= ring_len) u -= ring_len;
     }
-    ChunkColumn c;
-    c.idx = (e.x & 0x7fffffff) + u * stride;
-    c.mask = (uint32_t)e.y >> 16;
-    c.bias = __int_as_float(e.z);
-    return c;
+    return (e.x & 0x7fffffff) + u * stride;
+}
+
+// Issue the copies of one chunk: lane l owns stream column l % 16 (entry e).  Rows of both arrays are copied
+// in 16-byte pieces, C/8 pieces per lane and array; metadata is written by the owning lanes.
+template <int C, bool TRANSPOSED>
+__device__ __forceinline__ void stage_chunk(Stage<C>& st, const int4& e, int lane, int first, int ring_len, int stride,
+                                            const float* a_base, const float* b_base, const float* lse_base, const float* D_base) {
+    const int idx = partner_index(e, first, ring_len, stride);
+    constexpr int PIECES = C / 4;              // 16-byte pieces per row
+#pragma unroll
+    for (int j = 0; j < C / 8; ++j) {
+        const int i = lane + 32 * j;
+        const int row = i / PIECES, piece = i % PIECES;
+        const size_t off = (size_t)__shfl_sync(FULL, idx, row) * C + piece * 4;
+        cp_async16(&st.a[row][piece * 4], a_base + off);
+        cp_async16(&st.b[row][piece * 4], b_base + off);
+    }
+    if (lane < 16) {
+        st.mask[lane] = (uint32_t)e.y >> 16;
+        if (TRANSPOSED) {
+            cp_async4(&st.m0[lane], lse_base + idx);
+            cp_async4(&st.m1[lane], D_base + idx);
+        } else {
+            st.m0[lane] = __int_as_float(e.z);
+        }
+    }
+}
+
+template <int CPT, int PITCH>
+__device__ __forceinline__ void lds_row(const float (&arr)[16][PITCH], int row, int t, float (&x)[CPT]) {
+#pragma unroll
+    for (int j = 0; j < CPT / 4; ++j) {
+        const float4 v4 = *reinterpret_cast<const float4*>(&arr[row][t * CPT + 4 * j]);
+        x[4 * j] = v4.x; x[4 * j + 1] = v4.y; x[4 * j + 2] = v4.z; x[4 * j + 3] = v4.w;
+    }
+}
+template <int KS, int PITCH>
+__device__ __forceinline__ void lds_col(const float (&arr)[16][PITCH], int row, int g, float (&x)[KS]) {
+    if constexpr (KS % 4 == 0) {
+#pragma unroll
+        for (int j = 0; j < KS / 4; ++j) {
+            const float4 v4 = *reinterpret_cast<const float4*>(&arr[row][g * KS + 4 * j]);
+            x[4 * j] = v4.x; x[4 * j + 1] = v4.y; x[4 * j + 2] = v4.z; x[4 * j + 3] = v4.w;
+        }
+    } else {
+        const float2 v2 = *reinterpret_cast<const float2*>(&arr[row][g * KS]);
+        x[0] = v2.x; x[1] = v2.y;
+    }
 }
 
 // Decode a warp task into (slice n, rank of the ring row in heavy-first order, tile).
@@ -198,6 +264,28 @@ __device__ __forceinline__ void store_row(float* p, const float (&x)[CPT]) {
     for (int j = 0; j < CPT / 4; ++j) *reinterpret_cast<float4*>(p + 4 * j) = make_float4(x[4 * j], x[4 * j + 1], x[4 * j + 2], x[4 * j + 3]);
 }
 
+// The software pipeline shared by the three kernels: chunk c+1 is copied while chunk c is consumed.
+//   BODY(stage) consumes one staged chunk.
+template <int C, bool TRANSPOSED, typename Body>
+__device__ __forceinline__ void walk_stream(Stage<C>* stages, const int4* stream, int nchunks, int lane, int first, int ring_len,
+                                            int stride, const float* a_base, const float* b_base, const float* lse_base,
+                                            const float* D_base, Body&& body) {
+    if (nchunks <= 0) return;
+    int4 e = __ldg(stream + (lane & 15));
+    stage_chunk<C, TRANSPOSED>(stages[0], e, lane, first, ring_len, stride, a_base, b_base, lse_base, D_base);
+    cp_async_commit();
+    if (nchunks > 1) e = __ldg(stream + 16 + (lane & 15));
+    for (int c = 0; c < nchunks; ++c) {
+        if (c + 1 < nchunks) stage_chunk<C, TRANSPOSED>(stages[(c + 1) & 1], e, lane, first, ring_len, stride, a_base, b_base, lse_base, D_base);
+        cp_async_commit();
+        if (c + 2 < nchunks) e = __ldg(stream + (size_t)(c + 2) * 16 + (lane & 15));
+        cp_async_wait<1>();
+        __syncwarp();
+        body(stages[c & 1]);
+        __syncwarp();   // everyone is done with this stage before the next iteration refills it
+    }
+}
+
 // ---------------------------------------------------------------------------------------------------------
 // forward
 // ---------------------------------------------------------------------------------------------------------
@@ -206,6 +294,8 @@ __global__ void __launch_bounds__(THREADS)
 forward_mma_kernel(DevPlan p, const float* __restrict__ q, const float* __restrict__ k, const float* __restrict__ v,
                    float* __restrict__ out, float* __restrict__ lse, int N, float scale_log2, int tiles_per_row, long long total_tasks) {
     constexpr int CPT = C / 4, KS = C / 8;
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    Stage<C>* stages = reinterpret_cast<Stage<C>*>(smem_raw) + 2 * (threadIdx.x >> 5);
     const int lane = threadIdx.x & 31, g = lane >> 2, t = lane & 3;
     int n, rank, tile;
     if (!decode_task(N, tiles_per_row, total_tasks, n, rank, tile)) return;
@@ -221,32 +311,31 @@ forward_mma_kernel(DevPlan p, const float* __restrict__ q, const float* __restri
     for (int nt = 0; nt < KS; ++nt) o[nt][0] = o[nt][1] = o[nt][2] = o[nt][3] = 0.f;
     float m0 = -INFINITY, m1 = -INFINITY, l0 = 0.f, l1 = 0.f;
 
-    const float* kb = k + (size_t)n * p.nlat_in * p.nlon_in * C + t * CPT;
-    const float* vb = v + (size_t)n * p.nlat_in * p.nlon_in * C + g * KS;
+    const size_t slice = (size_t)n * p.nlat_in * p.nlon_in * C;
     const int4* stream = p.fwd_stream + (size_t)p.fwd_chunk_ptr[h] * 16;
     const int nchunks = p.fwd_chunk_ptr[h + 1] - p.fwd_chunk_ptr[h];
 
-    for (int c = 0; c < nchunks; ++c) {
-        const ChunkColumn col = load_chunk_column(stream + c * 16, lane, w0, p.nlon_out, p.ps);
+    walk_stream<C, false>(stages, stream, nchunks, lane, w0, p.nlon_out, p.ps, k + slice, v + slice, nullptr, nullptr, [&](const Stage<C>& st) {
         float s[2][4];
 #pragma unroll
         for (int tl = 0; tl < 2; ++tl) {
             float kr[CPT];
-            load_row<CPT>(kb + (size_t)__shfl_sync(FULL, col.idx, tl * 8 + g) * C, kr);
+            lds_row<CPT>(st.a, tl * 8 + g, t, kr);
             rows_dot_point<CPT>(s[tl], qh, ql, kr);
         }
         float vr[2][2][KS];
 #pragma unroll
-        for (int tl = 0; tl < 2; ++tl)
-#pragma unroll
-            for (int j = 0; j < 2; ++j) {
-                const int src = tl * 8 + 2 * t + j;
-                load_col<KS>(vb + (size_t)__shfl_sync(FULL, col.idx, src) * C, vr[tl][j]);
-                const float bias = __shfl_sync(FULL, col.bias, src);
-                const uint32_t mask = __shfl_sync(FULL, col.mask, src) >> g;
-                s[tl][j] = (mask & 1u) ? s[tl][j] + bias : -INFINITY;
-                s[tl][2 + j] = (mask & 0x100u) ? s[tl][2 + j] + bias : -INFINITY;
-            }
+        for (int tl = 0; tl < 2; ++tl) {
+            const uint2 mk = *reinterpret_cast<const uint2*>(&st.mask[tl * 8 + 2 * t]);
+            const float2 bs = *reinterpret_cast<const float2*>(&st.m0[tl * 8 + 2 * t]);
+            lds_col<KS>(st.b, tl * 8 + 2 * t, g, vr[tl][0]);
+            lds_col<KS>(st.b, tl * 8 + 2 * t + 1, g, vr[tl][1]);
+            const uint32_t ma = mk.x >> g, mb = mk.y >> g;
+            s[tl][0] = (ma & 1u) ? s[tl][0] + bs.x : -INFINITY;
+            s[tl][1] = (mb & 1u) ? s[tl][1] + bs.y : -INFINITY;
+            s[tl][2] = (ma & 0x100u) ? s[tl][2] + bs.x : -INFINITY;
+            s[tl][3] = (mb & 0x100u) ? s[tl][3] + bs.y : -INFINITY;
+        }
         // online softmax over the chunk (row maxima across the four threads of a group)
         float mx0 = fmaxf(fmaxf(s[0][0], s[0][1]), fmaxf(s[1][0], s[1][1]));
         float mx1 = fmaxf(fmaxf(s[0][2], s[0][3]), fmaxf(s[1][2], s[1][3]));
@@ -277,7 +366,7 @@ forward_mma_kernel(DevPlan p, const float* __restrict__ q, const float* __restri
             o[nt][0] = fmaf(o[nt][0], corr0, pv[nt][0]); o[nt][1] = fmaf(o[nt][1], corr0, pv[nt][1]);
             o[nt][2] = fmaf(o[nt][2], corr1, pv[nt][2]); o[nt][3] = fmaf(o[nt][3], corr1, pv[nt][3]);
         }
-    }
+    });
     // row sums across the four threads of a group, normalise, store
     l0 += __shfl_xor_sync(FULL, l0, 1); l1 += __shfl_xor_sync(FULL, l1, 1);
     l0 += __shfl_xor_sync(FULL, l0, 2); l1 += __shfl_xor_sync(FULL, l1, 2);
@@ -303,11 +392,13 @@ forward_mma_kernel(DevPlan p, const float* __restrict__ q, const float* __restri
 // `out` and `dq` may be the same buffer: a warp reads its own 16 rows of `out` before it writes them as dq.
 // ---------------------------------------------------------------------------------------------------------
 template <int C>
-__global__ void __launch_bounds__(THREADS, 1)
+__global__ void __launch_bounds__(THREADS)
 backward_dq_mma_kernel(DevPlan p, const float* __restrict__ q, const float* __restrict__ k, const float* __restrict__ v,
                        const float* __restrict__ dout, const float* out, const float* __restrict__ lse,
                        float* dq, float* __restrict__ Dws, int N, float scale, int tiles_per_row, long long total_tasks) {
     constexpr int CPT = C / 4, KS = C / 8;
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    Stage<C>* stages = reinterpret_cast<Stage<C>*>(smem_raw) + 2 * (threadIdx.x >> 5);
     const int lane = threadIdx.x & 31, g = lane >> 2, t = lane & 3;
     int n, rank, tile;
     if (!decode_task(N, tiles_per_row, total_tasks, n, rank, tile)) return;
@@ -343,38 +434,36 @@ backward_dq_mma_kernel(DevPlan p, const float* __restrict__ q, const float* __re
     for (int nt = 0; nt < KS; ++nt) acc[nt][0] = acc[nt][1] = acc[nt][2] = acc[nt][3] = 0.f;
 
     const size_t slice = (size_t)n * p.nlat_in * p.nlon_in * C;
-    const float* kb = k + slice + t * CPT;
-    const float* vb = v + slice + t * CPT;
-    const float* kc = k + slice + g * KS;
     const int4* stream = p.fwd_stream + (size_t)p.fwd_chunk_ptr[h] * 16;
     const int nchunks = p.fwd_chunk_ptr[h + 1] - p.fwd_chunk_ptr[h];
 
-    for (int c = 0; c < nchunks; ++c) {
-        const ChunkColumn col = load_chunk_column(stream + c * 16, lane, w0, p.nlon_out, p.ps);
+    walk_stream<C, false>(stages, stream, nchunks, lane, w0, p.nlon_out, p.ps, k + slice, v + slice, nullptr, nullptr, [&](const Stage<C>& st) {
         float s[2][4], tt[2][4];
 #pragma unroll
         for (int tl = 0; tl < 2; ++tl) {
-            const size_t off = (size_t)__shfl_sync(FULL, col.idx, tl * 8 + g) * C;
             float xr[CPT];
-            load_row<CPT>(kb + off, xr);
+            lds_row<CPT>(st.a, tl * 8 + g, t, xr);
             rows_dot_point<CPT>(s[tl], qh, ql, xr);
-            load_row<CPT>(vb + off, xr);
+            lds_row<CPT>(st.b, tl * 8 + g, t, xr);
             rows_dot_point<CPT>(tt[tl], yh, yl, xr);
         }
         float kr[2][2][KS];
 #pragma unroll
-        for (int tl = 0; tl < 2; ++tl)
-#pragma unroll
-            for (int j = 0; j < 2; ++j) {
-                const int src = tl * 8 + 2 * t + j;
-                load_col<KS>(kc + (size_t)__shfl_sync(FULL, col.idx, src) * C, kr[tl][j]);
-                const float bias = __shfl_sync(FULL, col.bias, src);
-                const uint32_t mask = __shfl_sync(FULL, col.mask, src) >> g;
-                const float p0 = (mask & 1u) ? ex2(s[tl][j] + bias + nl0) : 0.f;
-                const float p1 = (mask & 0x100u) ? ex2(s[tl][2 + j] + bias + nl1) : 0.f;
-                s[tl][j] = p0 * (tt[tl][j] - D0);          // ds
-                s[tl][2 + j] = p1 * (tt[tl][2 + j] - D1);
-            }
+        for (int tl = 0; tl < 2; ++tl) {
+            const uint2 mk = *reinterpret_cast<const uint2*>(&st.mask[tl * 8 + 2 * t]);
+            const float2 bs = *reinterpret_cast<const float2*>(&st.m0[tl * 8 + 2 * t]);
+            lds_col<KS>(st.a, tl * 8 + 2 * t, g, kr[tl][0]);
+            lds_col<KS>(st.a, tl * 8 + 2 * t + 1, g, kr[tl][1]);
+            const uint32_t ma = mk.x >> g, mb = mk.y >> g;
+            const float p00 = (ma & 1u) ? ex2(s[tl][0] + bs.x + nl0) : 0.f;
+            const float p01 = (mb & 1u) ? ex2(s[tl][1] + bs.y + nl0) : 0.f;
+            const float p10 = (ma & 0x100u) ? ex2(s[tl][2] + bs.x + nl1) : 0.f;
+            const float p11 = (mb & 0x100u) ? ex2(s[tl][3] + bs.y + nl1) : 0.f;
+            s[tl][0] = p00 * (tt[tl][0] - D0);   // ds
+            s[tl][1] = p01 * (tt[tl][1] - D0);
+            s[tl][2] = p10 * (tt[tl][2] - D1);
+            s[tl][3] = p11 * (tt[tl][3] - D1);
+        }
         uint32_t dh[2][4], dl[2][4];
         scores_as_a(s, dh, dl);
         float part[KS][4];
@@ -383,7 +472,7 @@ backward_dq_mma_kernel(DevPlan p, const float* __restrict__ q, const float* __re
         for (int nt = 0; nt < KS; ++nt) {
             acc[nt][0] += part[nt][0]; acc[nt][1] += part[nt][1]; acc[nt][2] += part[nt][2]; acc[nt][3] += part[nt][3];
         }
-    }
+    });
     float r0v[CPT], r1v[CPT];
 #pragma unroll
     for (int nt = 0; nt < KS; ++nt) {
@@ -400,11 +489,13 @@ backward_dq_mma_kernel(DevPlan p, const float* __restrict__ q, const float* __re
 // Tile rows are 16 input columns c = ps*(u0+i) + r of one input ring; stream columns are output points.
 // ---------------------------------------------------------------------------------------------------------
 template <int C>
-__global__ void __launch_bounds__(THREADS, 1)
+__global__ void __launch_bounds__(THREADS)
 backward_dkdv_mma_kernel(DevPlan p, const float* __restrict__ q, const float* __restrict__ k, const float* __restrict__ v,
                          const float* __restrict__ dout, const float* __restrict__ lse, const float* __restrict__ Dws,
                          float* __restrict__ dk, float* __restrict__ dv, int N, float scale, int tiles_per_row, long long total_tasks) {
     constexpr int CPT = C / 4, KS = C / 8;
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    Stage<C>* stages = reinterpret_cast<Stage<C>*>(smem_raw) + 2 * (threadIdx.x >> 5);
     const int lane = threadIdx.x & 31, g = lane >> 2, t = lane & 3;
     int n, rank, tile;
     if (!decode_task(N, tiles_per_row * p.ps, total_tasks, n, rank, tile)) return;
@@ -426,49 +517,42 @@ backward_dkdv_mma_kernel(DevPlan p, const float* __restrict__ q, const float* __
         gv[nt][0] = gv[nt][1] = gv[nt][2] = gv[nt][3] = 0.f;
     }
     const size_t oslice = (size_t)n * p.nlat_out * p.nlon_out;
-    const float* qb = q + oslice * C + t * CPT;
-    const float* yb = dout + oslice * C + t * CPT;
-    const float* qc = q + oslice * C + g * KS;
-    const float* yc = dout + oslice * C + g * KS;
-    const float* lse_n = lse + oslice;
-    const float* D_n = Dws + oslice;
     const int srow = hp * p.ps + r;
     const int4* stream = p.t_stream + (size_t)p.t_chunk_ptr[srow] * 16;
     const int nchunks = p.t_chunk_ptr[srow + 1] - p.t_chunk_ptr[srow];
 
-    for (int c = 0; c < nchunks; ++c) {
-        const ChunkColumn col = load_chunk_column(stream + c * 16, lane, u0, p.nlon_out, 1);
-        const float col_nl = fmaf(-__ldg(lse_n + col.idx), LOG2E, bias);   // -lse_i (log2) + log2 omega_j
-        const float col_D = __ldg(D_n + col.idx);
+    walk_stream<C, true>(stages, stream, nchunks, lane, u0, p.nlon_out, 1, q + oslice * C, dout + oslice * C, lse + oslice, Dws + oslice, [&](const Stage<C>& st) {
         float s[2][4], tt[2][4];
 #pragma unroll
         for (int tl = 0; tl < 2; ++tl) {
-            const size_t off = (size_t)__shfl_sync(FULL, col.idx, tl * 8 + g) * C;
             float xr[CPT];
-            load_row<CPT>(qb + off, xr);
+            lds_row<CPT>(st.a, tl * 8 + g, t, xr);
             rows_dot_point<CPT>(s[tl], kh, kl, xr);
-            load_row<CPT>(yb + off, xr);
+            lds_row<CPT>(st.b, tl * 8 + g, t, xr);
             rows_dot_point<CPT>(tt[tl], vh, vl, xr);
         }
         float qr[2][2][KS], yr[2][2][KS];
         float pr[2][4];
 #pragma unroll
-        for (int tl = 0; tl < 2; ++tl)
-#pragma unroll
-            for (int j = 0; j < 2; ++j) {
-                const int src = tl * 8 + 2 * t + j;
-                const size_t off = (size_t)__shfl_sync(FULL, col.idx, src) * C;
-                load_col<KS>(qc + off, qr[tl][j]);
-                load_col<KS>(yc + off, yr[tl][j]);
-                const float nl = __shfl_sync(FULL, col_nl, src);
-                const float Di = __shfl_sync(FULL, col_D, src);
-                const uint32_t mask = __shfl_sync(FULL, col.mask, src) >> g;
-                const float p0 = (mask & 1u) ? ex2(s[tl][j] + nl) : 0.f;
-                const float p1 = (mask & 0x100u) ? ex2(s[tl][2 + j] + nl) : 0.f;
-                pr[tl][j] = p0; pr[tl][2 + j] = p1;
-                s[tl][j] = p0 * (tt[tl][j] - Di);          // ds
-                s[tl][2 + j] = p1 * (tt[tl][2 + j] - Di);
-            }
+        for (int tl = 0; tl < 2; ++tl) {
+            const uint2 mk = *reinterpret_cast<const uint2*>(&st.mask[tl * 8 + 2 * t]);
+            const float2 ls = *reinterpret_cast<const float2*>(&st.m0[tl * 8 + 2 * t]);
+            const float2 Dd = *reinterpret_cast<const float2*>(&st.m1[tl * 8 + 2 * t]);
+            lds_col<KS>(st.a, tl * 8 + 2 * t, g, qr[tl][0]);
+            lds_col<KS>(st.a, tl * 8 + 2 * t + 1, g, qr[tl][1]);
+            lds_col<KS>(st.b, tl * 8 + 2 * t, g, yr[tl][0]);
+            lds_col<KS>(st.b, tl * 8 + 2 * t + 1, g, yr[tl][1]);
+            const float nla = fmaf(-ls.x, LOG2E, bias), nlb = fmaf(-ls.y, LOG2E, bias);   // -lse_i (log2) + log2 omega_j
+            const uint32_t ma = mk.x >> g, mb = mk.y >> g;
+            pr[tl][0] = (ma & 1u) ? ex2(s[tl][0] + nla) : 0.f;
+            pr[tl][1] = (mb & 1u) ? ex2(s[tl][1] + nlb) : 0.f;
+            pr[tl][2] = (ma & 0x100u) ? ex2(s[tl][2] + nla) : 0.f;
+            pr[tl][3] = (mb & 0x100u) ? ex2(s[tl][3] + nlb) : 0.f;
+            s[tl][0] = pr[tl][0] * (tt[tl][0] - Dd.x);   // ds
+            s[tl][1] = pr[tl][1] * (tt[tl][1] - Dd.y);
+            s[tl][2] = pr[tl][2] * (tt[tl][2] - Dd.x);
+            s[tl][3] = pr[tl][3] * (tt[tl][3] - Dd.y);
+        }
         uint32_t wh[2][4], wl[2][4];
         float part[KS][4];
         scores_as_a(pr, wh, wl);
@@ -479,7 +563,7 @@ backward_dkdv_mma_kernel(DevPlan p, const float* __restrict__ q, const float* __
         scores_times_points<KS>(part, wh, wl, qr);
 #pragma unroll
         for (int nt = 0; nt < KS; ++nt) { gk[nt][0] += part[nt][0]; gk[nt][1] += part[nt][1]; gk[nt][2] += part[nt][2]; gk[nt][3] += part[nt][3]; }
-    }
+    });
     // k was pre-multiplied by scale*log2e for the scores only; dk carries the plain scale
     float a0[CPT], a1[CPT], b0[CPT], b1[CPT];
 #pragma unroll
@@ -495,6 +579,16 @@ backward_dkdv_mma_kernel(DevPlan p, const float* __restrict__ q, const float* __
         store_row<CPT>(dk + (irow + (size_t)(u0 + g + 8) * p.ps) * C + t * CPT, a1);
         store_row<CPT>(dv + (irow + (size_t)(u0 + g + 8) * p.ps) * C + t * CPT, b1);
     }
+}
+
+template <int C>
+constexpr size_t smem_bytes() { return sizeof(Stage<C>) * 2 * WARPS; }
+
+// Dynamic shared memory above 48 KB needs an opt-in per kernel; it is requested on every launch (a cheap
+// host-side call) so that it holds on whichever device is current.
+template <typename K>
+cudaError_t prepare_kernel(K kernel, size_t bytes) {
+    return bytes > 48 * 1024 ? cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes) : cudaSuccess;
 }
 
 template <typename F>
@@ -521,7 +615,10 @@ cudaError_t launch_forward_mma(const DevPlan& p, const float* q, const float* k,
     const long long blocks = (tasks + WARPS - 1) / WARPS;
     if (blocks > 0x7fffffffLL) return cudaErrorInvalidValue;
     return dispatch_c(C, [&](auto c) {
-        forward_mma_kernel<decltype(c)::value><<<(unsigned)blocks, THREADS, 0, stream>>>(p, q, k, v, out, lse, N, scale_log2, tiles, tasks);
+        constexpr int CC = decltype(c)::value;
+        cudaError_t e = prepare_kernel(forward_mma_kernel<CC>, smem_bytes<CC>());
+        if (e != cudaSuccess) return e;
+        forward_mma_kernel<CC><<<(unsigned)blocks, THREADS, smem_bytes<CC>(), stream>>>(p, q, k, v, out, lse, N, scale_log2, tiles, tasks);
         return cudaGetLastError();
     });
 }
@@ -534,7 +631,10 @@ cudaError_t launch_backward_dq_mma(const DevPlan& p, const float* q, const float
     const long long blocks = (tasks + WARPS - 1) / WARPS;
     if (blocks > 0x7fffffffLL) return cudaErrorInvalidValue;
     return dispatch_c(C, [&](auto c) {
-        backward_dq_mma_kernel<decltype(c)::value><<<(unsigned)blocks, THREADS, 0, stream>>>(p, q, k, v, dout, out, lse, dq, Dws, N, scale, tiles, tasks);
+        constexpr int CC = decltype(c)::value;
+        cudaError_t e = prepare_kernel(backward_dq_mma_kernel<CC>, smem_bytes<CC>());
+        if (e != cudaSuccess) return e;
+        backward_dq_mma_kernel<CC><<<(unsigned)blocks, THREADS, smem_bytes<CC>(), stream>>>(p, q, k, v, dout, out, lse, dq, Dws, N, scale, tiles, tasks);
         return cudaGetLastError();
     });
 }
@@ -547,7 +647,10 @@ cudaError_t launch_backward_dkdv_mma(const DevPlan& p, const float* q, const flo
     const long long blocks = (tasks + WARPS - 1) / WARPS;
     if (blocks > 0x7fffffffLL) return cudaErrorInvalidValue;
     return dispatch_c(C, [&](auto c) {
-        backward_dkdv_mma_kernel<decltype(c)::value><<<(unsigned)blocks, THREADS, 0, stream>>>(p, q, k, v, dout, lse, Dws, dk, dv, N, scale, tiles, tasks);
+        constexpr int CC = decltype(c)::value;
+        cudaError_t e = prepare_kernel(backward_dkdv_mma_kernel<CC>, smem_bytes<CC>());
+        if (e != cudaSuccess) return e;
+        backward_dkdv_mma_kernel<CC><<<(unsigned)blocks, THREADS, smem_bytes<CC>(), stream>>>(p, q, k, v, dout, lse, Dws, dk, dv, N, scale, tiles, tasks);
         return cudaGetLastError();
     });
 }
