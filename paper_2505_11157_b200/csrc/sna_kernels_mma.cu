@@ -57,12 +57,12 @@ __device__ __forceinline__ void split_rn(float x, uint32_t& hi, uint32_t& lo) {
 // small correction terms lo*hi + hi*lo go first, the main terms hi*hi last, into a fragment that starts at
 // zero, and long sums are carried in fp32 FMAs outside the tensor core.
 __device__ __forceinline__ void mma_acc(float (&d)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
-    asm volatile("mma.sync.aligned.m16n8k8.row.col.f32.tf32.tf32.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+    asm("mma.sync.aligned.m16n8k8.row.col.f32.tf32.tf32.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
                  : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
                  : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
 }
 __device__ __forceinline__ void mma_zero(float (&d)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
-    asm volatile("mma.sync.aligned.m16n8k8.row.col.f32.tf32.tf32.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%10,%10,%10,%10};"
+    asm("mma.sync.aligned.m16n8k8.row.col.f32.tf32.tf32.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%10,%10,%10,%10};"
                  : "=f"(d[0]), "=f"(d[1]), "=f"(d[2]), "=f"(d[3])
                  : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1), "f"(0.f));
 }
@@ -108,21 +108,85 @@ __device__ __forceinline__ void make_a_operand(const float* p0, const float* p1,
     }
 }
 
-// d[16x8] = A (tile rows x channels) . B^T, B = row fragment `x` of the point in tile column g.
+// d[tl][16x8] = A (tile rows x channels) . B^T for the two 8-column tiles of a chunk; B = row fragment x[tl] of the
+// point in column g of tile tl.  The two dependent MMA chains are interleaved.
 template <int CPT>
-__device__ __forceinline__ void rows_dot_point(float (&d)[4], const uint32_t (&ah)[CPT / 2][4], const uint32_t (&al)[CPT / 2][4], const float (&x)[CPT]) {
-    uint32_t bh[CPT], bl[CPT];
+__device__ __forceinline__ void rows_dot_points(float (&d)[2][4], const uint32_t (&ah)[CPT / 2][4], const uint32_t (&al)[CPT / 2][4], const float (&x)[2][CPT]) {
+    uint32_t bh[2][CPT], bl[2][CPT];
 #pragma unroll
-    for (int j = 0; j < CPT; ++j) split_fast(x[j], bh[j], bl[j]);
-    mma_zero(d, al[0], bh[0], bh[1]);
-    mma_acc(d, ah[0], bl[0], bl[1]);
+    for (int tl = 0; tl < 2; ++tl)
+#pragma unroll
+        for (int j = 0; j < CPT; ++j) split_fast(x[tl][j], bh[tl][j], bl[tl][j]);
+    mma_zero(d[0], al[0], bh[0][0], bh[0][1]);
+    mma_zero(d[1], al[0], bh[1][0], bh[1][1]);
+    mma_acc(d[0], ah[0], bl[0][0], bl[0][1]);
+    mma_acc(d[1], ah[0], bl[1][0], bl[1][1]);
 #pragma unroll
     for (int ks = 1; ks < CPT / 2; ++ks) {
-        mma_acc(d, al[ks], bh[2 * ks], bh[2 * ks + 1]);
-        mma_acc(d, ah[ks], bl[2 * ks], bl[2 * ks + 1]);
+        mma_acc(d[0], al[ks], bh[0][2 * ks], bh[0][2 * ks + 1]);
+        mma_acc(d[1], al[ks], bh[1][2 * ks], bh[1][2 * ks + 1]);
+        mma_acc(d[0], ah[ks], bl[0][2 * ks], bl[0][2 * ks + 1]);
+        mma_acc(d[1], ah[ks], bl[1][2 * ks], bl[1][2 * ks + 1]);
     }
 #pragma unroll
-    for (int ks = 0; ks < CPT / 2; ++ks) mma_acc(d, ah[ks], bh[2 * ks], bh[2 * ks + 1]);
+    for (int ks = 0; ks < CPT / 2; ++ks) {
+        mma_acc(d[0], ah[ks], bh[0][2 * ks], bh[0][2 * ks + 1]);
+        mma_acc(d[1], ah[ks], bh[1][2 * ks], bh[1][2 * ks + 1]);
+    }
+}
+
+// The same contraction with the B operand already split (shared by several M-tiles).
+template <int CPT>
+__device__ __forceinline__ void split_rows(const float (&x)[2][CPT], uint32_t (&bh)[2][CPT], uint32_t (&bl)[2][CPT]) {
+#pragma unroll
+    for (int tl = 0; tl < 2; ++tl)
+#pragma unroll
+        for (int j = 0; j < CPT; ++j) split_fast(x[tl][j], bh[tl][j], bl[tl][j]);
+}
+template <int CPT>
+__device__ __forceinline__ void rows_dot_split(float (&d)[2][4], const uint32_t (&ah)[CPT / 2][4], const uint32_t (&al)[CPT / 2][4],
+                                               const uint32_t (&bh)[2][CPT], const uint32_t (&bl)[2][CPT]) {
+    mma_zero(d[0], al[0], bh[0][0], bh[0][1]);
+    mma_zero(d[1], al[0], bh[1][0], bh[1][1]);
+    mma_acc(d[0], ah[0], bl[0][0], bl[0][1]);
+    mma_acc(d[1], ah[0], bl[1][0], bl[1][1]);
+#pragma unroll
+    for (int ks = 1; ks < CPT / 2; ++ks) {
+        mma_acc(d[0], al[ks], bh[0][2 * ks], bh[0][2 * ks + 1]);
+        mma_acc(d[1], al[ks], bh[1][2 * ks], bh[1][2 * ks + 1]);
+        mma_acc(d[0], ah[ks], bl[0][2 * ks], bl[0][2 * ks + 1]);
+        mma_acc(d[1], ah[ks], bl[1][2 * ks], bl[1][2 * ks + 1]);
+    }
+#pragma unroll
+    for (int ks = 0; ks < CPT / 2; ++ks) {
+        mma_acc(d[0], ah[ks], bh[0][2 * ks], bh[0][2 * ks + 1]);
+        mma_acc(d[1], ah[ks], bh[1][2 * ks], bh[1][2 * ks + 1]);
+    }
+}
+template <int KS>
+__device__ __forceinline__ void split_cols(const float (&x)[2][2][KS], uint32_t (&xh)[2][2][KS], uint32_t (&xl)[2][2][KS]) {
+#pragma unroll
+    for (int tl = 0; tl < 2; ++tl)
+#pragma unroll
+        for (int j = 0; j < 2; ++j)
+#pragma unroll
+            for (int nt = 0; nt < KS; ++nt) split_fast(x[tl][j][nt], xh[tl][j][nt], xl[tl][j][nt]);
+}
+template <int KS>
+__device__ __forceinline__ void scores_times_split(float (&d)[KS][4], const uint32_t (&wh)[2][4], const uint32_t (&wl)[2][4],
+                                                   const uint32_t (&xh)[2][2][KS], const uint32_t (&xl)[2][2][KS]) {
+#pragma unroll
+    for (int nt = 0; nt < KS; ++nt) mma_zero(d[nt], wl[0], xh[0][0][nt], xh[0][1][nt]);
+#pragma unroll
+    for (int nt = 0; nt < KS; ++nt) mma_acc(d[nt], wh[0], xl[0][0][nt], xl[0][1][nt]);
+#pragma unroll
+    for (int nt = 0; nt < KS; ++nt) mma_acc(d[nt], wl[1], xh[1][0][nt], xh[1][1][nt]);
+#pragma unroll
+    for (int nt = 0; nt < KS; ++nt) mma_acc(d[nt], wh[1], xl[1][0][nt], xl[1][1][nt]);
+#pragma unroll
+    for (int nt = 0; nt < KS; ++nt) mma_acc(d[nt], wh[0], xh[0][0][nt], xh[0][1][nt]);
+#pragma unroll
+    for (int nt = 0; nt < KS; ++nt) mma_acc(d[nt], wh[1], xh[1][0][nt], xh[1][1][nt]);
 }
 
 // A operand from two score-layout fragments w[tl] (rows g, g+8; columns 2t, 2t+1 of 8-column tile tl).
@@ -148,14 +212,17 @@ __device__ __forceinline__ void scores_times_points(float (&d)[KS][4], const uin
 #pragma unroll
             for (int nt = 0; nt < KS; ++nt) split_fast(x[tl][j][nt], xh[tl][j][nt], xl[tl][j][nt]);
 #pragma unroll
-    for (int nt = 0; nt < KS; ++nt) {
-        mma_zero(d[nt], wl[0], xh[0][0][nt], xh[0][1][nt]);
-        mma_acc(d[nt], wh[0], xl[0][0][nt], xl[0][1][nt]);
-        mma_acc(d[nt], wl[1], xh[1][0][nt], xh[1][1][nt]);
-        mma_acc(d[nt], wh[1], xl[1][0][nt], xl[1][1][nt]);
-        mma_acc(d[nt], wh[0], xh[0][0][nt], xh[0][1][nt]);
-        mma_acc(d[nt], wh[1], xh[1][0][nt], xh[1][1][nt]);
-    }
+    for (int nt = 0; nt < KS; ++nt) mma_zero(d[nt], wl[0], xh[0][0][nt], xh[0][1][nt]);
+#pragma unroll
+    for (int nt = 0; nt < KS; ++nt) mma_acc(d[nt], wh[0], xl[0][0][nt], xl[0][1][nt]);
+#pragma unroll
+    for (int nt = 0; nt < KS; ++nt) mma_acc(d[nt], wl[1], xh[1][0][nt], xh[1][1][nt]);
+#pragma unroll
+    for (int nt = 0; nt < KS; ++nt) mma_acc(d[nt], wh[1], xl[1][0][nt], xl[1][1][nt]);
+#pragma unroll
+    for (int nt = 0; nt < KS; ++nt) mma_acc(d[nt], wh[0], xh[0][0][nt], xh[0][1][nt]);
+#pragma unroll
+    for (int nt = 0; nt < KS; ++nt) mma_acc(d[nt], wh[1], xh[1][0][nt], xh[1][1][nt]);
 }
 
 // ---------------------------------------------------------------------------------------------------------
@@ -171,58 +238,104 @@ struct Stage {
     uint32_t mask[16];   // tile rows that use the column
     float m0[16];        // forward stream: log2 omega of the partner ring; transposed stream: lse of the partner
     float m1[16];        // transposed stream: D of the partner
-    float pad[16];
+    uint32_t all_rows;   // 1 if every column of the chunk is used by all 16 tile rows (no masking needed)
+    uint32_t pad[15];
 };
 
-__device__ __forceinline__ void cp_async16(void* smem_dst, const void* gmem_src) {
-    const uint32_t d = (uint32_t)__cvta_generic_to_shared(smem_dst);
-    asm volatile("cp.async.ca.shared.global [%0], [%1], 16;" ::"r"(d), "l"(gmem_src) : "memory");
+__device__ __forceinline__ void cp_async16(uint32_t smem_dst, const void* gmem_src) {
+    asm volatile("cp.async.ca.shared.global [%0], [%1], 16;" ::"r"(smem_dst), "l"(gmem_src) : "memory");
 }
-__device__ __forceinline__ void cp_async4(void* smem_dst, const void* gmem_src) {
-    const uint32_t d = (uint32_t)__cvta_generic_to_shared(smem_dst);
-    asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(d), "l"(gmem_src) : "memory");
+__device__ __forceinline__ void cp_async4(uint32_t smem_dst, const void* gmem_src) {
+    asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(smem_dst), "l"(gmem_src) : "memory");
 }
 __device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
 template <int N>
 __device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
 
-// Flat index (inside one batch*head slice) of the partner point of stream entry e for a tile whose first point
-// is `first` on a ring of `ring_len` points; consecutive partners are `stride` apart in memory.
-__device__ __forceinline__ int partner_index(const int4& e, int first, int ring_len, int stride) {
-    int u = (int)(short)(e.y & 0xffff);
-    if (e.x >= 0) {   // offset relative to the tile's first point, wrapped around the ring
-        u += first;
-        if (u < 0) u += ring_len;
-        if (u >= ring_len) u -= ring_len;
-        if (u >= ring_len) u -= ring_len;
-    }
-    return (e.x & 0x7fffffff) + u * stride;
-}
-
-// Issue the copies of one chunk: lane l owns stream column l % 16 (entry e).  Rows of both arrays are copied
-// in 16-byte pieces, C/8 pieces per lane and array; metadata is written by the owning lanes.
+// Walks the column stream of one tile with a two-stage software pipeline: chunk c+1 is copied into shared
+// memory while chunk c is consumed by `body(stage)`.  Lane l owns stream column l % 16 (both half-warps compute
+// the same metadata, which keeps the code free of divergent branches).  Rows of the two point arrays are copied
+// in 16-byte pieces, C/8 pieces per lane and array; the pipeline is branch-free: past the end of the stream the
+// last chunk is simply staged again into the idle stage.
 template <int C, bool TRANSPOSED>
-__device__ __forceinline__ void stage_chunk(Stage<C>& st, const int4& e, int lane, int first, int ring_len, int stride,
-                                            const float* a_base, const float* b_base, const float* lse_base, const float* D_base) {
-    const int idx = partner_index(e, first, ring_len, stride);
-    constexpr int PIECES = C / 4;              // 16-byte pieces per row
-#pragma unroll
-    for (int j = 0; j < C / 8; ++j) {
-        const int i = lane + 32 * j;
-        const int row = i / PIECES, piece = i % PIECES;
-        const size_t off = (size_t)__shfl_sync(FULL, idx, row) * C + piece * 4;
-        cp_async16(&st.a[row][piece * 4], a_base + off);
-        cp_async16(&st.b[row][piece * 4], b_base + off);
-    }
-    if (lane < 16) {
-        st.mask[lane] = (uint32_t)e.y >> 16;
-        if (TRANSPOSED) {
-            cp_async4(&st.m0[lane], lse_base + idx);
-            cp_async4(&st.m1[lane], D_base + idx);
-        } else {
-            st.m0[lane] = __int_as_float(e.z);
+struct StreamWalker {
+    static constexpr int PIECES = C / 4;            // 16-byte pieces per point row
+    static constexpr int ROWS_PER_PASS = 32 / PIECES;
+    const int4* ent;          // this lane's entry of chunk 0
+    const float* a_lane;      // array bases advanced to this lane's piece
+    const float* b_lane;
+    const float* lse_base;
+    const float* D_base;
+    uint32_t stage_smem;      // shared address of stage 0
+    Stage<C>* stages;
+    int first, ring_len, stride, lane, row0;
+
+    __device__ __forceinline__ void issue(int slot, const int4& e) const {
+        int u = (int)(short)(e.y & 0xffff);
+        if (e.x >= 0) {   // offset relative to the tile's first point, wrapped around the ring
+            u += first;
+            if (u < 0) u += ring_len;
+            if (u >= ring_len) u -= ring_len;
+            if (u >= ring_len) u -= ring_len;
         }
+        const int idx = (e.x & 0x7fffffff) + u * stride;   // flat index of the partner point in its slice
+        const uint32_t sbase = stage_smem + slot * (uint32_t)sizeof(Stage<C>);
+        const uint32_t dst = sbase + (uint32_t)(row0 * Stage<C>::PITCH + (lane % PIECES) * 4) * 4u;
+#pragma unroll
+        for (int j = 0; j < C / 8; ++j) {
+            const uint32_t off = (uint32_t)__shfl_sync(FULL, idx, row0 + j * ROWS_PER_PASS) * C;   // < 2^32: checked on the host
+            cp_async16(dst + j * ROWS_PER_PASS * Stage<C>::PITCH * 4, a_lane + off);
+            cp_async16(dst + (16 + j * ROWS_PER_PASS) * Stage<C>::PITCH * 4, b_lane + off);
+        }
+        const uint32_t mask = (uint32_t)e.y >> 16;
+        const uint32_t meta = sbase + 2 * 16 * Stage<C>::PITCH * 4 + (lane & 15) * 4;
+        Stage<C>& st = stages[slot];
+        st.mask[lane & 15] = mask;
+        if (TRANSPOSED) {
+            cp_async4(meta + 64, lse_base + idx);
+            cp_async4(meta + 128, D_base + idx);
+        } else {
+            st.m0[lane & 15] = __int_as_float(e.z);
+        }
+        st.all_rows = __all_sync(FULL, mask == 0xffffu) ? 1u : 0u;
     }
+
+    template <typename Body>
+    __device__ __forceinline__ void run(int nchunks, Body&& body) const {
+        if (nchunks <= 0) return;
+        const int last = nchunks - 1;
+        int4 e = __ldg(ent);
+        issue(0, e);
+        cp_async_commit();
+        e = __ldg(ent + 16 * min(1, last));
+        for (int c = 0; c < nchunks; ++c) {
+            issue((c + 1) & 1, e);
+            cp_async_commit();
+            e = __ldg(ent + 16 * min(c + 2, last));
+            cp_async_wait<1>();
+            __syncwarp();
+            body(stages[c & 1]);
+            __syncwarp();   // everyone is done with this stage before the next iteration refills it
+        }
+        cp_async_wait<0>();
+    }
+};
+
+template <int C, bool TRANSPOSED>
+__device__ __forceinline__ StreamWalker<C, TRANSPOSED> make_walker(Stage<C>* stages, const int4* stream, int lane, int first, int ring_len,
+                                                                   int stride, const float* a_base, const float* b_base,
+                                                                   const float* lse_base, const float* D_base) {
+    StreamWalker<C, TRANSPOSED> w;
+    w.ent = stream + (lane & 15);
+    w.a_lane = a_base + (lane % (C / 4)) * 4;
+    w.b_lane = b_base + (lane % (C / 4)) * 4;
+    w.lse_base = lse_base;
+    w.D_base = D_base;
+    w.stages = stages;
+    w.stage_smem = (uint32_t)__cvta_generic_to_shared(stages);
+    w.first = first; w.ring_len = ring_len; w.stride = stride; w.lane = lane;
+    w.row0 = lane / (C / 4);
+    return w;
 }
 
 template <int CPT, int PITCH>
@@ -264,33 +377,11 @@ __device__ __forceinline__ void store_row(float* p, const float (&x)[CPT]) {
     for (int j = 0; j < CPT / 4; ++j) *reinterpret_cast<float4*>(p + 4 * j) = make_float4(x[4 * j], x[4 * j + 1], x[4 * j + 2], x[4 * j + 3]);
 }
 
-// The software pipeline shared by the three kernels: chunk c+1 is copied while chunk c is consumed.
-//   BODY(stage) consumes one staged chunk.
-template <int C, bool TRANSPOSED, typename Body>
-__device__ __forceinline__ void walk_stream(Stage<C>* stages, const int4* stream, int nchunks, int lane, int first, int ring_len,
-                                            int stride, const float* a_base, const float* b_base, const float* lse_base,
-                                            const float* D_base, Body&& body) {
-    if (nchunks <= 0) return;
-    int4 e = __ldg(stream + (lane & 15));
-    stage_chunk<C, TRANSPOSED>(stages[0], e, lane, first, ring_len, stride, a_base, b_base, lse_base, D_base);
-    cp_async_commit();
-    if (nchunks > 1) e = __ldg(stream + 16 + (lane & 15));
-    for (int c = 0; c < nchunks; ++c) {
-        if (c + 1 < nchunks) stage_chunk<C, TRANSPOSED>(stages[(c + 1) & 1], e, lane, first, ring_len, stride, a_base, b_base, lse_base, D_base);
-        cp_async_commit();
-        if (c + 2 < nchunks) e = __ldg(stream + (size_t)(c + 2) * 16 + (lane & 15));
-        cp_async_wait<1>();
-        __syncwarp();
-        body(stages[c & 1]);
-        __syncwarp();   // everyone is done with this stage before the next iteration refills it
-    }
-}
-
 // ---------------------------------------------------------------------------------------------------------
 // forward
 // ---------------------------------------------------------------------------------------------------------
 template <int C>
-__global__ void __launch_bounds__(THREADS)
+__global__ void __launch_bounds__(THREADS, 4)
 forward_mma_kernel(DevPlan p, const float* __restrict__ q, const float* __restrict__ k, const float* __restrict__ v,
                    float* __restrict__ out, float* __restrict__ lse, int N, float scale_log2, int tiles_per_row, long long total_tasks) {
     constexpr int CPT = C / 4, KS = C / 8;
@@ -315,26 +406,32 @@ forward_mma_kernel(DevPlan p, const float* __restrict__ q, const float* __restri
     const int4* stream = p.fwd_stream + (size_t)p.fwd_chunk_ptr[h] * 16;
     const int nchunks = p.fwd_chunk_ptr[h + 1] - p.fwd_chunk_ptr[h];
 
-    walk_stream<C, false>(stages, stream, nchunks, lane, w0, p.nlon_out, p.ps, k + slice, v + slice, nullptr, nullptr, [&](const Stage<C>& st) {
+    make_walker<C, false>(stages, stream, lane, w0, p.nlon_out, p.ps, k + slice, v + slice, nullptr, nullptr).run(nchunks, [&](const Stage<C>& st) {
         float s[2][4];
-#pragma unroll
-        for (int tl = 0; tl < 2; ++tl) {
-            float kr[CPT];
-            lds_row<CPT>(st.a, tl * 8 + g, t, kr);
-            rows_dot_point<CPT>(s[tl], qh, ql, kr);
+        {
+            float kr[2][CPT];
+            lds_row<CPT>(st.a, g, t, kr[0]);
+            lds_row<CPT>(st.a, 8 + g, t, kr[1]);
+            rows_dot_points<CPT>(s, qh, ql, kr);
         }
         float vr[2][2][KS];
 #pragma unroll
         for (int tl = 0; tl < 2; ++tl) {
-            const uint2 mk = *reinterpret_cast<const uint2*>(&st.mask[tl * 8 + 2 * t]);
             const float2 bs = *reinterpret_cast<const float2*>(&st.m0[tl * 8 + 2 * t]);
             lds_col<KS>(st.b, tl * 8 + 2 * t, g, vr[tl][0]);
             lds_col<KS>(st.b, tl * 8 + 2 * t + 1, g, vr[tl][1]);
-            const uint32_t ma = mk.x >> g, mb = mk.y >> g;
-            s[tl][0] = (ma & 1u) ? s[tl][0] + bs.x : -INFINITY;
-            s[tl][1] = (mb & 1u) ? s[tl][1] + bs.y : -INFINITY;
-            s[tl][2] = (ma & 0x100u) ? s[tl][2] + bs.x : -INFINITY;
-            s[tl][3] = (mb & 0x100u) ? s[tl][3] + bs.y : -INFINITY;
+            s[tl][0] += bs.x; s[tl][1] += bs.y; s[tl][2] += bs.x; s[tl][3] += bs.y;
+        }
+        if (!st.all_rows) {   // warp-uniform: some tile row skips some column of this chunk
+#pragma unroll
+            for (int tl = 0; tl < 2; ++tl) {
+                const uint2 mk = *reinterpret_cast<const uint2*>(&st.mask[tl * 8 + 2 * t]);
+                const uint32_t ma = mk.x >> g, mb = mk.y >> g;
+                if (!(ma & 1u)) s[tl][0] = -INFINITY;
+                if (!(mb & 1u)) s[tl][1] = -INFINITY;
+                if (!(ma & 0x100u)) s[tl][2] = -INFINITY;
+                if (!(mb & 0x100u)) s[tl][3] = -INFINITY;
+            }
         }
         // online softmax over the chunk (row maxima across the four threads of a group)
         float mx0 = fmaxf(fmaxf(s[0][0], s[0][1]), fmaxf(s[1][0], s[1][1]));
@@ -392,7 +489,7 @@ forward_mma_kernel(DevPlan p, const float* __restrict__ q, const float* __restri
 // `out` and `dq` may be the same buffer: a warp reads its own 16 rows of `out` before it writes them as dq.
 // ---------------------------------------------------------------------------------------------------------
 template <int C>
-__global__ void __launch_bounds__(THREADS)
+__global__ void __launch_bounds__(THREADS, 3)
 backward_dq_mma_kernel(DevPlan p, const float* __restrict__ q, const float* __restrict__ k, const float* __restrict__ v,
                        const float* __restrict__ dout, const float* out, const float* __restrict__ lse,
                        float* dq, float* __restrict__ Dws, int N, float scale, int tiles_per_row, long long total_tasks) {
@@ -437,15 +534,16 @@ backward_dq_mma_kernel(DevPlan p, const float* __restrict__ q, const float* __re
     const int4* stream = p.fwd_stream + (size_t)p.fwd_chunk_ptr[h] * 16;
     const int nchunks = p.fwd_chunk_ptr[h + 1] - p.fwd_chunk_ptr[h];
 
-    walk_stream<C, false>(stages, stream, nchunks, lane, w0, p.nlon_out, p.ps, k + slice, v + slice, nullptr, nullptr, [&](const Stage<C>& st) {
+    make_walker<C, false>(stages, stream, lane, w0, p.nlon_out, p.ps, k + slice, v + slice, nullptr, nullptr).run(nchunks, [&](const Stage<C>& st) {
         float s[2][4], tt[2][4];
-#pragma unroll
-        for (int tl = 0; tl < 2; ++tl) {
-            float xr[CPT];
-            lds_row<CPT>(st.a, tl * 8 + g, t, xr);
-            rows_dot_point<CPT>(s[tl], qh, ql, xr);
-            lds_row<CPT>(st.b, tl * 8 + g, t, xr);
-            rows_dot_point<CPT>(tt[tl], yh, yl, xr);
+        {
+            float xr[2][CPT];
+            lds_row<CPT>(st.a, g, t, xr[0]);
+            lds_row<CPT>(st.a, 8 + g, t, xr[1]);
+            rows_dot_points<CPT>(s, qh, ql, xr);
+            lds_row<CPT>(st.b, g, t, xr[0]);
+            lds_row<CPT>(st.b, 8 + g, t, xr[1]);
+            rows_dot_points<CPT>(tt, yh, yl, xr);
         }
         float kr[2][2][KS];
 #pragma unroll
@@ -489,7 +587,7 @@ backward_dq_mma_kernel(DevPlan p, const float* __restrict__ q, const float* __re
 // Tile rows are 16 input columns c = ps*(u0+i) + r of one input ring; stream columns are output points.
 // ---------------------------------------------------------------------------------------------------------
 template <int C>
-__global__ void __launch_bounds__(THREADS)
+__global__ void __launch_bounds__(THREADS, 3)
 backward_dkdv_mma_kernel(DevPlan p, const float* __restrict__ q, const float* __restrict__ k, const float* __restrict__ v,
                          const float* __restrict__ dout, const float* __restrict__ lse, const float* __restrict__ Dws,
                          float* __restrict__ dk, float* __restrict__ dv, int N, float scale, int tiles_per_row, long long total_tasks) {
@@ -521,15 +619,16 @@ backward_dkdv_mma_kernel(DevPlan p, const float* __restrict__ q, const float* __
     const int4* stream = p.t_stream + (size_t)p.t_chunk_ptr[srow] * 16;
     const int nchunks = p.t_chunk_ptr[srow + 1] - p.t_chunk_ptr[srow];
 
-    walk_stream<C, true>(stages, stream, nchunks, lane, u0, p.nlon_out, 1, q + oslice * C, dout + oslice * C, lse + oslice, Dws + oslice, [&](const Stage<C>& st) {
+    make_walker<C, true>(stages, stream, lane, u0, p.nlon_out, 1, q + oslice * C, dout + oslice * C, lse + oslice, Dws + oslice).run(nchunks, [&](const Stage<C>& st) {
         float s[2][4], tt[2][4];
-#pragma unroll
-        for (int tl = 0; tl < 2; ++tl) {
-            float xr[CPT];
-            lds_row<CPT>(st.a, tl * 8 + g, t, xr);
-            rows_dot_point<CPT>(s[tl], kh, kl, xr);
-            lds_row<CPT>(st.b, tl * 8 + g, t, xr);
-            rows_dot_point<CPT>(tt[tl], vh, vl, xr);
+        {
+            float xr[2][CPT];
+            lds_row<CPT>(st.a, g, t, xr[0]);
+            lds_row<CPT>(st.a, 8 + g, t, xr[1]);
+            rows_dot_points<CPT>(s, kh, kl, xr);
+            lds_row<CPT>(st.b, g, t, xr[0]);
+            lds_row<CPT>(st.b, 8 + g, t, xr[1]);
+            rows_dot_points<CPT>(tt, vh, vl, xr);
         }
         float qr[2][2][KS], yr[2][2][KS];
         float pr[2][4];
@@ -604,7 +703,8 @@ cudaError_t dispatch_c(int C, F&& f) {
 }  // namespace
 
 bool mma_path_supported(const DevPlan& p, int C) {
-    return p.fwd_stream != nullptr && (C == 16 || C == 32 || C == 64) && p.nlon_out >= 32 && p.nlon_out < 32768;
+    return p.fwd_stream != nullptr && (C == 16 || C == 32 || C == 64) && p.nlon_out >= 32 && p.nlon_out < 32768 &&
+           (long long)p.nlat_in * p.nlon_in * C < (1LL << 32) && (long long)p.nlat_out * p.nlon_out * C < (1LL << 32);
 }
 
 cudaError_t launch_forward_mma(const DevPlan& p, const float* q, const float* k, const float* v, float* out, float* lse,

@@ -11,7 +11,9 @@
 #include "sna_plan.hpp"
 
 #include <algorithm>
+#include <climits>
 #include <cmath>
+#include <cstdint>
 
 namespace sna {
 namespace {
