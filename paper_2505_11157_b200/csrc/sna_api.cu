@@ -128,9 +128,21 @@ static sna_status_t plan_create(int nlat_in, int nlon_in, int nlat_out, int nlon
     for (int h = 0; h < hp.nlat_in; ++h) log2_omega[h] = (float)std::log2(hp.omega[h]);
 
     sna::Stream fwd_stream, t_stream;
+    std::vector<int32_t> grp_order, t_grp_order;
     try {
         sna::build_forward_stream(hp, fwd_stream);
         sna::build_transposed_stream(hp, t_stream);
+        // heavy-first orders of the ring groups (by stream length; for the transposed stream summed over residues)
+        grp_order.resize(fwd_stream.chunk_ptr.size() - 1);
+        std::iota(grp_order.begin(), grp_order.end(), 0);
+        std::stable_sort(grp_order.begin(), grp_order.end(), [&](int a, int b) {
+            return fwd_stream.chunk_ptr[a + 1] - fwd_stream.chunk_ptr[a] > fwd_stream.chunk_ptr[b + 1] - fwd_stream.chunk_ptr[b];
+        });
+        t_grp_order.resize((t_stream.chunk_ptr.size() - 1) / hp.ps);
+        std::iota(t_grp_order.begin(), t_grp_order.end(), 0);
+        std::stable_sort(t_grp_order.begin(), t_grp_order.end(), [&](int a, int b) {
+            return t_stream.chunk_ptr[(a + 1) * hp.ps] - t_stream.chunk_ptr[a * hp.ps] > t_stream.chunk_ptr[(b + 1) * hp.ps] - t_stream.chunk_ptr[b * hp.ps];
+        });
     } catch (const std::bad_alloc&) {
         delete plan;
         set_error("out of host memory while building the column streams");
@@ -145,7 +157,8 @@ static sna_status_t plan_create(int nlat_in, int nlon_in, int nlat_out, int nlon
         {row_order.data(), row_order.size() * 4, 0}, {hp.t_row_ptr.data(), hp.t_row_ptr.size() * 4, 0}, {t_lat.data(), t_lat.size() * 4, 0},
         {t_m.data(), t_m.size() * 4, 0}, {t_row_order.data(), t_row_order.size() * 4, 0}, {log2_omega.data(), log2_omega.size() * 4, 0},
         {fwd_stream.entries.data(), fwd_stream.entries.size() * 16, 0}, {fwd_stream.chunk_ptr.data(), fwd_stream.chunk_ptr.size() * 4, 0},
-        {t_stream.entries.data(), t_stream.entries.size() * 16, 0}, {t_stream.chunk_ptr.data(), t_stream.chunk_ptr.size() * 4, 0}};
+        {t_stream.entries.data(), t_stream.entries.size() * 16, 0}, {t_stream.chunk_ptr.data(), t_stream.chunk_ptr.size() * 4, 0},
+        {grp_order.data(), grp_order.size() * 4, 0}, {t_grp_order.data(), t_grp_order.size() * 4, 0}};
     size_t total = 0;
     for (Piece& p : pieces) { p.offset = total; total += round256(p.bytes); }
     cudaError_t e = cudaGetDevice(&plan->device);
@@ -164,6 +177,7 @@ static sna_status_t plan_create(int nlat_in, int nlon_in, int nlat_out, int nlon
     d.log2_omega = (const float*)at(8);
     d.fwd_stream = (const int4*)at(9); d.fwd_chunk_ptr = at(10);
     d.t_stream = (const int4*)at(11); d.t_chunk_ptr = at(12);
+    d.grp_order = at(13); d.t_grp_order = at(14);
     *plan_out = plan;
     return SNA_OK;
 }

@@ -21,9 +21,11 @@ struct DevPlan {
     const float* log2_omega;    // [nlat_in] log2 of the per-point quadrature weight
     // column streams of the tensor-core kernels (see sna_plan.hpp); null if not built
     const int4* fwd_stream;         // 16 entries per chunk: {base|abs flag, e | mask<<16, bias, aux}
-    const int32_t* fwd_chunk_ptr;   // [nlat_out+1]
+    const int32_t* fwd_chunk_ptr;   // [groups of output latitudes + 1]
+    const int32_t* grp_order;       // groups of output latitudes, longest stream first
     const int4* t_stream;
-    const int32_t* t_chunk_ptr;     // [nlat_in*ps+1]
+    const int32_t* t_chunk_ptr;     // [groups of input latitudes * ps + 1]
+    const int32_t* t_grp_order;     // groups of input latitudes, longest stream first
 };
 
 // Tensor-core kernels (C = 16, 32 or 64, nlon_out >= 32); same contracts as the generic launchers.

@@ -27,6 +27,8 @@ namespace sna {
 namespace {
 
 constexpr int WARPS = 4;
+constexpr int TILE_LON = 8;   // a tile is 8 consecutive longitudes on each of 2 adjacent rings (must match the planner)
+constexpr int TILE_LAT = 2;
 constexpr int THREADS = WARPS * 32;
 constexpr float LOG2E = 1.4426950408889634f;
 constexpr float LN2 = 0.6931471805599453f;
@@ -390,21 +392,24 @@ forward_mma_kernel(DevPlan p, const float* __restrict__ q, const float* __restri
     const int lane = threadIdx.x & 31, g = lane >> 2, t = lane & 3;
     int n, rank, tile;
     if (!decode_task(N, tiles_per_row, total_tasks, n, rank, tile)) return;
-    const int h = p.row_order[rank];
-    const int w0 = tile * 16;
-    const int r0 = min(w0 + g, p.nlon_out - 1), r1 = min(w0 + g + 8, p.nlon_out - 1);   // clamped tile rows
-    const size_t orow = (size_t)(n * p.nlat_out + h) * p.nlon_out;
+    // tile rows g and g+8 of this thread: the same longitude on the two rings of the group
+    const int hg = p.grp_order[rank];
+    const int w0 = tile * TILE_LON;
+    const bool ok0 = w0 + g < p.nlon_out, ok1 = ok0 && hg * TILE_LAT + 1 < p.nlat_out;
+    const int wq = min(w0 + g, p.nlon_out - 1);
+    const size_t pt0 = (size_t)(n * p.nlat_out + hg * TILE_LAT) * p.nlon_out + wq;
+    const size_t pt1 = (size_t)(n * p.nlat_out + min(hg * TILE_LAT + 1, p.nlat_out - 1)) * p.nlon_out + wq;
 
     uint32_t qh[KS][4], ql[KS][4];   // q in the log2 domain
-    make_a_operand<CPT>(q + (orow + r0) * C + t * CPT, q + (orow + r1) * C + t * CPT, scale_log2, qh, ql);
+    make_a_operand<CPT>(q + pt0 * C + t * CPT, q + pt1 * C + t * CPT, scale_log2, qh, ql);
     float o[KS][4];
 #pragma unroll
     for (int nt = 0; nt < KS; ++nt) o[nt][0] = o[nt][1] = o[nt][2] = o[nt][3] = 0.f;
     float m0 = -INFINITY, m1 = -INFINITY, l0 = 0.f, l1 = 0.f;
 
     const size_t slice = (size_t)n * p.nlat_in * p.nlon_in * C;
-    const int4* stream = p.fwd_stream + (size_t)p.fwd_chunk_ptr[h] * 16;
-    const int nchunks = p.fwd_chunk_ptr[h + 1] - p.fwd_chunk_ptr[h];
+    const int4* stream = p.fwd_stream + (size_t)p.fwd_chunk_ptr[hg] * 16;
+    const int nchunks = p.fwd_chunk_ptr[hg + 1] - p.fwd_chunk_ptr[hg];
 
     make_walker<C, false>(stages, stream, lane, w0, p.nlon_out, p.ps, k + slice, v + slice, nullptr, nullptr).run(nchunks, [&](const Stage<C>& st) {
         float s[2][4];
@@ -475,12 +480,12 @@ forward_mma_kernel(DevPlan p, const float* __restrict__ q, const float* __restri
             r0v[nt] = o[nt][0] * inv0; r0v[KS + nt] = o[nt][1] * inv0;
             r1v[nt] = o[nt][2] * inv1; r1v[KS + nt] = o[nt][3] * inv1;
         }
-        if (w0 + g < p.nlon_out) store_row<CPT>(out + (orow + w0 + g) * C + t * CPT, r0v);
-        if (w0 + g + 8 < p.nlon_out) store_row<CPT>(out + (orow + w0 + g + 8) * C + t * CPT, r1v);
+        if (ok0) store_row<CPT>(out + pt0 * C + t * CPT, r0v);
+        if (ok1) store_row<CPT>(out + pt1 * C + t * CPT, r1v);
     }
     if (lse != nullptr && t == 0) {
-        if (w0 + g < p.nlon_out) lse[orow + w0 + g] = (m0 + log2f(l0)) * LN2;
-        if (w0 + g + 8 < p.nlon_out) lse[orow + w0 + g + 8] = (m1 + log2f(l1)) * LN2;
+        if (ok0) lse[pt0] = (m0 + log2f(l0)) * LN2;
+        if (ok1) lse[pt1] = (m1 + log2f(l1)) * LN2;
     }
 }
 
@@ -499,40 +504,42 @@ backward_dq_mma_kernel(DevPlan p, const float* __restrict__ q, const float* __re
     const int lane = threadIdx.x & 31, g = lane >> 2, t = lane & 3;
     int n, rank, tile;
     if (!decode_task(N, tiles_per_row, total_tasks, n, rank, tile)) return;
-    const int h = p.row_order[rank];
-    const int w0 = tile * 16;
-    const int r0 = min(w0 + g, p.nlon_out - 1), r1 = min(w0 + g + 8, p.nlon_out - 1);
-    const size_t orow = (size_t)(n * p.nlat_out + h) * p.nlon_out;
+    const int hg = p.grp_order[rank];
+    const int w0 = tile * TILE_LON;
+    const bool ok0 = w0 + g < p.nlon_out, ok1 = ok0 && hg * TILE_LAT + 1 < p.nlat_out;
+    const int wq = min(w0 + g, p.nlon_out - 1);
+    const size_t pt0 = (size_t)(n * p.nlat_out + hg * TILE_LAT) * p.nlon_out + wq;
+    const size_t pt1 = (size_t)(n * p.nlat_out + min(hg * TILE_LAT + 1, p.nlat_out - 1)) * p.nlon_out + wq;
     const float scale_log2 = scale * LOG2E;
 
     uint32_t qh[KS][4], ql[KS][4], yh[KS][4], yl[KS][4];
-    make_a_operand<CPT>(q + (orow + r0) * C + t * CPT, q + (orow + r1) * C + t * CPT, scale_log2, qh, ql);
-    make_a_operand<CPT>(dout + (orow + r0) * C + t * CPT, dout + (orow + r1) * C + t * CPT, 1.f, yh, yl);
+    make_a_operand<CPT>(q + pt0 * C + t * CPT, q + pt1 * C + t * CPT, scale_log2, qh, ql);
+    make_a_operand<CPT>(dout + pt0 * C + t * CPT, dout + pt1 * C + t * CPT, 1.f, yh, yl);
     // D of the two tile rows
     float D0 = 0.f, D1 = 0.f;
     {
         float a[CPT], b[CPT], ya[CPT], yb[CPT];
-        load_row<CPT>(out + (orow + r0) * C + t * CPT, a);
-        load_row<CPT>(out + (orow + r1) * C + t * CPT, b);
-        load_row<CPT>(dout + (orow + r0) * C + t * CPT, ya);
-        load_row<CPT>(dout + (orow + r1) * C + t * CPT, yb);
+        load_row<CPT>(out + pt0 * C + t * CPT, a);
+        load_row<CPT>(out + pt1 * C + t * CPT, b);
+        load_row<CPT>(dout + pt0 * C + t * CPT, ya);
+        load_row<CPT>(dout + pt1 * C + t * CPT, yb);
 #pragma unroll
         for (int j = 0; j < CPT; ++j) { D0 = fmaf(a[j], ya[j], D0); D1 = fmaf(b[j], yb[j], D1); }
         D0 += __shfl_xor_sync(FULL, D0, 1); D1 += __shfl_xor_sync(FULL, D1, 1);
         D0 += __shfl_xor_sync(FULL, D0, 2); D1 += __shfl_xor_sync(FULL, D1, 2);
         if (t == 0) {
-            if (w0 + g < p.nlon_out) Dws[orow + w0 + g] = D0;
-            if (w0 + g + 8 < p.nlon_out) Dws[orow + w0 + g + 8] = D1;
+            if (ok0) Dws[pt0] = D0;
+            if (ok1) Dws[pt1] = D1;
         }
     }
-    const float nl0 = -lse[orow + r0] * LOG2E, nl1 = -lse[orow + r1] * LOG2E;
+    const float nl0 = -lse[pt0] * LOG2E, nl1 = -lse[pt1] * LOG2E;
     float acc[KS][4];
 #pragma unroll
     for (int nt = 0; nt < KS; ++nt) acc[nt][0] = acc[nt][1] = acc[nt][2] = acc[nt][3] = 0.f;
 
     const size_t slice = (size_t)n * p.nlat_in * p.nlon_in * C;
-    const int4* stream = p.fwd_stream + (size_t)p.fwd_chunk_ptr[h] * 16;
-    const int nchunks = p.fwd_chunk_ptr[h + 1] - p.fwd_chunk_ptr[h];
+    const int4* stream = p.fwd_stream + (size_t)p.fwd_chunk_ptr[hg] * 16;
+    const int nchunks = p.fwd_chunk_ptr[hg + 1] - p.fwd_chunk_ptr[hg];
 
     make_walker<C, false>(stages, stream, lane, w0, p.nlon_out, p.ps, k + slice, v + slice, nullptr, nullptr).run(nchunks, [&](const Stage<C>& st) {
         float s[2][4], tt[2][4];
@@ -577,14 +584,15 @@ backward_dq_mma_kernel(DevPlan p, const float* __restrict__ q, const float* __re
         r0v[nt] = acc[nt][0] * scale; r0v[KS + nt] = acc[nt][1] * scale;
         r1v[nt] = acc[nt][2] * scale; r1v[KS + nt] = acc[nt][3] * scale;
     }
-    if (w0 + g < p.nlon_out) store_row<CPT>(dq + (orow + w0 + g) * C + t * CPT, r0v);
-    if (w0 + g + 8 < p.nlon_out) store_row<CPT>(dq + (orow + w0 + g + 8) * C + t * CPT, r1v);
+    if (ok0) store_row<CPT>(dq + pt0 * C + t * CPT, r0v);
+    if (ok1) store_row<CPT>(dq + pt1 * C + t * CPT, r1v);
 }
 
 // ---------------------------------------------------------------------------------------------------------
 // backward, dk and dv, gathered per input point over the transposed stream (no atomics):
 //   dk_j = scale * sum_i p_ij (t_ij - D_i) q_i,   dv_j = sum_i p_ij dout_i          (App. B.4)
-// Tile rows are 16 input columns c = ps*(u0+i) + r of one input ring; stream columns are output points.
+// Tile rows are the input columns c = ps*(u0+i) + r, i < 8, of the two rings of an input ring group; stream
+// columns are output points.
 // ---------------------------------------------------------------------------------------------------------
 template <int C>
 __global__ void __launch_bounds__(THREADS, 3)
@@ -597,17 +605,20 @@ backward_dkdv_mma_kernel(DevPlan p, const float* __restrict__ q, const float* __
     const int lane = threadIdx.x & 31, g = lane >> 2, t = lane & 3;
     int n, rank, tile;
     if (!decode_task(N, tiles_per_row * p.ps, total_tasks, n, rank, tile)) return;
-    const int hp = p.t_row_order[rank];
+    const int hg = p.t_grp_order[rank];
     const int r = tile % p.ps;
-    const int u0 = (tile / p.ps) * 16;
-    const int i0 = min(u0 + g, p.nlon_out - 1), i1 = min(u0 + g + 8, p.nlon_out - 1);   // clamped tile rows (units of ps columns)
-    const size_t irow = (size_t)(n * p.nlat_in + hp) * p.nlon_in + r;
+    const int u0 = (tile / p.ps) * TILE_LON;
+    const bool ok0 = u0 + g < p.nlon_out, ok1 = ok0 && hg * TILE_LAT + 1 < p.nlat_in;
+    const int uq = min(u0 + g, p.nlon_out - 1);   // tile row position in units of ps columns
+    const int hp0 = hg * TILE_LAT, hp1 = min(hg * TILE_LAT + 1, p.nlat_in - 1);
+    const size_t pt0 = (size_t)(n * p.nlat_in + hp0) * p.nlon_in + (size_t)uq * p.ps + r;
+    const size_t pt1 = (size_t)(n * p.nlat_in + hp1) * p.nlon_in + (size_t)uq * p.ps + r;
     const float scale_log2 = scale * LOG2E;
 
     uint32_t kh[KS][4], kl[KS][4], vh[KS][4], vl[KS][4];
-    make_a_operand<CPT>(k + (irow + (size_t)i0 * p.ps) * C + t * CPT, k + (irow + (size_t)i1 * p.ps) * C + t * CPT, scale_log2, kh, kl);
-    make_a_operand<CPT>(v + (irow + (size_t)i0 * p.ps) * C + t * CPT, v + (irow + (size_t)i1 * p.ps) * C + t * CPT, 1.f, vh, vl);
-    const float bias = p.log2_omega[hp];
+    make_a_operand<CPT>(k + pt0 * C + t * CPT, k + pt1 * C + t * CPT, scale_log2, kh, kl);
+    make_a_operand<CPT>(v + pt0 * C + t * CPT, v + pt1 * C + t * CPT, 1.f, vh, vl);
+    const float bias0 = p.log2_omega[hp0], bias1 = p.log2_omega[hp1];
     float gk[KS][4], gv[KS][4];
 #pragma unroll
     for (int nt = 0; nt < KS; ++nt) {
@@ -615,7 +626,7 @@ backward_dkdv_mma_kernel(DevPlan p, const float* __restrict__ q, const float* __
         gv[nt][0] = gv[nt][1] = gv[nt][2] = gv[nt][3] = 0.f;
     }
     const size_t oslice = (size_t)n * p.nlat_out * p.nlon_out;
-    const int srow = hp * p.ps + r;
+    const int srow = hg * p.ps + r;
     const int4* stream = p.t_stream + (size_t)p.t_chunk_ptr[srow] * 16;
     const int nchunks = p.t_chunk_ptr[srow + 1] - p.t_chunk_ptr[srow];
 
@@ -641,12 +652,12 @@ backward_dkdv_mma_kernel(DevPlan p, const float* __restrict__ q, const float* __
             lds_col<KS>(st.a, tl * 8 + 2 * t + 1, g, qr[tl][1]);
             lds_col<KS>(st.b, tl * 8 + 2 * t, g, yr[tl][0]);
             lds_col<KS>(st.b, tl * 8 + 2 * t + 1, g, yr[tl][1]);
-            const float nla = fmaf(-ls.x, LOG2E, bias), nlb = fmaf(-ls.y, LOG2E, bias);   // -lse_i (log2) + log2 omega_j
+            const float nla = -ls.x * LOG2E, nlb = -ls.y * LOG2E;   // -lse_i in the log2 domain
             const uint32_t ma = mk.x >> g, mb = mk.y >> g;
-            pr[tl][0] = (ma & 1u) ? ex2(s[tl][0] + nla) : 0.f;
-            pr[tl][1] = (mb & 1u) ? ex2(s[tl][1] + nlb) : 0.f;
-            pr[tl][2] = (ma & 0x100u) ? ex2(s[tl][2] + nla) : 0.f;
-            pr[tl][3] = (mb & 0x100u) ? ex2(s[tl][3] + nlb) : 0.f;
+            pr[tl][0] = (ma & 1u) ? ex2(s[tl][0] + nla + bias0) : 0.f;   // bias: log2 omega_j of the row's ring
+            pr[tl][1] = (mb & 1u) ? ex2(s[tl][1] + nlb + bias0) : 0.f;
+            pr[tl][2] = (ma & 0x100u) ? ex2(s[tl][2] + nla + bias1) : 0.f;
+            pr[tl][3] = (mb & 0x100u) ? ex2(s[tl][3] + nlb + bias1) : 0.f;
             s[tl][0] = pr[tl][0] * (tt[tl][0] - Dd.x);   // ds
             s[tl][1] = pr[tl][1] * (tt[tl][1] - Dd.y);
             s[tl][2] = pr[tl][2] * (tt[tl][2] - Dd.x);
@@ -670,13 +681,13 @@ backward_dkdv_mma_kernel(DevPlan p, const float* __restrict__ q, const float* __
         a0[nt] = gk[nt][0] * scale; a0[KS + nt] = gk[nt][1] * scale; a1[nt] = gk[nt][2] * scale; a1[KS + nt] = gk[nt][3] * scale;
         b0[nt] = gv[nt][0]; b0[KS + nt] = gv[nt][1]; b1[nt] = gv[nt][2]; b1[KS + nt] = gv[nt][3];
     }
-    if (u0 + g < p.nlon_out) {
-        store_row<CPT>(dk + (irow + (size_t)(u0 + g) * p.ps) * C + t * CPT, a0);
-        store_row<CPT>(dv + (irow + (size_t)(u0 + g) * p.ps) * C + t * CPT, b0);
+    if (ok0) {
+        store_row<CPT>(dk + pt0 * C + t * CPT, a0);
+        store_row<CPT>(dv + pt0 * C + t * CPT, b0);
     }
-    if (u0 + g + 8 < p.nlon_out) {
-        store_row<CPT>(dk + (irow + (size_t)(u0 + g + 8) * p.ps) * C + t * CPT, a1);
-        store_row<CPT>(dv + (irow + (size_t)(u0 + g + 8) * p.ps) * C + t * CPT, b1);
+    if (ok1) {
+        store_row<CPT>(dk + pt1 * C + t * CPT, a1);
+        store_row<CPT>(dv + pt1 * C + t * CPT, b1);
     }
 }
 
@@ -710,8 +721,8 @@ bool mma_path_supported(const DevPlan& p, int C) {
 cudaError_t launch_forward_mma(const DevPlan& p, const float* q, const float* k, const float* v, float* out, float* lse,
                                int N, int C, cudaStream_t stream) {
     const float scale_log2 = LOG2E / sqrtf((float)C);
-    const int tiles = (p.nlon_out + 15) / 16;
-    const long long tasks = (long long)tiles * p.nlat_out * N;
+    const int tiles = (p.nlon_out + TILE_LON - 1) / TILE_LON;
+    const long long tasks = (long long)tiles * ((p.nlat_out + TILE_LAT - 1) / TILE_LAT) * N;
     const long long blocks = (tasks + WARPS - 1) / WARPS;
     if (blocks > 0x7fffffffLL) return cudaErrorInvalidValue;
     return dispatch_c(C, [&](auto c) {
@@ -726,8 +737,8 @@ cudaError_t launch_forward_mma(const DevPlan& p, const float* q, const float* k,
 cudaError_t launch_backward_dq_mma(const DevPlan& p, const float* q, const float* k, const float* v, const float* dout,
                                    const float* out, const float* lse, float* dq, float* Dws, int N, int C, cudaStream_t stream) {
     const float scale = 1.0f / sqrtf((float)C);
-    const int tiles = (p.nlon_out + 15) / 16;
-    const long long tasks = (long long)tiles * p.nlat_out * N;
+    const int tiles = (p.nlon_out + TILE_LON - 1) / TILE_LON;
+    const long long tasks = (long long)tiles * ((p.nlat_out + TILE_LAT - 1) / TILE_LAT) * N;
     const long long blocks = (tasks + WARPS - 1) / WARPS;
     if (blocks > 0x7fffffffLL) return cudaErrorInvalidValue;
     return dispatch_c(C, [&](auto c) {
@@ -742,8 +753,8 @@ cudaError_t launch_backward_dq_mma(const DevPlan& p, const float* q, const float
 cudaError_t launch_backward_dkdv_mma(const DevPlan& p, const float* q, const float* k, const float* v, const float* dout,
                                      const float* lse, const float* Dws, float* dk, float* dv, int N, int C, cudaStream_t stream) {
     const float scale = 1.0f / sqrtf((float)C);
-    const int tiles = (p.nlon_out + 15) / 16;
-    const long long tasks = (long long)tiles * p.ps * p.nlat_in * N;
+    const int tiles = (p.nlon_out + TILE_LON - 1) / TILE_LON;
+    const long long tasks = (long long)tiles * p.ps * ((p.nlat_in + TILE_LAT - 1) / TILE_LAT) * N;
     const long long blocks = (tasks + WARPS - 1) / WARPS;
     if (blocks > 0x7fffffffLL) return cudaErrorInvalidValue;
     return dispatch_c(C, [&](auto c) {

@@ -192,21 +192,36 @@ namespace {
 inline int floor_div(int a, int b) { int q = a / b; return ((a % b != 0) && ((a < 0) != (b < 0))) ? q - 1 : q; }
 inline int ceil_div(int a, int b) { return -floor_div(-a, b); }
 
-// Appends the columns of one window (offsets e_lo..e_hi) or of a whole ring (count partners, absolute index).
-void append_window(std::vector<StreamEntry>& v, int32_t base, float bias, int32_t aux, bool whole, int e_lo, int e_hi, int count) {
-    if (whole) {
-        for (int u = 0; u < count; ++u)
-            v.push_back(StreamEntry{(int32_t)(base | (int32_t)0x80000000), (int32_t)((u & 0xffff) | (0xffff << 16)), bias, aux});
-        return;
+// One partner ring as seen from the rings of a group: per group ring either absent, a band of offsets, or whole.
+struct GroupRange {
+    bool present = false, whole = false;
+    int lo = 0, hi = -1;
+};
+
+// Appends the columns of one partner ring / residue for a ring group.
+void append_group_columns(std::vector<StreamEntry>& v, int32_t base, float bias, const GroupRange (&rg)[TILE_LAT], int whole_count) {
+    uint32_t whole_rows = 0, band_rows_any = 0;
+    for (int k = 0; k < TILE_LAT; ++k) {
+        if (rg[k].present && rg[k].whole) whole_rows |= ((1u << TILE_LON) - 1u) << (k * TILE_LON);
+        if (rg[k].present && !rg[k].whole && rg[k].hi >= rg[k].lo) band_rows_any |= 1u << k;
     }
-    const int E = e_hi - e_lo + 1;
-    if (E <= 0) return;
-    for (int x = 0; x < 15 + E; ++x) {
+    if (whole_rows) {   // absolute partner index: every partner of the ring, for the rings that take it whole
+        for (int u = 0; u < whole_count; ++u)
+            v.push_back(StreamEntry{(int32_t)(base | (int32_t)0x80000000), (int32_t)((u & 0xffff) | (whole_rows << 16)), bias, 0});
+    }
+    if (!band_rows_any) return;
+    int lo = INT32_MAX, hi = INT32_MIN;
+    for (int k = 0; k < TILE_LAT; ++k)
+        if (band_rows_any & (1u << k)) { lo = std::min(lo, rg[k].lo); hi = std::max(hi, rg[k].hi); }
+    for (int x = 0; x < TILE_LON - 1 + (hi - lo + 1); ++x) {
+        const int e_rel = lo + x;
         uint32_t mask = 0;
-        for (int i = 0; i < 16; ++i)
-            if (x - i >= 0 && x - i <= E - 1) mask |= 1u << i;
-        const int e_rel = e_lo + x;
-        v.push_back(StreamEntry{base, (int32_t)(((uint32_t)e_rel & 0xffffu) | (mask << 16)), bias, aux});
+        for (int k = 0; k < TILE_LAT; ++k) {
+            if (!(band_rows_any & (1u << k))) continue;
+            for (int i = 0; i < TILE_LON; ++i)
+                if (e_rel - i >= rg[k].lo && e_rel - i <= rg[k].hi) mask |= 1u << (k * TILE_LON + i);
+        }
+        if (mask) v.push_back(StreamEntry{base, (int32_t)(((uint32_t)e_rel & 0xffffu) | (mask << 16)), bias, 0});
     }
 }
 
@@ -218,43 +233,74 @@ void pad_row(std::vector<StreamEntry>& v, size_t row_start) {
     }
 }
 
+// Merges the window lists of the rings of a group (each sorted by partner ring) and calls
+// emit(partner_ring, m[TILE_LAT]) with m = -2 for "not in this ring's list".
+template <typename Emit>
+void merge_group(const std::vector<int32_t>& ptr, const std::vector<RingWindow>& win, int first_ring, int nrings, Emit&& emit) {
+    int pos[TILE_LAT], end[TILE_LAT];
+    for (int k = 0; k < TILE_LAT; ++k) {
+        const int ring = first_ring + k;
+        pos[k] = ring < nrings ? ptr[ring] : 0;
+        end[k] = ring < nrings ? ptr[ring + 1] : 0;
+    }
+    for (;;) {
+        int lat = INT32_MAX;
+        for (int k = 0; k < TILE_LAT; ++k)
+            if (pos[k] < end[k]) lat = std::min(lat, win[pos[k]].lat);
+        if (lat == INT32_MAX) break;
+        int m[TILE_LAT];
+        for (int k = 0; k < TILE_LAT; ++k) m[k] = (pos[k] < end[k] && win[pos[k]].lat == lat) ? win[pos[k]++].m : -2;
+        emit(lat, m);
+    }
+}
+
 }  // namespace
 
 void build_forward_stream(const HostPlan& P, Stream& S) {
-    S.chunk_ptr.assign(P.nlat_out + 1, 0);
+    const int groups = (P.nlat_out + TILE_LAT - 1) / TILE_LAT;
+    S.chunk_ptr.assign(groups + 1, 0);
     S.entries.clear();
-    for (int h = 0; h < P.nlat_out; ++h) {
+    for (int gi = 0; gi < groups; ++gi) {
         const size_t start = S.entries.size();
-        for (int e = P.row_ptr[h]; e < P.row_ptr[h + 1]; ++e) {
-            const RingWindow& w = P.windows[e];
-            const float bias = (float)std::log2(P.omega[w.lat]);
+        merge_group(P.row_ptr, P.windows, gi * TILE_LAT, P.nlat_out, [&](int lat, const int (&m)[TILE_LAT]) {
+            const float bias = (float)std::log2(P.omega[lat]);
             for (int r = 0; r < P.ps; ++r) {
-                const int32_t base = w.lat * P.nlon_in + r;
-                if (w.m < 0) append_window(S.entries, base, bias, 0, true, 0, 0, P.nlon_out);
-                else append_window(S.entries, base, bias, 0, false, ceil_div(-w.m - r, P.ps), floor_div(w.m - r, P.ps), 0);
+                GroupRange rg[TILE_LAT];
+                for (int k = 0; k < TILE_LAT; ++k) {
+                    if (m[k] == -2) continue;
+                    rg[k].present = true;
+                    if (m[k] < 0) rg[k].whole = true;
+                    else { rg[k].lo = ceil_div(-m[k] - r, P.ps); rg[k].hi = floor_div(m[k] - r, P.ps); }
+                }
+                append_group_columns(S.entries, lat * P.nlon_in + r, bias, rg, P.nlon_out);
             }
-        }
+        });
         pad_row(S.entries, start);
-        S.chunk_ptr[h + 1] = (int32_t)(S.entries.size() / 16);
+        S.chunk_ptr[gi + 1] = (int32_t)(S.entries.size() / 16);
     }
 }
 
 void build_transposed_stream(const HostPlan& P, Stream& S) {
-    // Row (h', r): tile rows are input columns c = ps*u + r, u = u0 + i.  Output point (h, w) is a partner iff
-    // c - w*ps in [-m, m]  <=>  w - u in [ceil((r - m)/ps), floor((r + m)/ps)].
-    S.chunk_ptr.assign((size_t)P.nlat_in * P.ps + 1, 0);
+    // Row (group of input rings, r): tile rows are input columns c = ps*u + r.  Output point (h, w) is a partner of
+    // column u of input ring h' iff c - w*ps in [-m, m]  <=>  w - u in [ceil((r - m)/ps), floor((r + m)/ps)].
+    const int groups = (P.nlat_in + TILE_LAT - 1) / TILE_LAT;
+    S.chunk_ptr.assign((size_t)groups * P.ps + 1, 0);
     S.entries.clear();
-    for (int hp = 0; hp < P.nlat_in; ++hp) {
+    for (int gi = 0; gi < groups; ++gi) {
         for (int r = 0; r < P.ps; ++r) {
             const size_t start = S.entries.size();
-            for (int e = P.t_row_ptr[hp]; e < P.t_row_ptr[hp + 1]; ++e) {
-                const RingWindow& w = P.t_windows[e];
-                const int32_t base = w.lat * P.nlon_out;
-                if (w.m < 0) append_window(S.entries, base, 0.f, w.lat, true, 0, 0, P.nlon_out);
-                else append_window(S.entries, base, 0.f, w.lat, false, ceil_div(r - w.m, P.ps), floor_div(r + w.m, P.ps), 0);
-            }
+            merge_group(P.t_row_ptr, P.t_windows, gi * TILE_LAT, P.nlat_in, [&](int lat, const int (&m)[TILE_LAT]) {
+                GroupRange rg[TILE_LAT];
+                for (int k = 0; k < TILE_LAT; ++k) {
+                    if (m[k] == -2) continue;
+                    rg[k].present = true;
+                    if (m[k] < 0) rg[k].whole = true;
+                    else { rg[k].lo = ceil_div(r - m[k], P.ps); rg[k].hi = floor_div(r + m[k], P.ps); }
+                }
+                append_group_columns(S.entries, lat * P.nlon_out, 0.f, rg, P.nlon_out);
+            });
             pad_row(S.entries, start);
-            S.chunk_ptr[(size_t)hp * P.ps + r + 1] = (int32_t)(S.entries.size() / 16);
+            S.chunk_ptr[(size_t)gi * P.ps + r + 1] = (int32_t)(S.entries.size() / 16);
         }
     }
 }

@@ -33,29 +33,35 @@ struct HostPlan {
     int window_count(const RingWindow& w) const { return w.m < 0 ? nlon_in : 2 * w.m + 1; }
 };
 
-// Column streams for the tensor-core kernels.  A warp owns a tile of 16 consecutive points of one ring
-// ("tile rows" i = 0..15, first point w0) and walks a stream of partner points ("columns"), 16 per step.
-// For a window with offsets e in [e_lo, e_hi] (in units of ps input columns for the forward table, of output
-// columns for the transposed one) the tile needs partners u = w0 + e_rel, e_rel = e_lo .. e_hi + 15, and tile
-// row i uses the column iff e_lo <= e_rel - i <= e_hi: that is the 16-bit row mask.  The stream of a ring row
-// is the concatenation of its windows' columns, padded to a multiple of 16 with mask-0 columns, and is the
-// same for every tile of the row, so it is built once on the host.
+// Column streams for the tensor-core kernels.  A warp owns a tile of 16 points: TILE_LON = 8 consecutive
+// longitudes on each of TILE_LAT = 2 adjacent rings (a "ring group"); tile row i is ring i / 8 of the group,
+// longitude first + i % 8.  Two adjacent rings see almost the same partner points, and 8-wide rows waste fewer
+// columns on the slanted band than 16-wide rows would.  The warp walks a stream of partner points ("columns"),
+// 16 per step.  For a window with offsets e in [e_lo, e_hi] (in units of ps input columns for the forward
+// table, of output columns for the transposed one) a row at longitude first + i uses partner first + e_rel iff
+// e_lo <= e_rel - i <= e_hi: that is the row's bit in the column's 16-bit mask.  The stream of a ring group is
+// the concatenation, over partner rings and residues, of the columns at least one row uses, padded to a
+// multiple of 16 with mask-0 columns; it is the same for every tile of the group, so it is built once on the host.
+constexpr int TILE_LON = 8;
+constexpr int TILE_LAT = 2;
+
 struct StreamEntry {
     int32_t base;      // flat row index of the partner ring plus the residue r; bit 31 set = e is absolute
     int32_t e_mask;    // low 16 bits: e_rel (signed) or the absolute partner index; high 16 bits: row mask
     float bias;        // forward: log2 of the partner ring's quadrature weight; transposed: unused (0)
-    int32_t aux;       // forward: unused; transposed: output ring index h (for lse / D lookups)
+    int32_t aux;       // unused
 };
 
 struct Stream {
-    std::vector<int32_t> chunk_ptr;     // [rows+1] first 16-column chunk of each row
+    std::vector<int32_t> chunk_ptr;     // [rows+1] first 16-column chunk of each stream row
     std::vector<StreamEntry> entries;   // 16 * chunk_ptr.back()
 };
 
-// Forward stream: rows = output latitudes, partners = input points; partner flat index = base + u*ps.
+// Forward stream: one row per group of output latitudes (ceil(nlat_out / TILE_LAT) rows); partners are input
+// points, flat index base + u*ps.
 void build_forward_stream(const HostPlan& plan, Stream& out);
-// Transposed stream for dk/dv: rows = (input latitude, residue r of the input column mod ps), tile rows are
-// input columns c = ps*(u0+i)+r, partners are output points (h, w).
+// Transposed stream for dk/dv: one row per (group of input latitudes, residue r of the input column mod ps);
+// tile rows are input columns c = ps*(first+i%8)+r of the group's rings, partners are output points (h, w).
 void build_transposed_stream(const HostPlan& plan, Stream& out);
 
 // Builds the plan.  On failure returns a status and fills `why`.
