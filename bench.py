@@ -33,6 +33,14 @@ if ROOT not in sys.path:
 
 import numpy as np  # noqa: E402
 
+# dram__bytes_read.sum + dram__bytes_write.sum per launch from the ncu capture summarised in
+# profiles/mma_kernels_c3_counters.md (bench.py cannot run ncu itself)
+NCU_DRAM_BYTES_PER_LAUNCH = {
+    ("c3", "forward"): 797289728 + 64207616,
+    ("c3", "backward_dq"): 967110144 + 65016832,
+    ("c3", "backward_dkdv"): 729955584 + 504659200,
+}
+
 METRIC = "fwd+bwd neighbor-pair-channels per second"
 UNIT = "pair*ch/s"
 FP32_LANES_PER_SM = 128
@@ -254,10 +262,13 @@ def run_ours(args, wl):
         props = torch.cuda.get_device_properties(local_rank)
         sm_max_mhz = (clocks or {}).get("sm_max_mhz") or 1965.0
         peak_tflops = props.multi_processor_count * FP32_LANES_PER_SM * 2 * sm_max_mhz * 1e6 / 1e12
-        kernels = {"forward": (ms_fwd, 4.0), "backward_dq": (ms_dq, 4.0), "backward_dkdv": (ms_dkdv, 6.0)}
+        # algorithmic flops per pair*channel credited to each kernel: forward 4 (s and p.v), dq kernel 6 (s, t, dq),
+        # dk/dv kernel 4 (dk, dv; its recomputation of s and t is not credited) -- 14 in total = 4 forward + 10 backward
+        kernels = {"forward": (ms_fwd, 4.0), "backward_dq": (ms_dq, 6.0), "backward_dkdv": (ms_dkdv, 4.0)}
         dominant = max(kernels, key=lambda n: kernels[n][0])
         dom_ms, dom_flops_per_unit = kernels[dominant]
         achieved = dom_flops_per_unit * units / (dom_ms * 1e-3) / 1e12
+        traffic = NCU_DRAM_BYTES_PER_LAUNCH.get((wl.name, dominant))
         ms_step = ms_total_max / args.steps
         roof_fwd_ms = 4.0 * units / (peak_tflops * 1e12) * 1e3
         roof_bwd_ms = 10.0 * units / (peak_tflops * 1e12) * 1e3
@@ -271,8 +282,10 @@ def run_ours(args, wl):
             "roofline_step": {"bound": "alu", "roofline_ms": roof_fwd_ms + roof_bwd_ms, "frac": (roof_fwd_ms + roof_bwd_ms) / ms_step,
                               "note": "algorithmic flops (4C fwd + 10C bwd per pair) at the FP32 FMA peak of measured-max clock"},
             "roofline": {"bound": "alu", "kernel": dominant, "achieved": achieved, "peak": peak_tflops, "unit": "TFLOP/s",
-                         "frac": achieved / peak_tflops, "traffic": None,
-                         "note": f"{dom_flops_per_unit:g}C flops per pair credited; peak = SMs x 128 lanes x 2 x max SM clock"},
+                         "frac": achieved / peak_tflops, "traffic": traffic,
+                         "note": f"{dom_flops_per_unit:g} flops per pair*channel credited; peak = SMs x 128 FP32 lanes x 2 x max SM clock "
+                                 "(of derived peak; a pure-FMA loop measured 127.7 of 128 FMA/clk/SM); contractions run on tensor cores "
+                                 "as 3xTF32 MMAs; traffic = ncu dram bytes read+written per launch (profiles/)"},
             "e2e": {"value": world * units / (ms_e2e_step_max * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
                     "d2h_bytes_per_step": d2h, "ms_per_step": ms_e2e_step_max},
             "gpu_launches": launches_per_step * args.steps,
