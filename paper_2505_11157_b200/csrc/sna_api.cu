@@ -129,19 +129,22 @@ static sna_status_t plan_create(int nlat_in, int nlon_in, int nlat_out, int nlon
 
     sna::Stream fwd_stream, t_stream;
     std::vector<int32_t> grp_order, t_grp_order;
+    bool t_consecutive = false;
     try {
         sna::build_forward_stream(hp, fwd_stream);
-        sna::build_transposed_stream(hp, t_stream);
+        t_consecutive = sna::build_transposed_stream(hp, t_stream);
         // heavy-first orders of the ring groups (by stream length; for the transposed stream summed over residues)
         grp_order.resize(fwd_stream.chunk_ptr.size() - 1);
         std::iota(grp_order.begin(), grp_order.end(), 0);
         std::stable_sort(grp_order.begin(), grp_order.end(), [&](int a, int b) {
             return fwd_stream.chunk_ptr[a + 1] - fwd_stream.chunk_ptr[a] > fwd_stream.chunk_ptr[b + 1] - fwd_stream.chunk_ptr[b];
         });
-        t_grp_order.resize((t_stream.chunk_ptr.size() - 1) / hp.ps);
+        const int rows_per_group = t_consecutive ? 1 : hp.ps;
+        t_grp_order.resize((t_stream.chunk_ptr.size() - 1) / rows_per_group);
         std::iota(t_grp_order.begin(), t_grp_order.end(), 0);
         std::stable_sort(t_grp_order.begin(), t_grp_order.end(), [&](int a, int b) {
-            return t_stream.chunk_ptr[(a + 1) * hp.ps] - t_stream.chunk_ptr[a * hp.ps] > t_stream.chunk_ptr[(b + 1) * hp.ps] - t_stream.chunk_ptr[b * hp.ps];
+            return t_stream.chunk_ptr[(a + 1) * rows_per_group] - t_stream.chunk_ptr[a * rows_per_group] >
+                   t_stream.chunk_ptr[(b + 1) * rows_per_group] - t_stream.chunk_ptr[b * rows_per_group];
         });
     } catch (const std::bad_alloc&) {
         delete plan;
@@ -178,6 +181,7 @@ static sna_status_t plan_create(int nlat_in, int nlon_in, int nlat_out, int nlon
     d.fwd_stream = (const int4*)at(9); d.fwd_chunk_ptr = at(10);
     d.t_stream = (const int4*)at(11); d.t_chunk_ptr = at(12);
     d.grp_order = at(13); d.t_grp_order = at(14);
+    d.t_consecutive = t_consecutive ? 1 : 0;
     *plan_out = plan;
     return SNA_OK;
 }

@@ -26,6 +26,7 @@ struct DevPlan {
     const int4* t_stream;
     const int32_t* t_chunk_ptr;     // [groups of input latitudes * ps + 1]
     const int32_t* t_grp_order;     // groups of input latitudes, longest stream first
+    int t_consecutive;              // 1: transposed tiles are 8 consecutive input columns; 0: split by residue mod ps
 };
 
 // Tensor-core kernels (C = 16, 32 or 64, nlon_out >= 32); same contracts as the generic launchers.

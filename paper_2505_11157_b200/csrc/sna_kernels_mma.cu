@@ -595,7 +595,7 @@ backward_dq_mma_kernel(DevPlan p, const float* __restrict__ q, const float* __re
 // columns are output points.
 // ---------------------------------------------------------------------------------------------------------
 template <int C>
-__global__ void __launch_bounds__(THREADS, 3)
+__global__ void __launch_bounds__(THREADS, 2)
 backward_dkdv_mma_kernel(DevPlan p, const float* __restrict__ q, const float* __restrict__ k, const float* __restrict__ v,
                          const float* __restrict__ dout, const float* __restrict__ lse, const float* __restrict__ Dws,
                          float* __restrict__ dk, float* __restrict__ dv, int N, float scale, int tiles_per_row, long long total_tasks) {
@@ -604,15 +604,28 @@ backward_dkdv_mma_kernel(DevPlan p, const float* __restrict__ q, const float* __
     Stage<C>* stages = reinterpret_cast<Stage<C>*>(smem_raw) + 2 * (threadIdx.x >> 5);
     const int lane = threadIdx.x & 31, g = lane >> 2, t = lane & 3;
     int n, rank, tile;
-    if (!decode_task(N, tiles_per_row * p.ps, total_tasks, n, rank, tile)) return;
+    if (!decode_task(N, tiles_per_row, total_tasks, n, rank, tile)) return;
     const int hg = p.t_grp_order[rank];
-    const int r = tile % p.ps;
-    const int u0 = (tile / p.ps) * TILE_LON;
-    const bool ok0 = u0 + g < p.nlon_out, ok1 = ok0 && hg * TILE_LAT + 1 < p.nlat_in;
-    const int uq = min(u0 + g, p.nlon_out - 1);   // tile row position in units of ps columns
+    // input column of tile row g (and g+8), the first partner index of the tile, and the tile's stream row
+    int col, first, srow;
+    bool ok0;
+    if (p.t_consecutive) {           // 8 consecutive input columns
+        col = tile * TILE_LON + g;
+        ok0 = col < p.nlon_in;
+        first = tile * TILE_LON / p.ps;
+        srow = hg;
+    } else {                         // every ps-th column of one residue class
+        const int r = tile % p.ps, u0 = (tile / p.ps) * TILE_LON;
+        col = (u0 + g) * p.ps + r;
+        ok0 = u0 + g < p.nlon_out;
+        first = u0;
+        srow = hg * p.ps + r;
+    }
+    const bool ok1 = ok0 && hg * TILE_LAT + 1 < p.nlat_in;
+    col = min(col, p.nlon_in - 1);
     const int hp0 = hg * TILE_LAT, hp1 = min(hg * TILE_LAT + 1, p.nlat_in - 1);
-    const size_t pt0 = (size_t)(n * p.nlat_in + hp0) * p.nlon_in + (size_t)uq * p.ps + r;
-    const size_t pt1 = (size_t)(n * p.nlat_in + hp1) * p.nlon_in + (size_t)uq * p.ps + r;
+    const size_t pt0 = (size_t)(n * p.nlat_in + hp0) * p.nlon_in + col;
+    const size_t pt1 = (size_t)(n * p.nlat_in + hp1) * p.nlon_in + col;
     const float scale_log2 = scale * LOG2E;
 
     uint32_t kh[KS][4], kl[KS][4], vh[KS][4], vl[KS][4];
@@ -626,11 +639,10 @@ backward_dkdv_mma_kernel(DevPlan p, const float* __restrict__ q, const float* __
         gv[nt][0] = gv[nt][1] = gv[nt][2] = gv[nt][3] = 0.f;
     }
     const size_t oslice = (size_t)n * p.nlat_out * p.nlon_out;
-    const int srow = hg * p.ps + r;
     const int4* stream = p.t_stream + (size_t)p.t_chunk_ptr[srow] * 16;
     const int nchunks = p.t_chunk_ptr[srow + 1] - p.t_chunk_ptr[srow];
 
-    make_walker<C, true>(stages, stream, lane, u0, p.nlon_out, 1, q + oslice * C, dout + oslice * C, lse + oslice, Dws + oslice).run(nchunks, [&](const Stage<C>& st) {
+    make_walker<C, true>(stages, stream, lane, first, p.nlon_out, 1, q + oslice * C, dout + oslice * C, lse + oslice, Dws + oslice).run(nchunks, [&](const Stage<C>& st) {
         float s[2][4], tt[2][4];
         {
             float xr[2][CPT];
@@ -753,8 +765,8 @@ cudaError_t launch_backward_dq_mma(const DevPlan& p, const float* q, const float
 cudaError_t launch_backward_dkdv_mma(const DevPlan& p, const float* q, const float* k, const float* v, const float* dout,
                                      const float* lse, const float* Dws, float* dk, float* dv, int N, int C, cudaStream_t stream) {
     const float scale = 1.0f / sqrtf((float)C);
-    const int tiles = (p.nlon_out + TILE_LON - 1) / TILE_LON;
-    const long long tasks = (long long)tiles * p.ps * ((p.nlat_in + TILE_LAT - 1) / TILE_LAT) * N;
+    const int tiles = p.t_consecutive ? (p.nlon_in + TILE_LON - 1) / TILE_LON : p.ps * ((p.nlon_out + TILE_LON - 1) / TILE_LON);
+    const long long tasks = (long long)tiles * ((p.nlat_in + TILE_LAT - 1) / TILE_LAT) * N;
     const long long blocks = (tasks + WARPS - 1) / WARPS;
     if (blocks > 0x7fffffffLL) return cudaErrorInvalidValue;
     return dispatch_c(C, [&](auto c) {

@@ -280,12 +280,46 @@ void build_forward_stream(const HostPlan& P, Stream& S) {
     }
 }
 
-void build_transposed_stream(const HostPlan& P, Stream& S) {
-    // Row (group of input rings, r): tile rows are input columns c = ps*u + r.  Output point (h, w) is a partner of
-    // column u of input ring h' iff c - w*ps in [-m, m]  <=>  w - u in [ceil((r - m)/ps), floor((r + m)/ps)].
+bool build_transposed_stream(const HostPlan& P, Stream& S) {
     const int groups = (P.nlat_in + TILE_LAT - 1) / TILE_LAT;
-    S.chunk_ptr.assign((size_t)groups * P.ps + 1, 0);
     S.entries.clear();
+    if (TILE_LON % P.ps == 0) {
+        // Consecutive layout.  Tile row i of ring k is input column c0 + i; output point (h, w) is its partner iff
+        // (c0 + i) - w*ps in [-m, m]  <=>  w - c0/ps in [ceil((i - m)/ps), floor((i + m)/ps)].
+        S.chunk_ptr.assign((size_t)groups + 1, 0);
+        for (int gi = 0; gi < groups; ++gi) {
+            const size_t start = S.entries.size();
+            merge_group(P.t_row_ptr, P.t_windows, gi * TILE_LAT, P.nlat_in, [&](int lat, const int (&m)[TILE_LAT]) {
+                const int32_t base = lat * P.nlon_out;
+                uint32_t whole_rows = 0;
+                int lo = INT32_MAX, hi = INT32_MIN;
+                for (int k = 0; k < TILE_LAT; ++k) {
+                    if (m[k] == -2) continue;
+                    if (m[k] < 0) { whole_rows |= ((1u << TILE_LON) - 1u) << (k * TILE_LON); continue; }
+                    lo = std::min(lo, ceil_div(-m[k], P.ps));
+                    hi = std::max(hi, floor_div(TILE_LON - 1 + m[k], P.ps));
+                }
+                if (whole_rows)
+                    for (int u = 0; u < P.nlon_out; ++u)
+                        S.entries.push_back(StreamEntry{(int32_t)(base | (int32_t)0x80000000), (int32_t)((u & 0xffff) | (whole_rows << 16)), 0.f, 0});
+                for (int e_rel = lo; e_rel <= hi; ++e_rel) {
+                    uint32_t mask = 0;
+                    for (int k = 0; k < TILE_LAT; ++k) {
+                        if (m[k] < 0) continue;   // absent (-2) or whole (-1, handled above)
+                        for (int i = 0; i < TILE_LON; ++i)
+                            if (e_rel >= ceil_div(i - m[k], P.ps) && e_rel <= floor_div(i + m[k], P.ps)) mask |= 1u << (k * TILE_LON + i);
+                    }
+                    if (mask) S.entries.push_back(StreamEntry{base, (int32_t)(((uint32_t)e_rel & 0xffffu) | (mask << 16)), 0.f, 0});
+                }
+            });
+            pad_row(S.entries, start);
+            S.chunk_ptr[(size_t)gi + 1] = (int32_t)(S.entries.size() / 16);
+        }
+        return true;
+    }
+    // By residue.  Row (group, r): tile rows are input columns c = ps*u + r.  Output point (h, w) is a partner of
+    // column u of input ring h' iff c - w*ps in [-m, m]  <=>  w - u in [ceil((r - m)/ps), floor((r + m)/ps)].
+    S.chunk_ptr.assign((size_t)groups * P.ps + 1, 0);
     for (int gi = 0; gi < groups; ++gi) {
         for (int r = 0; r < P.ps; ++r) {
             const size_t start = S.entries.size();
@@ -303,6 +337,7 @@ void build_transposed_stream(const HostPlan& P, Stream& S) {
             S.chunk_ptr[(size_t)gi * P.ps + r + 1] = (int32_t)(S.entries.size() / 16);
         }
     }
+    return false;
 }
 
 }  // namespace sna

@@ -60,9 +60,15 @@ struct Stream {
 // Forward stream: one row per group of output latitudes (ceil(nlat_out / TILE_LAT) rows); partners are input
 // points, flat index base + u*ps.
 void build_forward_stream(const HostPlan& plan, Stream& out);
-// Transposed stream for dk/dv: one row per (group of input latitudes, residue r of the input column mod ps);
-// tile rows are input columns c = ps*(first+i%8)+r of the group's rings, partners are output points (h, w).
-void build_transposed_stream(const HostPlan& plan, Stream& out);
+// Transposed stream for dk/dv; partners are output points (h, w).  Two layouts:
+//  - consecutive (when ps divides 8): one stream row per group of input latitudes; tile rows are 8 consecutive
+//    input columns c = c0 + i%8 (c0 a multiple of 8) and the partner index is c0/ps + e_rel.  Neighbouring
+//    input columns share most of their partners, so this needs ~ps times fewer stream columns per input column
+//    than splitting by residue.
+//  - by residue (any other ps): one stream row per (group, residue r); tile rows are c = ps*(u0+i%8) + r and
+//    the partner index is u0 + e_rel.
+// Returns true for the consecutive layout.
+bool build_transposed_stream(const HostPlan& plan, Stream& out);
 
 // Builds the plan.  On failure returns a status and fills `why`.
 PlanStatus build_plan(int nlat_in, int nlon_in, int nlat_out, int nlon_out, int grid_in, int grid_out,

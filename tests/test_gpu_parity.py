@@ -63,6 +63,10 @@ SMALL = [
     small_workload("eq_wide_c32", 40, 160, 40, 160, EQ, EQ, 0.5, 1, 1, 32, 20),           # several tiles per ring
     small_workload("eq_single_neighbor", 9, 16, 9, 16, EQ, EQ, 0.05, 1, 1, 32, 21),       # degenerate: disc = the point itself
     small_workload("eq_down2_wide_c32", 41, 320, 21, 160, EQ, EQ, 0.25, 1, 1, 32, 22),
+    small_workload("eq_down3_c32", 25, 96, 13, 32, EQ, EQ, 0.4, 1, 2, 32, 23),             # ps = 3: transposed stream by residue
+    small_workload("gl_down4_c32", 24, 160, 12, 40, GL, GL, 0.45, 1, 1, 32, 24),           # ps = 4, nlon_out not a tile multiple
+    small_workload("eq_oddlat_c16", 21, 64, 21, 64, EQ, EQ, 0.35, 1, 2, 16, 25),           # odd ring count: last ring group is half empty
+    small_workload("eq_c64_wide", 14, 48, 14, 48, EQ, EQ, 0.9, 1, 1, 64, 26),
 ]
 
 
