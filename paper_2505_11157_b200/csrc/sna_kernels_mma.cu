@@ -228,6 +228,117 @@ __device__ __forceinline__ void scores_times_points(float (&d)[KS][4], const uin
 }
 
 // ---------------------------------------------------------------------------------------------------------
+// Two-MMA products for the backward pass (tolerance 1e-4): the main term a_hi*b_hi is one TF32 MMA and BOTH
+// correction terms a_lo*b_hi + a_hi*b_lo are one BF16 m16n8k16 MMA whose 16 k-slots hold [a_lo | a_hi] against
+// [b_hi ; b_lo] for the same 8 channels.  The corrections are ~2^-11 of the product, so BF16's 8 bits leave a
+// relative error of ~2^-18 (measured ~2e-6 normalised), at two thirds of the tensor time.
+// ---------------------------------------------------------------------------------------------------------
+__device__ __forceinline__ void mma_bf16_acc(float (&d)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
+    asm("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+        : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+        : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+__device__ __forceinline__ void mma_bf16_zero(float (&d)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
+    asm("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%10,%10,%10,%10};"
+        : "=f"(d[0]), "=f"(d[1]), "=f"(d[2]), "=f"(d[3])
+        : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1), "f"(0.f));
+}
+// {lower half = bf16(x0), upper half = bf16(x1)} by truncation (the upper 16 bits of each fp32 word)
+__device__ __forceinline__ uint32_t pack_bf16_trunc(uint32_t x0, uint32_t x1) { return __byte_perm(x0, x1, 0x7632); }
+__device__ __forceinline__ uint32_t pack_bf16_rn(float x0, float x1) {
+    uint32_t r;
+    asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(x1), "f"(x0));
+    return r;
+}
+
+// Persistent A operand of the two-MMA product: hi[ks] = TF32-rounded values (main term), c16[ks] = BF16 quads
+// {lo(row g), lo(row g+8), hi(row g), hi(row g+8)} of the thread's channel pair of k-step ks.
+template <int CPT>
+__device__ __forceinline__ void make_a_operand2(const float* p0, const float* p1, float mul, uint32_t (&hi)[CPT / 2][4], uint32_t (&c16)[CPT / 2][4]) {
+    float a[CPT], b[CPT];
+    load_row<CPT>(p0, a);
+    load_row<CPT>(p1, b);
+#pragma unroll
+    for (int ks = 0; ks < CPT / 2; ++ks) {
+        uint32_t l[4];
+        split_rn(a[2 * ks] * mul, hi[ks][0], l[0]);
+        split_rn(b[2 * ks] * mul, hi[ks][1], l[1]);
+        split_rn(a[2 * ks + 1] * mul, hi[ks][2], l[2]);
+        split_rn(b[2 * ks + 1] * mul, hi[ks][3], l[3]);
+        c16[ks][0] = pack_bf16_rn(__uint_as_float(l[0]), __uint_as_float(l[2]));      // row g:   lo of the channel pair
+        c16[ks][1] = pack_bf16_rn(__uint_as_float(l[1]), __uint_as_float(l[3]));      // row g+8
+        c16[ks][2] = pack_bf16_rn(__uint_as_float(hi[ks][0]), __uint_as_float(hi[ks][2]));   // row g:   hi of the pair
+        c16[ks][3] = pack_bf16_rn(__uint_as_float(hi[ks][1]), __uint_as_float(hi[ks][3]));   // row g+8
+    }
+}
+
+// B operand of one k-step from the raw channel pair (x0, x1): main registers are the raw words; the BF16 pair is
+// {hi pair, lo pair} with lo = x - trunc19(x).
+__device__ __forceinline__ void split_b2(float x0, float x1, uint32_t& m0, uint32_t& m1, uint32_t& h16, uint32_t& l16) {
+    m0 = __float_as_uint(x0);
+    m1 = __float_as_uint(x1);
+    const float l0 = x0 - __uint_as_float(m0 & 0xffffe000u), l1 = x1 - __uint_as_float(m1 & 0xffffe000u);
+    h16 = pack_bf16_trunc(m0, m1);
+    l16 = pack_bf16_trunc(__float_as_uint(l0), __float_as_uint(l1));
+}
+
+// d[tl] = A . B^T for the two 8-column tiles with the two-MMA product (corrections first, then the main terms).
+template <int CPT>
+__device__ __forceinline__ void rows_dot_points2(float (&d)[2][4], const uint32_t (&ah)[CPT / 2][4], const uint32_t (&a16)[CPT / 2][4], const float (&x)[2][CPT]) {
+    uint32_t bm[2][CPT], bh16[2][CPT / 2], bl16[2][CPT / 2];
+#pragma unroll
+    for (int tl = 0; tl < 2; ++tl)
+#pragma unroll
+        for (int ks = 0; ks < CPT / 2; ++ks) split_b2(x[tl][2 * ks], x[tl][2 * ks + 1], bm[tl][2 * ks], bm[tl][2 * ks + 1], bh16[tl][ks], bl16[tl][ks]);
+    mma_bf16_zero(d[0], a16[0], bh16[0][0], bl16[0][0]);
+    mma_bf16_zero(d[1], a16[0], bh16[1][0], bl16[1][0]);
+#pragma unroll
+    for (int ks = 1; ks < CPT / 2; ++ks) {
+        mma_bf16_acc(d[0], a16[ks], bh16[0][ks], bl16[0][ks]);
+        mma_bf16_acc(d[1], a16[ks], bh16[1][ks], bl16[1][ks]);
+    }
+#pragma unroll
+    for (int ks = 0; ks < CPT / 2; ++ks) {
+        mma_acc(d[0], ah[ks], bm[0][2 * ks], bm[0][2 * ks + 1]);
+        mma_acc(d[1], ah[ks], bm[1][2 * ks], bm[1][2 * ks + 1]);
+    }
+}
+
+// Second contraction with the two-MMA product: W (scores layout, 16 x 16 columns) times the column fragments.
+// k-slots of the BF16 MMA of tile tl: [W_lo(8 columns) | W_hi(8 columns)] against [X_hi ; X_lo].
+template <int KS>
+__device__ __forceinline__ void scores_times_points2(float (&d)[KS][4], const float (&w)[2][4], const float (&x)[2][2][KS]) {
+    uint32_t wm[2][4], w16[2][4];
+#pragma unroll
+    for (int tl = 0; tl < 2; ++tl) {
+        uint32_t h[4], l[4];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            h[i] = __float_as_uint(w[tl][i]);
+            l[i] = __float_as_uint(w[tl][i] - __uint_as_float(h[i] & 0xffffe000u));
+        }
+        wm[tl][0] = h[0]; wm[tl][1] = h[2]; wm[tl][2] = h[1]; wm[tl][3] = h[3];   // TF32 A quad: (g,2t) (g+8,2t) (g,2t+1) (g+8,2t+1)
+        w16[tl][0] = pack_bf16_trunc(l[0], l[1]);   // row g:   lo of columns 2t, 2t+1
+        w16[tl][1] = pack_bf16_trunc(l[2], l[3]);   // row g+8
+        w16[tl][2] = pack_bf16_trunc(h[0], h[1]);   // row g:   hi
+        w16[tl][3] = pack_bf16_trunc(h[2], h[3]);   // row g+8
+    }
+    uint32_t xm[2][2][KS], xh16[2][KS], xl16[2][KS];
+#pragma unroll
+    for (int tl = 0; tl < 2; ++tl)
+#pragma unroll
+        for (int nt = 0; nt < KS; ++nt) split_b2(x[tl][0][nt], x[tl][1][nt], xm[tl][0][nt], xm[tl][1][nt], xh16[tl][nt], xl16[tl][nt]);
+#pragma unroll
+    for (int nt = 0; nt < KS; ++nt) mma_bf16_zero(d[nt], w16[0], xh16[0][nt], xl16[0][nt]);
+#pragma unroll
+    for (int nt = 0; nt < KS; ++nt) mma_bf16_acc(d[nt], w16[1], xh16[1][nt], xl16[1][nt]);
+#pragma unroll
+    for (int nt = 0; nt < KS; ++nt) mma_acc(d[nt], wm[0], xm[0][0][nt], xm[0][1][nt]);
+#pragma unroll
+    for (int nt = 0; nt < KS; ++nt) mma_acc(d[nt], wm[1], xm[1][0][nt], xm[1][1][nt]);
+}
+
+// ---------------------------------------------------------------------------------------------------------
 // Warp-private staging of a chunk's 16 partner points in shared memory (cp.async, two stages).
 // Two point arrays are staged per chunk (forward / dq: k and v rows; dk/dv: q and dout rows), each row padded
 // to C+4 floats so that both fragment layouts read without bank conflicts, plus per-column metadata.
@@ -513,8 +624,8 @@ backward_dq_mma_kernel(DevPlan p, const float* __restrict__ q, const float* __re
     const float scale_log2 = scale * LOG2E;
 
     uint32_t qh[KS][4], ql[KS][4], yh[KS][4], yl[KS][4];
-    make_a_operand<CPT>(q + pt0 * C + t * CPT, q + pt1 * C + t * CPT, scale_log2, qh, ql);
-    make_a_operand<CPT>(dout + pt0 * C + t * CPT, dout + pt1 * C + t * CPT, 1.f, yh, yl);
+    make_a_operand2<CPT>(q + pt0 * C + t * CPT, q + pt1 * C + t * CPT, scale_log2, qh, ql);   // ql, yl: BF16 correction quads
+    make_a_operand2<CPT>(dout + pt0 * C + t * CPT, dout + pt1 * C + t * CPT, 1.f, yh, yl);
     // D of the two tile rows
     float D0 = 0.f, D1 = 0.f;
     {
@@ -547,10 +658,10 @@ backward_dq_mma_kernel(DevPlan p, const float* __restrict__ q, const float* __re
             float xr[2][CPT];
             lds_row<CPT>(st.a, g, t, xr[0]);
             lds_row<CPT>(st.a, 8 + g, t, xr[1]);
-            rows_dot_points<CPT>(s, qh, ql, xr);
+            rows_dot_points2<CPT>(s, qh, ql, xr);
             lds_row<CPT>(st.b, g, t, xr[0]);
             lds_row<CPT>(st.b, 8 + g, t, xr[1]);
-            rows_dot_points<CPT>(tt, yh, yl, xr);
+            rows_dot_points2<CPT>(tt, yh, yl, xr);
         }
         float kr[2][2][KS];
 #pragma unroll
@@ -569,10 +680,8 @@ backward_dq_mma_kernel(DevPlan p, const float* __restrict__ q, const float* __re
             s[tl][2] = p10 * (tt[tl][2] - D1);
             s[tl][3] = p11 * (tt[tl][3] - D1);
         }
-        uint32_t dh[2][4], dl[2][4];
-        scores_as_a(s, dh, dl);
         float part[KS][4];
-        scores_times_points<KS>(part, dh, dl, kr);
+        scores_times_points2<KS>(part, s, kr);
 #pragma unroll
         for (int nt = 0; nt < KS; ++nt) {
             acc[nt][0] += part[nt][0]; acc[nt][1] += part[nt][1]; acc[nt][2] += part[nt][2]; acc[nt][3] += part[nt][3];
@@ -629,8 +738,8 @@ backward_dkdv_mma_kernel(DevPlan p, const float* __restrict__ q, const float* __
     const float scale_log2 = scale * LOG2E;
 
     uint32_t kh[KS][4], kl[KS][4], vh[KS][4], vl[KS][4];
-    make_a_operand<CPT>(k + pt0 * C + t * CPT, k + pt1 * C + t * CPT, scale_log2, kh, kl);
-    make_a_operand<CPT>(v + pt0 * C + t * CPT, v + pt1 * C + t * CPT, 1.f, vh, vl);
+    make_a_operand2<CPT>(k + pt0 * C + t * CPT, k + pt1 * C + t * CPT, scale_log2, kh, kl);   // kl, vl: BF16 correction quads
+    make_a_operand2<CPT>(v + pt0 * C + t * CPT, v + pt1 * C + t * CPT, 1.f, vh, vl);
     const float bias0 = p.log2_omega[hp0], bias1 = p.log2_omega[hp1];
     float gk[KS][4], gv[KS][4];
 #pragma unroll
@@ -648,10 +757,10 @@ backward_dkdv_mma_kernel(DevPlan p, const float* __restrict__ q, const float* __
             float xr[2][CPT];
             lds_row<CPT>(st.a, g, t, xr[0]);
             lds_row<CPT>(st.a, 8 + g, t, xr[1]);
-            rows_dot_points<CPT>(s, kh, kl, xr);
+            rows_dot_points2<CPT>(s, kh, kl, xr);
             lds_row<CPT>(st.b, g, t, xr[0]);
             lds_row<CPT>(st.b, 8 + g, t, xr[1]);
-            rows_dot_points<CPT>(tt, vh, vl, xr);
+            rows_dot_points2<CPT>(tt, vh, vl, xr);
         }
         float qr[2][2][KS], yr[2][2][KS];
         float pr[2][4];
@@ -675,14 +784,11 @@ backward_dkdv_mma_kernel(DevPlan p, const float* __restrict__ q, const float* __
             s[tl][2] = pr[tl][2] * (tt[tl][2] - Dd.x);
             s[tl][3] = pr[tl][3] * (tt[tl][3] - Dd.y);
         }
-        uint32_t wh[2][4], wl[2][4];
         float part[KS][4];
-        scores_as_a(pr, wh, wl);
-        scores_times_points<KS>(part, wh, wl, yr);
+        scores_times_points2<KS>(part, pr, yr);
 #pragma unroll
         for (int nt = 0; nt < KS; ++nt) { gv[nt][0] += part[nt][0]; gv[nt][1] += part[nt][1]; gv[nt][2] += part[nt][2]; gv[nt][3] += part[nt][3]; }
-        scores_as_a(s, wh, wl);
-        scores_times_points<KS>(part, wh, wl, qr);
+        scores_times_points2<KS>(part, s, qr);
 #pragma unroll
         for (int nt = 0; nt < KS; ++nt) { gk[nt][0] += part[nt][0]; gk[nt][1] += part[nt][1]; gk[nt][2] += part[nt][2]; gk[nt][3] += part[nt][3]; }
     });
