@@ -274,22 +274,25 @@ __device__ __forceinline__ void make_a_operand2(const float* p0, const float* p1
 
 // B operand of one k-step from the raw channel pair (x0, x1): main registers are the raw words; the BF16 pair is
 // {hi pair, lo pair} with lo = x - trunc19(x).
+template <bool RN = false>
 __device__ __forceinline__ void split_b2(float x0, float x1, uint32_t& m0, uint32_t& m1, uint32_t& h16, uint32_t& l16) {
     m0 = __float_as_uint(x0);
     m1 = __float_as_uint(x1);
     const float l0 = x0 - __uint_as_float(m0 & 0xffffe000u), l1 = x1 - __uint_as_float(m1 & 0xffffe000u);
     h16 = pack_bf16_trunc(m0, m1);
-    l16 = pack_bf16_trunc(__float_as_uint(l0), __float_as_uint(l1));
+    // the lo parts carry the larger correction (2^-10 of the value): rounding them to nearest instead of truncating
+    // brings the product's relative error from 2^-17 to below 2^-19, which the forward pass needs
+    l16 = RN ? pack_bf16_rn(l0, l1) : pack_bf16_trunc(__float_as_uint(l0), __float_as_uint(l1));
 }
 
 // d[tl] = A . B^T for the two 8-column tiles with the two-MMA product (corrections first, then the main terms).
-template <int CPT>
+template <int CPT, bool RN = false>
 __device__ __forceinline__ void rows_dot_points2(float (&d)[2][4], const uint32_t (&ah)[CPT / 2][4], const uint32_t (&a16)[CPT / 2][4], const float (&x)[2][CPT]) {
     uint32_t bm[2][CPT], bh16[2][CPT / 2], bl16[2][CPT / 2];
 #pragma unroll
     for (int tl = 0; tl < 2; ++tl)
 #pragma unroll
-        for (int ks = 0; ks < CPT / 2; ++ks) split_b2(x[tl][2 * ks], x[tl][2 * ks + 1], bm[tl][2 * ks], bm[tl][2 * ks + 1], bh16[tl][ks], bl16[tl][ks]);
+        for (int ks = 0; ks < CPT / 2; ++ks) split_b2<RN>(x[tl][2 * ks], x[tl][2 * ks + 1], bm[tl][2 * ks], bm[tl][2 * ks + 1], bh16[tl][ks], bl16[tl][ks]);
     mma_bf16_zero(d[0], a16[0], bh16[0][0], bl16[0][0]);
     mma_bf16_zero(d[1], a16[0], bh16[1][0], bl16[1][0]);
 #pragma unroll
@@ -306,7 +309,7 @@ __device__ __forceinline__ void rows_dot_points2(float (&d)[2][4], const uint32_
 
 // Second contraction with the two-MMA product: W (scores layout, 16 x 16 columns) times the column fragments.
 // k-slots of the BF16 MMA of tile tl: [W_lo(8 columns) | W_hi(8 columns)] against [X_hi ; X_lo].
-template <int KS>
+template <int KS, bool RN = false>
 __device__ __forceinline__ void scores_times_points2(float (&d)[KS][4], const float (&w)[2][4], const float (&x)[2][2][KS]) {
     uint32_t wm[2][4], w16[2][4];
 #pragma unroll
@@ -318,8 +321,8 @@ __device__ __forceinline__ void scores_times_points2(float (&d)[KS][4], const fl
             l[i] = __float_as_uint(w[tl][i] - __uint_as_float(h[i] & 0xffffe000u));
         }
         wm[tl][0] = h[0]; wm[tl][1] = h[2]; wm[tl][2] = h[1]; wm[tl][3] = h[3];   // TF32 A quad: (g,2t) (g+8,2t) (g,2t+1) (g+8,2t+1)
-        w16[tl][0] = pack_bf16_trunc(l[0], l[1]);   // row g:   lo of columns 2t, 2t+1
-        w16[tl][1] = pack_bf16_trunc(l[2], l[3]);   // row g+8
+        w16[tl][0] = RN ? pack_bf16_rn(__uint_as_float(l[0]), __uint_as_float(l[1])) : pack_bf16_trunc(l[0], l[1]);   // row g: lo of columns 2t, 2t+1
+        w16[tl][1] = RN ? pack_bf16_rn(__uint_as_float(l[2]), __uint_as_float(l[3])) : pack_bf16_trunc(l[2], l[3]);   // row g+8
         w16[tl][2] = pack_bf16_trunc(h[0], h[1]);   // row g:   hi
         w16[tl][3] = pack_bf16_trunc(h[2], h[3]);   // row g+8
     }
@@ -327,7 +330,7 @@ __device__ __forceinline__ void scores_times_points2(float (&d)[KS][4], const fl
 #pragma unroll
     for (int tl = 0; tl < 2; ++tl)
 #pragma unroll
-        for (int nt = 0; nt < KS; ++nt) split_b2(x[tl][0][nt], x[tl][1][nt], xm[tl][0][nt], xm[tl][1][nt], xh16[tl][nt], xl16[tl][nt]);
+        for (int nt = 0; nt < KS; ++nt) split_b2<RN>(x[tl][0][nt], x[tl][1][nt], xm[tl][0][nt], xm[tl][1][nt], xh16[tl][nt], xl16[tl][nt]);
 #pragma unroll
     for (int nt = 0; nt < KS; ++nt) mma_bf16_zero(d[nt], w16[0], xh16[0][nt], xl16[0][nt]);
 #pragma unroll
@@ -512,7 +515,7 @@ forward_mma_kernel(DevPlan p, const float* __restrict__ q, const float* __restri
     const size_t pt1 = (size_t)(n * p.nlat_out + min(hg * TILE_LAT + 1, p.nlat_out - 1)) * p.nlon_out + wq;
 
     uint32_t qh[KS][4], ql[KS][4];   // q in the log2 domain
-    make_a_operand<CPT>(q + pt0 * C + t * CPT, q + pt1 * C + t * CPT, scale_log2, qh, ql);
+    make_a_operand2<CPT>(q + pt0 * C + t * CPT, q + pt1 * C + t * CPT, scale_log2, qh, ql);   // ql: BF16 correction quads
     float o[KS][4];
 #pragma unroll
     for (int nt = 0; nt < KS; ++nt) o[nt][0] = o[nt][1] = o[nt][2] = o[nt][3] = 0.f;
@@ -528,7 +531,7 @@ forward_mma_kernel(DevPlan p, const float* __restrict__ q, const float* __restri
             float kr[2][CPT];
             lds_row<CPT>(st.a, g, t, kr[0]);
             lds_row<CPT>(st.a, 8 + g, t, kr[1]);
-            rows_dot_points<CPT>(s, qh, ql, kr);
+            rows_dot_points2<CPT, true>(s, qh, ql, kr);
         }
         float vr[2][2][KS];
 #pragma unroll
@@ -570,10 +573,8 @@ forward_mma_kernel(DevPlan p, const float* __restrict__ q, const float* __restri
         }
         l0 = fmaf(l0, corr0, ps0);
         l1 = fmaf(l1, corr1, ps1);
-        uint32_t ph[2][4], pl[2][4];
-        scores_as_a(s, ph, pl);
         float pv[KS][4];
-        scores_times_points<KS>(pv, ph, pl, vr);
+        scores_times_points2<KS, true>(pv, s, vr);
 #pragma unroll
         for (int nt = 0; nt < KS; ++nt) {
             o[nt][0] = fmaf(o[nt][0], corr0, pv[nt][0]); o[nt][1] = fmaf(o[nt][1], corr0, pv[nt][1]);
