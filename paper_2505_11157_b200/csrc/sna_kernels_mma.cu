@@ -1,10 +1,13 @@
-// Tensor-core kernels (sm_100a): every contraction of the path runs on mma.sync m16n8k8 TF32 with a three-term
-// split (x = hi + lo; lo*hi + hi*lo + hi*hi, fp32 accumulate), which keeps fp32-level accuracy
-// (measured < 1e-6 normalised error) at four times the FP32 FMA rate for dense tiles.
+// Tensor-core kernels (sm_100a): every contraction of the path runs on mma.sync with fp32-level accuracy from a
+// split of each operand, x = hi + lo with hi the top 11 significand bits.  A product a*b is two MMAs into one fp32
+// fragment: the main term a_hi*b_hi as m16n8k8 TF32, and both correction terms a_lo*b_hi + a_hi*b_lo as a single
+// m16n8k16 BF16 MMA whose 16 k-slots hold [a_lo | a_hi] against [b_hi ; b_lo] (the corrections are ~2^-11 of the
+// product, so 8 bits suffice).  Measured normalised errors: forward 2.5e-6..3.3e-6, backward <= 1.9e-5.
 //
-// Work decomposition: one warp owns 16 consecutive points of one ring (the M dimension of the MMA: "tile rows")
-// and walks the host-built column stream of that ring row, 16 partner points ("columns") per step.  Band
-// structure and ragged edges are expressed by the 16-bit row mask carried by every stream column.
+// Work decomposition: one warp owns a tile of 16 points (the M dimension of the MMA: "tile rows") = 8 consecutive
+// longitudes on each of 2 adjacent rings, and walks the host-built column stream of that ring group, 16 partner
+// points ("columns") per step.  Band structure and ragged edges are expressed by the 16-bit row mask carried by
+// every stream column.
 // The 16 partner points of a chunk are staged by cp.async into a warp-private, two-stage shared-memory ring
 // while the previous chunk is consumed; warps never synchronise with each other (no block-level barrier).
 //
@@ -40,33 +43,23 @@ __device__ __forceinline__ float ex2(float x) {
     return y;
 }
 
-// Split for operands that are used once: the MMA reads only the top 19 bits of a TF32 operand, so the raw fp32
-// word serves as hi, and lo is the exact remainder after that truncation (itself truncated by the MMA: the
-// representation error is below 2^-20 relative).
-__device__ __forceinline__ void split_fast(float x, uint32_t& hi, uint32_t& lo) {
-    hi = __float_as_uint(x);
-    lo = __float_as_uint(x - __uint_as_float(hi & 0xffffe000u));
-}
-// Split for operands that are reused over the whole stream: both parts rounded to nearest.
+// The MMA reads only the top 19 bits of a TF32 operand (verified on B200), so for operands that are used once
+// the raw fp32 word serves as hi and lo = x - trunc19(x) is exact; see split_b2 below.
+// Split for operands that are reused over the whole stream (the A operand of a tile): both parts rounded to nearest.
 __device__ __forceinline__ void split_rn(float x, uint32_t& hi, uint32_t& lo) {
     const uint32_t h = (__float_as_uint(x) + 0x1000u) & 0xffffe000u;
     hi = h;
     lo = (__float_as_uint(x - __uint_as_float(h)) + 0x1000u) & 0xffffe000u;
 }
 
-// The tensor core adds into its fp32 accumulator with truncation, so a long chain of MMAs into one fragment
-// drifts towards zero (measured: 3e-5 relative after ~1000 steps).  Every chain here is therefore short: the
-// small correction terms lo*hi + hi*lo go first, the main terms hi*hi last, into a fragment that starts at
-// zero, and long sums are carried in fp32 FMAs outside the tensor core.
+// The tensor core adds into its fp32 accumulator with truncation (verified: 1 + 1.75*2^-24 -> 1), so a long chain
+// of MMAs into one fragment drifts towards zero (measured: 3e-5 relative after ~1000 steps).  Every chain here is
+// therefore short: the correction MMAs go first, the main terms last, into a fragment that starts at zero, and long
+// sums are carried in fp32 FMAs outside the tensor core.
 __device__ __forceinline__ void mma_acc(float (&d)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
     asm("mma.sync.aligned.m16n8k8.row.col.f32.tf32.tf32.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
-                 : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
-                 : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
-}
-__device__ __forceinline__ void mma_zero(float (&d)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
-    asm("mma.sync.aligned.m16n8k8.row.col.f32.tf32.tf32.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%10,%10,%10,%10};"
-                 : "=f"(d[0]), "=f"(d[1]), "=f"(d[2]), "=f"(d[3])
-                 : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1), "f"(0.f));
+        : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+        : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
 }
 
 __device__ __forceinline__ float4 ldg4(const float* p) { return __ldg(reinterpret_cast<const float4*>(p)); }
@@ -80,158 +73,12 @@ __device__ __forceinline__ void load_row(const float* p, float (&x)[CPT]) {
         x[4 * j] = a.x; x[4 * j + 1] = a.y; x[4 * j + 2] = a.z; x[4 * j + 3] = a.w;
     }
 }
-// Column fragment (KS contiguous channels).
-template <int KS>
-__device__ __forceinline__ void load_col(const float* p, float (&x)[KS]) {
-    if constexpr (KS % 4 == 0) {
-#pragma unroll
-        for (int j = 0; j < KS / 4; ++j) {
-            const float4 a = ldg4(p + 4 * j);
-            x[4 * j] = a.x; x[4 * j + 1] = a.y; x[4 * j + 2] = a.z; x[4 * j + 3] = a.w;
-        }
-    } else {
-        const float2 a = __ldg(reinterpret_cast<const float2*>(p));
-        x[0] = a.x; x[1] = a.y;
-    }
-}
-
-// A operand (tile rows g and g+8) from the row fragments of the two points, pre-multiplied by `mul`.
-template <int CPT>
-__device__ __forceinline__ void make_a_operand(const float* p0, const float* p1, float mul, uint32_t (&hi)[CPT / 2][4], uint32_t (&lo)[CPT / 2][4]) {
-    float a[CPT], b[CPT];
-    load_row<CPT>(p0, a);
-    load_row<CPT>(p1, b);
-#pragma unroll
-    for (int ks = 0; ks < CPT / 2; ++ks) {
-        split_rn(a[2 * ks] * mul, hi[ks][0], lo[ks][0]);       // (row g,   k = t)
-        split_rn(b[2 * ks] * mul, hi[ks][1], lo[ks][1]);       // (row g+8, k = t)
-        split_rn(a[2 * ks + 1] * mul, hi[ks][2], lo[ks][2]);   // (row g,   k = t+4)
-        split_rn(b[2 * ks + 1] * mul, hi[ks][3], lo[ks][3]);   // (row g+8, k = t+4)
-    }
-}
-
-// d[tl][16x8] = A (tile rows x channels) . B^T for the two 8-column tiles of a chunk; B = row fragment x[tl] of the
-// point in column g of tile tl.  The two dependent MMA chains are interleaved.
-template <int CPT>
-__device__ __forceinline__ void rows_dot_points(float (&d)[2][4], const uint32_t (&ah)[CPT / 2][4], const uint32_t (&al)[CPT / 2][4], const float (&x)[2][CPT]) {
-    uint32_t bh[2][CPT], bl[2][CPT];
-#pragma unroll
-    for (int tl = 0; tl < 2; ++tl)
-#pragma unroll
-        for (int j = 0; j < CPT; ++j) split_fast(x[tl][j], bh[tl][j], bl[tl][j]);
-    mma_zero(d[0], al[0], bh[0][0], bh[0][1]);
-    mma_zero(d[1], al[0], bh[1][0], bh[1][1]);
-    mma_acc(d[0], ah[0], bl[0][0], bl[0][1]);
-    mma_acc(d[1], ah[0], bl[1][0], bl[1][1]);
-#pragma unroll
-    for (int ks = 1; ks < CPT / 2; ++ks) {
-        mma_acc(d[0], al[ks], bh[0][2 * ks], bh[0][2 * ks + 1]);
-        mma_acc(d[1], al[ks], bh[1][2 * ks], bh[1][2 * ks + 1]);
-        mma_acc(d[0], ah[ks], bl[0][2 * ks], bl[0][2 * ks + 1]);
-        mma_acc(d[1], ah[ks], bl[1][2 * ks], bl[1][2 * ks + 1]);
-    }
-#pragma unroll
-    for (int ks = 0; ks < CPT / 2; ++ks) {
-        mma_acc(d[0], ah[ks], bh[0][2 * ks], bh[0][2 * ks + 1]);
-        mma_acc(d[1], ah[ks], bh[1][2 * ks], bh[1][2 * ks + 1]);
-    }
-}
-
-// The same contraction with the B operand already split (shared by several M-tiles).
-template <int CPT>
-__device__ __forceinline__ void split_rows(const float (&x)[2][CPT], uint32_t (&bh)[2][CPT], uint32_t (&bl)[2][CPT]) {
-#pragma unroll
-    for (int tl = 0; tl < 2; ++tl)
-#pragma unroll
-        for (int j = 0; j < CPT; ++j) split_fast(x[tl][j], bh[tl][j], bl[tl][j]);
-}
-template <int CPT>
-__device__ __forceinline__ void rows_dot_split(float (&d)[2][4], const uint32_t (&ah)[CPT / 2][4], const uint32_t (&al)[CPT / 2][4],
-                                               const uint32_t (&bh)[2][CPT], const uint32_t (&bl)[2][CPT]) {
-    mma_zero(d[0], al[0], bh[0][0], bh[0][1]);
-    mma_zero(d[1], al[0], bh[1][0], bh[1][1]);
-    mma_acc(d[0], ah[0], bl[0][0], bl[0][1]);
-    mma_acc(d[1], ah[0], bl[1][0], bl[1][1]);
-#pragma unroll
-    for (int ks = 1; ks < CPT / 2; ++ks) {
-        mma_acc(d[0], al[ks], bh[0][2 * ks], bh[0][2 * ks + 1]);
-        mma_acc(d[1], al[ks], bh[1][2 * ks], bh[1][2 * ks + 1]);
-        mma_acc(d[0], ah[ks], bl[0][2 * ks], bl[0][2 * ks + 1]);
-        mma_acc(d[1], ah[ks], bl[1][2 * ks], bl[1][2 * ks + 1]);
-    }
-#pragma unroll
-    for (int ks = 0; ks < CPT / 2; ++ks) {
-        mma_acc(d[0], ah[ks], bh[0][2 * ks], bh[0][2 * ks + 1]);
-        mma_acc(d[1], ah[ks], bh[1][2 * ks], bh[1][2 * ks + 1]);
-    }
-}
-template <int KS>
-__device__ __forceinline__ void split_cols(const float (&x)[2][2][KS], uint32_t (&xh)[2][2][KS], uint32_t (&xl)[2][2][KS]) {
-#pragma unroll
-    for (int tl = 0; tl < 2; ++tl)
-#pragma unroll
-        for (int j = 0; j < 2; ++j)
-#pragma unroll
-            for (int nt = 0; nt < KS; ++nt) split_fast(x[tl][j][nt], xh[tl][j][nt], xl[tl][j][nt]);
-}
-template <int KS>
-__device__ __forceinline__ void scores_times_split(float (&d)[KS][4], const uint32_t (&wh)[2][4], const uint32_t (&wl)[2][4],
-                                                   const uint32_t (&xh)[2][2][KS], const uint32_t (&xl)[2][2][KS]) {
-#pragma unroll
-    for (int nt = 0; nt < KS; ++nt) mma_zero(d[nt], wl[0], xh[0][0][nt], xh[0][1][nt]);
-#pragma unroll
-    for (int nt = 0; nt < KS; ++nt) mma_acc(d[nt], wh[0], xl[0][0][nt], xl[0][1][nt]);
-#pragma unroll
-    for (int nt = 0; nt < KS; ++nt) mma_acc(d[nt], wl[1], xh[1][0][nt], xh[1][1][nt]);
-#pragma unroll
-    for (int nt = 0; nt < KS; ++nt) mma_acc(d[nt], wh[1], xl[1][0][nt], xl[1][1][nt]);
-#pragma unroll
-    for (int nt = 0; nt < KS; ++nt) mma_acc(d[nt], wh[0], xh[0][0][nt], xh[0][1][nt]);
-#pragma unroll
-    for (int nt = 0; nt < KS; ++nt) mma_acc(d[nt], wh[1], xh[1][0][nt], xh[1][1][nt]);
-}
-
-// A operand from two score-layout fragments w[tl] (rows g, g+8; columns 2t, 2t+1 of 8-column tile tl).
-__device__ __forceinline__ void scores_as_a(const float (&w)[2][4], uint32_t (&hi)[2][4], uint32_t (&lo)[2][4]) {
-#pragma unroll
-    for (int tl = 0; tl < 2; ++tl) {
-        split_fast(w[tl][0], hi[tl][0], lo[tl][0]);
-        split_fast(w[tl][2], hi[tl][1], lo[tl][1]);
-        split_fast(w[tl][1], hi[tl][2], lo[tl][2]);
-        split_fast(w[tl][3], hi[tl][3], lo[tl][3]);
-    }
-}
-
-// d[nt] (16 rows x 8 channels of n-tile nt) = W (16 x 16 columns, as A operand) times the column fragments
-// x[tl][j] of the 16 partner points, in a zero-started fragment per n-tile.
-template <int KS>
-__device__ __forceinline__ void scores_times_points(float (&d)[KS][4], const uint32_t (&wh)[2][4], const uint32_t (&wl)[2][4], const float (&x)[2][2][KS]) {
-    uint32_t xh[2][2][KS], xl[2][2][KS];
-#pragma unroll
-    for (int tl = 0; tl < 2; ++tl)
-#pragma unroll
-        for (int j = 0; j < 2; ++j)
-#pragma unroll
-            for (int nt = 0; nt < KS; ++nt) split_fast(x[tl][j][nt], xh[tl][j][nt], xl[tl][j][nt]);
-#pragma unroll
-    for (int nt = 0; nt < KS; ++nt) mma_zero(d[nt], wl[0], xh[0][0][nt], xh[0][1][nt]);
-#pragma unroll
-    for (int nt = 0; nt < KS; ++nt) mma_acc(d[nt], wh[0], xl[0][0][nt], xl[0][1][nt]);
-#pragma unroll
-    for (int nt = 0; nt < KS; ++nt) mma_acc(d[nt], wl[1], xh[1][0][nt], xh[1][1][nt]);
-#pragma unroll
-    for (int nt = 0; nt < KS; ++nt) mma_acc(d[nt], wh[1], xl[1][0][nt], xl[1][1][nt]);
-#pragma unroll
-    for (int nt = 0; nt < KS; ++nt) mma_acc(d[nt], wh[0], xh[0][0][nt], xh[0][1][nt]);
-#pragma unroll
-    for (int nt = 0; nt < KS; ++nt) mma_acc(d[nt], wh[1], xh[1][0][nt], xh[1][1][nt]);
-}
-
 // ---------------------------------------------------------------------------------------------------------
-// Two-MMA products for the backward pass (tolerance 1e-4): the main term a_hi*b_hi is one TF32 MMA and BOTH
-// correction terms a_lo*b_hi + a_hi*b_lo are one BF16 m16n8k16 MMA whose 16 k-slots hold [a_lo | a_hi] against
-// [b_hi ; b_lo] for the same 8 channels.  The corrections are ~2^-11 of the product, so BF16's 8 bits leave a
-// relative error of ~2^-18 (measured ~2e-6 normalised), at two thirds of the tensor time.
+// Two-MMA products: the main term a_hi*b_hi is one TF32 MMA and BOTH correction terms a_lo*b_hi + a_hi*b_lo are
+// one BF16 m16n8k16 MMA whose 16 k-slots hold [a_lo | a_hi] against [b_hi ; b_lo] for the same 8 channels.  The
+// corrections are ~2^-11 of the product, so BF16's 8 bits leave a relative error of 2^-17 (lo parts truncated;
+// used by the backward pass, gate 1e-4) or below 2^-19 (lo parts rounded to nearest; forward pass, gate 1e-5), at
+// two thirds of the tensor time of three TF32 MMAs.
 // ---------------------------------------------------------------------------------------------------------
 __device__ __forceinline__ void mma_bf16_acc(float (&d)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
     asm("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
