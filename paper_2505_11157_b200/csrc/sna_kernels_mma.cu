@@ -453,7 +453,7 @@ forward_mma_kernel(DevPlan p, const float* __restrict__ q, const float* __restri
 // `out` and `dq` may be the same buffer: a warp reads its own 16 rows of `out` before it writes them as dq.
 // ---------------------------------------------------------------------------------------------------------
 template <int C>
-__global__ void __launch_bounds__(THREADS, 3)
+__global__ void __launch_bounds__(THREADS, 2)
 backward_dq_mma_kernel(DevPlan p, const float* __restrict__ q, const float* __restrict__ k, const float* __restrict__ v,
                        const float* __restrict__ dout, const float* out, const float* __restrict__ lse,
                        float* dq, float* __restrict__ Dws, int N, float scale, int tiles_per_row, long long total_tasks) {

@@ -67,6 +67,10 @@ SMALL = [
     small_workload("gl_down4_c32", 24, 160, 12, 40, GL, GL, 0.45, 1, 1, 32, 24),           # ps = 4, nlon_out not a tile multiple
     small_workload("eq_oddlat_c16", 21, 64, 21, 64, EQ, EQ, 0.35, 1, 2, 16, 25),           # odd ring count: last ring group is half empty
     small_workload("eq_c64_wide", 14, 48, 14, 48, EQ, EQ, 0.9, 1, 1, 64, 26),
+    small_workload("gl_latratio_2p4_c32", 24, 64, 10, 32, GL, GL, 0.5, 1, 2, 32, 27),      # latitude grids do not nest
+    small_workload("eq_to_gl_up_lat_c32", 9, 40, 20, 40, EQ, GL, 0.6, 1, 1, 32, 28),       # more output than input rings
+    small_workload("eq_nearly_global_c32", 12, 32, 12, 32, EQ, EQ, 2.6, 1, 1, 32, 29),     # windows wider than half a ring
+    small_workload("eq_many_heads_c16", 10, 32, 10, 32, EQ, EQ, 0.5, 3, 7, 16, 30),        # 21 independent slices
 ]
 
 
