@@ -27,7 +27,7 @@
  *     calls that run concurrently do not share a workspace (see sna_backward).
  *   - Accuracy: results are fp32; against an fp64 evaluation of the same formulas the normalised maximum
  *     error max|x - ref| / max|ref| per tensor is below 1e-5 for out and below 1e-4 for dq, dk, dv
- *     (measured 3e-6 and 2e-5).  No atomics are used: the same call on the same inputs gives the same bits.
+ *     (measured 2e-6 and 2e-5).  No atomics are used: the same call on the same inputs gives the same bits.
  */
 #ifndef SNA_H
 #define SNA_H

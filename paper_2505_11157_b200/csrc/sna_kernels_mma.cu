@@ -2,7 +2,8 @@
 // split of each operand, x = hi + lo with hi the top 11 significand bits.  A product a*b is two MMAs into one fp32
 // fragment: the main term a_hi*b_hi as m16n8k8 TF32, and both correction terms a_lo*b_hi + a_hi*b_lo as a single
 // m16n8k16 BF16 MMA whose 16 k-slots hold [a_lo | a_hi] against [b_hi ; b_lo] (the corrections are ~2^-11 of the
-// product, so 8 bits suffice).  Measured normalised errors: forward 2.5e-6..3.3e-6, backward <= 1.9e-5.
+// product, so 8 bits suffice).  The scores of the forward pass, whose errors the softmax amplifies, use three TF32
+// MMAs instead.  Measured normalised errors: forward ~1e-6, backward <= 2e-5.
 //
 // Work decomposition: one warp owns a tile of 16 points (the M dimension of the MMA: "tile rows") = 8 consecutive
 // longitudes on each of 2 adjacent rings, and walks the host-built column stream of that ring group, 16 partner
@@ -73,6 +74,61 @@ __device__ __forceinline__ void load_row(const float* p, float (&x)[CPT]) {
         x[4 * j] = a.x; x[4 * j + 1] = a.y; x[4 * j + 2] = a.z; x[4 * j + 3] = a.w;
     }
 }
+// ---------------------------------------------------------------------------------------------------------
+// Three-MMA product, all TF32: a*b = a_lo*b_hi + a_hi*b_lo + a_hi*b_hi with ~2^-21 relative precision.  Used for
+// the scores of the forward pass: softmax turns an absolute score error e into a relative weight error e*ln 2, so
+// peaked softmaxes (|s| of tens) need the scores at full fp32-level precision.
+// ---------------------------------------------------------------------------------------------------------
+__device__ __forceinline__ void mma_zero(float (&d)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
+    asm("mma.sync.aligned.m16n8k8.row.col.f32.tf32.tf32.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%10,%10,%10,%10};"
+        : "=f"(d[0]), "=f"(d[1]), "=f"(d[2]), "=f"(d[3])
+        : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1), "f"(0.f));
+}
+// Persistent A operand (tile rows g and g+8) from the row fragments of the two points, pre-multiplied by `mul`:
+// TF32 hi and lo quads per k-step, both rounded to nearest.
+template <int CPT>
+__device__ __forceinline__ void make_a_operand3(const float* p0, const float* p1, float mul, uint32_t (&hi)[CPT / 2][4], uint32_t (&lo)[CPT / 2][4]) {
+    float a[CPT], b[CPT];
+    load_row<CPT>(p0, a);
+    load_row<CPT>(p1, b);
+#pragma unroll
+    for (int ks = 0; ks < CPT / 2; ++ks) {
+        split_rn(a[2 * ks] * mul, hi[ks][0], lo[ks][0]);       // (row g,   k = t)
+        split_rn(b[2 * ks] * mul, hi[ks][1], lo[ks][1]);       // (row g+8, k = t)
+        split_rn(a[2 * ks + 1] * mul, hi[ks][2], lo[ks][2]);   // (row g,   k = t+4)
+        split_rn(b[2 * ks + 1] * mul, hi[ks][3], lo[ks][3]);   // (row g+8, k = t+4)
+    }
+}
+// d[tl] = A . B^T for the two 8-column tiles of a chunk; B = row fragment x[tl] of the point in column g of tile
+// tl, used raw as hi (the MMA truncates it) with lo = x - trunc19(x).  Corrections first, main terms last.
+template <int CPT>
+__device__ __forceinline__ void rows_dot_points3(float (&d)[2][4], const uint32_t (&ah)[CPT / 2][4], const uint32_t (&al)[CPT / 2][4], const float (&x)[2][CPT]) {
+    uint32_t bh[2][CPT], bl[2][CPT];
+#pragma unroll
+    for (int tl = 0; tl < 2; ++tl)
+#pragma unroll
+        for (int j = 0; j < CPT; ++j) {
+            bh[tl][j] = __float_as_uint(x[tl][j]);
+            bl[tl][j] = __float_as_uint(x[tl][j] - __uint_as_float(bh[tl][j] & 0xffffe000u));
+        }
+    mma_zero(d[0], al[0], bh[0][0], bh[0][1]);
+    mma_zero(d[1], al[0], bh[1][0], bh[1][1]);
+    mma_acc(d[0], ah[0], bl[0][0], bl[0][1]);
+    mma_acc(d[1], ah[0], bl[1][0], bl[1][1]);
+#pragma unroll
+    for (int ks = 1; ks < CPT / 2; ++ks) {
+        mma_acc(d[0], al[ks], bh[0][2 * ks], bh[0][2 * ks + 1]);
+        mma_acc(d[1], al[ks], bh[1][2 * ks], bh[1][2 * ks + 1]);
+        mma_acc(d[0], ah[ks], bl[0][2 * ks], bl[0][2 * ks + 1]);
+        mma_acc(d[1], ah[ks], bl[1][2 * ks], bl[1][2 * ks + 1]);
+    }
+#pragma unroll
+    for (int ks = 0; ks < CPT / 2; ++ks) {
+        mma_acc(d[0], ah[ks], bh[0][2 * ks], bh[0][2 * ks + 1]);
+        mma_acc(d[1], ah[ks], bh[1][2 * ks], bh[1][2 * ks + 1]);
+    }
+}
+
 // ---------------------------------------------------------------------------------------------------------
 // Two-MMA products: the main term a_hi*b_hi is one TF32 MMA and BOTH correction terms a_lo*b_hi + a_hi*b_lo are
 // one BF16 m16n8k16 MMA whose 16 k-slots hold [a_lo | a_hi] against [b_hi ; b_lo] for the same 8 channels.  The
@@ -362,7 +418,7 @@ forward_mma_kernel(DevPlan p, const float* __restrict__ q, const float* __restri
     const size_t pt1 = (size_t)(n * p.nlat_out + min(hg * TILE_LAT + 1, p.nlat_out - 1)) * p.nlon_out + wq;
 
     uint32_t qh[KS][4], ql[KS][4];   // q in the log2 domain
-    make_a_operand2<CPT>(q + pt0 * C + t * CPT, q + pt1 * C + t * CPT, scale_log2, qh, ql);   // ql: BF16 correction quads
+    make_a_operand3<CPT>(q + pt0 * C + t * CPT, q + pt1 * C + t * CPT, scale_log2, qh, ql);
     float o[KS][4];
 #pragma unroll
     for (int nt = 0; nt < KS; ++nt) o[nt][0] = o[nt][1] = o[nt][2] = o[nt][3] = 0.f;
@@ -378,7 +434,7 @@ forward_mma_kernel(DevPlan p, const float* __restrict__ q, const float* __restri
             float kr[2][CPT];
             lds_row<CPT>(st.a, g, t, kr[0]);
             lds_row<CPT>(st.a, 8 + g, t, kr[1]);
-            rows_dot_points2<CPT, true>(s, qh, ql, kr);
+            rows_dot_points3<CPT>(s, qh, ql, kr);   // scores at full precision (three TF32 MMAs per product)
         }
         float vr[2][2][KS];
 #pragma unroll

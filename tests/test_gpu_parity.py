@@ -140,6 +140,27 @@ def test_benchmark_configurations_sampled(name, n_out, n_in):
     assert np.max(np.abs(dk64.sum((1, 2)))) <= 1e-4 * np.max(np.abs(dk64).sum((1, 2)))
 
 
+@pytest.mark.parametrize("q_scale, v_scale", [(12.0, 1.0), (1e-3, 50.0)], ids=["peaked_softmax", "flat_softmax_large_v"])
+def test_extreme_score_magnitudes(q_scale, v_scale):
+    """Scores of +-60 (softmax dominated by one neighbor; exp() overflows without the running maximum) and
+    scores of ~1e-3 (flat softmax) with large values: no overflow, and the gates still hold."""
+    wl = small_workload("extreme", 20, 64, 20, 64, EQ, EQ, 0.4, 1, 2, 32, 31)
+    g = _geometry(wl)
+    q, k, v, dout = make_inputs(wl)
+    q = (q * q_scale).astype(np.float32)
+    v = (v * v_scale).astype(np.float32)
+    with _plan(wl) as plan:
+        out, lse, dq, dk, dv = _run_gpu(plan, q, k, v, dout, True)
+    for a in (out, lse, dq, dk, dv):
+        assert np.isfinite(a).all()
+    ref_out = orc.forward(g, q, k, v)
+    rdq, rdk, rdv = orc.backward(g, q, k, v, dout)
+    assert nerr(out.reshape(ref_out.shape), ref_out) <= FWD_TOL
+    assert nerr(dq.reshape(rdq.shape), rdq) <= BWD_TOL
+    assert nerr(dk.reshape(rdk.shape), rdk) <= BWD_TOL
+    assert nerr(dv.reshape(rdv.shape), rdv) <= BWD_TOL
+
+
 def test_global_limit_against_dense_oracle():
     wl = small_workload("global", 16, 32, 16, 32, EQ, EQ, math.pi, 1, 2, 32, 30)
     g = _geometry(wl)
