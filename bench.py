@@ -276,6 +276,7 @@ def run_ours(args, wl):
         dom_ms, dom_flops_per_unit = kernels[dominant]
         achieved = dom_flops_per_unit * units / (dom_ms * 1e-3) / 1e12
         traffic = NCU_DRAM_BYTES_PER_LAUNCH.get((wl.name, dominant))
+        peak_measured = sna.sna_measure_fp32_fma_peak()   # pure-FMA loop on this device, TFLOP/s
         ms_step = ms_total_max / args.steps
         roof_fwd_ms = 4.0 * units / (peak_tflops * 1e12) * 1e3
         roof_bwd_ms = 10.0 * units / (peak_tflops * 1e12) * 1e3
@@ -287,6 +288,8 @@ def run_ours(args, wl):
             "ms_forward": ms_fwd, "ms_backward": ms_dq + ms_dkdv, "ms_backward_dq": ms_dq, "ms_backward_dkdv": ms_dkdv,
             "pairs_per_step": pairs,
             "roofline_step": {"bound": "alu", "roofline_ms": roof_fwd_ms + roof_bwd_ms, "frac": (roof_fwd_ms + roof_bwd_ms) / ms_step,
+                              "peak_derived_tflops": peak_tflops, "peak_fma_measured_tflops": peak_measured,
+                              "frac_of_measured_peak": (roof_fwd_ms + roof_bwd_ms) * (peak_tflops / peak_measured) / ms_step,
                               "note": "algorithmic flops (4C fwd + 10C bwd per pair) at the FP32 FMA peak of measured-max clock"},
             "roofline": {"bound": "alu", "kernel": dominant, "achieved": achieved, "peak": peak_tflops, "unit": "TFLOP/s",
                          "frac": achieved / peak_tflops, "traffic": traffic,

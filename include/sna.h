@@ -192,6 +192,14 @@ sna_status_t sna_backward_static(const sna_plan_t* plan, const float* q, const f
                                  const float* dout, float* dq, float* dk, float* dv,
                                  int B, int H, int C, void* cuda_stream);
 
+/*
+ * Measurement aid (the paper has no counterpart): runs a pure FP32 fused-multiply-add loop on every SM of the
+ * current device and returns the sustained rate in TFLOP/s (2 flops per FMA) in *tflops (host).  It is the
+ * denominator check for the roofline, which is stated against the FP32 FMA peak (SMs x 128 lanes x 2 x clock).
+ * Blocks until the probe has finished (about a millisecond); allocates a few KB of device memory for its result.
+ */
+sna_status_t sna_measure_fp32_fma_peak(double* tflops);
+
 /* Human-readable name of a status code (static string). */
 const char* sna_status_string(sna_status_t status);
 /* Detail of the most recent failure on the calling thread (static thread-local buffer; "" if none). */

@@ -56,6 +56,7 @@ _SIGNATURES = {
     "sna_backward_dq": (_i, [_vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _i, _i, _i, _vp]),
     "sna_backward_dkdv": (_i, [_vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _i, _i, _i, _vp]),
     "sna_backward_static": (_i, [_vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _i, _i, _i, _vp]),
+    "sna_measure_fp32_fma_peak": (_i, [ctypes.POINTER(ctypes.c_double)]),
     "sna_status_string": (ctypes.c_char_p, [_i]),
     "sna_last_error_message": (ctypes.c_char_p, []),
 }
@@ -164,6 +165,13 @@ def sna_backward_static(plan, q, k, v, dout, dq, dk, dv, B, H, C, stream=None):
     overlaps share that array and must be serialised."""
     _check(_lib.sna_backward_static(plan, _ptr(q), _ptr(k), _ptr(v), _ptr(dout), _ptr(dq), _ptr(dk), _ptr(dv),
                                     B, H, C, _stream(stream)))
+
+
+def sna_measure_fp32_fma_peak() -> float:
+    """Sustained FP32 FMA rate of the current device in TFLOP/s (a pure-FMA loop on every SM)."""
+    t = ctypes.c_double()
+    _check(_lib.sna_measure_fp32_fma_peak(ctypes.byref(t)))
+    return t.value
 
 
 # ---- convenience wrapper -----------------------------------------------------------------------------------

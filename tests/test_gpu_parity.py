@@ -218,6 +218,13 @@ def test_argument_errors_launch_nothing():
         torch.cuda.synchronize()
 
 
+def test_fp32_fma_peak_probe_is_plausible():
+    props = torch.cuda.get_device_properties(0)
+    nominal = props.multi_processor_count * 128 * 2 * 1.965e9 / 1e12      # B200: 148 SMs -> 74.4 TFLOP/s
+    measured = sna.sna_measure_fp32_fma_peak()
+    assert 0.5 * nominal < measured < 1.1 * nominal
+
+
 def test_runs_on_a_side_stream():
     wl = SMALL[0]
     g = _geometry(wl)
