@@ -36,7 +36,7 @@ import numpy as np  # noqa: E402
 # dram__bytes_read.sum + dram__bytes_write.sum per launch from the ncu capture summarised in
 # profiles/mma_kernels_c3_counters.md (bench.py cannot run ncu itself)
 NCU_DRAM_BYTES_PER_LAUNCH = {
-    ("c3", "forward"): 816557312 + 63465472,
+    ("c3", "forward"): 816768768 + 63346432,
     ("c3", "backward_dq"): 980778752 + 66266112,
     ("c3", "backward_dkdv"): 715740160 + 502913024,
 }
