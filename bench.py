@@ -49,7 +49,7 @@ FP32_LANES_PER_SM = 128
 def parse_args():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=30)
+    ap.add_argument("--steps", type=int, default=100)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--workload", default="c3")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
@@ -237,7 +237,6 @@ def run_ours(args, wl):
         marks[i][3].record(stream)
     t_end.record(stream)
     barrier()
-    clocks = sampler.stop() if rank == 0 else None
     ms_total = t_start.elapsed_time(t_end)
     ms_fwd = statistics.mean(m[0].elapsed_time(m[1]) for m in marks)
     ms_dq = statistics.mean(m[1].elapsed_time(m[2]) for m in marks)
@@ -260,6 +259,7 @@ def run_ours(args, wl):
     e1.record(stream)
     barrier()
     ms_e2e = e0.elapsed_time(e1)
+    clocks = sampler.stop() if rank == 0 else None   # sampled over the device-resident and the end-to-end timed regions
     h2d = sum(h.numel() * 4 for h in host)
     d2h = sum(h.numel() * 4 for h in host_out)
 
