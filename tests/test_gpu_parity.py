@@ -225,6 +225,24 @@ def test_fp32_fma_peak_probe_is_plausible():
     assert 0.5 * nominal < measured < 1.1 * nominal
 
 
+def test_autograd_wrapper_matches_oracle_gradients():
+    from paper_2505_11157_b200.autograd import spherical_neighborhood_attention
+    wl = SMALL[2]
+    g = _geometry(wl)
+    q, k, v, dout = make_inputs(wl)
+    with _plan(wl) as plan:
+        qd, kd, vd, dd = _dev(q, k, v, dout)
+        for t in (qd, kd, vd):
+            t.requires_grad_(True)
+        out = spherical_neighborhood_attention(plan, qd, kd, vd)
+        (out * dd).sum().backward()
+        torch.cuda.synchronize()
+        got = [t.grad.cpu().numpy() for t in (qd, kd, vd)]
+    refs = orc.backward(g, q, k, v, dout)
+    for x, r in zip(got, refs):
+        assert nerr(x.reshape(r.shape), r) <= BWD_TOL
+
+
 def test_runs_on_a_side_stream():
     wl = SMALL[0]
     g = _geometry(wl)
