@@ -90,6 +90,11 @@ sna_status_t sna_plan_create_host_only(int nlat_in, int nlon_in, int nlat_out, i
 /* Free the plan's host and device memory (including a workspace it may have grown).  NULL is accepted. */
 sna_status_t sna_plan_destroy(sna_plan_t* plan);
 
+/* Waits for the plan's device to finish and reports whether any kernel launched through this plan gave up on one of
+ * its bounded waits (SNA_ERR_CUDA; its outputs would be incomplete).  Kernels never spin without limit; this is the
+ * way to find out that a limit was hit.  Not expected to happen. */
+sna_status_t sna_plan_check(const sna_plan_t* plan);
+
 /* ---- introspection into caller-owned HOST buffers ------------------------------------------------------ */
 
 /* Number of (lat_in, lon_off) entries in the table. */

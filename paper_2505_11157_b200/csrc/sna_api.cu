@@ -127,12 +127,21 @@ static sna_status_t plan_create(int nlat_in, int nlon_in, int nlat_out, int nlon
     std::vector<float> log2_omega(hp.nlat_in);
     for (int h = 0; h < hp.nlat_in; ++h) log2_omega[h] = (float)std::log2(hp.omega[h]);
 
-    sna::Stream fwd_stream, t_stream;
-    std::vector<int32_t> grp_order, t_grp_order;
+    sna::Stream fwd_stream, t_stream, fwdb_stream;
+    sna::DenseLists dense;
+    std::vector<int32_t> grp_order, t_grp_order, grpb_order;
+    const int32_t zero_status[64] = {};
     bool t_consecutive = false;
     try {
         sna::build_forward_stream(hp, fwd_stream);
         t_consecutive = sna::build_transposed_stream(hp, t_stream);
+        sna::build_dense_lists(hp, dense);
+        sna::build_forward_stream(hp, fwdb_stream, /*include_whole=*/false);
+        grpb_order.resize(fwdb_stream.chunk_ptr.size() - 1);
+        std::iota(grpb_order.begin(), grpb_order.end(), 0);
+        std::stable_sort(grpb_order.begin(), grpb_order.end(), [&](int a, int b) {
+            return fwdb_stream.chunk_ptr[a + 1] - fwdb_stream.chunk_ptr[a] > fwdb_stream.chunk_ptr[b + 1] - fwdb_stream.chunk_ptr[b];
+        });
         // heavy-first orders of the ring groups (by stream length; for the transposed stream summed over residues)
         grp_order.resize(fwd_stream.chunk_ptr.size() - 1);
         std::iota(grp_order.begin(), grp_order.end(), 0);
@@ -161,7 +170,10 @@ static sna_status_t plan_create(int nlat_in, int nlon_in, int nlat_out, int nlon
         {t_m.data(), t_m.size() * 4, 0}, {t_row_order.data(), t_row_order.size() * 4, 0}, {log2_omega.data(), log2_omega.size() * 4, 0},
         {fwd_stream.entries.data(), fwd_stream.entries.size() * 16, 0}, {fwd_stream.chunk_ptr.data(), fwd_stream.chunk_ptr.size() * 4, 0},
         {t_stream.entries.data(), t_stream.entries.size() * 16, 0}, {t_stream.chunk_ptr.data(), t_stream.chunk_ptr.size() * 4, 0},
-        {grp_order.data(), grp_order.size() * 4, 0}, {t_grp_order.data(), t_grp_order.size() * 4, 0}};
+        {grp_order.data(), grp_order.size() * 4, 0}, {t_grp_order.data(), t_grp_order.size() * 4, 0},
+        {fwdb_stream.entries.data(), fwdb_stream.entries.size() * 16, 0}, {fwdb_stream.chunk_ptr.data(), fwdb_stream.chunk_ptr.size() * 4, 0},
+        {grpb_order.data(), grpb_order.size() * 4, 0}, {dense.ptr.data(), dense.ptr.size() * 4, 0},
+        {dense.lat.data(), dense.lat.size() * 4, 0}, {dense.rows.data(), dense.rows.size() * 4, 0}, {zero_status, sizeof(zero_status), 0}};
     size_t total = 0;
     for (Piece& p : pieces) { p.offset = total; total += round256(p.bytes); }
     cudaError_t e = cudaGetDevice(&plan->device);
@@ -169,6 +181,7 @@ static sna_status_t plan_create(int nlat_in, int nlon_in, int nlat_out, int nlon
     e = cudaMalloc(&plan->dev_blob, total);
     if (e != cudaSuccess) { delete plan; set_error("cudaMalloc of %zu bytes: %s", total, cudaGetErrorString(e)); return SNA_ERR_ALLOC; }
     for (const Piece& p : pieces) {
+        if (p.bytes == 0) continue;
         e = cudaMemcpy((char*)plan->dev_blob + p.offset, p.src, p.bytes, cudaMemcpyHostToDevice);
         if (e != cudaSuccess) { cudaFree(plan->dev_blob); delete plan; return cuda_fail(e, "cudaMemcpy of plan tables"); }
     }
@@ -182,6 +195,10 @@ static sna_status_t plan_create(int nlat_in, int nlon_in, int nlat_out, int nlon
     d.t_stream = (const int4*)at(11); d.t_chunk_ptr = at(12);
     d.grp_order = at(13); d.t_grp_order = at(14);
     d.t_consecutive = t_consecutive ? 1 : 0;
+    d.fwdb_stream = (const int4*)at(15); d.fwdb_chunk_ptr = at(16); d.grpb_order = at(17);
+    d.dense_ptr = at(18); d.dense_lat = at(19); d.dense_rows = at(20);
+    d.n_dense_rows = (int)dense.rows.size();
+    d.dev_status = (int*)((char*)plan->dev_blob + pieces[21].offset);
     *plan_out = plan;
     return SNA_OK;
 }
@@ -203,6 +220,18 @@ sna_status_t sna_plan_destroy(sna_plan_t* plan) {
     delete plan;
     if (e1 != cudaSuccess) return cuda_fail(e1, "cudaFree");
     if (e2 != cudaSuccess) return cuda_fail(e2, "cudaFree");
+    return SNA_OK;
+}
+
+sna_status_t sna_plan_check(const sna_plan_t* plan) {
+    if (!plan) { set_error("plan is NULL"); return SNA_ERR_INVALID_ARG; }
+    if (plan->dev_blob == nullptr) return SNA_OK;
+    cudaError_t e = cudaDeviceSynchronize();
+    if (e != cudaSuccess) return cuda_fail(e, "cudaDeviceSynchronize");
+    int status = 0;
+    e = cudaMemcpy(&status, plan->dev.dev_status, sizeof(int), cudaMemcpyDeviceToHost);
+    if (e != cudaSuccess) return cuda_fail(e, "cudaMemcpy of the device status word");
+    if (status != 0) { set_error("a kernel gave up on a bounded wait; its outputs are incomplete"); return SNA_ERR_CUDA; }
     return SNA_OK;
 }
 
@@ -279,9 +308,16 @@ sna_status_t sna_forward_ex(const sna_plan_t* plan, const float* q, const float*
     if (st != SNA_OK) return st;
     if (!q || !k || !v || !out) { set_error("q, k, v and out must not be NULL"); return SNA_ERR_INVALID_ARG; }
     if (!all_aligned(q, k, v, out) || (reinterpret_cast<uintptr_t>(lse) & 3u)) { set_error("device pointers must be 16-byte aligned"); return SNA_ERR_INVALID_ARG; }
-    cudaError_t e = sna::mma_path_supported(plan->dev, C)
-                        ? sna::launch_forward_mma(plan->dev, q, k, v, out, lse, B * H, C, (cudaStream_t)cuda_stream)
-                        : sna::launch_forward_generic(plan->dev, q, k, v, out, lse, B * H, C, (cudaStream_t)cuda_stream);
+    cudaError_t e;
+    if (lse != nullptr && sna::dense_path_supported(plan->dev, C)) {
+        // whole-ring windows on the tcgen05 kernel (its partial result travels in out / lse), the rest on the band kernel
+        e = sna::launch_forward_dense(plan->dev, q, k, v, out, lse, B * H, C, (cudaStream_t)cuda_stream);
+        if (e == cudaSuccess) e = sna::launch_forward_mma_band(plan->dev, q, k, v, out, lse, B * H, C, (cudaStream_t)cuda_stream);
+    } else if (sna::mma_path_supported(plan->dev, C)) {
+        e = sna::launch_forward_mma(plan->dev, q, k, v, out, lse, B * H, C, (cudaStream_t)cuda_stream);
+    } else {
+        e = sna::launch_forward_generic(plan->dev, q, k, v, out, lse, B * H, C, (cudaStream_t)cuda_stream);
+    }
     if (e != cudaSuccess) return cuda_fail(e, "forward launch");
     return SNA_OK;
 }

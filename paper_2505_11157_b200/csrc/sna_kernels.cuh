@@ -23,6 +23,15 @@ struct DevPlan {
     const int4* fwd_stream;         // 16 entries per chunk: {base|abs flag, e | mask<<16, bias, aux}
     const int32_t* fwd_chunk_ptr;   // [groups of output latitudes + 1]
     const int32_t* grp_order;       // groups of output latitudes, longest stream first
+    // band-only forward stream (whole-ring windows left to the dense kernel) and the dense kernel's lists
+    const int4* fwdb_stream;
+    const int32_t* fwdb_chunk_ptr;
+    const int32_t* grpb_order;
+    const int32_t* dense_ptr;       // [nlat_out+1] whole-ring windows per output latitude
+    const int32_t* dense_lat;       // their input rings
+    const int32_t* dense_rows;      // output latitudes with at least one whole-ring window
+    int n_dense_rows;
+    int* dev_status;                // set to non-zero by a kernel whose bounded wait ran out
     const int4* t_stream;
     const int32_t* t_chunk_ptr;     // [groups of input latitudes * ps + 1]
     const int32_t* t_grp_order;     // groups of input latitudes, longest stream first
@@ -33,6 +42,14 @@ struct DevPlan {
 bool mma_path_supported(const DevPlan& p, int C);
 cudaError_t launch_forward_mma(const DevPlan& p, const float* q, const float* k, const float* v, float* out, float* lse,
                                int N, int C, cudaStream_t stream);
+// Dense (tcgen05) forward over the whole-ring windows only: writes the partial result (normalised out, lse) of the
+// output latitudes in p.dense_rows; launch_forward_mma_band then continues from it with the banded windows.
+// Both need lse != null.  dense_path_supported tells whether the pair may be used for this problem.
+bool dense_path_supported(const DevPlan& p, int C);
+cudaError_t launch_forward_dense(const DevPlan& p, const float* q, const float* k, const float* v, float* out, float* lse,
+                                 int N, int C, cudaStream_t stream);
+cudaError_t launch_forward_mma_band(const DevPlan& p, const float* q, const float* k, const float* v, float* out, float* lse,
+                                    int N, int C, cudaStream_t stream);
 // out is required (D_i = dout_i . out_i); out and dq may be the same buffer.
 cudaError_t launch_backward_dq_mma(const DevPlan& p, const float* q, const float* k, const float* v, const float* dout,
                                    const float* out, const float* lse, float* dq, float* Dws, int N, int C, cudaStream_t stream);

@@ -1,0 +1,291 @@
+// Dense forward kernel for whole-ring windows on the 5th-generation tensor cores (tcgen05 / TMEM), sm_100a.
+//
+// Near the poles, and in the global limit theta_cutoff = pi, an output ring attends to EVERY point of an input
+// ring.  That part of Eq. (s2_attention_discrete_detailed) is an ordinary dense attention block, so it runs as
+// UMMA GEMMs: one CTA owns 128 consecutive output longitudes of one ring (the M = 128 rows of the MMA), walks the
+// ring's whole input rings in blocks of 64 columns, and for every block
+//   1. splits the k and v rows into hi = top 11 significand bits and lo = remainder and writes them to shared
+//      memory in the K-major 128-byte-swizzle layout (v transposed, so that the columns are its K dimension),
+//   2. S = Q K^T as three TF32 UMMAs per k-step (q_lo k_hi + q_hi k_lo + q_hi k_hi) into TMEM,
+//   3. reads its row of S from TMEM (thread r owns tile row r), does the online softmax in registers and writes
+//      P_hi and P_lo back to TMEM,
+//   4. O_block = P V with the A operand taken from TMEM, again three UMMAs per k-step,
+//   5. folds O_block into fp32 register accumulators (the tensor core's accumulate truncates, so chains stay short).
+// The result (normalised out and lse of the dense part) is the initial state of the band kernel.
+// Every wait on an mbarrier is bounded; a wait that runs out sets the plan's device status word and the CTA leaves.
+#include "sna_kernels.cuh"
+
+#include <cstdint>
+
+namespace sna {
+namespace {
+
+constexpr int DM = 128;        // tile rows (output longitudes)
+constexpr int DBN = 64;        // columns per block
+constexpr int DC = 32;         // channels
+constexpr int TMEM_COLS = 256; // S 64 | P_hi 64 | P_lo 64 | O 32 (power of two allocation)
+constexpr size_t DENSE_SMEM = 100 * 1024;   // 64 KB of tiles + alignment; sized so that two CTAs share an SM (and its 512 TMEM columns)
+constexpr float LOG2E_D = 1.4426950408889634f;
+constexpr float LN2_D = 0.6931471805599453f;
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ float ex2d(float x) { float y; asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x)); return y; }
+
+// Shared-memory matrix descriptor, K-major, 128-byte swizzle: rows of 128 bytes, 8-row groups 1024 bytes apart.
+__device__ __forceinline__ uint64_t umma_desc(uint32_t saddr) {
+    return (uint64_t)((saddr >> 4) & 0x3fff) | ((uint64_t)1 << 16) | ((uint64_t)(1024 >> 4) << 32) | ((uint64_t)1 << 46) | ((uint64_t)2 << 61);
+}
+// Instruction descriptor: fp32 accumulator, TF32 operands, both K-major, M = 128, N = n.
+__device__ __forceinline__ uint32_t umma_idesc(int n) {
+    return (1u << 4) | (2u << 7) | (2u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(DM >> 4) << 24);
+}
+__device__ __forceinline__ void umma_ss(uint32_t d, uint64_t a, uint64_t b, uint32_t idesc, uint32_t acc) {
+    asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\ttcgen05.mma.cta_group::1.kind::tf32 [%0], %1, %2, %3, {%5, %5, %5, %5}, p;\n\t}\n"
+                 ::"r"(d), "l"(a), "l"(b), "r"(idesc), "r"(acc), "r"(0u));
+}
+__device__ __forceinline__ void umma_ts(uint32_t d, uint32_t a_tmem, uint64_t b, uint32_t idesc, uint32_t acc) {
+    asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\ttcgen05.mma.cta_group::1.kind::tf32 [%0], [%1], %2, %3, {%5, %5, %5, %5}, p;\n\t}\n"
+                 ::"r"(d), "r"(a_tmem), "l"(b), "r"(idesc), "r"(acc), "r"(0u));
+}
+__device__ __forceinline__ void umma_commit(uint32_t bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ bool wait_bar(uint32_t bar, uint32_t parity) {
+    uint32_t done = 0;
+    for (int it = 0; it < (1 << 20) && !done; ++it)
+        asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}\n"
+                     : "=r"(done) : "r"(bar), "r"(parity) : "memory");
+    return done != 0;
+}
+__device__ __forceinline__ void tmem_ld32(uint32_t (&r)[32], uint32_t addr) {
+    asm volatile("tcgen05.ld.sync.aligned.32x32b.x32.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
+        : "=r"(r[0]),"=r"(r[1]),"=r"(r[2]),"=r"(r[3]),"=r"(r[4]),"=r"(r[5]),"=r"(r[6]),"=r"(r[7]),"=r"(r[8]),"=r"(r[9]),"=r"(r[10]),"=r"(r[11]),"=r"(r[12]),"=r"(r[13]),"=r"(r[14]),"=r"(r[15]),
+          "=r"(r[16]),"=r"(r[17]),"=r"(r[18]),"=r"(r[19]),"=r"(r[20]),"=r"(r[21]),"=r"(r[22]),"=r"(r[23]),"=r"(r[24]),"=r"(r[25]),"=r"(r[26]),"=r"(r[27]),"=r"(r[28]),"=r"(r[29]),"=r"(r[30]),"=r"(r[31]) : "r"(addr));
+    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_st32(uint32_t addr, const uint32_t (&r)[32]) {
+    asm volatile("tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31,%32};"
+        :: "r"(addr), "r"(r[0]),"r"(r[1]),"r"(r[2]),"r"(r[3]),"r"(r[4]),"r"(r[5]),"r"(r[6]),"r"(r[7]),"r"(r[8]),"r"(r[9]),"r"(r[10]),"r"(r[11]),"r"(r[12]),"r"(r[13]),"r"(r[14]),"r"(r[15]),
+           "r"(r[16]),"r"(r[17]),"r"(r[18]),"r"(r[19]),"r"(r[20]),"r"(r[21]),"r"(r[22]),"r"(r[23]),"r"(r[24]),"r"(r[25]),"r"(r[26]),"r"(r[27]),"r"(r[28]),"r"(r[29]),"r"(r[30]),"r"(r[31]) : "memory");
+}
+// Byte offset of the 16-byte chunk c4 of row r inside a [rows x 128 B] swizzled block.
+__device__ __forceinline__ int sw_chunk(int r, int c4) { return r * 128 + ((c4 ^ (r & 7)) << 4); }
+
+__global__ void __launch_bounds__(DM)
+forward_dense_kernel(DevPlan p, const float* __restrict__ q, const float* __restrict__ k, const float* __restrict__ v,
+                     float* __restrict__ out, float* __restrict__ lse, int N, float scale_log2, int blocks_per_row) {
+    extern __shared__ unsigned char dense_raw[];
+    unsigned char* base = (unsigned char*)(((uintptr_t)dense_raw + 1023) & ~(uintptr_t)1023);
+    unsigned char *sQh = base, *sQl = base + 16384, *sKh = base + 32768, *sKl = base + 40960, *sVh = base + 49152, *sVl = base + 57344;
+    __shared__ uint64_t mbar;
+    __shared__ uint32_t tmem_base;
+    const int tid = threadIdx.x, warp = tid >> 5;
+    const int lb = blockIdx.x % blocks_per_row;
+    const int rest = blockIdx.x / blocks_per_row;
+    const int n = rest % N;
+    const int h = p.dense_rows[rest / N];
+    const int w = lb * DM + tid;
+    const bool row_ok = w < p.nlon_out;
+    const size_t opt = (size_t)(n * p.nlat_out + h) * p.nlon_out + min(w, p.nlon_out - 1);
+
+    {   // this thread's q row, in the log2 domain, split and stored as tile row tid
+        const float4* src = reinterpret_cast<const float4*>(q + opt * DC);
+#pragma unroll
+        for (int c4 = 0; c4 < DC / 4; ++c4) {
+            float4 x = __ldg(src + c4);
+            x.x *= scale_log2; x.y *= scale_log2; x.z *= scale_log2; x.w *= scale_log2;
+            float4 hi;
+            hi.x = __uint_as_float(__float_as_uint(x.x) & 0xffffe000u); hi.y = __uint_as_float(__float_as_uint(x.y) & 0xffffe000u);
+            hi.z = __uint_as_float(__float_as_uint(x.z) & 0xffffe000u); hi.w = __uint_as_float(__float_as_uint(x.w) & 0xffffe000u);
+            *reinterpret_cast<float4*>(sQh + sw_chunk(tid, c4)) = hi;
+            *reinterpret_cast<float4*>(sQl + sw_chunk(tid, c4)) = make_float4(x.x - hi.x, x.y - hi.y, x.z - hi.z, x.w - hi.w);
+        }
+    }
+    if (tid == 0) {
+        asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(smem_u32(&mbar)));
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 0) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base)), "r"(TMEM_COLS));
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::);
+    }
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    const uint32_t tm = tmem_base, lanebits = (uint32_t)(warp * 32) << 16;
+    const uint32_t tS = tm, tPh = tm + 64, tPl = tm + 128, tO = tm + 192;
+    const uint32_t idS = umma_idesc(DBN), idO = umma_idesc(DC), bar = smem_u32(&mbar);
+    uint32_t phase = 0;
+    bool ok = true;
+    float m = -INFINITY, l = 0.f, o[DC];
+#pragma unroll
+    for (int i = 0; i < DC; ++i) o[i] = 0.f;
+
+    const int col = tid >> 1, half = tid & 1;      // this thread's share of a 64-column block: one column, 16 channels
+    const int nblk = (p.nlon_in + DBN - 1) / DBN;
+    const int e_begin = p.dense_ptr[h], e_end = p.dense_ptr[h + 1];
+    const int total = (e_end - e_begin) * nblk;    // blocks of this tile, over all its whole input rings
+    // raw k / v rows of the next block travel in registers while the current block's MMAs and softmax run
+    float4 kraw[4], vraw[4];
+    auto fetch = [&](int it) {
+        const int hp = p.dense_lat[e_begin + it / nblk];
+        const size_t pt = ((size_t)(n * p.nlat_in + hp) * p.nlon_in + min((it % nblk) * DBN + col, p.nlon_in - 1)) * DC + half * 16;
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            kraw[j] = __ldg(reinterpret_cast<const float4*>(k + pt) + j);
+            vraw[j] = __ldg(reinterpret_cast<const float4*>(v + pt) + j);
+        }
+    };
+    if (total > 0) fetch(0);
+    for (int it = 0; it < total && ok; ++it) {
+        const float bias = p.log2_omega[p.dense_lat[e_begin + it / nblk]];
+        {
+            const int c0 = (it % nblk) * DBN;
+            {   // split this block's k rows, and v rows transposed (row = channel, K index = column)
+                const int kb = col >> 5, kc = col & 31;
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    const float4 x = kraw[j];
+                    float4 hi;
+                    hi.x = __uint_as_float(__float_as_uint(x.x) & 0xffffe000u); hi.y = __uint_as_float(__float_as_uint(x.y) & 0xffffe000u);
+                    hi.z = __uint_as_float(__float_as_uint(x.z) & 0xffffe000u); hi.w = __uint_as_float(__float_as_uint(x.w) & 0xffffe000u);
+                    *reinterpret_cast<float4*>(sKh + sw_chunk(col, half * 4 + j)) = hi;
+                    *reinterpret_cast<float4*>(sKl + sw_chunk(col, half * 4 + j)) = make_float4(x.x - hi.x, x.y - hi.y, x.z - hi.z, x.w - hi.w);
+                    const float4 y = vraw[j];
+                    const float yv[4] = {y.x, y.y, y.z, y.w};
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) {
+                        const int ch = half * 16 + 4 * j + i;
+                        const int off = kb * (DC * 128) + sw_chunk(ch, kc >> 2) + (kc & 3) * 4;
+                        const float g = __uint_as_float(__float_as_uint(yv[i]) & 0xffffe000u);
+                        *reinterpret_cast<float*>(sVh + off) = g;
+                        *reinterpret_cast<float*>(sVl + off) = yv[i] - g;
+                    }
+                }
+            }
+            if (it + 1 < total) fetch(it + 1);
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+            asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+            __syncthreads();
+            if (tid == 0) {
+                asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                const uint64_t qh = umma_desc(smem_u32(sQh)), ql = umma_desc(smem_u32(sQl)), kh = umma_desc(smem_u32(sKh)), kl = umma_desc(smem_u32(sKl));
+#pragma unroll
+                for (int ks2 = 0; ks2 < DC / 8; ++ks2) umma_ss(tS, ql + 2 * ks2, kh + 2 * ks2, idS, ks2 > 0);
+#pragma unroll
+                for (int ks2 = 0; ks2 < DC / 8; ++ks2) umma_ss(tS, qh + 2 * ks2, kl + 2 * ks2, idS, 1);
+#pragma unroll
+                for (int ks2 = 0; ks2 < DC / 8; ++ks2) umma_ss(tS, qh + 2 * ks2, kh + 2 * ks2, idS, 1);
+                umma_commit(bar);
+            }
+            ok = wait_bar(bar, phase);
+            phase ^= 1;
+            asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+            float corr = 1.f;
+            if (ok) {
+                uint32_t s0[32], s1[32], lo[32];
+                tmem_ld32(s0, tS + lanebits);
+                tmem_ld32(s1, tS + lanebits + 32);
+                const int nvalid = p.nlon_in - c0;   // columns of this block that exist (>= 64 except in the last block)
+                float mx = m;
+                if (nvalid >= DBN) {
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) {
+                        const float a = __uint_as_float(s0[j]) + bias, b = __uint_as_float(s1[j]) + bias;
+                        s0[j] = __float_as_uint(a); s1[j] = __float_as_uint(b);
+                        mx = fmaxf(mx, fmaxf(a, b));
+                    }
+                } else {
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) {
+                        const float a = j < nvalid ? __uint_as_float(s0[j]) + bias : -INFINITY;
+                        const float b = j + 32 < nvalid ? __uint_as_float(s1[j]) + bias : -INFINITY;
+                        s0[j] = __float_as_uint(a); s1[j] = __float_as_uint(b);
+                        mx = fmaxf(mx, fmaxf(a, b));
+                    }
+                }
+                corr = ex2d(m - mx);
+                m = mx;
+                float ps = 0.f;
+#pragma unroll
+                for (int j = 0; j < 32; ++j) {
+                    const float pj = ex2d(__uint_as_float(s0[j]) - m);
+                    ps += pj;
+                    s0[j] = __float_as_uint(pj);
+                    lo[j] = __float_as_uint(pj - __uint_as_float(s0[j] & 0xffffe000u));
+                }
+                tmem_st32(tPh + lanebits, s0);
+                tmem_st32(tPl + lanebits, lo);
+#pragma unroll
+                for (int j = 0; j < 32; ++j) {
+                    const float pj = ex2d(__uint_as_float(s1[j]) - m);
+                    ps += pj;
+                    s1[j] = __float_as_uint(pj);
+                    lo[j] = __float_as_uint(pj - __uint_as_float(s1[j] & 0xffffe000u));
+                }
+                tmem_st32(tPh + lanebits + 32, s1);
+                tmem_st32(tPl + lanebits + 32, lo);
+                asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
+                l = l * corr + ps;
+            }
+            asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+            __syncthreads();
+            if (tid == 0 && ok) {
+                asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                const uint64_t vh0 = umma_desc(smem_u32(sVh)), vl0 = umma_desc(smem_u32(sVl));
+#pragma unroll
+                for (int ks2 = 0; ks2 < DBN / 8; ++ks2) umma_ts(tO, tPl + ks2 * 8, vh0 + (uint64_t)((ks2 >> 2) * (DC * 128 >> 4) + (ks2 & 3) * 2), idO, ks2 > 0);
+#pragma unroll
+                for (int ks2 = 0; ks2 < DBN / 8; ++ks2) umma_ts(tO, tPh + ks2 * 8, vl0 + (uint64_t)((ks2 >> 2) * (DC * 128 >> 4) + (ks2 & 3) * 2), idO, 1);
+#pragma unroll
+                for (int ks2 = 0; ks2 < DBN / 8; ++ks2) umma_ts(tO, tPh + ks2 * 8, vh0 + (uint64_t)((ks2 >> 2) * (DC * 128 >> 4) + (ks2 & 3) * 2), idO, 1);
+                umma_commit(bar);
+            }
+            if (ok) {
+                ok = wait_bar(bar, phase);
+                phase ^= 1;
+            }
+            asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+            if (ok) {
+                uint32_t ob[32];
+                tmem_ld32(ob, tO + lanebits);
+#pragma unroll
+                for (int j = 0; j < DC; ++j) o[j] = fmaf(o[j], corr, __uint_as_float(ob[j]));
+            }
+            asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+            __syncthreads();   // the tiles and the TMEM blocks are free for the next block
+        }
+    }
+    if (!ok && tid == 0) atomicExch(p.dev_status, 1);
+    if (ok && row_ok) {
+        const float inv = 1.f / l;
+        float4* dst = reinterpret_cast<float4*>(out + opt * DC);
+#pragma unroll
+        for (int c4 = 0; c4 < DC / 4; ++c4) dst[c4] = make_float4(o[4 * c4] * inv, o[4 * c4 + 1] * inv, o[4 * c4 + 2] * inv, o[4 * c4 + 3] * inv);
+        lse[opt] = (m + log2f(l)) * LN2_D;
+    }
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    if (warp == 0) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tm), "r"(TMEM_COLS));
+}
+
+}  // namespace
+
+bool dense_path_supported(const DevPlan& p, int C) {
+    return C == DC && p.dense_ptr != nullptr && p.n_dense_rows > 0 && p.fwdb_stream != nullptr && mma_path_supported(p, C);
+}
+
+cudaError_t launch_forward_dense(const DevPlan& p, const float* q, const float* k, const float* v, float* out, float* lse,
+                                 int N, int C, cudaStream_t stream) {
+    if (C != DC || lse == nullptr) return cudaErrorInvalidValue;
+    const int blocks_per_row = (p.nlon_out + DM - 1) / DM;
+    const long long blocks = (long long)blocks_per_row * p.n_dense_rows * N;
+    if (blocks <= 0) return cudaSuccess;
+    if (blocks > 0x7fffffffLL) return cudaErrorInvalidValue;
+    cudaError_t e = cudaFuncSetAttribute(forward_dense_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)DENSE_SMEM);
+    if (e != cudaSuccess) return e;
+    forward_dense_kernel<<<(unsigned)blocks, DM, DENSE_SMEM, stream>>>(p, q, k, v, out, lse, N, LOG2E_D / sqrtf((float)C), blocks_per_row);
+    return cudaGetLastError();
+}
+
+}  // namespace sna

@@ -396,13 +396,22 @@ __device__ __forceinline__ void store_row(float* p, const float (&x)[CPT]) {
     for (int j = 0; j < CPT / 4; ++j) *reinterpret_cast<float4*>(p + 4 * j) = make_float4(x[4 * j], x[4 * j + 1], x[4 * j + 2], x[4 * j + 3]);
 }
 
+// The column stream a forward launch walks: the full one, or the band-only one when the dense kernel has already
+// produced the whole-ring part (dense_ptr != null: rows with whole-ring windows start from that partial result).
+struct FwdView {
+    const int4* stream;
+    const int32_t* chunk_ptr;
+    const int32_t* order;
+    const int32_t* dense_ptr;
+};
+
 // ---------------------------------------------------------------------------------------------------------
 // forward
 // ---------------------------------------------------------------------------------------------------------
 template <int C>
 __global__ void __launch_bounds__(THREADS, 4)
-forward_mma_kernel(DevPlan p, const float* __restrict__ q, const float* __restrict__ k, const float* __restrict__ v,
-                   float* __restrict__ out, float* __restrict__ lse, int N, float scale_log2, int tiles_per_row, long long total_tasks) {
+forward_mma_kernel(DevPlan p, FwdView fv, const float* __restrict__ q, const float* __restrict__ k, const float* __restrict__ v,
+                   float* out, float* lse, int N, float scale_log2, int tiles_per_row, long long total_tasks) {
     constexpr int CPT = C / 4, KS = C / 8;
     extern __shared__ __align__(16) unsigned char smem_raw[];
     Stage<C>* stages = reinterpret_cast<Stage<C>*>(smem_raw) + 2 * (threadIdx.x >> 5);
@@ -410,7 +419,7 @@ forward_mma_kernel(DevPlan p, const float* __restrict__ q, const float* __restri
     int n, rank, tile;
     if (!decode_task(N, tiles_per_row, total_tasks, n, rank, tile)) return;
     // tile rows g and g+8 of this thread: the same longitude on the two rings of the group
-    const int hg = p.grp_order[rank];
+    const int hg = fv.order[rank];
     const int w0 = tile * TILE_LON;
     const bool ok0 = w0 + g < p.nlon_out, ok1 = ok0 && hg * TILE_LAT + 1 < p.nlat_out;
     const int wq = min(w0 + g, p.nlon_out - 1);
@@ -423,10 +432,30 @@ forward_mma_kernel(DevPlan p, const float* __restrict__ q, const float* __restri
 #pragma unroll
     for (int nt = 0; nt < KS; ++nt) o[nt][0] = o[nt][1] = o[nt][2] = o[nt][3] = 0.f;
     float m0 = -INFINITY, m1 = -INFINITY, l0 = 0.f, l1 = 0.f;
+    if (fv.dense_ptr != nullptr) {
+        // continue from the dense kernel's partial result of this row (normalised out and lse): m = lse, l = 1
+        const int ha = hg * TILE_LAT, hb = min(hg * TILE_LAT + 1, p.nlat_out - 1);
+        if (fv.dense_ptr[ha + 1] > fv.dense_ptr[ha]) {
+            float r[CPT];
+            load_row<CPT>(out + pt0 * C + t * CPT, r);
+#pragma unroll
+            for (int nt = 0; nt < KS; ++nt) { o[nt][0] = r[nt]; o[nt][1] = r[KS + nt]; }
+            m0 = lse[pt0] * LOG2E;
+            l0 = t == 0 ? 1.f : 0.f;
+        }
+        if (fv.dense_ptr[hb + 1] > fv.dense_ptr[hb]) {
+            float r[CPT];
+            load_row<CPT>(out + pt1 * C + t * CPT, r);
+#pragma unroll
+            for (int nt = 0; nt < KS; ++nt) { o[nt][2] = r[nt]; o[nt][3] = r[KS + nt]; }
+            m1 = lse[pt1] * LOG2E;
+            l1 = t == 0 ? 1.f : 0.f;
+        }
+    }
 
     const size_t slice = (size_t)n * p.nlat_in * p.nlon_in * C;
-    const int4* stream = p.fwd_stream + (size_t)p.fwd_chunk_ptr[hg] * 16;
-    const int nchunks = p.fwd_chunk_ptr[hg + 1] - p.fwd_chunk_ptr[hg];
+    const int4* stream = fv.stream + (size_t)fv.chunk_ptr[hg] * 16;
+    const int nchunks = fv.chunk_ptr[hg + 1] - fv.chunk_ptr[hg];
 
     make_walker<C, false>(stages, stream, lane, w0, p.nlon_out, p.ps, k + slice, v + slice, nullptr, nullptr).run(nchunks, [&](const Stage<C>& st) {
         float s[2][4];
@@ -740,8 +769,8 @@ bool mma_path_supported(const DevPlan& p, int C) {
            (long long)p.nlat_in * p.nlon_in * C < (1LL << 32) && (long long)p.nlat_out * p.nlon_out * C < (1LL << 32);
 }
 
-cudaError_t launch_forward_mma(const DevPlan& p, const float* q, const float* k, const float* v, float* out, float* lse,
-                               int N, int C, cudaStream_t stream) {
+static cudaError_t launch_forward_view(const DevPlan& p, const FwdView& fv, const float* q, const float* k, const float* v, float* out,
+                                       float* lse, int N, int C, cudaStream_t stream) {
     const float scale_log2 = LOG2E / sqrtf((float)C);
     const int tiles = (p.nlon_out + TILE_LON - 1) / TILE_LON;
     const long long tasks = (long long)tiles * ((p.nlat_out + TILE_LAT - 1) / TILE_LAT) * N;
@@ -751,9 +780,21 @@ cudaError_t launch_forward_mma(const DevPlan& p, const float* q, const float* k,
         constexpr int CC = decltype(c)::value;
         cudaError_t e = prepare_kernel(forward_mma_kernel<CC>, smem_bytes<CC>());
         if (e != cudaSuccess) return e;
-        forward_mma_kernel<CC><<<(unsigned)blocks, THREADS, smem_bytes<CC>(), stream>>>(p, q, k, v, out, lse, N, scale_log2, tiles, tasks);
+        forward_mma_kernel<CC><<<(unsigned)blocks, THREADS, smem_bytes<CC>(), stream>>>(p, fv, q, k, v, out, lse, N, scale_log2, tiles, tasks);
         return cudaGetLastError();
     });
+}
+
+cudaError_t launch_forward_mma(const DevPlan& p, const float* q, const float* k, const float* v, float* out, float* lse,
+                               int N, int C, cudaStream_t stream) {
+    const FwdView fv{p.fwd_stream, p.fwd_chunk_ptr, p.grp_order, nullptr};
+    return launch_forward_view(p, fv, q, k, v, out, lse, N, C, stream);
+}
+
+cudaError_t launch_forward_mma_band(const DevPlan& p, const float* q, const float* k, const float* v, float* out, float* lse,
+                                    int N, int C, cudaStream_t stream) {
+    const FwdView fv{p.fwdb_stream, p.fwdb_chunk_ptr, p.grpb_order, p.dense_ptr};
+    return launch_forward_view(p, fv, q, k, v, out, lse, N, C, stream);
 }
 
 cudaError_t launch_backward_dq_mma(const DevPlan& p, const float* q, const float* k, const float* v, const float* dout,

@@ -256,7 +256,19 @@ void merge_group(const std::vector<int32_t>& ptr, const std::vector<RingWindow>&
 
 }  // namespace
 
-void build_forward_stream(const HostPlan& P, Stream& S) {
+void build_dense_lists(const HostPlan& P, DenseLists& D) {
+    D.ptr.assign(P.nlat_out + 1, 0);
+    D.lat.clear();
+    D.rows.clear();
+    for (int h = 0; h < P.nlat_out; ++h) {
+        for (int e = P.row_ptr[h]; e < P.row_ptr[h + 1]; ++e)
+            if (P.windows[e].m < 0) D.lat.push_back(P.windows[e].lat);
+        D.ptr[h + 1] = (int32_t)D.lat.size();
+        if (D.ptr[h + 1] > D.ptr[h]) D.rows.push_back(h);
+    }
+}
+
+void build_forward_stream(const HostPlan& P, Stream& S, bool include_whole) {
     const int groups = (P.nlat_out + TILE_LAT - 1) / TILE_LAT;
     S.chunk_ptr.assign(groups + 1, 0);
     S.entries.clear();
@@ -268,6 +280,7 @@ void build_forward_stream(const HostPlan& P, Stream& S) {
                 GroupRange rg[TILE_LAT];
                 for (int k = 0; k < TILE_LAT; ++k) {
                     if (m[k] == -2) continue;
+                    if (m[k] < 0 && !include_whole) continue;   // served by the dense kernel
                     rg[k].present = true;
                     if (m[k] < 0) rg[k].whole = true;
                     else { rg[k].lo = ceil_div(-m[k] - r, P.ps); rg[k].hi = floor_div(m[k] - r, P.ps); }

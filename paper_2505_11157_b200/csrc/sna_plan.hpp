@@ -59,7 +59,18 @@ struct Stream {
 
 // Forward stream: one row per group of output latitudes (ceil(nlat_out / TILE_LAT) rows); partners are input
 // points, flat index base + u*ps.
-void build_forward_stream(const HostPlan& plan, Stream& out);
+// With include_whole = false the columns of windows that cover a whole input ring are left out: those are
+// served by the dense kernel (see DenseLists), and the stream only carries the banded windows.
+void build_forward_stream(const HostPlan& plan, Stream& out, bool include_whole = true);
+
+// Whole-ring windows per output latitude, for the dense (tcgen05) forward kernel: ring h attends to every point
+// of the input rings lat[ptr[h]] .. lat[ptr[h+1]-1].
+struct DenseLists {
+    std::vector<int32_t> ptr;    // [nlat_out+1]
+    std::vector<int32_t> lat;    // input rings
+    std::vector<int32_t> rows;   // output latitudes that have at least one whole-ring window
+};
+void build_dense_lists(const HostPlan& plan, DenseLists& out);
 // Transposed stream for dk/dv; partners are output points (h, w).  Two layouts:
 //  - consecutive (when ps divides 8): one stream row per group of input latitudes; tile rows are 8 consecutive
 //    input columns c = c0 + i%8 (c0 a multiple of 8) and the partner index is c0/ps + e_rel.  Neighbouring

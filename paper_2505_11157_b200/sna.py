@@ -43,6 +43,7 @@ _SIGNATURES = {
     "sna_plan_create": (_i, [_i, _i, _i, _i, _i, _i, _d, ctypes.POINTER(_vp)]),
     "sna_plan_create_host_only": (_i, [_i, _i, _i, _i, _i, _i, _d, ctypes.POINTER(_vp)]),
     "sna_plan_destroy": (_i, [_vp]),
+    "sna_plan_check": (_i, [_vp]),
     "sna_plan_get_nnz": (_i, [_vp, ctypes.POINTER(ctypes.c_int64)]),
     "sna_plan_get_colatitudes": (_i, [_vp, _vp, _vp]),
     "sna_plan_get_quad_weights": (_i, [_vp, _vp]),
@@ -116,6 +117,11 @@ def sna_plan_create_host_only(nlat_in, nlon_in, nlat_out, nlon_out, grid_in, gri
 
 def sna_plan_destroy(plan: int):
     _check(_lib.sna_plan_destroy(plan))
+
+
+def sna_plan_check(plan: int):
+    """Synchronise and raise if a kernel of this plan gave up on a bounded wait."""
+    _check(_lib.sna_plan_check(plan))
 
 
 def sna_plan_get_nnz(plan: int) -> int:

@@ -45,6 +45,7 @@ def _run_gpu(plan, q, k, v, dout, reuse_forward_state=True):
     else:
         dq, dk, dv = plan.backward(qd, kd, vd, dd)
     torch.cuda.synchronize()
+    sna.sna_plan_check(plan.handle)      # no kernel gave up on a bounded wait
     return [t.cpu().numpy() for t in (out, lse, dq, dk, dv)]
 
 
