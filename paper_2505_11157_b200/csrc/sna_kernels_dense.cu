@@ -126,15 +126,20 @@ forward_dense_kernel(DevPlan p, const float* __restrict__ q, const float* __rest
     const int e_begin = p.dense_ptr[h], e_end = p.dense_ptr[h + 1];
     const int total = (e_end - e_begin) * nblk;    // blocks of this tile, over all its whole input rings
     // raw k / v rows of the next block travel in registers while the current block's MMAs and softmax run
-    float4 kraw[4], vraw[4];
+    // k: thread = (column tid/2, 16 channels); v: thread = (channel lane, 16 columns of group warp), so that the
+    // transposed v rows are written with vector stores and read from global memory as whole 128-byte rows per warp
+    float4 kraw[4];
+    float vraw[16];
+    const int lane = tid & 31;
     auto fetch = [&](int it) {
         const int hp = p.dense_lat[e_begin + it / nblk];
-        const size_t pt = ((size_t)(n * p.nlat_in + hp) * p.nlon_in + min((it % nblk) * DBN + col, p.nlon_in - 1)) * DC + half * 16;
+        const size_t ring0 = (size_t)(n * p.nlat_in + hp) * p.nlon_in;
+        const int c0n = (it % nblk) * DBN;
+        const size_t pt = (ring0 + min(c0n + col, p.nlon_in - 1)) * DC + half * 16;
 #pragma unroll
-        for (int j = 0; j < 4; ++j) {
-            kraw[j] = __ldg(reinterpret_cast<const float4*>(k + pt) + j);
-            vraw[j] = __ldg(reinterpret_cast<const float4*>(v + pt) + j);
-        }
+        for (int j = 0; j < 4; ++j) kraw[j] = __ldg(reinterpret_cast<const float4*>(k + pt) + j);
+#pragma unroll
+        for (int jj = 0; jj < 16; ++jj) vraw[jj] = __ldg(v + (ring0 + min(c0n + warp * 16 + jj, p.nlon_in - 1)) * DC + lane);
     };
     if (total > 0) fetch(0);
     for (int it = 0; it < total && ok; ++it) {
@@ -142,7 +147,6 @@ forward_dense_kernel(DevPlan p, const float* __restrict__ q, const float* __rest
         {
             const int c0 = (it % nblk) * DBN;
             {   // split this block's k rows, and v rows transposed (row = channel, K index = column)
-                const int kb = col >> 5, kc = col & 31;
 #pragma unroll
                 for (int j = 0; j < 4; ++j) {
                     const float4 x = kraw[j];
@@ -151,16 +155,19 @@ forward_dense_kernel(DevPlan p, const float* __restrict__ q, const float* __rest
                     hi.z = __uint_as_float(__float_as_uint(x.z) & 0xffffe000u); hi.w = __uint_as_float(__float_as_uint(x.w) & 0xffffe000u);
                     *reinterpret_cast<float4*>(sKh + sw_chunk(col, half * 4 + j)) = hi;
                     *reinterpret_cast<float4*>(sKl + sw_chunk(col, half * 4 + j)) = make_float4(x.x - hi.x, x.y - hi.y, x.z - hi.z, x.w - hi.w);
-                    const float4 y = vraw[j];
-                    const float yv[4] = {y.x, y.y, y.z, y.w};
+                }
+                // columns warp*16 .. +15 of channel `lane`: K block warp/2, 16-byte chunks (warp%2)*4 .. +3 of row `lane`
+#pragma unroll
+                for (int g4 = 0; g4 < 4; ++g4) {
+                    float hi[4], lo[4];
 #pragma unroll
                     for (int i = 0; i < 4; ++i) {
-                        const int ch = half * 16 + 4 * j + i;
-                        const int off = kb * (DC * 128) + sw_chunk(ch, kc >> 2) + (kc & 3) * 4;
-                        const float g = __uint_as_float(__float_as_uint(yv[i]) & 0xffffe000u);
-                        *reinterpret_cast<float*>(sVh + off) = g;
-                        *reinterpret_cast<float*>(sVl + off) = yv[i] - g;
+                        hi[i] = __uint_as_float(__float_as_uint(vraw[4 * g4 + i]) & 0xffffe000u);
+                        lo[i] = vraw[4 * g4 + i] - hi[i];
                     }
+                    const int off = (warp >> 1) * (DC * 128) + sw_chunk(lane, (warp & 1) * 4 + g4);
+                    *reinterpret_cast<float4*>(sVh + off) = make_float4(hi[0], hi[1], hi[2], hi[3]);
+                    *reinterpret_cast<float4*>(sVl + off) = make_float4(lo[0], lo[1], lo[2], lo[3]);
                 }
             }
             if (it + 1 < total) fetch(it + 1);
