@@ -216,7 +216,7 @@ def run_ours(args, wl):
         if marks is not None:
             marks[2].record(stream)
         sna.sna_backward_dkdv(plan.handle, q, k, v, dout, lse, Dst, dk, dv, B, H, C, stream)
-    launches_per_step = 3
+    launches_per_step = sna.sna_forward_kernel_count(plan.handle, C, True) + 2   # forward (dense + band, or one) + dq + dk/dv
 
     for _ in range(max(args.warmup, 3)):
         step()

@@ -302,6 +302,11 @@ size_t sna_workspace_bytes(const sna_plan_t* plan, int B, int H, int C) {
     return round256(2 * stats_elems(plan, B, H) * sizeof(float));
 }
 
+int sna_forward_kernel_count(const sna_plan_t* plan, int C, int with_lse) {
+    if (plan == nullptr || plan->dev_blob == nullptr || !supported_C(C)) return 0;
+    return (with_lse && sna::dense_path_supported(plan->dev, C)) ? 2 : 1;
+}
+
 sna_status_t sna_forward_ex(const sna_plan_t* plan, const float* q, const float* k, const float* v, float* out,
                             float* lse, int B, int H, int C, void* cuda_stream) {
     sna_status_t st = check_problem(plan, B, H, C);

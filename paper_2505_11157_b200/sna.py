@@ -50,6 +50,7 @@ _SIGNATURES = {
     "sna_plan_get_table": (_i, [_vp, _vp, _vp, _vp]),
     "sna_plan_get_table_transposed": (_i, [_vp, _vp, _vp, _vp]),
     "sna_workspace_bytes": (_sz, [_vp, _i, _i, _i]),
+    "sna_forward_kernel_count": (_i, [_vp, _i, _i]),
     "sna_forward": (_i, [_vp, _vp, _vp, _vp, _vp, _i, _i, _i, _vp]),
     "sna_forward_ex": (_i, [_vp, _vp, _vp, _vp, _vp, _vp, _i, _i, _i, _vp]),
     "sna_backward": (_i, [_vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _i, _i, _i, _vp]),
@@ -132,6 +133,10 @@ def sna_plan_get_nnz(plan: int) -> int:
 
 def sna_workspace_bytes(plan: int, B: int, H: int, C: int) -> int:
     return int(_lib.sna_workspace_bytes(plan, B, H, C))
+
+
+def sna_forward_kernel_count(plan: int, C: int, with_lse: bool) -> int:
+    return int(_lib.sna_forward_kernel_count(plan, C, 1 if with_lse else 0))
 
 
 def sna_forward(plan, q, k, v, out, B, H, C, stream=None):
