@@ -198,6 +198,11 @@ static sna_status_t plan_create(int nlat_in, int nlon_in, int nlat_out, int nlon
     d.fwdb_stream = (const int4*)at(15); d.fwdb_chunk_ptr = at(16); d.grpb_order = at(17);
     d.dense_ptr = at(18); d.dense_lat = at(19); d.dense_rows = at(20);
     d.n_dense_rows = (int)dense.rows.size();
+    {
+        size_t whole = 0;
+        for (const sna::StreamEntry& en : fwd_stream.entries) whole += en.base < 0;
+        d.dense_fraction = fwd_stream.entries.empty() ? 0.f : (float)whole / (float)fwd_stream.entries.size();
+    }
     d.dev_status = (int*)((char*)plan->dev_blob + pieces[21].offset);
     *plan_out = plan;
     return SNA_OK;
@@ -339,9 +344,18 @@ sna_status_t sna_backward_dq(const sna_plan_t* plan, const float* q, const float
     if (st != SNA_OK) return st;
     if (!q || !k || !v || !dout || !lse || !dq || !D) { set_error("q, k, v, dout, lse, dq and D must not be NULL"); return SNA_ERR_INVALID_ARG; }
     if (!all_aligned(q, k, v, dout, dq, out) || ((reinterpret_cast<uintptr_t>(lse) | reinterpret_cast<uintptr_t>(D)) & 3u)) { set_error("device pointers must be 16-byte aligned"); return SNA_ERR_INVALID_ARG; }
-    cudaError_t e = (out != nullptr && sna::mma_path_supported(plan->dev, C))
-                        ? sna::launch_backward_dq_mma(plan->dev, q, k, v, dout, out, lse, dq, D, B * H, C, (cudaStream_t)cuda_stream)
-                        : sna::launch_backward_dq_generic(plan->dev, q, k, v, dout, out, lse, dq, D, B * H, C, (cudaStream_t)cuda_stream);
+    cudaError_t e;
+    // The dense dq kernel pays off when whole-ring windows are a large share of the work (measured: 1.5x on the
+    // global limit, -3 % at a 25 % share), so it is used from a 35 % share on.
+    if (out != nullptr && out != dq && plan->dev.dense_fraction >= 0.35f && sna::dense_path_supported(plan->dev, C)) {
+        // whole-ring windows on the tcgen05 kernel (its part of dq is written first), the banded rest is added by the band kernel
+        e = sna::launch_backward_dq_dense(plan->dev, q, k, v, dout, out, lse, dq, B * H, C, (cudaStream_t)cuda_stream);
+        if (e == cudaSuccess) e = sna::launch_backward_dq_mma_band(plan->dev, q, k, v, dout, out, lse, dq, D, B * H, C, (cudaStream_t)cuda_stream);
+    } else if (out != nullptr && sna::mma_path_supported(plan->dev, C)) {
+        e = sna::launch_backward_dq_mma(plan->dev, q, k, v, dout, out, lse, dq, D, B * H, C, (cudaStream_t)cuda_stream);
+    } else {
+        e = sna::launch_backward_dq_generic(plan->dev, q, k, v, dout, out, lse, dq, D, B * H, C, (cudaStream_t)cuda_stream);
+    }
     if (e != cudaSuccess) return cuda_fail(e, "backward dq launch");
     return SNA_OK;
 }

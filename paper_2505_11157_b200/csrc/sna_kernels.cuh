@@ -31,6 +31,7 @@ struct DevPlan {
     const int32_t* dense_lat;       // their input rings
     const int32_t* dense_rows;      // output latitudes with at least one whole-ring window
     int n_dense_rows;
+    float dense_fraction;           // share of the full forward stream's columns that belong to whole-ring windows
     int* dev_status;                // set to non-zero by a kernel whose bounded wait ran out
     const int4* t_stream;
     const int32_t* t_chunk_ptr;     // [groups of input latitudes * ps + 1]
@@ -48,6 +49,12 @@ cudaError_t launch_forward_mma(const DevPlan& p, const float* q, const float* k,
 bool dense_path_supported(const DevPlan& p, int C);
 cudaError_t launch_forward_dense(const DevPlan& p, const float* q, const float* k, const float* v, float* out, float* lse,
                                  int N, int C, cudaStream_t stream);
+// The same split for the dq stage: the dense kernel writes the whole-ring part of dq (out and dq must be different
+// buffers), the band kernel adds its banded part to it.
+cudaError_t launch_backward_dq_dense(const DevPlan& p, const float* q, const float* k, const float* v, const float* dout,
+                                     const float* out, const float* lse, float* dq, int N, int C, cudaStream_t stream);
+cudaError_t launch_backward_dq_mma_band(const DevPlan& p, const float* q, const float* k, const float* v, const float* dout,
+                                        const float* out, const float* lse, float* dq, float* Dws, int N, int C, cudaStream_t stream);
 cudaError_t launch_forward_mma_band(const DevPlan& p, const float* q, const float* k, const float* v, float* out, float* lse,
                                     int N, int C, cudaStream_t stream);
 // out is required (D_i = dout_i . out_i); out and dq may be the same buffer.

@@ -276,6 +276,199 @@ forward_dense_kernel(DevPlan p, const float* __restrict__ q, const float* __rest
     if (warp == 0) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tm), "r"(TMEM_COLS));
 }
 
+
+// ---------------------------------------------------------------------------------------------------------
+// Dense part of the dq stage (App. B.4): for the whole input rings of an output ring,
+//   p = exp2(s + log2 omega - lse),  ds = p (t - D),  dq += scale * dS K,   s = q.k (log2 domain),  t = dout.v.
+// Same tiling as the forward kernel.  S and T go to TMEM as three TF32 UMMAs per k-step each; every thread turns
+// its row of (S, T) into dS, split in hi and lo, in place; the k tile is then written transposed into the space
+// of the v tile (dead once T is complete) and dq_block = dS K runs with A from TMEM.
+// ---------------------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(DM)
+backward_dq_dense_kernel(DevPlan p, const float* __restrict__ q, const float* __restrict__ k, const float* __restrict__ v,
+                         const float* __restrict__ dout, const float* __restrict__ out, const float* __restrict__ lse,
+                         float* __restrict__ dq, int N, float scale, int blocks_per_row) {
+    extern __shared__ unsigned char dense_raw[];
+    unsigned char* base = (unsigned char*)(((uintptr_t)dense_raw + 1023) & ~(uintptr_t)1023);
+    unsigned char *sQh = base, *sQl = base + 16384, *sYh = base + 32768, *sYl = base + 49152;
+    unsigned char *sKh = base + 65536, *sKl = base + 73728, *sVh = base + 81920, *sVl = base + 90112;   // v tiles, later k transposed
+    __shared__ uint64_t mbar;
+    __shared__ uint32_t tmem_base;
+    const int tid = threadIdx.x, warp = tid >> 5;
+    const int lb = blockIdx.x % blocks_per_row;
+    const int rest = blockIdx.x / blocks_per_row;
+    const int n = rest % N;
+    const int h = p.dense_rows[rest / N];
+    const int w = lb * DM + tid;
+    const bool row_ok = w < p.nlon_out;
+    const size_t opt = (size_t)(n * p.nlat_out + h) * p.nlon_out + min(w, p.nlon_out - 1);
+    const float scale_log2 = scale * LOG2E_D;
+
+    float D = 0.f;
+    {   // this thread's q row (log2 domain) and dout row as tile row tid; D = dout . out
+        const float4* qs = reinterpret_cast<const float4*>(q + opt * DC);
+        const float4* ys = reinterpret_cast<const float4*>(dout + opt * DC);
+        const float4* os = reinterpret_cast<const float4*>(out + opt * DC);
+#pragma unroll
+        for (int c4 = 0; c4 < DC / 4; ++c4) {
+            float4 x = __ldg(qs + c4);
+            x.x *= scale_log2; x.y *= scale_log2; x.z *= scale_log2; x.w *= scale_log2;
+            float4 hi;
+            hi.x = __uint_as_float(__float_as_uint(x.x) & 0xffffe000u); hi.y = __uint_as_float(__float_as_uint(x.y) & 0xffffe000u);
+            hi.z = __uint_as_float(__float_as_uint(x.z) & 0xffffe000u); hi.w = __uint_as_float(__float_as_uint(x.w) & 0xffffe000u);
+            *reinterpret_cast<float4*>(sQh + sw_chunk(tid, c4)) = hi;
+            *reinterpret_cast<float4*>(sQl + sw_chunk(tid, c4)) = make_float4(x.x - hi.x, x.y - hi.y, x.z - hi.z, x.w - hi.w);
+            const float4 y = __ldg(ys + c4), o4 = __ldg(os + c4);
+            D = fmaf(y.x, o4.x, fmaf(y.y, o4.y, fmaf(y.z, o4.z, fmaf(y.w, o4.w, D))));
+            hi.x = __uint_as_float(__float_as_uint(y.x) & 0xffffe000u); hi.y = __uint_as_float(__float_as_uint(y.y) & 0xffffe000u);
+            hi.z = __uint_as_float(__float_as_uint(y.z) & 0xffffe000u); hi.w = __uint_as_float(__float_as_uint(y.w) & 0xffffe000u);
+            *reinterpret_cast<float4*>(sYh + sw_chunk(tid, c4)) = hi;
+            *reinterpret_cast<float4*>(sYl + sw_chunk(tid, c4)) = make_float4(y.x - hi.x, y.y - hi.y, y.z - hi.z, y.w - hi.w);
+        }
+    }
+    const float nl = -__ldg(lse + opt) * LOG2E_D;
+    if (tid == 0) {
+        asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(smem_u32(&mbar)));
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 0) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base)), "r"(TMEM_COLS));
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::);
+    }
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    const uint32_t tm = tmem_base, lanebits = (uint32_t)(warp * 32) << 16;
+    const uint32_t tS = tm, tT = tm + 64, tG = tm + 128;
+    const uint32_t idS = umma_idesc(DBN), idO = umma_idesc(DC), bar = smem_u32(&mbar);
+    uint32_t phase = 0;
+    bool ok = true;
+    float acc[DC];
+#pragma unroll
+    for (int i = 0; i < DC; ++i) acc[i] = 0.f;
+
+    const int col = tid >> 1, half = tid & 1;      // this thread's share of a 64-column block: one column, 16 channels
+    const int nblk = (p.nlon_in + DBN - 1) / DBN;
+    const int e_begin = p.dense_ptr[h], e_end = p.dense_ptr[h + 1];
+    const int total = (e_end - e_begin) * nblk;
+    float4 kcur[4], vcur[4], knext[4], vnext[4];
+    auto fetch = [&](int it, float4 (&kk)[4], float4 (&vv)[4]) {
+        const int hp = p.dense_lat[e_begin + it / nblk];
+        const size_t pt = ((size_t)(n * p.nlat_in + hp) * p.nlon_in + min((it % nblk) * DBN + col, p.nlon_in - 1)) * DC + half * 16;
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            kk[j] = __ldg(reinterpret_cast<const float4*>(k + pt) + j);
+            vv[j] = __ldg(reinterpret_cast<const float4*>(v + pt) + j);
+        }
+    };
+    auto hi4 = [](const float4& x) {
+        return make_float4(__uint_as_float(__float_as_uint(x.x) & 0xffffe000u), __uint_as_float(__float_as_uint(x.y) & 0xffffe000u),
+                           __uint_as_float(__float_as_uint(x.z) & 0xffffe000u), __uint_as_float(__float_as_uint(x.w) & 0xffffe000u));
+    };
+    if (total > 0) fetch(0, kcur, vcur);
+    for (int it = 0; it < total && ok; ++it) {
+        const float bias = p.log2_omega[p.dense_lat[e_begin + it / nblk]] + nl;
+        const int c0 = (it % nblk) * DBN;
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {   // k and v rows of this block, both with the channels as K dimension
+            const float4 kh = hi4(kcur[j]), vh = hi4(vcur[j]);
+            *reinterpret_cast<float4*>(sKh + sw_chunk(col, half * 4 + j)) = kh;
+            *reinterpret_cast<float4*>(sKl + sw_chunk(col, half * 4 + j)) = make_float4(kcur[j].x - kh.x, kcur[j].y - kh.y, kcur[j].z - kh.z, kcur[j].w - kh.w);
+            *reinterpret_cast<float4*>(sVh + sw_chunk(col, half * 4 + j)) = vh;
+            *reinterpret_cast<float4*>(sVl + sw_chunk(col, half * 4 + j)) = make_float4(vcur[j].x - vh.x, vcur[j].y - vh.y, vcur[j].z - vh.z, vcur[j].w - vh.w);
+        }
+        if (it + 1 < total) fetch(it + 1, knext, vnext);
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+        __syncthreads();
+        if (tid == 0) {
+            asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+            const uint64_t qh = umma_desc(smem_u32(sQh)), ql = umma_desc(smem_u32(sQl)), yh = umma_desc(smem_u32(sYh)), yl = umma_desc(smem_u32(sYl));
+            const uint64_t kh = umma_desc(smem_u32(sKh)), kl = umma_desc(smem_u32(sKl)), vh = umma_desc(smem_u32(sVh)), vl = umma_desc(smem_u32(sVl));
+#pragma unroll
+            for (int ks2 = 0; ks2 < DC / 8; ++ks2) { umma_ss(tS, ql + 2 * ks2, kh + 2 * ks2, idS, ks2 > 0); umma_ss(tT, yl + 2 * ks2, vh + 2 * ks2, idS, ks2 > 0); }
+#pragma unroll
+            for (int ks2 = 0; ks2 < DC / 8; ++ks2) { umma_ss(tS, qh + 2 * ks2, kl + 2 * ks2, idS, 1); umma_ss(tT, yh + 2 * ks2, vl + 2 * ks2, idS, 1); }
+#pragma unroll
+            for (int ks2 = 0; ks2 < DC / 8; ++ks2) { umma_ss(tS, qh + 2 * ks2, kh + 2 * ks2, idS, 1); umma_ss(tT, yh + 2 * ks2, vh + 2 * ks2, idS, 1); }
+            umma_commit(bar);
+        }
+        ok = wait_bar(bar, phase);
+        phase ^= 1;
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        if (ok) {
+            const int nvalid = p.nlon_in - c0;
+#pragma unroll
+            for (int hf = 0; hf < 2; ++hf) {   // dS = p (t - D), split, in place over this row of S (hi) and T (lo)
+                uint32_t sv[32], tv[32];
+                tmem_ld32(sv, tS + lanebits + hf * 32);
+                tmem_ld32(tv, tT + lanebits + hf * 32);
+#pragma unroll
+                for (int j = 0; j < 32; ++j) {
+                    const float pj = hf * 32 + j < nvalid ? ex2d(__uint_as_float(sv[j]) + bias) : 0.f;
+                    const float ds = pj * (__uint_as_float(tv[j]) - D);
+                    sv[j] = __float_as_uint(ds);
+                    tv[j] = __float_as_uint(ds - __uint_as_float(sv[j] & 0xffffe000u));
+                }
+                tmem_st32(tS + lanebits + hf * 32, sv);
+                tmem_st32(tT + lanebits + hf * 32, tv);
+            }
+            asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
+            // k transposed (row = channel, K index = column) into the v tiles, which the completed T MMAs no longer read
+            const int kb = col >> 5, kc = col & 31;
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                const float xv[4] = {kcur[j].x, kcur[j].y, kcur[j].z, kcur[j].w};
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    const int ch = half * 16 + 4 * j + i;
+                    const int off = kb * (DC * 128) + sw_chunk(ch, kc >> 2) + (kc & 3) * 4;
+                    const float g = __uint_as_float(__float_as_uint(xv[i]) & 0xffffe000u);
+                    *reinterpret_cast<float*>(sVh + off) = g;
+                    *reinterpret_cast<float*>(sVl + off) = xv[i] - g;
+                }
+            }
+        }
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+        __syncthreads();
+        if (tid == 0 && ok) {
+            asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+            const uint64_t th0 = umma_desc(smem_u32(sVh)), tl0 = umma_desc(smem_u32(sVl));
+#pragma unroll
+            for (int ks2 = 0; ks2 < DBN / 8; ++ks2) umma_ts(tG, tT + ks2 * 8, th0 + (uint64_t)((ks2 >> 2) * (DC * 128 >> 4) + (ks2 & 3) * 2), idO, ks2 > 0);
+#pragma unroll
+            for (int ks2 = 0; ks2 < DBN / 8; ++ks2) umma_ts(tG, tS + ks2 * 8, tl0 + (uint64_t)((ks2 >> 2) * (DC * 128 >> 4) + (ks2 & 3) * 2), idO, 1);
+#pragma unroll
+            for (int ks2 = 0; ks2 < DBN / 8; ++ks2) umma_ts(tG, tS + ks2 * 8, th0 + (uint64_t)((ks2 >> 2) * (DC * 128 >> 4) + (ks2 & 3) * 2), idO, 1);
+            umma_commit(bar);
+        }
+        if (ok) {
+            ok = wait_bar(bar, phase);
+            phase ^= 1;
+        }
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        if (ok) {
+            uint32_t gb[32];
+            tmem_ld32(gb, tG + lanebits);
+#pragma unroll
+            for (int j = 0; j < DC; ++j) acc[j] += __uint_as_float(gb[j]);
+        }
+#pragma unroll
+        for (int j = 0; j < 4; ++j) { kcur[j] = knext[j]; vcur[j] = vnext[j]; }
+        asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+        __syncthreads();
+    }
+    if (!ok && tid == 0) atomicExch(p.dev_status, 1);
+    if (ok && row_ok) {
+        float4* dst = reinterpret_cast<float4*>(dq + opt * DC);
+#pragma unroll
+        for (int c4 = 0; c4 < DC / 4; ++c4) dst[c4] = make_float4(acc[4 * c4] * scale, acc[4 * c4 + 1] * scale, acc[4 * c4 + 2] * scale, acc[4 * c4 + 3] * scale);
+    }
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    if (warp == 0) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tm), "r"(TMEM_COLS));
+}
 }  // namespace
 
 bool dense_path_supported(const DevPlan& p, int C) {
@@ -292,6 +485,19 @@ cudaError_t launch_forward_dense(const DevPlan& p, const float* q, const float* 
     cudaError_t e = cudaFuncSetAttribute(forward_dense_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)DENSE_SMEM);
     if (e != cudaSuccess) return e;
     forward_dense_kernel<<<(unsigned)blocks, DM, DENSE_SMEM, stream>>>(p, q, k, v, out, lse, N, LOG2E_D / sqrtf((float)C), blocks_per_row);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_backward_dq_dense(const DevPlan& p, const float* q, const float* k, const float* v, const float* dout,
+                                     const float* out, const float* lse, float* dq, int N, int C, cudaStream_t stream) {
+    if (C != DC || out == nullptr || lse == nullptr || out == dq) return cudaErrorInvalidValue;
+    const int blocks_per_row = (p.nlon_out + DM - 1) / DM;
+    const long long blocks = (long long)blocks_per_row * p.n_dense_rows * N;
+    if (blocks <= 0) return cudaSuccess;
+    if (blocks > 0x7fffffffLL) return cudaErrorInvalidValue;
+    cudaError_t e = cudaFuncSetAttribute(backward_dq_dense_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)DENSE_SMEM);
+    if (e != cudaSuccess) return e;
+    backward_dq_dense_kernel<<<(unsigned)blocks, DM, DENSE_SMEM, stream>>>(p, q, k, v, dout, out, lse, dq, N, 1.0f / sqrtf((float)C), blocks_per_row);
     return cudaGetLastError();
 }
 

@@ -538,8 +538,8 @@ forward_mma_kernel(DevPlan p, FwdView fv, const float* __restrict__ q, const flo
 // `out` and `dq` may be the same buffer: a warp reads its own 16 rows of `out` before it writes them as dq.
 // ---------------------------------------------------------------------------------------------------------
 template <int C>
-__global__ void __launch_bounds__(THREADS, 2)
-backward_dq_mma_kernel(DevPlan p, const float* __restrict__ q, const float* __restrict__ k, const float* __restrict__ v,
+__global__ void __launch_bounds__(THREADS, 3)
+backward_dq_mma_kernel(DevPlan p, FwdView fv, const float* __restrict__ q, const float* __restrict__ k, const float* __restrict__ v,
                        const float* __restrict__ dout, const float* out, const float* __restrict__ lse,
                        float* dq, float* __restrict__ Dws, int N, float scale, int tiles_per_row, long long total_tasks) {
     constexpr int CPT = C / 4, KS = C / 8;
@@ -548,7 +548,7 @@ backward_dq_mma_kernel(DevPlan p, const float* __restrict__ q, const float* __re
     const int lane = threadIdx.x & 31, g = lane >> 2, t = lane & 3;
     int n, rank, tile;
     if (!decode_task(N, tiles_per_row, total_tasks, n, rank, tile)) return;
-    const int hg = p.grp_order[rank];
+    const int hg = fv.order[rank];
     const int w0 = tile * TILE_LON;
     const bool ok0 = w0 + g < p.nlon_out, ok1 = ok0 && hg * TILE_LAT + 1 < p.nlat_out;
     const int wq = min(w0 + g, p.nlon_out - 1);
@@ -582,8 +582,8 @@ backward_dq_mma_kernel(DevPlan p, const float* __restrict__ q, const float* __re
     for (int nt = 0; nt < KS; ++nt) acc[nt][0] = acc[nt][1] = acc[nt][2] = acc[nt][3] = 0.f;
 
     const size_t slice = (size_t)n * p.nlat_in * p.nlon_in * C;
-    const int4* stream = p.fwd_stream + (size_t)p.fwd_chunk_ptr[hg] * 16;
-    const int nchunks = p.fwd_chunk_ptr[hg + 1] - p.fwd_chunk_ptr[hg];
+    const int4* stream = fv.stream + (size_t)fv.chunk_ptr[hg] * 16;
+    const int nchunks = fv.chunk_ptr[hg + 1] - fv.chunk_ptr[hg];
 
     make_walker<C, false>(stages, stream, lane, w0, p.nlon_out, p.ps, k + slice, v + slice, nullptr, nullptr).run(nchunks, [&](const Stage<C>& st) {
         float s[2][4], tt[2][4];
@@ -625,6 +625,22 @@ backward_dq_mma_kernel(DevPlan p, const float* __restrict__ q, const float* __re
     for (int nt = 0; nt < KS; ++nt) {
         r0v[nt] = acc[nt][0] * scale; r0v[KS + nt] = acc[nt][1] * scale;
         r1v[nt] = acc[nt][2] * scale; r1v[KS + nt] = acc[nt][3] * scale;
+    }
+    if (fv.dense_ptr != nullptr) {
+        // the dense kernel has already written the whole-ring part of dq for rows that have such windows: add it
+        const int ha = hg * TILE_LAT, hb = min(hg * TILE_LAT + 1, p.nlat_out - 1);
+        if (fv.dense_ptr[ha + 1] > fv.dense_ptr[ha]) {
+            float r[CPT];
+            load_row<CPT>(dq + pt0 * C + t * CPT, r);
+#pragma unroll
+            for (int j = 0; j < CPT; ++j) r0v[j] += r[j];
+        }
+        if (fv.dense_ptr[hb + 1] > fv.dense_ptr[hb]) {
+            float r[CPT];
+            load_row<CPT>(dq + pt1 * C + t * CPT, r);
+#pragma unroll
+            for (int j = 0; j < CPT; ++j) r1v[j] += r[j];
+        }
     }
     if (ok0) store_row<CPT>(dq + pt0 * C + t * CPT, r0v);
     if (ok1) store_row<CPT>(dq + pt1 * C + t * CPT, r1v);
@@ -797,8 +813,8 @@ cudaError_t launch_forward_mma_band(const DevPlan& p, const float* q, const floa
     return launch_forward_view(p, fv, q, k, v, out, lse, N, C, stream);
 }
 
-cudaError_t launch_backward_dq_mma(const DevPlan& p, const float* q, const float* k, const float* v, const float* dout,
-                                   const float* out, const float* lse, float* dq, float* Dws, int N, int C, cudaStream_t stream) {
+static cudaError_t launch_backward_dq_view(const DevPlan& p, const FwdView& fv, const float* q, const float* k, const float* v, const float* dout,
+                                           const float* out, const float* lse, float* dq, float* Dws, int N, int C, cudaStream_t stream) {
     const float scale = 1.0f / sqrtf((float)C);
     const int tiles = (p.nlon_out + TILE_LON - 1) / TILE_LON;
     const long long tasks = (long long)tiles * ((p.nlat_out + TILE_LAT - 1) / TILE_LAT) * N;
@@ -808,9 +824,21 @@ cudaError_t launch_backward_dq_mma(const DevPlan& p, const float* q, const float
         constexpr int CC = decltype(c)::value;
         cudaError_t e = prepare_kernel(backward_dq_mma_kernel<CC>, smem_bytes<CC>());
         if (e != cudaSuccess) return e;
-        backward_dq_mma_kernel<CC><<<(unsigned)blocks, THREADS, smem_bytes<CC>(), stream>>>(p, q, k, v, dout, out, lse, dq, Dws, N, scale, tiles, tasks);
+        backward_dq_mma_kernel<CC><<<(unsigned)blocks, THREADS, smem_bytes<CC>(), stream>>>(p, fv, q, k, v, dout, out, lse, dq, Dws, N, scale, tiles, tasks);
         return cudaGetLastError();
     });
+}
+
+cudaError_t launch_backward_dq_mma(const DevPlan& p, const float* q, const float* k, const float* v, const float* dout,
+                                   const float* out, const float* lse, float* dq, float* Dws, int N, int C, cudaStream_t stream) {
+    const FwdView fv{p.fwd_stream, p.fwd_chunk_ptr, p.grp_order, nullptr};
+    return launch_backward_dq_view(p, fv, q, k, v, dout, out, lse, dq, Dws, N, C, stream);
+}
+
+cudaError_t launch_backward_dq_mma_band(const DevPlan& p, const float* q, const float* k, const float* v, const float* dout,
+                                        const float* out, const float* lse, float* dq, float* Dws, int N, int C, cudaStream_t stream) {
+    const FwdView fv{p.fwdb_stream, p.fwdb_chunk_ptr, p.grpb_order, p.dense_ptr};
+    return launch_backward_dq_view(p, fv, q, k, v, dout, out, lse, dq, Dws, N, C, stream);
 }
 
 cudaError_t launch_backward_dkdv_mma(const DevPlan& p, const float* q, const float* k, const float* v, const float* dout,

@@ -72,6 +72,11 @@ SMALL = [
     small_workload("eq_to_gl_up_lat_c32", 9, 40, 20, 40, EQ, GL, 0.6, 1, 1, 32, 28),       # more output than input rings
     small_workload("eq_nearly_global_c32", 12, 32, 12, 32, EQ, EQ, 2.6, 1, 1, 32, 29),     # windows wider than half a ring
     small_workload("eq_many_heads_c16", 10, 32, 10, 32, EQ, EQ, 0.5, 3, 7, 16, 30),        # 21 independent slices
+    # whole-ring windows everywhere: both dense tensor-core kernels do all the work
+    small_workload("global_c32_dense", 14, 64, 14, 64, EQ, EQ, math.pi, 1, 2, 32, 33),
+    small_workload("global_ragged_dense", 10, 80, 10, 80, GL, GL, math.pi, 2, 1, 32, 34),  # 80 columns: partial last block; 80 rows < 128
+    small_workload("global_down2_dense", 12, 288, 7, 144, EQ, EQ, math.pi, 1, 1, 32, 35),  # 144 rows: two row blocks, the second ragged
+    small_workload("polar_heavy_c32", 16, 64, 16, 64, EQ, EQ, 1.2, 1, 2, 32, 36),          # dense and banded windows mixed in every row
 ]
 
 
