@@ -127,9 +127,9 @@ static sna_status_t plan_create(int nlat_in, int nlon_in, int nlat_out, int nlon
     std::vector<float> log2_omega(hp.nlat_in);
     for (int h = 0; h < hp.nlat_in; ++h) log2_omega[h] = (float)std::log2(hp.omega[h]);
 
-    sna::Stream fwd_stream, t_stream, fwdb_stream;
-    sna::DenseLists dense;
-    std::vector<int32_t> grp_order, t_grp_order, grpb_order;
+    sna::Stream fwd_stream, t_stream, fwdb_stream, tb_stream;
+    sna::DenseLists dense, t_dense;
+    std::vector<int32_t> grp_order, t_grp_order, grpb_order, tb_grp_order;
     const int32_t zero_status[64] = {};
     bool t_consecutive = false;
     try {
@@ -148,7 +148,15 @@ static sna_status_t plan_create(int nlat_in, int nlon_in, int nlat_out, int nlon
         std::stable_sort(grp_order.begin(), grp_order.end(), [&](int a, int b) {
             return fwd_stream.chunk_ptr[a + 1] - fwd_stream.chunk_ptr[a] > fwd_stream.chunk_ptr[b + 1] - fwd_stream.chunk_ptr[b];
         });
+        sna::build_transposed_dense_lists(hp, t_dense);
+        sna::build_transposed_stream(hp, tb_stream, /*include_whole=*/false);
         const int rows_per_group = t_consecutive ? 1 : hp.ps;
+        tb_grp_order.resize((tb_stream.chunk_ptr.size() - 1) / rows_per_group);
+        std::iota(tb_grp_order.begin(), tb_grp_order.end(), 0);
+        std::stable_sort(tb_grp_order.begin(), tb_grp_order.end(), [&](int a, int b) {
+            return tb_stream.chunk_ptr[(a + 1) * rows_per_group] - tb_stream.chunk_ptr[a * rows_per_group] >
+                   tb_stream.chunk_ptr[(b + 1) * rows_per_group] - tb_stream.chunk_ptr[b * rows_per_group];
+        });
         t_grp_order.resize((t_stream.chunk_ptr.size() - 1) / rows_per_group);
         std::iota(t_grp_order.begin(), t_grp_order.end(), 0);
         std::stable_sort(t_grp_order.begin(), t_grp_order.end(), [&](int a, int b) {
@@ -173,7 +181,10 @@ static sna_status_t plan_create(int nlat_in, int nlon_in, int nlat_out, int nlon
         {grp_order.data(), grp_order.size() * 4, 0}, {t_grp_order.data(), t_grp_order.size() * 4, 0},
         {fwdb_stream.entries.data(), fwdb_stream.entries.size() * 16, 0}, {fwdb_stream.chunk_ptr.data(), fwdb_stream.chunk_ptr.size() * 4, 0},
         {grpb_order.data(), grpb_order.size() * 4, 0}, {dense.ptr.data(), dense.ptr.size() * 4, 0},
-        {dense.lat.data(), dense.lat.size() * 4, 0}, {dense.rows.data(), dense.rows.size() * 4, 0}, {zero_status, sizeof(zero_status), 0}};
+        {dense.lat.data(), dense.lat.size() * 4, 0}, {dense.rows.data(), dense.rows.size() * 4, 0}, {zero_status, sizeof(zero_status), 0},
+        {tb_stream.entries.data(), tb_stream.entries.size() * 16, 0}, {tb_stream.chunk_ptr.data(), tb_stream.chunk_ptr.size() * 4, 0},
+        {tb_grp_order.data(), tb_grp_order.size() * 4, 0}, {t_dense.ptr.data(), t_dense.ptr.size() * 4, 0},
+        {t_dense.lat.data(), t_dense.lat.size() * 4, 0}, {t_dense.rows.data(), t_dense.rows.size() * 4, 0}};
     size_t total = 0;
     for (Piece& p : pieces) { p.offset = total; total += round256(p.bytes); }
     cudaError_t e = cudaGetDevice(&plan->device);
@@ -204,6 +215,9 @@ static sna_status_t plan_create(int nlat_in, int nlon_in, int nlat_out, int nlon
         d.dense_fraction = fwd_stream.entries.empty() ? 0.f : (float)whole / (float)fwd_stream.entries.size();
     }
     d.dev_status = (int*)((char*)plan->dev_blob + pieces[21].offset);
+    d.tb_stream = (const int4*)at(22); d.tb_chunk_ptr = at(23); d.tb_grp_order = at(24);
+    d.t_dense_ptr = at(25); d.t_dense_lat = at(26); d.t_dense_rows = at(27);
+    d.n_t_dense_rows = (int)t_dense.rows.size();
     *plan_out = plan;
     return SNA_OK;
 }
@@ -367,9 +381,16 @@ sna_status_t sna_backward_dkdv(const sna_plan_t* plan, const float* q, const flo
     if (st != SNA_OK) return st;
     if (!q || !k || !v || !dout || !lse || !D || !dk || !dv) { set_error("q, k, v, dout, lse, D, dk and dv must not be NULL"); return SNA_ERR_INVALID_ARG; }
     if (!all_aligned(q, k, v, dout, dk, dv) || ((reinterpret_cast<uintptr_t>(lse) | reinterpret_cast<uintptr_t>(D)) & 3u)) { set_error("device pointers must be 16-byte aligned"); return SNA_ERR_INVALID_ARG; }
-    cudaError_t e = sna::mma_path_supported(plan->dev, C)
-                        ? sna::launch_backward_dkdv_mma(plan->dev, q, k, v, dout, lse, D, dk, dv, B * H, C, (cudaStream_t)cuda_stream)
-                        : sna::launch_backward_dkdv_generic(plan->dev, q, k, v, dout, lse, D, dk, dv, B * H, C, (cudaStream_t)cuda_stream);
+    cudaError_t e;
+    if (plan->dev.dense_fraction >= 0.35f && plan->dev.n_t_dense_rows > 0 && sna::dense_path_supported(plan->dev, C)) {
+        // whole-ring partners on the tcgen05 kernel (its part of dk, dv is written first), the band kernel adds the rest
+        e = sna::launch_backward_dkdv_dense(plan->dev, q, k, v, dout, lse, D, dk, dv, B * H, C, (cudaStream_t)cuda_stream);
+        if (e == cudaSuccess) e = sna::launch_backward_dkdv_mma_band(plan->dev, q, k, v, dout, lse, D, dk, dv, B * H, C, (cudaStream_t)cuda_stream);
+    } else if (sna::mma_path_supported(plan->dev, C)) {
+        e = sna::launch_backward_dkdv_mma(plan->dev, q, k, v, dout, lse, D, dk, dv, B * H, C, (cudaStream_t)cuda_stream);
+    } else {
+        e = sna::launch_backward_dkdv_generic(plan->dev, q, k, v, dout, lse, D, dk, dv, B * H, C, (cudaStream_t)cuda_stream);
+    }
     if (e != cudaSuccess) return cuda_fail(e, "backward dk/dv launch");
     return SNA_OK;
 }

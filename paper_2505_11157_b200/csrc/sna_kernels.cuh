@@ -31,6 +31,15 @@ struct DevPlan {
     const int32_t* dense_lat;       // their input rings
     const int32_t* dense_rows;      // output latitudes with at least one whole-ring window
     int n_dense_rows;
+    // the same for the transposed side (dk/dv): band-only transposed stream and, per input latitude, the output rings
+    // that attend to it as a whole
+    const int4* tb_stream;
+    const int32_t* tb_chunk_ptr;
+    const int32_t* tb_grp_order;
+    const int32_t* t_dense_ptr;     // [nlat_in+1]
+    const int32_t* t_dense_lat;     // output rings
+    const int32_t* t_dense_rows;    // input latitudes with at least one such output ring
+    int n_t_dense_rows;
     float dense_fraction;           // share of the full forward stream's columns that belong to whole-ring windows
     int* dev_status;                // set to non-zero by a kernel whose bounded wait ran out
     const int4* t_stream;
@@ -55,6 +64,10 @@ cudaError_t launch_backward_dq_dense(const DevPlan& p, const float* q, const flo
                                      const float* out, const float* lse, float* dq, int N, int C, cudaStream_t stream);
 cudaError_t launch_backward_dq_mma_band(const DevPlan& p, const float* q, const float* k, const float* v, const float* dout,
                                         const float* out, const float* lse, float* dq, float* Dws, int N, int C, cudaStream_t stream);
+cudaError_t launch_backward_dkdv_dense(const DevPlan& p, const float* q, const float* k, const float* v, const float* dout,
+                                       const float* lse, const float* Dws, float* dk, float* dv, int N, int C, cudaStream_t stream);
+cudaError_t launch_backward_dkdv_mma_band(const DevPlan& p, const float* q, const float* k, const float* v, const float* dout,
+                                          const float* lse, const float* Dws, float* dk, float* dv, int N, int C, cudaStream_t stream);
 cudaError_t launch_forward_mma_band(const DevPlan& p, const float* q, const float* k, const float* v, float* out, float* lse,
                                     int N, int C, cudaStream_t stream);
 // out is required (D_i = dout_i . out_i); out and dq may be the same buffer.

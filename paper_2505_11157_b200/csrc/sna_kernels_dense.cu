@@ -469,6 +469,238 @@ backward_dq_dense_kernel(DevPlan p, const float* __restrict__ q, const float* __
     __syncthreads();
     if (warp == 0) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tm), "r"(TMEM_COLS));
 }
+
+// ---------------------------------------------------------------------------------------------------------
+// Dense part of the dk/dv stage (App. B.4), transposed roles: one CTA owns 128 consecutive input columns of an input
+// ring (tile row = input point j) and walks, in blocks of 64, the output points i of the output rings that attend to
+// this input ring as a whole:
+//   S^T = K Q^T, T^T = V dY^T (TF32 UMMAs into TMEM);  p = exp2(s + log2 omega_j - lse_i),  ds = p (t - D_i);
+//   dV += P^T dY,  dK += scale * dS^T Q   (A from TMEM, the q / dout tiles rewritten transposed once S^T, T^T are done).
+// TMEM budget (256 columns): P_hi over S, P_lo over T, raw dS in a third block; after the dV MMAs dS_lo replaces P_lo
+// and the raw dS block itself serves as dS_hi (the MMA reads only its top 19 bits).
+// ---------------------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(DM)
+backward_dkdv_dense_kernel(DevPlan p, const float* __restrict__ q, const float* __restrict__ k, const float* __restrict__ v,
+                           const float* __restrict__ dout, const float* __restrict__ lse, const float* __restrict__ Dws,
+                           float* __restrict__ dk, float* __restrict__ dv, int N, float scale, int blocks_per_row) {
+    extern __shared__ unsigned char dense_raw[];
+    unsigned char* base = (unsigned char*)(((uintptr_t)dense_raw + 1023) & ~(uintptr_t)1023);
+    unsigned char *sKh = base, *sKl = base + 16384, *sVh = base + 32768, *sVl = base + 49152;                 // persistent A tiles
+    unsigned char *sQh = base + 65536, *sQl = base + 73728, *sYh = base + 81920, *sYl = base + 90112;         // per block, later transposed
+    __shared__ uint64_t mbar;
+    __shared__ uint32_t tmem_base;
+    __shared__ float s_nl[DBN], s_D[DBN];     // per partner column: -lse (log2) and D
+    const int tid = threadIdx.x, warp = tid >> 5;
+    const int lb = blockIdx.x % blocks_per_row;
+    const int rest = blockIdx.x / blocks_per_row;
+    const int n = rest % N;
+    const int hp = p.t_dense_rows[rest / N];
+    const int c = lb * DM + tid;
+    const bool row_ok = c < p.nlon_in;
+    const size_t ipt = (size_t)(n * p.nlat_in + hp) * p.nlon_in + min(c, p.nlon_in - 1);
+    const float scale_log2 = scale * LOG2E_D;
+    const float bias = p.log2_omega[hp];
+
+    {   // this thread's k row (log2 domain) and v row as tile row tid
+        const float4* ks = reinterpret_cast<const float4*>(k + ipt * DC);
+        const float4* vs = reinterpret_cast<const float4*>(v + ipt * DC);
+#pragma unroll
+        for (int c4 = 0; c4 < DC / 4; ++c4) {
+            float4 x = __ldg(ks + c4);
+            x.x *= scale_log2; x.y *= scale_log2; x.z *= scale_log2; x.w *= scale_log2;
+            float4 hi;
+            hi.x = __uint_as_float(__float_as_uint(x.x) & 0xffffe000u); hi.y = __uint_as_float(__float_as_uint(x.y) & 0xffffe000u);
+            hi.z = __uint_as_float(__float_as_uint(x.z) & 0xffffe000u); hi.w = __uint_as_float(__float_as_uint(x.w) & 0xffffe000u);
+            *reinterpret_cast<float4*>(sKh + sw_chunk(tid, c4)) = hi;
+            *reinterpret_cast<float4*>(sKl + sw_chunk(tid, c4)) = make_float4(x.x - hi.x, x.y - hi.y, x.z - hi.z, x.w - hi.w);
+            const float4 y = __ldg(vs + c4);
+            hi.x = __uint_as_float(__float_as_uint(y.x) & 0xffffe000u); hi.y = __uint_as_float(__float_as_uint(y.y) & 0xffffe000u);
+            hi.z = __uint_as_float(__float_as_uint(y.z) & 0xffffe000u); hi.w = __uint_as_float(__float_as_uint(y.w) & 0xffffe000u);
+            *reinterpret_cast<float4*>(sVh + sw_chunk(tid, c4)) = hi;
+            *reinterpret_cast<float4*>(sVl + sw_chunk(tid, c4)) = make_float4(y.x - hi.x, y.y - hi.y, y.z - hi.z, y.w - hi.w);
+        }
+    }
+    if (tid == 0) {
+        asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(smem_u32(&mbar)));
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 0) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base)), "r"(TMEM_COLS));
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::);
+    }
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    const uint32_t tm = tmem_base, lanebits = (uint32_t)(warp * 32) << 16;
+    const uint32_t tS = tm, tT = tm + 64, tX = tm + 128, tGv = tm + 192, tGk = tm + 224;
+    const uint32_t idS = umma_idesc(DBN), idO = umma_idesc(DC), bar = smem_u32(&mbar);
+    uint32_t phase = 0;
+    bool ok = true;
+    float gk[DC], gv[DC];
+#pragma unroll
+    for (int i = 0; i < DC; ++i) { gk[i] = 0.f; gv[i] = 0.f; }
+    const int col = tid >> 1, half = tid & 1;      // this thread's share of a 64-partner block: one output point, 16 channels
+    const int nblk = (p.nlon_out + DBN - 1) / DBN;
+    const int e_begin = p.t_dense_ptr[hp], e_end = p.t_dense_ptr[hp + 1];
+    const int total = (e_end - e_begin) * nblk;
+    float4 qcur[4], ycur[4], qnext[4], ynext[4];
+    auto fetch = [&](int it, float4 (&qq)[4], float4 (&yy)[4]) {
+        const int h = p.t_dense_lat[e_begin + it / nblk];
+        const size_t pt = ((size_t)(n * p.nlat_out + h) * p.nlon_out + min((it % nblk) * DBN + col, p.nlon_out - 1)) * DC + half * 16;
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            qq[j] = __ldg(reinterpret_cast<const float4*>(q + pt) + j);
+            yy[j] = __ldg(reinterpret_cast<const float4*>(dout + pt) + j);
+        }
+    };
+    auto hi4 = [](const float4& x) {
+        return make_float4(__uint_as_float(__float_as_uint(x.x) & 0xffffe000u), __uint_as_float(__float_as_uint(x.y) & 0xffffe000u),
+                           __uint_as_float(__float_as_uint(x.z) & 0xffffe000u), __uint_as_float(__float_as_uint(x.w) & 0xffffe000u));
+    };
+    // element (row = channel, K index = partner column) of a transposed 32 x 64 tile
+    auto st_t = [&](unsigned char* th, unsigned char* tl, int ch, float x) {
+        const int off = (col >> 5) * (DC * 128) + sw_chunk(ch, (col & 31) >> 2) + (col & 3) * 4;
+        const float g = __uint_as_float(__float_as_uint(x) & 0xffffe000u);
+        *reinterpret_cast<float*>(th + off) = g;
+        *reinterpret_cast<float*>(tl + off) = x - g;
+    };
+    if (total > 0) fetch(0, qcur, ycur);
+    for (int it = 0; it < total && ok; ++it) {
+        const int h = p.t_dense_lat[e_begin + it / nblk];
+        const int w0 = (it % nblk) * DBN;
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {   // q and dout rows of the partner points, channels as K dimension
+            const float4 qh = hi4(qcur[j]), yh = hi4(ycur[j]);
+            *reinterpret_cast<float4*>(sQh + sw_chunk(col, half * 4 + j)) = qh;
+            *reinterpret_cast<float4*>(sQl + sw_chunk(col, half * 4 + j)) = make_float4(qcur[j].x - qh.x, qcur[j].y - qh.y, qcur[j].z - qh.z, qcur[j].w - qh.w);
+            *reinterpret_cast<float4*>(sYh + sw_chunk(col, half * 4 + j)) = yh;
+            *reinterpret_cast<float4*>(sYl + sw_chunk(col, half * 4 + j)) = make_float4(ycur[j].x - yh.x, ycur[j].y - yh.y, ycur[j].z - yh.z, ycur[j].w - yh.w);
+        }
+        if (tid < DBN) {
+            const size_t o = (size_t)(n * p.nlat_out + h) * p.nlon_out + min(w0 + tid, p.nlon_out - 1);
+            s_nl[tid] = fmaf(-__ldg(lse + o), LOG2E_D, bias);
+            s_D[tid] = __ldg(Dws + o);
+        }
+        if (it + 1 < total) fetch(it + 1, qnext, ynext);
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+        __syncthreads();
+        if (tid == 0) {
+            asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+            const uint64_t kh = umma_desc(smem_u32(sKh)), kl = umma_desc(smem_u32(sKl)), vh = umma_desc(smem_u32(sVh)), vl = umma_desc(smem_u32(sVl));
+            const uint64_t qh = umma_desc(smem_u32(sQh)), ql = umma_desc(smem_u32(sQl)), yh = umma_desc(smem_u32(sYh)), yl = umma_desc(smem_u32(sYl));
+#pragma unroll
+            for (int ks2 = 0; ks2 < DC / 8; ++ks2) { umma_ss(tS, kl + 2 * ks2, qh + 2 * ks2, idS, ks2 > 0); umma_ss(tT, vl + 2 * ks2, yh + 2 * ks2, idS, ks2 > 0); }
+#pragma unroll
+            for (int ks2 = 0; ks2 < DC / 8; ++ks2) { umma_ss(tS, kh + 2 * ks2, ql + 2 * ks2, idS, 1); umma_ss(tT, vh + 2 * ks2, yl + 2 * ks2, idS, 1); }
+#pragma unroll
+            for (int ks2 = 0; ks2 < DC / 8; ++ks2) { umma_ss(tS, kh + 2 * ks2, qh + 2 * ks2, idS, 1); umma_ss(tT, vh + 2 * ks2, yh + 2 * ks2, idS, 1); }
+            umma_commit(bar);
+        }
+        ok = wait_bar(bar, phase);
+        phase ^= 1;
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        if (ok) {
+            const int nvalid = p.nlon_out - w0;
+#pragma unroll
+            for (int hf = 0; hf < 2; ++hf) {   // P (hi over S, lo over T) and raw dS for this row
+                uint32_t sv[32], tv[32], xv[32];
+                tmem_ld32(sv, tS + lanebits + hf * 32);
+                tmem_ld32(tv, tT + lanebits + hf * 32);
+#pragma unroll
+                for (int j = 0; j < 32; ++j) {
+                    const float pj = hf * 32 + j < nvalid ? ex2d(__uint_as_float(sv[j]) + s_nl[hf * 32 + j]) : 0.f;
+                    xv[j] = __float_as_uint(pj * (__uint_as_float(tv[j]) - s_D[hf * 32 + j]));
+                    sv[j] = __float_as_uint(pj);
+                    tv[j] = __float_as_uint(pj - __uint_as_float(sv[j] & 0xffffe000u));
+                }
+                tmem_st32(tS + lanebits + hf * 32, sv);
+                tmem_st32(tT + lanebits + hf * 32, tv);
+                tmem_st32(tX + lanebits + hf * 32, xv);
+            }
+            asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
+            // the q / dout tiles are dead: rewrite them transposed (row = channel, K index = partner)
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                const float qv[4] = {qcur[j].x, qcur[j].y, qcur[j].z, qcur[j].w}, yv[4] = {ycur[j].x, ycur[j].y, ycur[j].z, ycur[j].w};
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    st_t(sQh, sQl, half * 16 + 4 * j + i, qv[i]);
+                    st_t(sYh, sYl, half * 16 + 4 * j + i, yv[i]);
+                }
+            }
+        }
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+        __syncthreads();
+        const auto tdesc = [](uint64_t d0, int ks2) { return d0 + (uint64_t)((ks2 >> 2) * (DC * 128 >> 4) + (ks2 & 3) * 2); };
+        if (tid == 0 && ok) {   // dV_block = P^T dY
+            asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+            const uint64_t yh = umma_desc(smem_u32(sYh)), yl = umma_desc(smem_u32(sYl));
+#pragma unroll
+            for (int ks2 = 0; ks2 < DBN / 8; ++ks2) umma_ts(tGv, tT + ks2 * 8, tdesc(yh, ks2), idO, ks2 > 0);
+#pragma unroll
+            for (int ks2 = 0; ks2 < DBN / 8; ++ks2) umma_ts(tGv, tS + ks2 * 8, tdesc(yl, ks2), idO, 1);
+#pragma unroll
+            for (int ks2 = 0; ks2 < DBN / 8; ++ks2) umma_ts(tGv, tS + ks2 * 8, tdesc(yh, ks2), idO, 1);
+            umma_commit(bar);
+        }
+        if (ok) { ok = wait_bar(bar, phase); phase ^= 1; }
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        if (ok) {   // dS_lo replaces P_lo; the raw dS block is dS_hi
+#pragma unroll
+            for (int hf = 0; hf < 2; ++hf) {
+                uint32_t xv[32];
+                tmem_ld32(xv, tX + lanebits + hf * 32);
+#pragma unroll
+                for (int j = 0; j < 32; ++j) xv[j] = __float_as_uint(__uint_as_float(xv[j]) - __uint_as_float(xv[j] & 0xffffe000u));
+                tmem_st32(tT + lanebits + hf * 32, xv);
+            }
+            asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
+        }
+        asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+        __syncthreads();
+        if (tid == 0 && ok) {   // dK_block = dS^T Q
+            asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+            const uint64_t qh = umma_desc(smem_u32(sQh)), ql = umma_desc(smem_u32(sQl));
+#pragma unroll
+            for (int ks2 = 0; ks2 < DBN / 8; ++ks2) umma_ts(tGk, tT + ks2 * 8, tdesc(qh, ks2), idO, ks2 > 0);
+#pragma unroll
+            for (int ks2 = 0; ks2 < DBN / 8; ++ks2) umma_ts(tGk, tX + ks2 * 8, tdesc(ql, ks2), idO, 1);
+#pragma unroll
+            for (int ks2 = 0; ks2 < DBN / 8; ++ks2) umma_ts(tGk, tX + ks2 * 8, tdesc(qh, ks2), idO, 1);
+            umma_commit(bar);
+        }
+        if (ok) { ok = wait_bar(bar, phase); phase ^= 1; }
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        if (ok) {
+            uint32_t gb[32];
+            tmem_ld32(gb, tGv + lanebits);
+#pragma unroll
+            for (int j = 0; j < DC; ++j) gv[j] += __uint_as_float(gb[j]);
+            tmem_ld32(gb, tGk + lanebits);
+#pragma unroll
+            for (int j = 0; j < DC; ++j) gk[j] += __uint_as_float(gb[j]);
+        }
+#pragma unroll
+        for (int j = 0; j < 4; ++j) { qcur[j] = qnext[j]; ycur[j] = ynext[j]; }
+        asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+        __syncthreads();
+    }
+    if (!ok && tid == 0) atomicExch(p.dev_status, 1);
+    if (ok && row_ok) {
+        float4* dkp = reinterpret_cast<float4*>(dk + ipt * DC);
+        float4* dvp = reinterpret_cast<float4*>(dv + ipt * DC);
+#pragma unroll
+        for (int c4 = 0; c4 < DC / 4; ++c4) {
+            dkp[c4] = make_float4(gk[4 * c4] * scale, gk[4 * c4 + 1] * scale, gk[4 * c4 + 2] * scale, gk[4 * c4 + 3] * scale);
+            dvp[c4] = make_float4(gv[4 * c4], gv[4 * c4 + 1], gv[4 * c4 + 2], gv[4 * c4 + 3]);
+        }
+    }
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    if (warp == 0) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tm), "r"(TMEM_COLS));
+}
 }  // namespace
 
 bool dense_path_supported(const DevPlan& p, int C) {
@@ -498,6 +730,19 @@ cudaError_t launch_backward_dq_dense(const DevPlan& p, const float* q, const flo
     cudaError_t e = cudaFuncSetAttribute(backward_dq_dense_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)DENSE_SMEM);
     if (e != cudaSuccess) return e;
     backward_dq_dense_kernel<<<(unsigned)blocks, DM, DENSE_SMEM, stream>>>(p, q, k, v, dout, out, lse, dq, N, 1.0f / sqrtf((float)C), blocks_per_row);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_backward_dkdv_dense(const DevPlan& p, const float* q, const float* k, const float* v, const float* dout,
+                                       const float* lse, const float* Dws, float* dk, float* dv, int N, int C, cudaStream_t stream) {
+    if (C != DC) return cudaErrorInvalidValue;
+    const int blocks_per_row = (p.nlon_in + DM - 1) / DM;
+    const long long blocks = (long long)blocks_per_row * p.n_t_dense_rows * N;
+    if (blocks <= 0) return cudaSuccess;
+    if (blocks > 0x7fffffffLL) return cudaErrorInvalidValue;
+    cudaError_t e = cudaFuncSetAttribute(backward_dkdv_dense_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)DENSE_SMEM);
+    if (e != cudaSuccess) return e;
+    backward_dkdv_dense_kernel<<<(unsigned)blocks, DM, DENSE_SMEM, stream>>>(p, q, k, v, dout, lse, Dws, dk, dv, N, 1.0f / sqrtf((float)C), blocks_per_row);
     return cudaGetLastError();
 }
 

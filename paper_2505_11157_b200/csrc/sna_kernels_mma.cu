@@ -654,16 +654,16 @@ backward_dq_mma_kernel(DevPlan p, FwdView fv, const float* __restrict__ q, const
 // ---------------------------------------------------------------------------------------------------------
 template <int C>
 __global__ void __launch_bounds__(THREADS, 2)
-backward_dkdv_mma_kernel(DevPlan p, const float* __restrict__ q, const float* __restrict__ k, const float* __restrict__ v,
+backward_dkdv_mma_kernel(DevPlan p, FwdView tv, const float* __restrict__ q, const float* __restrict__ k, const float* __restrict__ v,
                          const float* __restrict__ dout, const float* __restrict__ lse, const float* __restrict__ Dws,
-                         float* __restrict__ dk, float* __restrict__ dv, int N, float scale, int tiles_per_row, long long total_tasks) {
+                         float* dk, float* dv, int N, float scale, int tiles_per_row, long long total_tasks) {
     constexpr int CPT = C / 4, KS = C / 8;
     extern __shared__ __align__(16) unsigned char smem_raw[];
     Stage<C>* stages = reinterpret_cast<Stage<C>*>(smem_raw) + 2 * (threadIdx.x >> 5);
     const int lane = threadIdx.x & 31, g = lane >> 2, t = lane & 3;
     int n, rank, tile;
     if (!decode_task(N, tiles_per_row, total_tasks, n, rank, tile)) return;
-    const int hg = p.t_grp_order[rank];
+    const int hg = tv.order[rank];
     // input column of tile row g (and g+8), the first partner index of the tile, and the tile's stream row
     int col, first, srow;
     bool ok0;
@@ -697,8 +697,8 @@ backward_dkdv_mma_kernel(DevPlan p, const float* __restrict__ q, const float* __
         gv[nt][0] = gv[nt][1] = gv[nt][2] = gv[nt][3] = 0.f;
     }
     const size_t oslice = (size_t)n * p.nlat_out * p.nlon_out;
-    const int4* stream = p.t_stream + (size_t)p.t_chunk_ptr[srow] * 16;
-    const int nchunks = p.t_chunk_ptr[srow + 1] - p.t_chunk_ptr[srow];
+    const int4* stream = tv.stream + (size_t)tv.chunk_ptr[srow] * 16;
+    const int nchunks = tv.chunk_ptr[srow + 1] - tv.chunk_ptr[srow];
 
     make_walker<C, true>(stages, stream, lane, first, p.nlon_out, 1, q + oslice * C, dout + oslice * C, lse + oslice, Dws + oslice).run(nchunks, [&](const Stage<C>& st) {
         float s[2][4], tt[2][4];
@@ -747,6 +747,27 @@ backward_dkdv_mma_kernel(DevPlan p, const float* __restrict__ q, const float* __
     for (int nt = 0; nt < KS; ++nt) {
         a0[nt] = gk[nt][0] * scale; a0[KS + nt] = gk[nt][1] * scale; a1[nt] = gk[nt][2] * scale; a1[KS + nt] = gk[nt][3] * scale;
         b0[nt] = gv[nt][0]; b0[KS + nt] = gv[nt][1]; b1[nt] = gv[nt][2]; b1[KS + nt] = gv[nt][3];
+    }
+    if (tv.dense_ptr != nullptr) {
+        // the dense kernel has already written the whole-ring part of dk, dv for input rings that have such partners
+        if (tv.dense_ptr[hp0 + 1] > tv.dense_ptr[hp0]) {
+            float r[CPT];
+            load_row<CPT>(dk + pt0 * C + t * CPT, r);
+#pragma unroll
+            for (int j = 0; j < CPT; ++j) a0[j] += r[j];
+            load_row<CPT>(dv + pt0 * C + t * CPT, r);
+#pragma unroll
+            for (int j = 0; j < CPT; ++j) b0[j] += r[j];
+        }
+        if (tv.dense_ptr[hp1 + 1] > tv.dense_ptr[hp1]) {
+            float r[CPT];
+            load_row<CPT>(dk + pt1 * C + t * CPT, r);
+#pragma unroll
+            for (int j = 0; j < CPT; ++j) a1[j] += r[j];
+            load_row<CPT>(dv + pt1 * C + t * CPT, r);
+#pragma unroll
+            for (int j = 0; j < CPT; ++j) b1[j] += r[j];
+        }
     }
     if (ok0) {
         store_row<CPT>(dk + pt0 * C + t * CPT, a0);
@@ -841,8 +862,8 @@ cudaError_t launch_backward_dq_mma_band(const DevPlan& p, const float* q, const 
     return launch_backward_dq_view(p, fv, q, k, v, dout, out, lse, dq, Dws, N, C, stream);
 }
 
-cudaError_t launch_backward_dkdv_mma(const DevPlan& p, const float* q, const float* k, const float* v, const float* dout,
-                                     const float* lse, const float* Dws, float* dk, float* dv, int N, int C, cudaStream_t stream) {
+static cudaError_t launch_backward_dkdv_view(const DevPlan& p, const FwdView& tv, const float* q, const float* k, const float* v, const float* dout,
+                                             const float* lse, const float* Dws, float* dk, float* dv, int N, int C, cudaStream_t stream) {
     const float scale = 1.0f / sqrtf((float)C);
     const int tiles = p.t_consecutive ? (p.nlon_in + TILE_LON - 1) / TILE_LON : p.ps * ((p.nlon_out + TILE_LON - 1) / TILE_LON);
     const long long tasks = (long long)tiles * ((p.nlat_in + TILE_LAT - 1) / TILE_LAT) * N;
@@ -852,9 +873,21 @@ cudaError_t launch_backward_dkdv_mma(const DevPlan& p, const float* q, const flo
         constexpr int CC = decltype(c)::value;
         cudaError_t e = prepare_kernel(backward_dkdv_mma_kernel<CC>, smem_bytes<CC>());
         if (e != cudaSuccess) return e;
-        backward_dkdv_mma_kernel<CC><<<(unsigned)blocks, THREADS, smem_bytes<CC>(), stream>>>(p, q, k, v, dout, lse, Dws, dk, dv, N, scale, tiles, tasks);
+        backward_dkdv_mma_kernel<CC><<<(unsigned)blocks, THREADS, smem_bytes<CC>(), stream>>>(p, tv, q, k, v, dout, lse, Dws, dk, dv, N, scale, tiles, tasks);
         return cudaGetLastError();
     });
+}
+
+cudaError_t launch_backward_dkdv_mma(const DevPlan& p, const float* q, const float* k, const float* v, const float* dout,
+                                     const float* lse, const float* Dws, float* dk, float* dv, int N, int C, cudaStream_t stream) {
+    const FwdView tv{p.t_stream, p.t_chunk_ptr, p.t_grp_order, nullptr};
+    return launch_backward_dkdv_view(p, tv, q, k, v, dout, lse, Dws, dk, dv, N, C, stream);
+}
+
+cudaError_t launch_backward_dkdv_mma_band(const DevPlan& p, const float* q, const float* k, const float* v, const float* dout,
+                                          const float* lse, const float* Dws, float* dk, float* dv, int N, int C, cudaStream_t stream) {
+    const FwdView tv{p.tb_stream, p.tb_chunk_ptr, p.tb_grp_order, p.t_dense_ptr};
+    return launch_backward_dkdv_view(p, tv, q, k, v, dout, lse, Dws, dk, dv, N, C, stream);
 }
 
 }  // namespace sna

@@ -268,6 +268,18 @@ void build_dense_lists(const HostPlan& P, DenseLists& D) {
     }
 }
 
+void build_transposed_dense_lists(const HostPlan& P, DenseLists& D) {
+    D.ptr.assign(P.nlat_in + 1, 0);
+    D.lat.clear();
+    D.rows.clear();
+    for (int hp = 0; hp < P.nlat_in; ++hp) {
+        for (int e = P.t_row_ptr[hp]; e < P.t_row_ptr[hp + 1]; ++e)
+            if (P.t_windows[e].m < 0) D.lat.push_back(P.t_windows[e].lat);
+        D.ptr[hp + 1] = (int32_t)D.lat.size();
+        if (D.ptr[hp + 1] > D.ptr[hp]) D.rows.push_back(hp);
+    }
+}
+
 void build_forward_stream(const HostPlan& P, Stream& S, bool include_whole) {
     const int groups = (P.nlat_out + TILE_LAT - 1) / TILE_LAT;
     S.chunk_ptr.assign(groups + 1, 0);
@@ -293,7 +305,7 @@ void build_forward_stream(const HostPlan& P, Stream& S, bool include_whole) {
     }
 }
 
-bool build_transposed_stream(const HostPlan& P, Stream& S) {
+bool build_transposed_stream(const HostPlan& P, Stream& S, bool include_whole) {
     const int groups = (P.nlat_in + TILE_LAT - 1) / TILE_LAT;
     S.entries.clear();
     if (TILE_LON % P.ps == 0) {
@@ -308,7 +320,7 @@ bool build_transposed_stream(const HostPlan& P, Stream& S) {
                 int lo = INT32_MAX, hi = INT32_MIN;
                 for (int k = 0; k < TILE_LAT; ++k) {
                     if (m[k] == -2) continue;
-                    if (m[k] < 0) { whole_rows |= ((1u << TILE_LON) - 1u) << (k * TILE_LON); continue; }
+                    if (m[k] < 0) { if (include_whole) whole_rows |= ((1u << TILE_LON) - 1u) << (k * TILE_LON); continue; }
                     lo = std::min(lo, ceil_div(-m[k], P.ps));
                     hi = std::max(hi, floor_div(TILE_LON - 1 + m[k], P.ps));
                 }
@@ -340,6 +352,7 @@ bool build_transposed_stream(const HostPlan& P, Stream& S) {
                 GroupRange rg[TILE_LAT];
                 for (int k = 0; k < TILE_LAT; ++k) {
                     if (m[k] == -2) continue;
+                    if (m[k] < 0 && !include_whole) continue;   // served by the dense kernel
                     rg[k].present = true;
                     if (m[k] < 0) rg[k].whole = true;
                     else { rg[k].lo = ceil_div(r - m[k], P.ps); rg[k].hi = floor_div(r + m[k], P.ps); }

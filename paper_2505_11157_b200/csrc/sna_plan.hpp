@@ -71,6 +71,9 @@ struct DenseLists {
     std::vector<int32_t> rows;   // output latitudes that have at least one whole-ring window
 };
 void build_dense_lists(const HostPlan& plan, DenseLists& out);
+// The transposed lists for the dense dk/dv kernel: input ring h' is attended to as a whole by the output rings
+// lat[ptr[h']] .. lat[ptr[h'+1]-1]; rows = input latitudes with at least one such output ring.
+void build_transposed_dense_lists(const HostPlan& plan, DenseLists& out);
 // Transposed stream for dk/dv; partners are output points (h, w).  Two layouts:
 //  - consecutive (when ps divides 8): one stream row per group of input latitudes; tile rows are 8 consecutive
 //    input columns c = c0 + i%8 (c0 a multiple of 8) and the partner index is c0/ps + e_rel.  Neighbouring
@@ -79,7 +82,7 @@ void build_dense_lists(const HostPlan& plan, DenseLists& out);
 //  - by residue (any other ps): one stream row per (group, residue r); tile rows are c = ps*(u0+i%8) + r and
 //    the partner index is u0 + e_rel.
 // Returns true for the consecutive layout.
-bool build_transposed_stream(const HostPlan& plan, Stream& out);
+bool build_transposed_stream(const HostPlan& plan, Stream& out, bool include_whole = true);
 
 // Builds the plan.  On failure returns a status and fills `why`.
 PlanStatus build_plan(int nlat_in, int nlon_in, int nlat_out, int nlon_out, int grid_in, int grid_out,
