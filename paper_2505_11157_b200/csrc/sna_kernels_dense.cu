@@ -68,8 +68,63 @@ __device__ __forceinline__ void tmem_st32(uint32_t addr, const uint32_t (&r)[32]
         :: "r"(addr), "r"(r[0]),"r"(r[1]),"r"(r[2]),"r"(r[3]),"r"(r[4]),"r"(r[5]),"r"(r[6]),"r"(r[7]),"r"(r[8]),"r"(r[9]),"r"(r[10]),"r"(r[11]),"r"(r[12]),"r"(r[13]),"r"(r[14]),"r"(r[15]),
            "r"(r[16]),"r"(r[17]),"r"(r[18]),"r"(r[19]),"r"(r[20]),"r"(r[21]),"r"(r[22]),"r"(r[23]),"r"(r[24]),"r"(r[25]),"r"(r[26]),"r"(r[27]),"r"(r[28]),"r"(r[29]),"r"(r[30]),"r"(r[31]) : "memory");
 }
+// BF16 UMMA (K = 16 per instruction) for the stacked correction terms: the 16 k-slots of a step hold
+// [a_lo(8) | a_hi(8)] on the A side against [b_hi(8) ; b_lo(8)] on the B side, so one instruction adds
+// a_lo*b_hi + a_hi*b_lo for 8 contraction indices.  A step is 32 bytes, like a TF32 step.
+__device__ __forceinline__ uint32_t umma_idesc16(int n) {
+    return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(DM >> 4) << 24);
+}
+__device__ __forceinline__ void umma_ss16(uint32_t d, uint64_t a, uint64_t b, uint32_t idesc, uint32_t acc) {
+    asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\ttcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, {%5, %5, %5, %5}, p;\n\t}\n"
+                 ::"r"(d), "l"(a), "l"(b), "r"(idesc), "r"(acc), "r"(0u));
+}
+__device__ __forceinline__ void umma_ts16(uint32_t d, uint32_t a_tmem, uint64_t b, uint32_t idesc, uint32_t acc) {
+    asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\ttcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, {%5, %5, %5, %5}, p;\n\t}\n"
+                 ::"r"(d), "r"(a_tmem), "l"(b), "r"(idesc), "r"(acc), "r"(0u));
+}
+// {low half = bf16(x0), high half = bf16(x1)}, round to nearest
+__device__ __forceinline__ uint32_t bf16x2(float x0, float x1) {
+    uint32_t r;
+    asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(x1), "f"(x0));
+    return r;
+}
+__device__ __forceinline__ float trunc19(float x) { return __uint_as_float(__float_as_uint(x) & 0xffffe000u); }
+// Eight values as one 16-byte chunk of BF16.
+__device__ __forceinline__ uint4 bf16x8(const float (&x)[8]) {
+    return make_uint4(bf16x2(x[0], x[1]), bf16x2(x[2], x[3]), bf16x2(x[4], x[5]), bf16x2(x[6], x[7]));
+}
+// A operand in TMEM for the stacked product: per group of 8 columns, 4 words of lo pairs then 4 words of hi pairs.
+// src holds the fp32 values of 32 columns, dst receives the 32 packed words.
+__device__ __forceinline__ void pack_a16(const uint32_t (&src)[32], uint32_t (&dst)[32]) {
+#pragma unroll
+    for (int gq = 0; gq < 4; ++gq) {
+        float hi[8], lo[8];
+#pragma unroll
+        for (int i = 0; i < 8; ++i) { hi[i] = trunc19(__uint_as_float(src[gq * 8 + i])); lo[i] = __uint_as_float(src[gq * 8 + i]) - hi[i]; }
+#pragma unroll
+        for (int i = 0; i < 4; ++i) { dst[gq * 8 + i] = bf16x2(lo[2 * i], lo[2 * i + 1]); dst[gq * 8 + 4 + i] = bf16x2(hi[2 * i], hi[2 * i + 1]); }
+    }
+}
 // Byte offset of the 16-byte chunk c4 of row r inside a [rows x 128 B] swizzled block.
 __device__ __forceinline__ int sw_chunk(int r, int c4) { return r * 128 + ((c4 ^ (r & 7)) << 4); }
+// Eight consecutive channels (group grp) of a point as the two chunks of a stacked BF16 row tile.  A operand: lo then hi;
+// B operand: hi then lo.
+__device__ __forceinline__ void st_stacked8(unsigned char* tile, int row, int grp, const float (&x)[8], bool a_side) {
+    float hi[8], lo[8];
+#pragma unroll
+    for (int i = 0; i < 8; ++i) { hi[i] = trunc19(x[i]); lo[i] = x[i] - hi[i]; }
+    *reinterpret_cast<uint4*>(tile + sw_chunk(row, 2 * grp)) = a_side ? bf16x8(lo) : bf16x8(hi);
+    *reinterpret_cast<uint4*>(tile + sw_chunk(row, 2 * grp + 1)) = a_side ? bf16x8(hi) : bf16x8(lo);
+}
+// Element (row = channel ch, partner column col) of a transposed stacked BF16 tile (B operand of a second contraction):
+// per group of 8 columns 16 slots [hi(8) | lo(8)], 64 slots (32 columns) per 128-byte block.
+__device__ __forceinline__ void st_stacked_t(unsigned char* tile, int ch, int col, float x) {
+    const float hi = trunc19(x);
+    const int kbytes = ((col >> 3) & 3) * 32 + (col & 7) * 2;
+    unsigned char* blk = tile + (col >> 5) * (DC * 128);
+    *reinterpret_cast<unsigned short*>(blk + sw_chunk(ch, kbytes >> 4) + (kbytes & 15)) = (unsigned short)(bf16x2(hi, 0.f) & 0xffffu);
+    *reinterpret_cast<unsigned short*>(blk + sw_chunk(ch, (kbytes + 16) >> 4) + (kbytes & 15)) = (unsigned short)(bf16x2(x - hi, 0.f) & 0xffffu);
+}
 
 __global__ void __launch_bounds__(DM)
 forward_dense_kernel(DevPlan p, const float* __restrict__ q, const float* __restrict__ k, const float* __restrict__ v,
@@ -159,15 +214,21 @@ forward_dense_kernel(DevPlan p, const float* __restrict__ q, const float* __rest
                 // columns warp*16 .. +15 of channel `lane`: K block warp/2, 16-byte chunks (warp%2)*4 .. +3 of row `lane`
 #pragma unroll
                 for (int g4 = 0; g4 < 4; ++g4) {
-                    float hi[4], lo[4];
+                    float hi[4];
 #pragma unroll
-                    for (int i = 0; i < 4; ++i) {
-                        hi[i] = __uint_as_float(__float_as_uint(vraw[4 * g4 + i]) & 0xffffe000u);
-                        lo[i] = vraw[4 * g4 + i] - hi[i];
-                    }
+                    for (int i = 0; i < 4; ++i) hi[i] = trunc19(vraw[4 * g4 + i]);
                     const int off = (warp >> 1) * (DC * 128) + sw_chunk(lane, (warp & 1) * 4 + g4);
                     *reinterpret_cast<float4*>(sVh + off) = make_float4(hi[0], hi[1], hi[2], hi[3]);
-                    *reinterpret_cast<float4*>(sVl + off) = make_float4(lo[0], lo[1], lo[2], lo[3]);
+                }
+                // stacked BF16 tile (row = channel): per group of 8 columns a 16-byte chunk of hi, then one of lo
+#pragma unroll
+                for (int g8 = 0; g8 < 2; ++g8) {
+                    float hi[8], lo[8];
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) { hi[i] = trunc19(vraw[8 * g8 + i]); lo[i] = vraw[8 * g8 + i] - hi[i]; }
+                    const int chunk = ((warp & 1) * 2 + g8) * 2;
+                    *reinterpret_cast<uint4*>(sVl + (warp >> 1) * (DC * 128) + sw_chunk(lane, chunk)) = bf16x8(hi);
+                    *reinterpret_cast<uint4*>(sVl + (warp >> 1) * (DC * 128) + sw_chunk(lane, chunk + 1)) = bf16x8(lo);
                 }
             }
             if (it + 1 < total) fetch(it + 1);
@@ -219,8 +280,8 @@ forward_dense_kernel(DevPlan p, const float* __restrict__ q, const float* __rest
                     const float pj = ex2d(__uint_as_float(s0[j]) - m);
                     ps += pj;
                     s0[j] = __float_as_uint(pj);
-                    lo[j] = __float_as_uint(pj - __uint_as_float(s0[j] & 0xffffe000u));
                 }
+                pack_a16(s0, lo);
                 tmem_st32(tPh + lanebits, s0);
                 tmem_st32(tPl + lanebits, lo);
 #pragma unroll
@@ -228,8 +289,8 @@ forward_dense_kernel(DevPlan p, const float* __restrict__ q, const float* __rest
                     const float pj = ex2d(__uint_as_float(s1[j]) - m);
                     ps += pj;
                     s1[j] = __float_as_uint(pj);
-                    lo[j] = __float_as_uint(pj - __uint_as_float(s1[j] & 0xffffe000u));
                 }
+                pack_a16(s1, lo);
                 tmem_st32(tPh + lanebits + 32, s1);
                 tmem_st32(tPl + lanebits + 32, lo);
                 asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
@@ -240,10 +301,9 @@ forward_dense_kernel(DevPlan p, const float* __restrict__ q, const float* __rest
             if (tid == 0 && ok) {
                 asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
                 const uint64_t vh0 = umma_desc(smem_u32(sVh)), vl0 = umma_desc(smem_u32(sVl));
+                // corrections p_lo v_hi + p_hi v_lo: one BF16 UMMA per 8 columns; main term p_hi v_hi: one TF32 UMMA per 8 columns
 #pragma unroll
-                for (int ks2 = 0; ks2 < DBN / 8; ++ks2) umma_ts(tO, tPl + ks2 * 8, vh0 + (uint64_t)((ks2 >> 2) * (DC * 128 >> 4) + (ks2 & 3) * 2), idO, ks2 > 0);
-#pragma unroll
-                for (int ks2 = 0; ks2 < DBN / 8; ++ks2) umma_ts(tO, tPh + ks2 * 8, vl0 + (uint64_t)((ks2 >> 2) * (DC * 128 >> 4) + (ks2 & 3) * 2), idO, 1);
+                for (int ks2 = 0; ks2 < DBN / 8; ++ks2) umma_ts16(tO, tPl + ks2 * 8, vl0 + (uint64_t)((ks2 >> 2) * (DC * 128 >> 4) + (ks2 & 3) * 2), umma_idesc16(DC), ks2 > 0);
 #pragma unroll
                 for (int ks2 = 0; ks2 < DBN / 8; ++ks2) umma_ts(tO, tPh + ks2 * 8, vh0 + (uint64_t)((ks2 >> 2) * (DC * 128 >> 4) + (ks2 & 3) * 2), idO, 1);
                 umma_commit(bar);
@@ -305,25 +365,24 @@ backward_dq_dense_kernel(DevPlan p, const float* __restrict__ q, const float* __
     const float scale_log2 = scale * LOG2E_D;
 
     float D = 0.f;
-    {   // this thread's q row (log2 domain) and dout row as tile row tid; D = dout . out
+    {   // this thread's q row (log2 domain) and dout row as tile row tid (fp32 hi tile + stacked BF16 tile); D = dout . out
         const float4* qs = reinterpret_cast<const float4*>(q + opt * DC);
         const float4* ys = reinterpret_cast<const float4*>(dout + opt * DC);
         const float4* os = reinterpret_cast<const float4*>(out + opt * DC);
 #pragma unroll
-        for (int c4 = 0; c4 < DC / 4; ++c4) {
-            float4 x = __ldg(qs + c4);
-            x.x *= scale_log2; x.y *= scale_log2; x.z *= scale_log2; x.w *= scale_log2;
-            float4 hi;
-            hi.x = __uint_as_float(__float_as_uint(x.x) & 0xffffe000u); hi.y = __uint_as_float(__float_as_uint(x.y) & 0xffffe000u);
-            hi.z = __uint_as_float(__float_as_uint(x.z) & 0xffffe000u); hi.w = __uint_as_float(__float_as_uint(x.w) & 0xffffe000u);
-            *reinterpret_cast<float4*>(sQh + sw_chunk(tid, c4)) = hi;
-            *reinterpret_cast<float4*>(sQl + sw_chunk(tid, c4)) = make_float4(x.x - hi.x, x.y - hi.y, x.z - hi.z, x.w - hi.w);
-            const float4 y = __ldg(ys + c4), o4 = __ldg(os + c4);
-            D = fmaf(y.x, o4.x, fmaf(y.y, o4.y, fmaf(y.z, o4.z, fmaf(y.w, o4.w, D))));
-            hi.x = __uint_as_float(__float_as_uint(y.x) & 0xffffe000u); hi.y = __uint_as_float(__float_as_uint(y.y) & 0xffffe000u);
-            hi.z = __uint_as_float(__float_as_uint(y.z) & 0xffffe000u); hi.w = __uint_as_float(__float_as_uint(y.w) & 0xffffe000u);
-            *reinterpret_cast<float4*>(sYh + sw_chunk(tid, c4)) = hi;
-            *reinterpret_cast<float4*>(sYl + sw_chunk(tid, c4)) = make_float4(y.x - hi.x, y.y - hi.y, y.z - hi.z, y.w - hi.w);
+        for (int grp = 0; grp < DC / 8; ++grp) {
+            float x[8], y[8];
+#pragma unroll
+            for (int hh = 0; hh < 2; ++hh) {
+                const float4 a = __ldg(qs + 2 * grp + hh), b = __ldg(ys + 2 * grp + hh), o4 = __ldg(os + 2 * grp + hh);
+                x[4 * hh] = a.x * scale_log2; x[4 * hh + 1] = a.y * scale_log2; x[4 * hh + 2] = a.z * scale_log2; x[4 * hh + 3] = a.w * scale_log2;
+                y[4 * hh] = b.x; y[4 * hh + 1] = b.y; y[4 * hh + 2] = b.z; y[4 * hh + 3] = b.w;
+                D = fmaf(b.x, o4.x, fmaf(b.y, o4.y, fmaf(b.z, o4.z, fmaf(b.w, o4.w, D))));
+                *reinterpret_cast<float4*>(sQh + sw_chunk(tid, 2 * grp + hh)) = make_float4(trunc19(x[4 * hh]), trunc19(x[4 * hh + 1]), trunc19(x[4 * hh + 2]), trunc19(x[4 * hh + 3]));
+                *reinterpret_cast<float4*>(sYh + sw_chunk(tid, 2 * grp + hh)) = make_float4(trunc19(b.x), trunc19(b.y), trunc19(b.z), trunc19(b.w));
+            }
+            st_stacked8(sQl, tid, grp, x, true);
+            st_stacked8(sYl, tid, grp, y, true);
         }
     }
     const float nl = -__ldg(lse + opt) * LOG2E_D;
@@ -370,12 +429,18 @@ backward_dq_dense_kernel(DevPlan p, const float* __restrict__ q, const float* __
         const float bias = p.log2_omega[p.dense_lat[e_begin + it / nblk]] + nl;
         const int c0 = (it % nblk) * DBN;
 #pragma unroll
-        for (int j = 0; j < 4; ++j) {   // k and v rows of this block, both with the channels as K dimension
-            const float4 kh = hi4(kcur[j]), vh = hi4(vcur[j]);
-            *reinterpret_cast<float4*>(sKh + sw_chunk(col, half * 4 + j)) = kh;
-            *reinterpret_cast<float4*>(sKl + sw_chunk(col, half * 4 + j)) = make_float4(kcur[j].x - kh.x, kcur[j].y - kh.y, kcur[j].z - kh.z, kcur[j].w - kh.w);
-            *reinterpret_cast<float4*>(sVh + sw_chunk(col, half * 4 + j)) = vh;
-            *reinterpret_cast<float4*>(sVl + sw_chunk(col, half * 4 + j)) = make_float4(vcur[j].x - vh.x, vcur[j].y - vh.y, vcur[j].z - vh.z, vcur[j].w - vh.w);
+        for (int g2 = 0; g2 < 2; ++g2) {   // k and v rows of this block (channels as K dimension): fp32 hi tile + stacked BF16 tile
+            float kx[8], vx[8];
+#pragma unroll
+            for (int hh = 0; hh < 2; ++hh) {
+                const float4 a = kcur[2 * g2 + hh], b = vcur[2 * g2 + hh];
+                kx[4 * hh] = a.x; kx[4 * hh + 1] = a.y; kx[4 * hh + 2] = a.z; kx[4 * hh + 3] = a.w;
+                vx[4 * hh] = b.x; vx[4 * hh + 1] = b.y; vx[4 * hh + 2] = b.z; vx[4 * hh + 3] = b.w;
+                *reinterpret_cast<float4*>(sKh + sw_chunk(col, half * 4 + 2 * g2 + hh)) = hi4(a);
+                *reinterpret_cast<float4*>(sVh + sw_chunk(col, half * 4 + 2 * g2 + hh)) = hi4(b);
+            }
+            st_stacked8(sKl, col, half * 2 + g2, kx, false);
+            st_stacked8(sVl, col, half * 2 + g2, vx, false);
         }
         if (it + 1 < total) fetch(it + 1, knext, vnext);
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -385,10 +450,9 @@ backward_dq_dense_kernel(DevPlan p, const float* __restrict__ q, const float* __
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
             const uint64_t qh = umma_desc(smem_u32(sQh)), ql = umma_desc(smem_u32(sQl)), yh = umma_desc(smem_u32(sYh)), yl = umma_desc(smem_u32(sYl));
             const uint64_t kh = umma_desc(smem_u32(sKh)), kl = umma_desc(smem_u32(sKl)), vh = umma_desc(smem_u32(sVh)), vl = umma_desc(smem_u32(sVl));
+            // per 8 channels: one BF16 UMMA for both correction terms, one TF32 UMMA for the main term
 #pragma unroll
-            for (int ks2 = 0; ks2 < DC / 8; ++ks2) { umma_ss(tS, ql + 2 * ks2, kh + 2 * ks2, idS, ks2 > 0); umma_ss(tT, yl + 2 * ks2, vh + 2 * ks2, idS, ks2 > 0); }
-#pragma unroll
-            for (int ks2 = 0; ks2 < DC / 8; ++ks2) { umma_ss(tS, qh + 2 * ks2, kl + 2 * ks2, idS, 1); umma_ss(tT, yh + 2 * ks2, vl + 2 * ks2, idS, 1); }
+            for (int ks2 = 0; ks2 < DC / 8; ++ks2) { umma_ss16(tS, ql + 2 * ks2, kl + 2 * ks2, umma_idesc16(DBN), ks2 > 0); umma_ss16(tT, yl + 2 * ks2, vl + 2 * ks2, umma_idesc16(DBN), ks2 > 0); }
 #pragma unroll
             for (int ks2 = 0; ks2 < DC / 8; ++ks2) { umma_ss(tS, qh + 2 * ks2, kh + 2 * ks2, idS, 1); umma_ss(tT, yh + 2 * ks2, vh + 2 * ks2, idS, 1); }
             umma_commit(bar);
@@ -408,8 +472,8 @@ backward_dq_dense_kernel(DevPlan p, const float* __restrict__ q, const float* __
                     const float pj = hf * 32 + j < nvalid ? ex2d(__uint_as_float(sv[j]) + bias) : 0.f;
                     const float ds = pj * (__uint_as_float(tv[j]) - D);
                     sv[j] = __float_as_uint(ds);
-                    tv[j] = __float_as_uint(ds - __uint_as_float(sv[j] & 0xffffe000u));
                 }
+                pack_a16(sv, tv);
                 tmem_st32(tS + lanebits + hf * 32, sv);
                 tmem_st32(tT + lanebits + hf * 32, tv);
             }
@@ -422,10 +486,8 @@ backward_dq_dense_kernel(DevPlan p, const float* __restrict__ q, const float* __
 #pragma unroll
                 for (int i = 0; i < 4; ++i) {
                     const int ch = half * 16 + 4 * j + i;
-                    const int off = kb * (DC * 128) + sw_chunk(ch, kc >> 2) + (kc & 3) * 4;
-                    const float g = __uint_as_float(__float_as_uint(xv[i]) & 0xffffe000u);
-                    *reinterpret_cast<float*>(sVh + off) = g;
-                    *reinterpret_cast<float*>(sVl + off) = xv[i] - g;
+                    *reinterpret_cast<float*>(sVh + kb * (DC * 128) + sw_chunk(ch, kc >> 2) + (kc & 3) * 4) = trunc19(xv[i]);
+                    st_stacked_t(sVl, ch, col, xv[i]);
                 }
             }
         }
@@ -436,9 +498,7 @@ backward_dq_dense_kernel(DevPlan p, const float* __restrict__ q, const float* __
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
             const uint64_t th0 = umma_desc(smem_u32(sVh)), tl0 = umma_desc(smem_u32(sVl));
 #pragma unroll
-            for (int ks2 = 0; ks2 < DBN / 8; ++ks2) umma_ts(tG, tT + ks2 * 8, th0 + (uint64_t)((ks2 >> 2) * (DC * 128 >> 4) + (ks2 & 3) * 2), idO, ks2 > 0);
-#pragma unroll
-            for (int ks2 = 0; ks2 < DBN / 8; ++ks2) umma_ts(tG, tS + ks2 * 8, tl0 + (uint64_t)((ks2 >> 2) * (DC * 128 >> 4) + (ks2 & 3) * 2), idO, 1);
+            for (int ks2 = 0; ks2 < DBN / 8; ++ks2) umma_ts16(tG, tT + ks2 * 8, tl0 + (uint64_t)((ks2 >> 2) * (DC * 128 >> 4) + (ks2 & 3) * 2), umma_idesc16(DC), ks2 > 0);
 #pragma unroll
             for (int ks2 = 0; ks2 < DBN / 8; ++ks2) umma_ts(tG, tS + ks2 * 8, th0 + (uint64_t)((ks2 >> 2) * (DC * 128 >> 4) + (ks2 & 3) * 2), idO, 1);
             umma_commit(bar);
@@ -501,23 +561,22 @@ backward_dkdv_dense_kernel(DevPlan p, const float* __restrict__ q, const float* 
     const float scale_log2 = scale * LOG2E_D;
     const float bias = p.log2_omega[hp];
 
-    {   // this thread's k row (log2 domain) and v row as tile row tid
+    {   // this thread's k row (log2 domain) and v row as tile row tid: fp32 hi tile + stacked BF16 tile
         const float4* ks = reinterpret_cast<const float4*>(k + ipt * DC);
         const float4* vs = reinterpret_cast<const float4*>(v + ipt * DC);
 #pragma unroll
-        for (int c4 = 0; c4 < DC / 4; ++c4) {
-            float4 x = __ldg(ks + c4);
-            x.x *= scale_log2; x.y *= scale_log2; x.z *= scale_log2; x.w *= scale_log2;
-            float4 hi;
-            hi.x = __uint_as_float(__float_as_uint(x.x) & 0xffffe000u); hi.y = __uint_as_float(__float_as_uint(x.y) & 0xffffe000u);
-            hi.z = __uint_as_float(__float_as_uint(x.z) & 0xffffe000u); hi.w = __uint_as_float(__float_as_uint(x.w) & 0xffffe000u);
-            *reinterpret_cast<float4*>(sKh + sw_chunk(tid, c4)) = hi;
-            *reinterpret_cast<float4*>(sKl + sw_chunk(tid, c4)) = make_float4(x.x - hi.x, x.y - hi.y, x.z - hi.z, x.w - hi.w);
-            const float4 y = __ldg(vs + c4);
-            hi.x = __uint_as_float(__float_as_uint(y.x) & 0xffffe000u); hi.y = __uint_as_float(__float_as_uint(y.y) & 0xffffe000u);
-            hi.z = __uint_as_float(__float_as_uint(y.z) & 0xffffe000u); hi.w = __uint_as_float(__float_as_uint(y.w) & 0xffffe000u);
-            *reinterpret_cast<float4*>(sVh + sw_chunk(tid, c4)) = hi;
-            *reinterpret_cast<float4*>(sVl + sw_chunk(tid, c4)) = make_float4(y.x - hi.x, y.y - hi.y, y.z - hi.z, y.w - hi.w);
+        for (int grp = 0; grp < DC / 8; ++grp) {
+            float x[8], y[8];
+#pragma unroll
+            for (int hh = 0; hh < 2; ++hh) {
+                const float4 a = __ldg(ks + 2 * grp + hh), b = __ldg(vs + 2 * grp + hh);
+                x[4 * hh] = a.x * scale_log2; x[4 * hh + 1] = a.y * scale_log2; x[4 * hh + 2] = a.z * scale_log2; x[4 * hh + 3] = a.w * scale_log2;
+                y[4 * hh] = b.x; y[4 * hh + 1] = b.y; y[4 * hh + 2] = b.z; y[4 * hh + 3] = b.w;
+                *reinterpret_cast<float4*>(sKh + sw_chunk(tid, 2 * grp + hh)) = make_float4(trunc19(x[4 * hh]), trunc19(x[4 * hh + 1]), trunc19(x[4 * hh + 2]), trunc19(x[4 * hh + 3]));
+                *reinterpret_cast<float4*>(sVh + sw_chunk(tid, 2 * grp + hh)) = make_float4(trunc19(b.x), trunc19(b.y), trunc19(b.z), trunc19(b.w));
+            }
+            st_stacked8(sKl, tid, grp, x, true);
+            st_stacked8(sVl, tid, grp, y, true);
         }
     }
     if (tid == 0) {
@@ -557,24 +616,28 @@ backward_dkdv_dense_kernel(DevPlan p, const float* __restrict__ q, const float* 
         return make_float4(__uint_as_float(__float_as_uint(x.x) & 0xffffe000u), __uint_as_float(__float_as_uint(x.y) & 0xffffe000u),
                            __uint_as_float(__float_as_uint(x.z) & 0xffffe000u), __uint_as_float(__float_as_uint(x.w) & 0xffffe000u));
     };
-    // element (row = channel, K index = partner column) of a transposed 32 x 64 tile
+    // element (row = channel, K index = partner column) of a transposed tile: fp32 hi tile and stacked BF16 tile
     auto st_t = [&](unsigned char* th, unsigned char* tl, int ch, float x) {
-        const int off = (col >> 5) * (DC * 128) + sw_chunk(ch, (col & 31) >> 2) + (col & 3) * 4;
-        const float g = __uint_as_float(__float_as_uint(x) & 0xffffe000u);
-        *reinterpret_cast<float*>(th + off) = g;
-        *reinterpret_cast<float*>(tl + off) = x - g;
+        *reinterpret_cast<float*>(th + (col >> 5) * (DC * 128) + sw_chunk(ch, (col & 31) >> 2) + (col & 3) * 4) = trunc19(x);
+        st_stacked_t(tl, ch, col, x);
     };
     if (total > 0) fetch(0, qcur, ycur);
     for (int it = 0; it < total && ok; ++it) {
         const int h = p.t_dense_lat[e_begin + it / nblk];
         const int w0 = (it % nblk) * DBN;
 #pragma unroll
-        for (int j = 0; j < 4; ++j) {   // q and dout rows of the partner points, channels as K dimension
-            const float4 qh = hi4(qcur[j]), yh = hi4(ycur[j]);
-            *reinterpret_cast<float4*>(sQh + sw_chunk(col, half * 4 + j)) = qh;
-            *reinterpret_cast<float4*>(sQl + sw_chunk(col, half * 4 + j)) = make_float4(qcur[j].x - qh.x, qcur[j].y - qh.y, qcur[j].z - qh.z, qcur[j].w - qh.w);
-            *reinterpret_cast<float4*>(sYh + sw_chunk(col, half * 4 + j)) = yh;
-            *reinterpret_cast<float4*>(sYl + sw_chunk(col, half * 4 + j)) = make_float4(ycur[j].x - yh.x, ycur[j].y - yh.y, ycur[j].z - yh.z, ycur[j].w - yh.w);
+        for (int g2 = 0; g2 < 2; ++g2) {   // q and dout rows of the partner points (channels as K dimension)
+            float qx[8], yx[8];
+#pragma unroll
+            for (int hh = 0; hh < 2; ++hh) {
+                const float4 a = qcur[2 * g2 + hh], b = ycur[2 * g2 + hh];
+                qx[4 * hh] = a.x; qx[4 * hh + 1] = a.y; qx[4 * hh + 2] = a.z; qx[4 * hh + 3] = a.w;
+                yx[4 * hh] = b.x; yx[4 * hh + 1] = b.y; yx[4 * hh + 2] = b.z; yx[4 * hh + 3] = b.w;
+                *reinterpret_cast<float4*>(sQh + sw_chunk(col, half * 4 + 2 * g2 + hh)) = hi4(a);
+                *reinterpret_cast<float4*>(sYh + sw_chunk(col, half * 4 + 2 * g2 + hh)) = hi4(b);
+            }
+            st_stacked8(sQl, col, half * 2 + g2, qx, false);
+            st_stacked8(sYl, col, half * 2 + g2, yx, false);
         }
         if (tid < DBN) {
             const size_t o = (size_t)(n * p.nlat_out + h) * p.nlon_out + min(w0 + tid, p.nlon_out - 1);
@@ -590,9 +653,7 @@ backward_dkdv_dense_kernel(DevPlan p, const float* __restrict__ q, const float* 
             const uint64_t kh = umma_desc(smem_u32(sKh)), kl = umma_desc(smem_u32(sKl)), vh = umma_desc(smem_u32(sVh)), vl = umma_desc(smem_u32(sVl));
             const uint64_t qh = umma_desc(smem_u32(sQh)), ql = umma_desc(smem_u32(sQl)), yh = umma_desc(smem_u32(sYh)), yl = umma_desc(smem_u32(sYl));
 #pragma unroll
-            for (int ks2 = 0; ks2 < DC / 8; ++ks2) { umma_ss(tS, kl + 2 * ks2, qh + 2 * ks2, idS, ks2 > 0); umma_ss(tT, vl + 2 * ks2, yh + 2 * ks2, idS, ks2 > 0); }
-#pragma unroll
-            for (int ks2 = 0; ks2 < DC / 8; ++ks2) { umma_ss(tS, kh + 2 * ks2, ql + 2 * ks2, idS, 1); umma_ss(tT, vh + 2 * ks2, yl + 2 * ks2, idS, 1); }
+            for (int ks2 = 0; ks2 < DC / 8; ++ks2) { umma_ss16(tS, kl + 2 * ks2, ql + 2 * ks2, umma_idesc16(DBN), ks2 > 0); umma_ss16(tT, vl + 2 * ks2, yl + 2 * ks2, umma_idesc16(DBN), ks2 > 0); }
 #pragma unroll
             for (int ks2 = 0; ks2 < DC / 8; ++ks2) { umma_ss(tS, kh + 2 * ks2, qh + 2 * ks2, idS, 1); umma_ss(tT, vh + 2 * ks2, yh + 2 * ks2, idS, 1); }
             umma_commit(bar);
@@ -612,8 +673,8 @@ backward_dkdv_dense_kernel(DevPlan p, const float* __restrict__ q, const float* 
                     const float pj = hf * 32 + j < nvalid ? ex2d(__uint_as_float(sv[j]) + s_nl[hf * 32 + j]) : 0.f;
                     xv[j] = __float_as_uint(pj * (__uint_as_float(tv[j]) - s_D[hf * 32 + j]));
                     sv[j] = __float_as_uint(pj);
-                    tv[j] = __float_as_uint(pj - __uint_as_float(sv[j] & 0xffffe000u));
                 }
+                pack_a16(sv, tv);
                 tmem_st32(tS + lanebits + hf * 32, sv);
                 tmem_st32(tT + lanebits + hf * 32, tv);
                 tmem_st32(tX + lanebits + hf * 32, xv);
@@ -638,23 +699,20 @@ backward_dkdv_dense_kernel(DevPlan p, const float* __restrict__ q, const float* 
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
             const uint64_t yh = umma_desc(smem_u32(sYh)), yl = umma_desc(smem_u32(sYl));
 #pragma unroll
-            for (int ks2 = 0; ks2 < DBN / 8; ++ks2) umma_ts(tGv, tT + ks2 * 8, tdesc(yh, ks2), idO, ks2 > 0);
-#pragma unroll
-            for (int ks2 = 0; ks2 < DBN / 8; ++ks2) umma_ts(tGv, tS + ks2 * 8, tdesc(yl, ks2), idO, 1);
+            for (int ks2 = 0; ks2 < DBN / 8; ++ks2) umma_ts16(tGv, tT + ks2 * 8, tdesc(yl, ks2), umma_idesc16(DC), ks2 > 0);
 #pragma unroll
             for (int ks2 = 0; ks2 < DBN / 8; ++ks2) umma_ts(tGv, tS + ks2 * 8, tdesc(yh, ks2), idO, 1);
             umma_commit(bar);
         }
         if (ok) { ok = wait_bar(bar, phase); phase ^= 1; }
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-        if (ok) {   // dS_lo replaces P_lo; the raw dS block is dS_hi
+        if (ok) {   // the stacked packs of dS replace those of P; the raw dS block is the main-term operand
 #pragma unroll
             for (int hf = 0; hf < 2; ++hf) {
-                uint32_t xv[32];
+                uint32_t xv[32], pk[32];
                 tmem_ld32(xv, tX + lanebits + hf * 32);
-#pragma unroll
-                for (int j = 0; j < 32; ++j) xv[j] = __float_as_uint(__uint_as_float(xv[j]) - __uint_as_float(xv[j] & 0xffffe000u));
-                tmem_st32(tT + lanebits + hf * 32, xv);
+                pack_a16(xv, pk);
+                tmem_st32(tT + lanebits + hf * 32, pk);
             }
             asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
         }
@@ -664,9 +722,7 @@ backward_dkdv_dense_kernel(DevPlan p, const float* __restrict__ q, const float* 
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
             const uint64_t qh = umma_desc(smem_u32(sQh)), ql = umma_desc(smem_u32(sQl));
 #pragma unroll
-            for (int ks2 = 0; ks2 < DBN / 8; ++ks2) umma_ts(tGk, tT + ks2 * 8, tdesc(qh, ks2), idO, ks2 > 0);
-#pragma unroll
-            for (int ks2 = 0; ks2 < DBN / 8; ++ks2) umma_ts(tGk, tX + ks2 * 8, tdesc(ql, ks2), idO, 1);
+            for (int ks2 = 0; ks2 < DBN / 8; ++ks2) umma_ts16(tGk, tT + ks2 * 8, tdesc(ql, ks2), umma_idesc16(DC), ks2 > 0);
 #pragma unroll
             for (int ks2 = 0; ks2 < DBN / 8; ++ks2) umma_ts(tGk, tX + ks2 * 8, tdesc(qh, ks2), idO, 1);
             umma_commit(bar);
