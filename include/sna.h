@@ -19,7 +19,9 @@
  *         k, v, dk, dv     : [B][H][nlat_in ][nlon_in ][C]
  *         lse, and each half of the workspace : [B][H][nlat_out][nlon_out]
  *     Device pointers must be 16-byte aligned.  B*H heads are independent problems.
- *   - C must be one of 4, 8, 16, 32, 64, 128 (SNA_ERR_UNSUPPORTED otherwise).
+ *   - C must be a multiple of 4 between 4 and 128 (SNA_ERR_UNSUPPORTED otherwise).
+ *   - Compute calls must be made with the plan's device current; otherwise they return SNA_ERR_INVALID_ARG and
+ *     launch nothing.
  *   - Compute calls enqueue work on the given CUDA stream (a cudaStream_t passed as void*; NULL is the
  *     default stream) and return without synchronising.  They validate arguments on the host first and
  *     launch nothing if validation fails.  Outputs are overwritten, never accumulated into.

@@ -13,6 +13,9 @@ from . import sna
 class _SphericalNeighborhoodAttention(torch.autograd.Function):
     @staticmethod
     def forward(ctx, plan: "sna.Plan", q, k, v):
+        if q.dtype != torch.float32 or k.dtype != torch.float32 or v.dtype != torch.float32:
+            raise ValueError("spherical_neighborhood_attention computes in float32: cast q, k, v first "
+                             "(autocast does not apply to this operator)")
         q, k, v = q.contiguous(), k.contiguous(), v.contiguous()
         out, lse = plan.forward(q, k, v, return_lse=True)
         ctx.plan = plan
@@ -22,7 +25,7 @@ class _SphericalNeighborhoodAttention(torch.autograd.Function):
     @staticmethod
     def backward(ctx, dout):
         q, k, v, out, lse = ctx.saved_tensors
-        dq, dk, dv = ctx.plan.backward(q, k, v, dout.contiguous(), out=out, lse=lse)
+        dq, dk, dv = ctx.plan.backward(q, k, v, dout.contiguous().float(), out=out, lse=lse)
         return None, dq, dk, dv
 
 

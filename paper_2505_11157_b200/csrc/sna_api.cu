@@ -47,23 +47,24 @@ struct sna_plan {
     mutable std::mutex ws_mutex;
     mutable void* ws = nullptr;        // workspace grown on demand by sna_backward
     mutable size_t ws_bytes = 0;
-    // The dense (tcgen05) kernels run beside the band kernels on a stream of the plan's own and leave their part of the
-    // result in plan-owned scratch; a merge kernel on the caller's stream combines the two.
-    cudaStream_t side = nullptr;
-    cudaEvent_t ev_fork = nullptr, ev_join = nullptr;
-    mutable void* dscratch = nullptr;
-    mutable size_t dscratch_bytes = 0;
 };
 
 namespace {
 
-bool supported_C(int C) { return C == 4 || C == 8 || C == 16 || C == 32 || C == 64 || C == 128; }
+bool supported_C(int C) { return C >= 4 && C <= 128 && C % 4 == 0; }
 
 sna_status_t check_problem(const sna_plan_t* plan, int B, int H, int C) {
     if (plan == nullptr) { set_error("plan is NULL"); return SNA_ERR_INVALID_ARG; }
     if (plan->dev_blob == nullptr) { set_error("plan was created host-only; it cannot compute"); return SNA_ERR_INVALID_ARG; }
     if (B <= 0 || H <= 0 || C <= 0) { set_error("B, H and C must be positive"); return SNA_ERR_INVALID_ARG; }
-    if (!supported_C(C)) { set_error("C=%d unsupported (4, 8, 16, 32, 64 or 128)", C); return SNA_ERR_UNSUPPORTED; }
+    if (!supported_C(C)) { set_error("C=%d unsupported (a multiple of 4 between 4 and 128)", C); return SNA_ERR_UNSUPPORTED; }
+    // The plan's tables, and by contract the caller's tensors, live on the device the plan was created on; launching
+    // with another device current would hand that device foreign addresses.
+    int current = -1;
+    if (cudaGetDevice(&current) != cudaSuccess || current != plan->device) {
+        set_error("the current CUDA device (%d) is not the plan's device (%d)", current, plan->device);
+        return SNA_ERR_INVALID_ARG;
+    }
     const long long N = (long long)B * H;
     const long long big = std::max((long long)plan->host.nlat_in * plan->host.nlon_in,
                                    (long long)plan->host.nlat_out * plan->host.nlon_out);
@@ -78,34 +79,6 @@ size_t stats_elems(const sna_plan_t* plan, int B, int H) {
     return (size_t)B * H * plan->host.nlat_out * plan->host.nlon_out;
 }
 size_t round256(size_t x) { return (x + 255) / 256 * 256; }
-
-// Plan-owned scratch of the dense kernels, grown on demand (a growing call waits for the device first).
-sna_status_t ensure_dense_scratch(const sna_plan_t* plan, size_t bytes, float** out) {
-    std::lock_guard<std::mutex> lock(plan->ws_mutex);
-    if (plan->dscratch_bytes < bytes) {
-        cudaError_t e = cudaDeviceSynchronize();
-        if (e != cudaSuccess) return cuda_fail(e, "cudaDeviceSynchronize");
-        if (plan->dscratch) cudaFree(plan->dscratch);
-        plan->dscratch = nullptr;
-        plan->dscratch_bytes = 0;
-        e = cudaMalloc(&plan->dscratch, bytes);
-        if (e != cudaSuccess) { set_error("cudaMalloc of %zu bytes of dense scratch: %s", bytes, cudaGetErrorString(e)); return SNA_ERR_ALLOC; }
-        plan->dscratch_bytes = bytes;
-    }
-    *out = static_cast<float*>(plan->dscratch);
-    return SNA_OK;
-}
-
-// The side stream starts after everything already enqueued on the caller's stream ...
-cudaError_t fork_side(const sna_plan_t* plan, cudaStream_t main_stream) {
-    cudaError_t e = cudaEventRecord(plan->ev_fork, main_stream);
-    return e != cudaSuccess ? e : cudaStreamWaitEvent(plan->side, plan->ev_fork, 0);
-}
-// ... and the caller's stream continues only after the side stream's work.
-cudaError_t join_side(const sna_plan_t* plan, cudaStream_t main_stream) {
-    cudaError_t e = cudaEventRecord(plan->ev_join, plan->side);
-    return e != cudaSuccess ? e : cudaStreamWaitEvent(main_stream, plan->ev_join, 0);
-}
 
 }  // namespace
 
@@ -252,13 +225,6 @@ static sna_status_t plan_create(int nlat_in, int nlon_in, int nlat_out, int nlon
     d.tb_stream = (const int4*)at(22); d.tb_chunk_ptr = at(23); d.tb_grp_order = at(24);
     d.t_dense_ptr = at(25); d.t_dense_lat = at(26); d.t_dense_rows = at(27);
     d.n_t_dense_rows = (int)t_dense.rows.size();
-    if (cudaStreamCreateWithFlags(&plan->side, cudaStreamNonBlocking) != cudaSuccess ||
-        cudaEventCreateWithFlags(&plan->ev_fork, cudaEventDisableTiming) != cudaSuccess ||
-        cudaEventCreateWithFlags(&plan->ev_join, cudaEventDisableTiming) != cudaSuccess) {
-        sna_plan_destroy(plan);
-        set_error("could not create the plan's side stream and events");
-        return SNA_ERR_CUDA;
-    }
     *plan_out = plan;
     return SNA_OK;
 }
@@ -275,10 +241,6 @@ sna_status_t sna_plan_create_host_only(int nlat_in, int nlon_in, int nlat_out, i
 
 sna_status_t sna_plan_destroy(sna_plan_t* plan) {
     if (plan == nullptr) return SNA_OK;
-    if (plan->side) { cudaStreamSynchronize(plan->side); cudaStreamDestroy(plan->side); }
-    if (plan->ev_fork) cudaEventDestroy(plan->ev_fork);
-    if (plan->ev_join) cudaEventDestroy(plan->ev_join);
-    if (plan->dscratch) cudaFree(plan->dscratch);
     cudaError_t e1 = plan->dev_blob ? cudaFree(plan->dev_blob) : cudaSuccess;
     cudaError_t e2 = plan->ws ? cudaFree(plan->ws) : cudaSuccess;
     delete plan;

@@ -1,5 +1,7 @@
-// Generic kernels: correct for every supported channel count; LP = C/4 lanes hold one grid point, each lane
-// a float4 of channels.  Dot products are reduced with warp shuffles, the softmax is kept online in registers.
+// Generic kernels: correct for every supported channel count (any multiple of 4 up to 128).  A group of LP lanes
+// holds one grid point, each lane a float4 of channels; LP is C/4 rounded up to a power of two, and the surplus
+// lanes of a group carry zeros and store nothing.  Dot products are reduced with warp shuffles, the softmax is kept
+// online in registers.
 // Forward: Eq. (s2_attention_discrete_detailed); backward: App. B.4.
 #include "sna_kernels.cuh"
 
@@ -26,6 +28,8 @@ __device__ __forceinline__ void axpy4(float4& acc, float a, const float4& x) {
 }
 __device__ __forceinline__ void scale4(float4& acc, float a) { acc.x *= a; acc.y *= a; acc.z *= a; acc.w *= a; }
 __device__ __forceinline__ float4 ldg4(const float* p) { return __ldg(reinterpret_cast<const float4*>(p)); }
+// the float4 of a lane that holds channels, zeros for a padding lane
+__device__ __forceinline__ float4 ldg4(const float* p, bool lane_ok) { return lane_ok ? ldg4(p) : make_float4(0.f, 0.f, 0.f, 0.f); }
 
 // Decode a block index into (slice n, output/input latitude, first longitude of the block's tile); the
 // latitudes with the most work come first so the long polar rows do not form the tail of the grid.
@@ -39,17 +43,18 @@ __device__ __forceinline__ void decode_block(int b, int N, int tiles, const int3
 template <int LP>
 __global__ void __launch_bounds__(THREADS)
 forward_generic_kernel(DevPlan p, const float* __restrict__ q, const float* __restrict__ k, const float* __restrict__ v,
-                       float* __restrict__ out, float* __restrict__ lse, int N, float scale_log2) {
-    constexpr int C = LP * 4, PPB = THREADS / LP;
+                       float* __restrict__ out, float* __restrict__ lse, int N, int C, float scale_log2) {
+    constexpr int PPB = THREADS / LP;
     const int tiles = (p.nlon_out + PPB - 1) / PPB;
     int n, h, tile;
     decode_block(blockIdx.x, N, tiles, p.row_order, n, h, tile);
     const int lane = threadIdx.x % LP;
+    const bool lane_ok = lane * 4 < C;
     const int w = tile * PPB + threadIdx.x / LP;
     const bool active = w < p.nlon_out;
     const int wc = active ? w : p.nlon_out - 1;      // inactive groups shadow a valid point (shuffles stay converged)
     const size_t oi = ((size_t)(n * p.nlat_out + h) * p.nlon_out + wc);
-    const float4 qv = ldg4(q + oi * C + lane * 4);
+    const float4 qv = ldg4(q + oi * C + lane * 4, lane_ok);
     float m = -INFINITY, Z = 0.f;
     float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
     const int c0 = wc * p.ps;
@@ -64,8 +69,8 @@ forward_generic_kernel(DevPlan p, const float* __restrict__ q, const float* __re
         for (int j = 0; j < cnt; j += 2) {
             const bool two = j + 1 < cnt;
             int col1 = col + 1; if (col1 >= p.nlon_in) col1 -= p.nlon_in;
-            const float4 k0 = ldg4(kr + (size_t)col * C);
-            const float4 k1 = ldg4(kr + (size_t)(two ? col1 : col) * C);
+            const float4 k0 = ldg4(kr + (size_t)col * C, lane_ok);
+            const float4 k1 = ldg4(kr + (size_t)(two ? col1 : col) * C, lane_ok);
             float s0 = group_sum<LP>(dot4(qv, k0)) * scale_log2 + bias;
             float s1 = two ? group_sum<LP>(dot4(qv, k1)) * scale_log2 + bias : -INFINITY;
             const float mn = fmaxf(m, fmaxf(s0, s1));
@@ -74,8 +79,8 @@ forward_generic_kernel(DevPlan p, const float* __restrict__ q, const float* __re
             Z = fmaf(Z, corr, p0 + p1);
             m = mn;
             if (out != nullptr) {
-                const float4 v0 = ldg4(vr + (size_t)col * C);
-                const float4 v1 = ldg4(vr + (size_t)(two ? col1 : col) * C);
+                const float4 v0 = ldg4(vr + (size_t)col * C, lane_ok);
+                const float4 v1 = ldg4(vr + (size_t)(two ? col1 : col) * C, lane_ok);
                 scale4(acc, corr);
                 axpy4(acc, p0, v0);
                 axpy4(acc, p1, v1);
@@ -84,7 +89,7 @@ forward_generic_kernel(DevPlan p, const float* __restrict__ q, const float* __re
         }
     }
     if (!active) return;
-    if (out != nullptr) {
+    if (out != nullptr && lane_ok) {
         const float inv = 1.f / Z;
         scale4(acc, inv);
         *reinterpret_cast<float4*>(out + oi * C + lane * 4) = acc;
@@ -96,21 +101,22 @@ template <int LP, bool HAVE_OUT>
 __global__ void __launch_bounds__(THREADS)
 backward_dq_generic_kernel(DevPlan p, const float* __restrict__ q, const float* __restrict__ k, const float* __restrict__ v,
                            const float* __restrict__ dout, const float* __restrict__ out, const float* __restrict__ lse,
-                           float* __restrict__ dq, float* __restrict__ Dws, int N, float scale, float scale_log2) {
-    constexpr int C = LP * 4, PPB = THREADS / LP;
+                           float* __restrict__ dq, float* __restrict__ Dws, int N, int C, float scale, float scale_log2) {
+    constexpr int PPB = THREADS / LP;
     const int tiles = (p.nlon_out + PPB - 1) / PPB;
     int n, h, tile;
     decode_block(blockIdx.x, N, tiles, p.row_order, n, h, tile);
     const int lane = threadIdx.x % LP;
+    const bool lane_ok = lane * 4 < C;
     const int w = tile * PPB + threadIdx.x / LP;
     const bool active = w < p.nlon_out;
     const int wc = active ? w : p.nlon_out - 1;
     const size_t oi = ((size_t)(n * p.nlat_out + h) * p.nlon_out + wc);
-    const float4 qv = ldg4(q + oi * C + lane * 4);
-    const float4 dy = ldg4(dout + oi * C + lane * 4);
+    const float4 qv = ldg4(q + oi * C + lane * 4, lane_ok);
+    const float4 dy = ldg4(dout + oi * C + lane * 4, lane_ok);
     const float lse2 = lse[oi] * LOG2E;
     float D = 0.f;
-    if (HAVE_OUT) D = group_sum<LP>(dot4(dy, ldg4(out + oi * C + lane * 4)));
+    if (HAVE_OUT) D = group_sum<LP>(dot4(dy, ldg4(out + oi * C + lane * 4, lane_ok)));
     float4 a1 = make_float4(0.f, 0.f, 0.f, 0.f), a2 = make_float4(0.f, 0.f, 0.f, 0.f);
     float Dacc = 0.f;
     const int c0 = wc * p.ps;
@@ -123,8 +129,8 @@ backward_dq_generic_kernel(DevPlan p, const float* __restrict__ q, const float* 
         const float* kr = k + (size_t)(n * p.nlat_in + hp) * p.nlon_in * C + lane * 4;
         const float* vr = v + (size_t)(n * p.nlat_in + hp) * p.nlon_in * C + lane * 4;
         for (int j = 0; j < cnt; ++j) {
-            const float4 kj = ldg4(kr + (size_t)col * C);
-            const float4 vj = ldg4(vr + (size_t)col * C);
+            const float4 kj = ldg4(kr + (size_t)col * C, lane_ok);
+            const float4 vj = ldg4(vr + (size_t)col * C, lane_ok);
             float s = dot4(qv, kj), t = dot4(dy, vj);
 #pragma unroll
             for (int sh = LP / 2; sh > 0; sh >>= 1) {
@@ -148,7 +154,7 @@ backward_dq_generic_kernel(DevPlan p, const float* __restrict__ q, const float* 
         a1.x -= D * a2.x; a1.y -= D * a2.y; a1.z -= D * a2.z; a1.w -= D * a2.w;
     }
     scale4(a1, scale);
-    *reinterpret_cast<float4*>(dq + oi * C + lane * 4) = a1;
+    if (lane_ok) *reinterpret_cast<float4*>(dq + oi * C + lane * 4) = a1;
     if (lane == 0) Dws[oi] = D;
 }
 
@@ -158,18 +164,19 @@ template <int LP>
 __global__ void __launch_bounds__(THREADS)
 backward_dkdv_generic_kernel(DevPlan p, const float* __restrict__ q, const float* __restrict__ k, const float* __restrict__ v,
                              const float* __restrict__ dout, const float* __restrict__ lse, const float* __restrict__ Dws,
-                             float* __restrict__ dk, float* __restrict__ dv, int N, float scale, float scale_log2) {
-    constexpr int C = LP * 4, PPB = THREADS / LP;
+                             float* __restrict__ dk, float* __restrict__ dv, int N, int C, float scale, float scale_log2) {
+    constexpr int PPB = THREADS / LP;
     const int tiles = (p.nlon_in + PPB - 1) / PPB;
     int n, hp, tile;
     decode_block(blockIdx.x, N, tiles, p.t_row_order, n, hp, tile);
     const int lane = threadIdx.x % LP;
+    const bool lane_ok = lane * 4 < C;
     const int c = tile * PPB + threadIdx.x / LP;
     const bool active = c < p.nlon_in;
     const int cc = active ? c : p.nlon_in - 1;
     const size_t ji = ((size_t)(n * p.nlat_in + hp) * p.nlon_in + cc);
-    const float4 kj = ldg4(k + ji * C + lane * 4);
-    const float4 vj = ldg4(v + ji * C + lane * 4);
+    const float4 kj = ldg4(k + ji * C + lane * 4, lane_ok);
+    const float4 vj = ldg4(v + ji * C + lane * 4, lane_ok);
     const float bias = p.log2_omega[hp];
     float4 gk = make_float4(0.f, 0.f, 0.f, 0.f), gv = make_float4(0.f, 0.f, 0.f, 0.f);
     for (int e = p.t_row_ptr[hp]; e < p.t_row_ptr[hp + 1]; ++e) {
@@ -189,8 +196,8 @@ backward_dkdv_generic_kernel(DevPlan p, const float* __restrict__ q, const float
         for (int j = 0; j < cnt_uniform; ++j) {
             const bool valid = j < cnt;
             const size_t oi = rowbase + w;
-            const float4 qi = ldg4(q + oi * C + lane * 4);
-            const float4 dy = ldg4(dout + oi * C + lane * 4);
+            const float4 qi = ldg4(q + oi * C + lane * 4, lane_ok);
+            const float4 dy = ldg4(dout + oi * C + lane * 4, lane_ok);
             float s = dot4(qi, kj), t = dot4(dy, vj);
 #pragma unroll
             for (int sh = LP / 2; sh > 0; sh >>= 1) {
@@ -205,21 +212,22 @@ backward_dkdv_generic_kernel(DevPlan p, const float* __restrict__ q, const float
     }
     if (!active) return;
     scale4(gk, scale);
-    *reinterpret_cast<float4*>(dk + ji * C + lane * 4) = gk;
-    *reinterpret_cast<float4*>(dv + ji * C + lane * 4) = gv;
+    if (lane_ok) {
+        *reinterpret_cast<float4*>(dk + ji * C + lane * 4) = gk;
+        *reinterpret_cast<float4*>(dv + ji * C + lane * 4) = gv;
+    }
 }
 
 template <typename F>
 cudaError_t dispatch_lp(int C, F&& f) {
-    switch (C) {
-        case 4: return f(std::integral_constant<int, 1>());
-        case 8: return f(std::integral_constant<int, 2>());
-        case 16: return f(std::integral_constant<int, 4>());
-        case 32: return f(std::integral_constant<int, 8>());
-        case 64: return f(std::integral_constant<int, 16>());
-        case 128: return f(std::integral_constant<int, 32>());
-        default: return cudaErrorInvalidValue;
-    }
+    if (C < 4 || C > 128 || C % 4 != 0) return cudaErrorInvalidValue;
+    const int lanes = C / 4;   // rounded up to a power of two
+    if (lanes <= 1) return f(std::integral_constant<int, 1>());
+    if (lanes <= 2) return f(std::integral_constant<int, 2>());
+    if (lanes <= 4) return f(std::integral_constant<int, 4>());
+    if (lanes <= 8) return f(std::integral_constant<int, 8>());
+    if (lanes <= 16) return f(std::integral_constant<int, 16>());
+    return f(std::integral_constant<int, 32>());
 }
 
 }  // namespace
@@ -232,7 +240,7 @@ cudaError_t launch_forward_generic(const DevPlan& p, const float* q, const float
         const int tiles = (p.nlon_out + THREADS / LP - 1) / (THREADS / LP);
         const long long blocks = (long long)tiles * p.nlat_out * N;
         if (blocks > 0x7fffffffLL) return cudaErrorInvalidValue;
-        forward_generic_kernel<LP><<<(unsigned)blocks, THREADS, 0, stream>>>(p, q, k, v, out, lse, N, scale_log2);
+        forward_generic_kernel<LP><<<(unsigned)blocks, THREADS, 0, stream>>>(p, q, k, v, out, lse, N, C, scale_log2);
         return cudaGetLastError();
     });
 }
@@ -247,9 +255,9 @@ cudaError_t launch_backward_dq_generic(const DevPlan& p, const float* q, const f
         const long long blocks = (long long)tiles * p.nlat_out * N;
         if (blocks > 0x7fffffffLL) return cudaErrorInvalidValue;
         if (out != nullptr)
-            backward_dq_generic_kernel<LP, true><<<(unsigned)blocks, THREADS, 0, stream>>>(p, q, k, v, dout, out, lse, dq, Dws, N, scale, scale_log2);
+            backward_dq_generic_kernel<LP, true><<<(unsigned)blocks, THREADS, 0, stream>>>(p, q, k, v, dout, out, lse, dq, Dws, N, C, scale, scale_log2);
         else
-            backward_dq_generic_kernel<LP, false><<<(unsigned)blocks, THREADS, 0, stream>>>(p, q, k, v, dout, out, lse, dq, Dws, N, scale, scale_log2);
+            backward_dq_generic_kernel<LP, false><<<(unsigned)blocks, THREADS, 0, stream>>>(p, q, k, v, dout, out, lse, dq, Dws, N, C, scale, scale_log2);
         return cudaGetLastError();
     });
 }
@@ -263,7 +271,7 @@ cudaError_t launch_backward_dkdv_generic(const DevPlan& p, const float* q, const
         const int tiles = (p.nlon_in + THREADS / LP - 1) / (THREADS / LP);
         const long long blocks = (long long)tiles * p.nlat_in * N;
         if (blocks > 0x7fffffffLL) return cudaErrorInvalidValue;
-        backward_dkdv_generic_kernel<LP><<<(unsigned)blocks, THREADS, 0, stream>>>(p, q, k, v, dout, lse, Dws, dk, dv, N, scale, scale_log2);
+        backward_dkdv_generic_kernel<LP><<<(unsigned)blocks, THREADS, 0, stream>>>(p, q, k, v, dout, lse, Dws, dk, dv, N, C, scale, scale_log2);
         return cudaGetLastError();
     });
 }

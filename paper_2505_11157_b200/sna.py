@@ -257,12 +257,37 @@ class Plan:
             raise ValueError("tensor shapes do not match the plan")
         return B, H, C
 
+    def _validate(self, q, **tensors):
+        """The kernels read raw pointers as contiguous fp32 of the plan's shapes: refuse anything else here, on the
+        host, instead of letting a kernel run past an allocation.  Keyword names select the expected shape:
+        out-grid tensors (q, out, dout, dq), in-grid tensors (k, v, dk, dv) and per-point statistics (lse)."""
+        import torch
+        B, H, C = q.shape[0], q.shape[1], q.shape[4]
+        out_shape = (B, H, self.nlat_out, self.nlon_out, C)
+        in_shape = (B, H, self.nlat_in, self.nlon_in, C)
+        expected = {"q": out_shape, "out": out_shape, "dout": out_shape, "dq": out_shape,
+                    "k": in_shape, "v": in_shape, "dk": in_shape, "dv": in_shape, "lse": out_shape[:-1]}
+        given = {name: t for name, t in dict(q=q, **tensors).items() if t is not None}
+        for name, t in given.items():
+            if not isinstance(t, torch.Tensor):
+                raise ValueError(f"{name} must be a torch.Tensor")
+            if t.dtype != torch.float32:
+                raise ValueError(f"{name} must be float32, got {t.dtype}")
+            if tuple(t.shape) != expected[name]:
+                raise ValueError(f"{name} has shape {tuple(t.shape)}, expected {expected[name]}")
+            if not t.is_contiguous():
+                raise ValueError(f"{name} must be contiguous")
+        for name, t in given.items():
+            if not t.is_cuda or t.device != q.device:
+                raise ValueError(f"{name} must be a CUDA tensor on the device of q ({q.device}), got {t.device}")
+
     def workspace_bytes(self, B, H, C) -> int:
         return sna_workspace_bytes(self.handle, B, H, C)
 
     def forward(self, q, k, v, out=None, lse=None, return_lse=False, stream=None):
         import torch
         B, H, C = self._bhc(q, k)
+        self._validate(q, k=k, v=v, out=out, lse=lse)
         if out is None:
             out = torch.empty_like(q)
         if return_lse and lse is None:
@@ -273,6 +298,9 @@ class Plan:
     def backward(self, q, k, v, dout, out=None, lse=None, dq=None, dk=None, dv=None, workspace=None, stream=None):
         import torch
         B, H, C = self._bhc(q, k)
+        self._validate(q, k=k, v=v, dout=dout, out=out, lse=lse, dq=dq, dk=dk, dv=dv)
+        if workspace is not None and (not workspace.is_cuda or workspace.device != q.device or not workspace.is_contiguous()):
+            raise ValueError("workspace must be a contiguous CUDA tensor on the device of q")
         dq = torch.empty_like(q) if dq is None else dq
         dk = torch.empty_like(k) if dk is None else dk
         dv = torch.empty_like(k) if dv is None else dv
@@ -282,5 +310,5 @@ class Plan:
             need = self.workspace_bytes(B, H, C)
             if workspace is None:
                 workspace = torch.empty(need, dtype=torch.uint8, device=q.device)
-            sna_backward_ex(self.handle, q, k, v, dout, out, lse, dq, dk, dv, workspace, workspace.numel(), B, H, C, stream)
+            sna_backward_ex(self.handle, q, k, v, dout, out, lse, dq, dk, dv, workspace, workspace.numel() * workspace.element_size(), B, H, C, stream)
         return dq, dk, dv

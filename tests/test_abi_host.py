@@ -112,3 +112,33 @@ def test_host_only_plan_refuses_to_compute():
         assert sna._lib.sna_forward(None, 16, 16, 16, 16, 1, 1, 4, None) == sna.SNA_ERR_INVALID_ARG
         assert sna.sna_workspace_bytes(p.handle, 2, 3, 4) == 2 * 3 * 8 * 16 * 2 * 4
         assert sna.sna_workspace_bytes(p.handle, 0, 3, 4) == 0
+
+
+def test_binding_refuses_wrong_dtype_shape_and_device_before_any_launch():
+    """The kernels trust raw pointers, so the binding must stop malformed tensors on the host.  Nothing is
+    launched here: the plan is host-only and every call fails validation first."""
+    import torch
+    with sna.Plan(8, 16, 8, 16, EQ, EQ, 0.9, host_only=True) as p:
+        q = torch.zeros(1, 2, 8, 16, 8)
+        k = torch.zeros(1, 2, 8, 16, 8)
+        with pytest.raises(ValueError, match="float32"):
+            p.forward(q, k, k.half())
+        with pytest.raises(ValueError, match="float32"):
+            p.backward(q, k, k, q.double())
+        with pytest.raises(ValueError, match="shape"):
+            p.forward(q, k, torch.zeros(1, 2, 8, 15, 8))
+        with pytest.raises(ValueError, match="shape"):
+            p.backward(q, k, k, q, lse=torch.zeros(1, 2, 8, 15))
+        with pytest.raises(ValueError, match="shape"):
+            p.backward(q, k, k, q, dk=torch.zeros(1, 2, 8, 16, 4))
+        with pytest.raises(ValueError, match="do not match the plan"):
+            p.forward(torch.zeros(1, 2, 8, 15, 8), k, k)
+        with pytest.raises(ValueError, match="CUDA"):
+            p.forward(q, k, k)          # right dtype and shape, but host memory
+
+
+def test_unsupported_channel_counts_are_refused_on_the_host():
+    with sna.Plan(8, 16, 8, 16, EQ, EQ, 0.9, host_only=True) as p:
+        for C in (0, 3, 6, 130, 132):
+            st = sna._lib.sna_forward(p.handle, 16, 16, 16, 16, 1, 1, C, None)
+            assert st in (sna.SNA_ERR_INVALID_ARG, sna.SNA_ERR_UNSUPPORTED), C

@@ -77,6 +77,10 @@ SMALL = [
     small_workload("global_ragged_dense", 10, 80, 10, 80, GL, GL, math.pi, 2, 1, 32, 34),  # 80 columns: partial last block; 80 rows < 128
     small_workload("global_down2_dense", 12, 288, 7, 144, EQ, EQ, math.pi, 1, 1, 32, 35),  # 144 rows: two row blocks, the second ragged
     small_workload("polar_heavy_c32", 16, 64, 16, 64, EQ, EQ, 1.2, 1, 2, 32, 36),          # dense and banded windows mixed in every row
+    # channel counts that are multiples of 4 but not powers of two (lane groups padded with zero lanes)
+    small_workload("eq_c12", 12, 24, 12, 24, EQ, EQ, 0.6, 1, 2, 12, 37),
+    small_workload("gl_down2_c24", 17, 64, 9, 32, GL, GL, 0.5, 2, 1, 24, 38),
+    small_workload("eq_c48", 10, 40, 10, 40, EQ, EQ, 0.7, 1, 1, 48, 39),
 ]
 
 
@@ -99,7 +103,7 @@ def test_small_cases_full_comparison(wl, reuse):
     assert nerr(dv.reshape(rdv.shape), rdv) <= BWD_TOL
 
 
-@pytest.mark.parametrize("name", ["c2", "c3"])
+@pytest.mark.parametrize("name", ["c2", "c3", "c4", "c5"])
 def test_benchmark_configurations_full_comparison(name):
     wl = WORKLOADS[name]
     g = _geometry(wl)
@@ -208,7 +212,7 @@ def test_argument_errors_launch_nothing():
         qd, kd, vd, dd = _dev(q, k, v, dout)
         out = torch.empty_like(qd)
         with pytest.raises(sna.SnaError) as e:
-            sna.sna_forward(plan.handle, qd, kd, vd, out, wl.B, wl.H, 12)
+            sna.sna_forward(plan.handle, qd, kd, vd, out, wl.B, wl.H, 6)
         assert e.value.status == sna.SNA_ERR_UNSUPPORTED
         with pytest.raises(sna.SnaError) as e:
             sna.sna_forward(plan.handle, qd.data_ptr() + 4, kd, vd, out, wl.B, wl.H, wl.C)
@@ -222,6 +226,31 @@ def test_argument_errors_launch_nothing():
                                 torch.empty_like(kd), ws, ws.numel(), wl.B, wl.H, wl.C)
         assert e.value.status == sna.SNA_ERR_WORKSPACE
         torch.cuda.synchronize()
+
+
+def test_call_with_another_device_current_is_refused_on_the_host():
+    """A plan belongs to the device it was created on.  With another device current the call must fail validation
+    (the check runs on the host before any launch), not launch with the first device's addresses."""
+    if torch.cuda.device_count() < 2:
+        pytest.skip("needs two visible GPUs")
+    wl = SMALL[0]
+    q, k, v, dout = make_inputs(wl)
+    with torch.cuda.device(0):
+        plan = _plan(wl)
+        qd, kd, vd, dd = _dev(q, k, v, dout)
+        out = torch.empty_like(qd)
+    try:
+        with torch.cuda.device(1):
+            with pytest.raises(sna.SnaError) as e:
+                sna.sna_forward(plan.handle, qd, kd, vd, out, wl.B, wl.H, wl.C, stream=0)
+            assert e.value.status == sna.SNA_ERR_INVALID_ARG
+            with pytest.raises(sna.SnaError) as e:
+                sna.sna_backward_static(plan.handle, qd, kd, vd, dd, out, torch.empty_like(kd), torch.empty_like(kd),
+                                        wl.B, wl.H, wl.C, stream=0)
+            assert e.value.status == sna.SNA_ERR_INVALID_ARG
+    finally:
+        with torch.cuda.device(0):
+            plan.close()
 
 
 def test_fp32_fma_peak_probe_is_plausible():
