@@ -225,6 +225,8 @@ static sna_status_t plan_create(int nlat_in, int nlon_in, int nlat_out, int nlon
     d.tb_stream = (const int4*)at(22); d.tb_chunk_ptr = at(23); d.tb_grp_order = at(24);
     d.t_dense_ptr = at(25); d.t_dense_lat = at(26); d.t_dense_rows = at(27);
     d.n_t_dense_rows = (int)t_dense.rows.size();
+    e = sna::dense2_prepare_device();
+    if (e != cudaSuccess) { sna_plan_destroy(plan); return cuda_fail(e, "cudaFuncSetAttribute"); }
     *plan_out = plan;
     return SNA_OK;
 }
@@ -342,7 +344,9 @@ sna_status_t sna_forward_ex(const sna_plan_t* plan, const float* q, const float*
     cudaError_t e;
     if (lse != nullptr && sna::dense_path_supported(plan->dev, C)) {
         // whole-ring windows on the tcgen05 kernel (its partial result travels in out / lse), the rest on the band kernel
-        e = sna::launch_forward_dense(plan->dev, q, k, v, out, lse, B * H, C, (cudaStream_t)cuda_stream);
+        e = sna::dense2_path_supported(plan->dev, C)
+                ? sna::launch_forward_dense2(plan->dev, q, k, v, out, lse, B * H, C, (cudaStream_t)cuda_stream)
+                : sna::launch_forward_dense(plan->dev, q, k, v, out, lse, B * H, C, (cudaStream_t)cuda_stream);
         if (e == cudaSuccess) e = sna::launch_forward_mma_band(plan->dev, q, k, v, out, lse, B * H, C, (cudaStream_t)cuda_stream);
     } else if (sna::mma_path_supported(plan->dev, C)) {
         e = sna::launch_forward_mma(plan->dev, q, k, v, out, lse, B * H, C, (cudaStream_t)cuda_stream);
@@ -511,3 +515,4 @@ extern "C" sna_status_t sna_backward_static(const sna_plan_t* plan, const float*
     return sna_backward_ex(plan, q, k, v, dout, nullptr, nullptr, dq, dk, dv, scratch,
                            sizeof(float) * 2 * (size_t)SNA_STATIC_SCRATCH_MAX_POINTS, B, H, C, cuda_stream);
 }
+

@@ -58,6 +58,11 @@ cudaError_t launch_forward_mma(const DevPlan& p, const float* q, const float* k,
 bool dense_path_supported(const DevPlan& p, int C);
 cudaError_t launch_forward_dense(const DevPlan& p, const float* q, const float* k, const float* v, float* out, float* lse,
                                  int N, int C, cudaStream_t stream);
+// Pipelined version of the dense forward kernel (TMA loads, warp-specialised, see sna_kernels_dense2.cu); same contract.
+cudaError_t dense2_prepare_device();   // once per device: opt in to the kernel's shared-memory size
+bool dense2_path_supported(const DevPlan& p, int C);
+cudaError_t launch_forward_dense2(const DevPlan& p, const float* q, const float* k, const float* v, float* out, float* lse,
+                                  int N, int C, cudaStream_t stream);
 // The same split for the dq stage: the dense kernel writes the whole-ring part of dq (out and dq must be different
 // buffers), the band kernel adds its banded part to it.
 cudaError_t launch_backward_dq_dense(const DevPlan& p, const float* q, const float* k, const float* v, const float* dout,

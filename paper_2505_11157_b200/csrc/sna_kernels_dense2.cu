@@ -1,0 +1,467 @@
+// Pipelined dense forward kernel for whole-ring windows on tcgen05 / TMEM (sm_100a, C = 32).
+//
+// Near the poles, and in the global limit theta_cutoff = pi, an output ring attends to EVERY point of an input ring:
+// that part of Eq. (s2_attention_discrete_detailed) is a dense attention block with the additive bias log omega of
+// App. B.2.  One thread block owns 128 consecutive output longitudes of one ring (the M = 128 rows of the MMA) and walks
+// the ring's whole input rings in blocks of 128 columns.  Unlike the serial kernel in sna_kernels_dense.cu the work of a
+// block is spread over specialised warps that run concurrently, coupled only by mbarriers:
+//
+//   warp 8 (one thread)  TMA: raw k and v tiles of the next blocks, 128 points x 128 bytes, 128-byte swizzle
+//   warps 16-19          convert: k_lo = k - trunc19(k) (same layout as the raw tile), and v transposed and split into
+//                        v_hi^T, v_lo^T (row = channel, K index = column), the K-major form the second GEMM needs
+//   warp 9 (one thread)  S = Q K^T into one of two TMEM buffers: q_lo k + q k_lo + q k as TF32 UMMAs (the raw fp32 tiles
+//                        serve as the hi parts: the tensor core reads only the top 19 bits)
+//   warps 0-3 and 4-7    two softmax groups; thread (half, r) owns tile row r for one half of every block's columns, with
+//                        its own running maximum, sum and output: it reads S from TMEM, scales, adds the bias, writes P
+//                        over S and P_lo = P - trunc19(P) beside it, and folds the previous block's P V into its registers;
+//                        the two halves of a row are merged at the end (a TMEM round trip costs ~130 cycles and one warp
+//                        per scheduler cannot hide it, hence two groups)
+//   warps 12-15 (1 each) O_part = P V over one quarter of the block's columns each (A operand from TMEM), into their own
+//                        accumulators; the row's thread adds its two parts in a fixed order
+//
+// While the softmax threads work on block j, the tensor core computes S of block j+1 and P V of block j-1, TMA loads block
+// j+2 and the converters prepare block j+1.  Every accumulator has exactly one issuing thread and all sums are taken in a
+// fixed order, so results are reproducible bit for bit.  Every wait is bounded; a wait that runs out sets the plan's
+// device status word and the block leaves.
+#include <cuda.h>
+
+#include "sna_kernels.cuh"
+
+#include <cstdint>
+
+namespace sna {
+namespace {
+
+constexpr int M2 = 128;          // tile rows
+constexpr int BN2 = 128;         // columns per block
+constexpr int C2 = 32;           // channels
+constexpr int THREADS2 = 640;        // five warpgroups: softmax (two column halves) | TMA, S issuer | four P V issuers | converters
+constexpr int WAIT2 = 1 << 17;     // polls of one wait (each may suspend for up to ~2 us) before the thread gives up
+constexpr float LOG2E_2 = 1.4426950408889634f;
+constexpr float LN2_2 = 0.6931471805599453f;
+
+// shared-memory map (bytes from a 1024-aligned base)
+constexpr int TILE_B = BN2 * 128;                 // 16 KB: 128 points x 128 bytes
+constexpr int OFF_Q = 0, OFF_QLO = TILE_B;
+constexpr int OFF_K = 2 * TILE_B;                 // 2 stages x (raw, lo)
+constexpr int OFF_VRAW = OFF_K + 4 * TILE_B;      // 2 stages
+constexpr int OFF_VT = OFF_VRAW + 2 * TILE_B;     // 2 stages x (hi^T, lo^T)
+constexpr int OFF_END = OFF_VT + 4 * TILE_B;      // 12 tiles = 192 KB
+constexpr size_t DENSE2_SMEM = OFF_END + 1024;
+
+// TMEM columns
+constexpr int T_S0 = 0, T_S1 = 128, T_PLO = 256, T_O = 384, T_COLS = 512;   // T_O: four 32-column accumulators, one per P V issuer
+constexpr int PV_ISSUERS = 4;
+
+enum { B_KFULL = 0, B_KCONV = 2, B_KFREE = 4, B_VFULL = 6, B_VRAWFREE = 8, B_VCONV = 10, B_PVDONE = 12 /* [half][stage] */, B_SFULL = 16, B_PREADY = 18 /* [half] */, B_QFULL = 20, B_COUNT = 21 };
+
+__device__ __forceinline__ uint32_t s32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ float ex2f(float x) { float y; asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x)); return y; }
+__device__ __forceinline__ float trunc19f(float x) { return __uint_as_float(__float_as_uint(x) & 0xffffe000u); }
+
+__device__ __forceinline__ void mb_init(uint32_t bar, uint32_t count) { asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory"); }
+__device__ __forceinline__ void mb_arrive(uint32_t bar) { asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory"); }
+__device__ __forceinline__ void mb_expect(uint32_t bar, uint32_t bytes) { asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory"); }
+// Bounded wait.  try_wait suspends the thread in hardware for up to the hinted time, so a waiting warp takes few issue
+// slots from the warps that share its scheduler.  Once a wait has run out (`healthy` false) later waits give up at once.
+__device__ __forceinline__ bool mb_wait(uint32_t bar, uint32_t parity, bool healthy) {
+    uint32_t done = 0;
+    const int limit = healthy ? WAIT2 : 4;
+    for (int it = 0; it < limit && !done; ++it)
+        asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\tselp.u32 %0, 1, 0, p;\n\t}\n"
+                     : "=r"(done) : "r"(bar), "r"(parity), "r"(2000u) : "memory");
+    return done != 0;
+}
+__device__ __forceinline__ void tma_tile(uint32_t dst, const CUtensorMap* map, int col, int ring, uint32_t bar) {
+    asm volatile("cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];"
+                 ::"r"(dst), "l"(map), "r"(0), "r"(col), "r"(ring), "r"(bar) : "memory");
+}
+// K-major, 128-byte swizzle: rows of 128 bytes, 8-row groups 1024 bytes apart
+__device__ __forceinline__ uint64_t desc_k(uint32_t saddr) {
+    return (uint64_t)((saddr >> 4) & 0x3fff) | ((uint64_t)1 << 16) | ((uint64_t)(1024 >> 4) << 32) | ((uint64_t)1 << 46) | ((uint64_t)2 << 61);
+}
+__device__ __forceinline__ uint32_t idesc_tf32(int n) {
+    return (1u << 4) | (2u << 7) | (2u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(M2 >> 4) << 24);
+}
+__device__ __forceinline__ void mma_ss(uint32_t d, uint64_t a, uint64_t b, uint32_t idesc, uint32_t acc) {
+    asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\ttcgen05.mma.cta_group::1.kind::tf32 [%0], %1, %2, %3, {%5, %5, %5, %5}, p;\n\t}\n"
+                 ::"r"(d), "l"(a), "l"(b), "r"(idesc), "r"(acc), "r"(0u));
+}
+__device__ __forceinline__ void mma_ts(uint32_t d, uint32_t a_tmem, uint64_t b, uint32_t idesc, uint32_t acc) {
+    asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\ttcgen05.mma.cta_group::1.kind::tf32 [%0], [%1], %2, %3, {%5, %5, %5, %5}, p;\n\t}\n"
+                 ::"r"(d), "r"(a_tmem), "l"(b), "r"(idesc), "r"(acc), "r"(0u));
+}
+__device__ __forceinline__ void mma_commit(uint32_t bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void tm_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+// issue only: the registers are valid after tm_ld_wait()
+__device__ __forceinline__ void tm_ld32_issue(uint32_t (&r)[32], uint32_t addr) {
+    asm volatile("tcgen05.ld.sync.aligned.32x32b.x32.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
+        : "=r"(r[0]),"=r"(r[1]),"=r"(r[2]),"=r"(r[3]),"=r"(r[4]),"=r"(r[5]),"=r"(r[6]),"=r"(r[7]),"=r"(r[8]),"=r"(r[9]),"=r"(r[10]),"=r"(r[11]),"=r"(r[12]),"=r"(r[13]),"=r"(r[14]),"=r"(r[15]),
+          "=r"(r[16]),"=r"(r[17]),"=r"(r[18]),"=r"(r[19]),"=r"(r[20]),"=r"(r[21]),"=r"(r[22]),"=r"(r[23]),"=r"(r[24]),"=r"(r[25]),"=r"(r[26]),"=r"(r[27]),"=r"(r[28]),"=r"(r[29]),"=r"(r[30]),"=r"(r[31]) : "r"(addr) : "memory");
+}
+__device__ __forceinline__ void tm_ld16_issue(uint32_t (&r)[16], uint32_t addr) {
+    asm volatile("tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
+        : "=r"(r[0]),"=r"(r[1]),"=r"(r[2]),"=r"(r[3]),"=r"(r[4]),"=r"(r[5]),"=r"(r[6]),"=r"(r[7]),"=r"(r[8]),"=r"(r[9]),"=r"(r[10]),"=r"(r[11]),"=r"(r[12]),"=r"(r[13]),"=r"(r[14]),"=r"(r[15]) : "r"(addr) : "memory");
+}
+__device__ __forceinline__ void tm_st16(uint32_t addr, const uint32_t (&r)[16]) {
+    asm volatile("tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16};"
+        :: "r"(addr), "r"(r[0]),"r"(r[1]),"r"(r[2]),"r"(r[3]),"r"(r[4]),"r"(r[5]),"r"(r[6]),"r"(r[7]),"r"(r[8]),"r"(r[9]),"r"(r[10]),"r"(r[11]),"r"(r[12]),"r"(r[13]),"r"(r[14]),"r"(r[15]) : "memory");
+}
+__device__ __forceinline__ int sw_off(int row, int c4) { return row * 128 + ((c4 ^ (row & 7)) << 4); }
+
+__global__ void __launch_bounds__(THREADS2, 1)
+forward_dense2_kernel(DevPlan p, const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
+                      const __grid_constant__ CUtensorMap map_v, float* __restrict__ out, float* __restrict__ lse, int N,
+                      float scale_log2, int tiles_per_row) {
+    extern __shared__ unsigned char dense2_raw[];
+    unsigned char* base = (unsigned char*)(((uintptr_t)dense2_raw + 1023) & ~(uintptr_t)1023);
+    __shared__ unsigned long long bars[B_COUNT];
+    __shared__ uint32_t tmem_base_s;
+    __shared__ int fail_s;
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int tile = blockIdx.x % tiles_per_row;
+    const int rest = blockIdx.x / tiles_per_row;
+    const int n = rest % N;
+    const int h = p.dense_rows[rest / N];
+    const int w0 = tile * M2;
+    const int nblk = (p.nlon_in + BN2 - 1) / BN2;
+    const int e_begin = p.dense_ptr[h], e_end = p.dense_ptr[h + 1];
+    const int total = (e_end - e_begin) * nblk;
+
+    if (tid == 0) {
+        for (int s = 0; s < 2; ++s) {
+            mb_init(s32(&bars[B_KFULL + s]), 1);
+            mb_init(s32(&bars[B_KCONV + s]), 128);
+            mb_init(s32(&bars[B_KFREE + s]), 1);
+            mb_init(s32(&bars[B_VFULL + s]), 1);
+            mb_init(s32(&bars[B_VRAWFREE + s]), 128);
+            mb_init(s32(&bars[B_VCONV + s]), 128);
+            mb_init(s32(&bars[B_PVDONE + s]), 2);        // column half 0: two issuers
+            mb_init(s32(&bars[B_PVDONE + 2 + s]), 2);    // column half 1
+            mb_init(s32(&bars[B_SFULL + s]), 1);
+            mb_init(s32(&bars[B_PREADY + s]), 128);      // one per column half (index = half)
+        }
+        mb_init(s32(&bars[B_QFULL]), 1);
+        fail_s = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 0) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(s32(&tmem_base_s)), "r"(T_COLS));
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::);
+    }
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    const uint32_t tm = tmem_base_s;
+    const uint32_t sbase = s32(base);
+    bool ok = true;
+
+    if (warp < 8) {
+        asm volatile("setmaxnreg.inc.sync.aligned.u32 152;");
+        // ------------------------------------------------------------------ softmax: two groups of 128 threads; thread (half, r)
+        // owns tile row r for the columns [64 half, 64 half + 64) of every block, with its own running maximum, sum and output
+        const int half = warp >> 2, r = tid & 127;
+        const uint32_t lanebits = (uint32_t)((warp & 3) * 32) << 16;
+        const int w = w0 + r;
+        const bool row_ok = w < p.nlon_out;
+        constexpr int HC = BN2 / 2;                       // columns per thread and block
+        float m = -INFINITY, l = 0.f, o[C2];
+#pragma unroll
+        for (int i = 0; i < C2; ++i) o[i] = 0.f;
+        float corr_prev = 1.f;
+        for (int it = 0; it <= total && ok; ++it) {
+            float corr = 1.f;
+            if (it > 0) {
+                // fold P V of the previous block (this half's two partial results, fixed order); waiting for it here also
+                // frees this half's P_lo columns and accumulators
+                const int bp = (it - 1) & 1, up = (it - 1) >> 1;
+                ok = mb_wait(s32(&bars[B_PVDONE + 2 * half + bp]), up & 1, ok) && ok;
+                asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                uint32_t oa[32], ob[32];
+                tm_ld32_issue(oa, tm + T_O + half * 64 + lanebits);
+                tm_ld32_issue(ob, tm + T_O + half * 64 + 32 + lanebits);
+                tm_ld_wait();
+#pragma unroll
+                for (int j = 0; j < C2; ++j) o[j] = fmaf(o[j], corr_prev, __uint_as_float(oa[j]) + __uint_as_float(ob[j]));
+            }
+            if (it < total) {
+                const int b = it & 1, u = it >> 1;
+                const int hp = p.dense_lat[e_begin + it / nblk];
+                const float bias = p.log2_omega[hp];
+                const int nvalid = p.nlon_in - (it % nblk) * BN2 - half * HC;     // columns of this thread's half that exist
+                ok = mb_wait(s32(&bars[B_SFULL + b]), u & 1, ok) && ok;
+                asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                const uint32_t tS = tm + (b ? T_S1 : T_S0) + half * HC + lanebits;
+                // pass 1: maximum of the raw scores (the scale is positive and the bias is the same for the whole block)
+                float mxr[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+                {
+                    uint32_t sa[32], sb[32];
+                    tm_ld32_issue(sa, tS);
+                    tm_ld32_issue(sb, tS + 32);
+                    tm_ld_wait();
+                    if (nvalid >= HC) {
+#pragma unroll
+                        for (int j = 0; j < 32; ++j) mxr[j & 3] = fmaxf(mxr[j & 3], fmaxf(__uint_as_float(sa[j]), __uint_as_float(sb[j])));
+                    } else {
+#pragma unroll
+                        for (int j = 0; j < 32; ++j) {
+                            if (j < nvalid) mxr[j & 3] = fmaxf(mxr[j & 3], __uint_as_float(sa[j]));
+                            if (32 + j < nvalid) mxr[j & 3] = fmaxf(mxr[j & 3], __uint_as_float(sb[j]));
+                        }
+                    }
+                }
+                // (a half without any valid column keeps its state: exp2(-inf) = 0 below, and m stays -inf only if nothing was ever seen)
+                const float mblk = fmaf(fmaxf(fmaxf(mxr[0], mxr[1]), fmaxf(mxr[2], mxr[3])), scale_log2, bias);
+                const float mx = fmaxf(m, mblk);
+                const float msafe = mx == -INFINITY ? 0.f : mx;
+                corr = ex2f(m - msafe);
+                m = mx;
+                const float nb = bias - msafe;
+                // pass 2: P over S (its top 19 bits are the hi part) and P_lo = P - trunc19(P) beside it
+                float ps[4] = {0.f, 0.f, 0.f, 0.f};
+                uint32_t bufa[16], bufb[16];
+                auto softmax16 = [&](uint32_t (&x)[16], int c0) {
+                    uint32_t lo[16];
+#pragma unroll
+                    for (int j = 0; j < 16; ++j) {
+                        float pj = ex2f(fmaf(__uint_as_float(x[j]), scale_log2, nb));
+                        if (nvalid < HC && c0 + j >= nvalid) pj = 0.f;
+                        ps[j & 3] += pj;
+                        x[j] = __float_as_uint(pj);
+                        lo[j] = __float_as_uint(pj - trunc19f(pj));
+                    }
+                    tm_st16(tS + c0, x);
+                    tm_st16(tm + T_PLO + half * HC + lanebits + c0, lo);
+                };
+                tm_ld16_issue(bufa, tS);
+#pragma unroll
+                for (int c0 = 0; c0 < HC; c0 += 32) {
+                    tm_ld_wait();
+                    tm_ld16_issue(bufb, tS + c0 + 16);            // in flight while the first 16 columns are processed
+                    softmax16(bufa, c0);
+                    tm_ld_wait();
+                    if (c0 + 32 < HC) tm_ld16_issue(bufa, tS + c0 + 32);
+                    softmax16(bufb, c0 + 16);
+                }
+                l = fmaf(l, corr, (ps[0] + ps[1]) + (ps[2] + ps[3]));
+                asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
+                asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+                mb_arrive(s32(&bars[B_PREADY + half]));
+            }
+            corr_prev = corr;
+        }
+        // merge the two column halves of every row: half 1 hands its state over through shared memory
+        float* xs = reinterpret_cast<float*>(base + OFF_K);         // [34][128] floats in the k stages, which are dead by now
+        if (half == 1) {
+#pragma unroll
+            for (int j = 0; j < C2; ++j) xs[j * 128 + r] = o[j];
+            xs[C2 * 128 + r] = m;
+            xs[(C2 + 1) * 128 + r] = l;
+        }
+        asm volatile("bar.sync 1, 256;" ::: "memory");             // the two softmax groups only
+        if (half == 0 && ok && row_ok) {
+            const float m1 = xs[C2 * 128 + r], l1 = xs[(C2 + 1) * 128 + r];
+            const float mm = fmaxf(m, m1);
+            const float c0 = ex2f(m - mm), c1 = ex2f(m1 - mm);      // mm is finite: half 0 always has valid columns
+            const float lt = l * c0 + l1 * c1;
+            const size_t opt = (size_t)(n * p.nlat_out + h) * p.nlon_out + w;
+            const float inv = 1.f / lt;
+            float4* dst = reinterpret_cast<float4*>(out + opt * C2);
+#pragma unroll
+            for (int c4 = 0; c4 < C2 / 4; ++c4) {
+                float rr[4];
+#pragma unroll
+                for (int i = 0; i < 4; ++i) rr[i] = (o[4 * c4 + i] * c0 + xs[(4 * c4 + i) * 128 + r] * c1) * inv;
+                dst[c4] = make_float4(rr[0], rr[1], rr[2], rr[3]);
+            }
+            lse[opt] = (mm + log2f(lt)) * LN2_2;
+        }
+    } else if (warp < 12) {
+        asm volatile("setmaxnreg.dec.sync.aligned.u32 48;");
+        // ------------------------------------------------------------------ TMA producer
+        if (warp == 8 && lane == 0) {
+            mb_expect(s32(&bars[B_QFULL]), TILE_B);
+            tma_tile(sbase + OFF_Q, &map_q, w0, n * p.nlat_out + h, s32(&bars[B_QFULL]));
+            for (int it = 0; it < total && ok; ++it) {
+                const int s = it & 1, u = it >> 1;
+                const int hp = p.dense_lat[e_begin + it / nblk];
+                const int c0 = (it % nblk) * BN2;
+                if (u > 0) {
+                    ok = mb_wait(s32(&bars[B_KFREE + s]), (u - 1) & 1, ok);
+                    ok = mb_wait(s32(&bars[B_VRAWFREE + s]), (u - 1) & 1, ok) && ok;
+                }
+                mb_expect(s32(&bars[B_KFULL + s]), TILE_B);
+                tma_tile(sbase + OFF_K + s * 2 * TILE_B, &map_k, c0, n * p.nlat_in + hp, s32(&bars[B_KFULL + s]));
+                mb_expect(s32(&bars[B_VFULL + s]), TILE_B);
+                tma_tile(sbase + OFF_VRAW + s * TILE_B, &map_v, c0, n * p.nlat_in + hp, s32(&bars[B_VFULL + s]));
+            }
+        }
+        // ------------------------------------------------------------------ S = Q K^T
+        if (warp == 9 && lane == 0) {
+            ok = mb_wait(s32(&bars[B_QFULL]), 0, ok);
+            // q_lo is written by the converter warps before their first k tile: covered by KCONV of block 0
+            const uint32_t idS = idesc_tf32(BN2);
+            const uint64_t dq = desc_k(sbase + OFF_Q), dql = desc_k(sbase + OFF_QLO);
+            for (int it = 0; it < total && ok; ++it) {
+                const int s = it & 1, u = it >> 1;
+                ok = mb_wait(s32(&bars[B_KFULL + s]), u & 1, ok);
+                ok = mb_wait(s32(&bars[B_KCONV + s]), u & 1, ok) && ok;
+                if (u > 0) {   // P of block it-2 (in this S buffer) has been consumed by both column halves
+                    ok = mb_wait(s32(&bars[B_PVDONE + s]), (u - 1) & 1, ok) && ok;
+                    ok = mb_wait(s32(&bars[B_PVDONE + 2 + s]), (u - 1) & 1, ok) && ok;
+                }
+                asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                const uint64_t dk = desc_k(sbase + OFF_K + s * 2 * TILE_B), dkl = desc_k(sbase + OFF_K + s * 2 * TILE_B + TILE_B);
+                const uint32_t tS = tm + (s ? T_S1 : T_S0);
+#pragma unroll
+                for (int ks = 0; ks < C2 / 8; ++ks) mma_ss(tS, dql + 2 * ks, dk + 2 * ks, idS, ks > 0);
+#pragma unroll
+                for (int ks = 0; ks < C2 / 8; ++ks) mma_ss(tS, dq + 2 * ks, dkl + 2 * ks, idS, 1);
+#pragma unroll
+                for (int ks = 0; ks < C2 / 8; ++ks) mma_ss(tS, dq + 2 * ks, dk + 2 * ks, idS, 1);
+                mma_commit(s32(&bars[B_SFULL + s]));
+                mma_commit(s32(&bars[B_KFREE + s]));
+            }
+        }
+    } else if (warp < 16) {
+        asm volatile("setmaxnreg.dec.sync.aligned.u32 48;");
+        // ------------------------------------------------------------------ O_part = P V over one quarter of the block's columns
+        if (lane == 0) {
+            const int part = warp - 12, half = part >> 1;
+            constexpr int STEPS = BN2 / 8 / PV_ISSUERS;                              // 8-column steps per issuer
+            const uint32_t idO = idesc_tf32(C2);
+            const uint32_t tO = tm + T_O + part * 32;
+            for (int it = 0; it < total && ok; ++it) {
+                const int s = it & 1, u = it >> 1;
+                ok = mb_wait(s32(&bars[B_VCONV + s]), u & 1, ok);
+                ok = mb_wait(s32(&bars[B_PREADY + half]), it & 1, ok) && ok;
+                asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                const uint32_t tP = tm + (s ? T_S1 : T_S0), tPl = tm + T_PLO;
+                const uint32_t vt = sbase + OFF_VT + s * 2 * TILE_B;
+#pragma unroll
+                for (int k8 = 0; k8 < STEPS; ++k8) {
+                    const int ks = part * STEPS + k8;                               // 8-column step within the block
+                    const uint32_t off = (uint32_t)(ks >> 2) * (C2 * 128) + (uint32_t)(ks & 3) * 32;
+                    const uint64_t dvh = desc_k(vt + off), dvl = desc_k(vt + TILE_B + off);
+                    mma_ts(tO, tPl + ks * 8, dvh, idO, k8 > 0);
+                    mma_ts(tO, tP + ks * 8, dvl, idO, 1);
+                    mma_ts(tO, tP + ks * 8, dvh, idO, 1);
+                }
+                mma_commit(s32(&bars[B_PVDONE + 2 * half + s]));
+            }
+        }
+    } else {
+        asm volatile("setmaxnreg.dec.sync.aligned.u32 80;");
+        // ------------------------------------------------------------------ converters (warps 16-19, 128 threads)
+        const int ct = tid - 512, cw = ct >> 5;
+        // q_lo once
+        ok = mb_wait(s32(&bars[B_QFULL]), 0, ok);
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+            const int off = (j * 128 + ct) * 16;
+            const float4 x = *reinterpret_cast<const float4*>(base + OFF_Q + off);
+            *reinterpret_cast<float4*>(base + OFF_QLO + off) = make_float4(x.x - trunc19f(x.x), x.y - trunc19f(x.y), x.z - trunc19f(x.z), x.w - trunc19f(x.w));
+        }
+        for (int it = 0; it < total && ok; ++it) {
+            const int s = it & 1, u = it >> 1;
+            // k_lo: same swizzled position as the raw element
+            ok = mb_wait(s32(&bars[B_KFULL + s]), u & 1, ok);
+            unsigned char* kraw = base + OFF_K + s * 2 * TILE_B;
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+                const int off = (j * 128 + ct) * 16;
+                const float4 x = *reinterpret_cast<const float4*>(kraw + off);
+                *reinterpret_cast<float4*>(kraw + TILE_B + off) = make_float4(x.x - trunc19f(x.x), x.y - trunc19f(x.y), x.z - trunc19f(x.z), x.w - trunc19f(x.w));
+            }
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+            mb_arrive(s32(&bars[B_KCONV + s]));
+            // v transposed: this warp takes the 32 columns [32 cw, 32 cw + 32) (one K block of the transposed tiles), lane = channel
+            ok = mb_wait(s32(&bars[B_VFULL + s]), u & 1, ok) && ok;
+            if (u > 0) {   // the transposed tiles of block it-2 have been consumed by all four issuers
+                ok = mb_wait(s32(&bars[B_PVDONE + s]), (u - 1) & 1, ok) && ok;
+                ok = mb_wait(s32(&bars[B_PVDONE + 2 + s]), (u - 1) & 1, ok) && ok;
+            }
+            const unsigned char* vraw = base + OFF_VRAW + s * TILE_B;
+            unsigned char* vth = base + OFF_VT + s * 2 * TILE_B + cw * (C2 * 128);
+#pragma unroll
+            for (int c8 = 0; c8 < 8; ++c8) {
+                float hi[4], lo[4];
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    const int col = cw * 32 + c8 * 4 + i;
+                    const float x = *reinterpret_cast<const float*>(vraw + sw_off(col, lane >> 2) + (lane & 3) * 4);
+                    hi[i] = trunc19f(x);
+                    lo[i] = x - hi[i];
+                }
+                *reinterpret_cast<float4*>(vth + sw_off(lane, c8)) = make_float4(hi[0], hi[1], hi[2], hi[3]);
+                *reinterpret_cast<float4*>(vth + TILE_B + sw_off(lane, c8)) = make_float4(lo[0], lo[1], lo[2], lo[3]);
+            }
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+            mb_arrive(s32(&bars[B_VRAWFREE + s]));
+            mb_arrive(s32(&bars[B_VCONV + s]));
+        }
+    }
+    if (!ok) atomicExch(&fail_s, 1);
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    if (fail_s && tid == 0) atomicExch(p.dev_status, 1);
+    if (warp == 0) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tm), "r"(T_COLS));
+}
+
+using EncodeFn2 = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                               const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                               CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+EncodeFn2 encode_fn2() {
+    static EncodeFn2 fn = [] {
+        void* sym = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &sym, cudaEnableDefault, &qres) != cudaSuccess ||
+            qres != cudaDriverEntryPointSuccess)
+            sym = nullptr;
+        return reinterpret_cast<EncodeFn2>(sym);
+    }();
+    return fn;
+}
+// Tensor map over a channels-last array [slices * rings][nlon][32] with boxes of 128 points x 32 channels.
+cudaError_t make_map2(CUtensorMap* map, const float* base, int rings_total, int nlon) {
+    EncodeFn2 fn = encode_fn2();
+    if (fn == nullptr) return cudaErrorNotSupported;
+    const cuuint64_t dims[3] = {(cuuint64_t)C2, (cuuint64_t)nlon, (cuuint64_t)rings_total};
+    const cuuint64_t strides[2] = {(cuuint64_t)C2 * 4, (cuuint64_t)nlon * C2 * 4};
+    const cuuint32_t box[3] = {(cuuint32_t)C2, (cuuint32_t)BN2, 1};
+    const cuuint32_t estr[3] = {1, 1, 1};
+    const CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, const_cast<float*>(base), dims, strides, box, estr,
+                          CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                          CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS ? cudaSuccess : cudaErrorInvalidValue;
+}
+
+}  // namespace
+
+cudaError_t dense2_prepare_device() {
+    return cudaFuncSetAttribute(forward_dense2_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)DENSE2_SMEM);
+}
+
+bool dense2_path_supported(const DevPlan& p, int C) {
+    return dense_path_supported(p, C) && encode_fn2() != nullptr;
+}
+
+cudaError_t launch_forward_dense2(const DevPlan& p, const float* q, const float* k, const float* v, float* out, float* lse,
+                                  int N, int C, cudaStream_t stream) {
+    if (C != C2 || lse == nullptr) return cudaErrorInvalidValue;
+    const int tiles_per_row = (p.nlon_out + M2 - 1) / M2;
+    const long long blocks = (long long)tiles_per_row * p.n_dense_rows * N;
+    if (blocks <= 0) return cudaSuccess;
+    if (blocks > 0x7fffffffLL) return cudaErrorInvalidValue;
+    CUtensorMap mq, mk, mv;
+    cudaError_t e = make_map2(&mq, q, N * p.nlat_out, p.nlon_out);
+    if (e == cudaSuccess) e = make_map2(&mk, k, N * p.nlat_in, p.nlon_in);
+    if (e == cudaSuccess) e = make_map2(&mv, v, N * p.nlat_in, p.nlon_in);
+    if (e != cudaSuccess) return e;
+    forward_dense2_kernel<<<(unsigned)blocks, THREADS2, DENSE2_SMEM, stream>>>(p, mq, mk, mv, out, lse, N, LOG2E_2 / sqrtf((float)C), tiles_per_row);
+    return cudaGetLastError();
+}
+
+}  // namespace sna
