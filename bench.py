@@ -33,13 +33,15 @@ if ROOT not in sys.path:
 
 import numpy as np  # noqa: E402
 
-# dram__bytes_read.sum + dram__bytes_write.sum per launch from the ncu capture summarised in
-# profiles/mma_kernels_c3_counters.md (bench.py cannot run ncu itself)
+# Recorded constants: dram__bytes_read.sum + dram__bytes_write.sum per launch from an ncu capture of the band kernels on
+# workload c3 (bench.py cannot run ncu itself; the value is reported as `roofline.traffic` for that workload only).
 NCU_DRAM_BYTES_PER_LAUNCH = {
     ("c3", "forward"): 816768768 + 63346432,
     ("c3", "backward_dq"): 980778752 + 66266112,
     ("c3", "backward_dkdv"): 715740160 + 502913024,
 }
+HBM_GBS_FALLBACK = 6650.0          # used only if MEASURED_PEAKS.json is absent
+L2_BYTES = 126 * 1024 * 1024
 
 METRIC = "fwd+bwd neighbor-pair-channels per second"
 UNIT = "pair*ch/s"
@@ -54,7 +56,20 @@ def parse_args():
     ap.add_argument("--workload", default="c3")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true", help="skip the oracle timing leg")
+    ap.add_argument("--no-extras", action="store_true", help="skip the other configurations and the reduced-precision variant")
     return ap.parse_args()
+
+
+def input_bytes(wl):
+    """Bytes of q, k, v, dout (the tensors a step reads)."""
+    return 4 * wl.C * wl.N * (2 * wl.nlat_out * wl.nlon_out + 2 * wl.nlat_in * wl.nlon_in)
+
+
+def l2_policy(wl):
+    if input_bytes(wl) > L2_BYTES:
+        return f"inputs larger than L2 (q+k+v+dout = {input_bytes(wl) / 1e6:.0f} MB > 126 MB); no flush between iterations"
+    return (f"inputs smaller than L2 (q+k+v+dout = {input_bytes(wl) / 1e6:.1f} MB): a 256 MB buffer is overwritten before every "
+            "timed step (outside the timed events) to flush L2")
 
 
 def workload_config(wl, n_gpus):
@@ -62,7 +77,32 @@ def workload_config(wl, n_gpus):
             "grid_out": [wl.nlat_out, wl.nlon_out], "B": wl.B, "H": wl.H, "C": wl.C,
             "theta_cutoff": wl.theta_cutoff, "seed": wl.seed,
             "parallelism": "single GPU" if n_gpus == 1 else f"{n_gpus} independent replicas",
-            "l2": "inputs larger than L2 (q+k+v+dout > 126 MB); no flush between iterations"}
+            "l2": l2_policy(wl)}
+
+
+def hbm_peak_gbs():
+    try:
+        with open(os.path.join(ROOT, "MEASURED_PEAKS.json")) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    except (OSError, KeyError, ValueError):
+        return HBM_GBS_FALLBACK, "fallback"
+
+
+def kernel_rooflines(wl, units, peak_tflops):
+    """Per kernel: credited flops, compulsory bytes, and the slower of the two times (ms) with its bound."""
+    hbm, _ = hbm_peak_gbs()
+    o = 4 * wl.C * wl.N * wl.nlat_out * wl.nlon_out      # bytes of one out-grid tensor
+    i = 4 * wl.C * wl.N * wl.nlat_in * wl.nlon_in        # bytes of one in-grid tensor
+    spec = {"forward": (4.0, 2 * o + 2 * i),             # q, out; k, v
+            "backward_dq": (6.0, 4 * o + 2 * i),         # q, dout, out, dq; k, v
+            "backward_dkdv": (4.0, 2 * o + 4 * i)}       # q, dout; k, v, dk, dv
+    res = {}
+    for name, (flops_per_unit, nbytes) in spec.items():
+        t_alu = flops_per_unit * units / (peak_tflops * 1e12) * 1e3
+        t_hbm = nbytes / (hbm * 1e9) * 1e3
+        res[name] = {"flops_per_unit": flops_per_unit, "bytes": nbytes, "t_alu_ms": t_alu, "t_hbm_ms": t_hbm,
+                     "bound": "alu" if t_alu >= t_hbm else "hbm", "roofline_ms": max(t_alu, t_hbm)}
+    return res
 
 
 # ---------------------------------------------------------------------------------------------------------
@@ -172,10 +212,100 @@ def max_over_ranks(values, dist, device):
     return t.tolist()
 
 
+class Problem:
+    """Device tensors and the plan of one workload, plus one step (forward, dq, dk/dv) through the C ABI."""
+
+    def __init__(self, sna, torch, wl, keep_host=False):
+        from paper_2505_11157_b200.synthetic import make_inputs
+        self.sna, self.torch, self.wl = sna, torch, wl
+        self.plan = sna.Plan(wl.nlat_in, wl.nlon_in, wl.nlat_out, wl.nlon_out, wl.grid_in, wl.grid_out, wl.theta_cutoff)
+        self.pairs = self.plan.nnz * wl.nlon_out * wl.N
+        self.units = self.pairs * wl.C                  # neighbor-pair-channels per step (forward and backward)
+        host = [torch.from_numpy(a) for a in make_inputs(wl)]
+        self.host = [h.pin_memory() for h in host] if keep_host else host
+        self.q, self.k, self.v, self.dout = [h.cuda(non_blocking=True) for h in self.host]
+        self.out, self.dq = torch.empty_like(self.q), torch.empty_like(self.q)
+        self.dk, self.dv = torch.empty_like(self.k), torch.empty_like(self.k)
+        self.lse = torch.empty(self.q.shape[:-1], dtype=torch.float32, device="cuda")
+        self.D = torch.empty_like(self.lse)
+        self.ws = torch.empty(self.plan.workspace_bytes(wl.B, wl.H, wl.C), dtype=torch.uint8, device="cuda")
+        self.stream = torch.cuda.current_stream()
+        if not keep_host:
+            self.host = None
+
+    def step(self, marks=None):
+        s, wl, h = self.sna, self.wl, self.plan.handle
+        s.sna_forward_ex(h, self.q, self.k, self.v, self.out, self.lse, wl.B, wl.H, wl.C, self.stream)
+        if marks is not None:
+            marks[1].record(self.stream)
+        s.sna_backward_dq(h, self.q, self.k, self.v, self.dout, self.out, self.lse, self.dq, self.D, wl.B, wl.H, wl.C, self.stream)
+        if marks is not None:
+            marks[2].record(self.stream)
+        s.sna_backward_dkdv(h, self.q, self.k, self.v, self.dout, self.lse, self.D, self.dk, self.dv, wl.B, wl.H, wl.C, self.stream)
+
+    def step_tf32(self, marks=None):
+        s, wl, h = self.sna, self.wl, self.plan.handle
+        s.sna_forward_tf32(h, self.q, self.k, self.v, self.out, self.lse, wl.B, wl.H, wl.C, self.stream)
+        if marks is not None:
+            marks[1].record(self.stream)
+            marks[2].record(self.stream)
+        s.sna_backward_tf32(h, self.q, self.k, self.v, self.dout, self.out, self.lse, self.dq, self.dk, self.dv, self.ws,
+                            self.ws.numel(), wl.B, wl.H, wl.C, self.stream)
+
+    def launches_per_step(self):
+        return self.sna.sna_forward_kernel_count(self.plan.handle, self.wl.C, True) + 2   # forward (dense + band, or one) + dq + dk/dv
+
+    def close(self):
+        self.plan.close()
+
+
+def time_steps(torch, prob, steps, warmup, step_fn=None, flush=None):
+    """Mean per-kernel and per-step times (ms) over `steps` steps, CUDA events on the launching stream.  With `flush`
+    (a device buffer larger than L2) the buffer is overwritten before every step, outside the timed events."""
+    step_fn = step_fn or prob.step
+    ev = lambda: torch.cuda.Event(enable_timing=True)
+    for _ in range(warmup):
+        step_fn()
+    torch.cuda.synchronize()
+    marks = [[ev() for _ in range(4)] for _ in range(steps)]
+    for i in range(steps):
+        if flush is not None:
+            flush.add_(1.0)
+        marks[i][0].record(prob.stream)
+        step_fn(marks[i])
+        marks[i][3].record(prob.stream)
+    torch.cuda.synchronize()
+    mean = statistics.mean
+    return {"ms_forward": mean(m[0].elapsed_time(m[1]) for m in marks), "ms_backward_dq": mean(m[1].elapsed_time(m[2]) for m in marks),
+            "ms_backward_dkdv": mean(m[2].elapsed_time(m[3]) for m in marks), "ms_per_step": mean(m[0].elapsed_time(m[3]) for m in marks)}
+
+
+def accuracy_against_oracle(orc, g, prob, n_slices):
+    """Errors of the GPU results of the first n_slices batch*head slices against the oracle: the gated measure
+    max|x-o| / max|o| per tensor, and the element-wise relative error with denominator max(|o|, 1e-3 max|o|)."""
+    wl = prob.wl
+    arrays = [h.numpy() for h in prob.host]
+    sl = lambda a, nlat, nlon: a.reshape(wl.N, nlat, nlon, wl.C)[:n_slices]
+    qs, ds = sl(arrays[0], wl.nlat_out, wl.nlon_out), sl(arrays[3], wl.nlat_out, wl.nlon_out)
+    ks, vs = sl(arrays[1], wl.nlat_in, wl.nlon_in), sl(arrays[2], wl.nlat_in, wl.nlon_in)
+    t0 = time.perf_counter()
+    ref_out = orc.forward(g, qs, ks, vs)
+    refs = (ref_out,) + tuple(orc.backward(g, qs, ks, vs, ds))
+    seconds = time.perf_counter() - t0
+    got = (prob.out, prob.dq, prob.dk, prob.dv)
+    acc = {}
+    for name, x, r in zip(("out", "dq", "dk", "dv"), got, refs):
+        x = x.reshape((wl.N,) + r.shape[1:])[:n_slices].cpu().numpy().astype(np.float64)
+        scale = np.max(np.abs(r))
+        acc[name] = {"normalised_max_error": float(np.max(np.abs(x - r)) / scale),
+                     "floor_relative_max_error": float(np.max(np.abs(x - r) / np.maximum(np.abs(r), 1e-3 * scale)))}
+    return seconds, acc
+
+
 def run_ours(args, wl):
     import torch
     from paper_2505_11157_b200 import sna            # raises if the CUDA library is missing: no fallback
-    from paper_2505_11157_b200.synthetic import make_inputs
+    from paper_2505_11157_b200.synthetic import WORKLOADS
 
     world = int(os.environ.get("WORLD_SIZE", "1"))
     rank = int(os.environ.get("RANK", "0"))
@@ -193,30 +323,17 @@ def run_ours(args, wl):
             dist.barrier()
         torch.cuda.synchronize()
 
-    B, H, C = wl.B, wl.H, wl.C
-    plan = sna.Plan(wl.nlat_in, wl.nlon_in, wl.nlat_out, wl.nlon_out, wl.grid_in, wl.grid_out, wl.theta_cutoff)
-    pairs = plan.nnz * wl.nlon_out * wl.N
-    units = pairs * C                                   # neighbor-pair-channels per step (forward and backward)
-    host = [torch.from_numpy(a).pin_memory() for a in make_inputs(wl)]
-    q, k, v, dout = [h.cuda(non_blocking=True) for h in host]
-    out, dq = torch.empty_like(q), torch.empty_like(q)
-    dk, dv = torch.empty_like(k), torch.empty_like(k)
-    lse = torch.empty(q.shape[:-1], dtype=torch.float32, device="cuda")
-    Dst = torch.empty_like(lse)
+    C = wl.C
+    prob = Problem(sna, torch, wl, keep_host=True)
+    units, pairs = prob.units, prob.pairs
+    q, k, v, dout, out, dq, dk, dv = prob.q, prob.k, prob.v, prob.dout, prob.out, prob.dq, prob.dk, prob.dv
+    host = prob.host
     host_out = [torch.empty_like(t, device="cpu").pin_memory() for t in (out, dq, dk, dv)]
-    stream = torch.cuda.current_stream()
-
+    stream = prob.stream
+    step = prob.step
+    flush = None if input_bytes(wl) > L2_BYTES else torch.zeros(64 * 1024 * 1024, dtype=torch.float32, device="cuda")
+    launches_per_step = prob.launches_per_step()
     ev = lambda: torch.cuda.Event(enable_timing=True)
-
-    def step(marks=None):
-        sna.sna_forward_ex(plan.handle, q, k, v, out, lse, B, H, C, stream)
-        if marks is not None:
-            marks[1].record(stream)
-        sna.sna_backward_dq(plan.handle, q, k, v, dout, out, lse, dq, Dst, B, H, C, stream)
-        if marks is not None:
-            marks[2].record(stream)
-        sna.sna_backward_dkdv(plan.handle, q, k, v, dout, lse, Dst, dk, dv, B, H, C, stream)
-    launches_per_step = sna.sna_forward_kernel_count(plan.handle, C, True) + 2   # forward (dense + band, or one) + dq + dk/dv
 
     for _ in range(max(args.warmup, 3)):
         step()
@@ -232,15 +349,18 @@ def run_ours(args, wl):
     t_start, t_end = ev(), ev()
     t_start.record(stream)
     for i in range(args.steps):
+        if flush is not None:
+            flush.add_(1.0)
         marks[i][0].record(stream)
         step(marks[i])
         marks[i][3].record(stream)
     t_end.record(stream)
     barrier()
-    ms_total = t_start.elapsed_time(t_end)
     ms_fwd = statistics.mean(m[0].elapsed_time(m[1]) for m in marks)
     ms_dq = statistics.mean(m[1].elapsed_time(m[2]) for m in marks)
     ms_dkdv = statistics.mean(m[2].elapsed_time(m[3]) for m in marks)
+    # with an L2 flush between steps the flush itself is outside the per-step events; without one the K steps run back to back
+    ms_total = t_start.elapsed_time(t_end) if flush is None else sum(m[0].elapsed_time(m[3]) for m in marks)
 
     # ---- end to end: pinned host -> device, compute, device -> pinned host ------------------------------
     def e2e_step():
@@ -269,17 +389,25 @@ def run_ours(args, wl):
         props = torch.cuda.get_device_properties(local_rank)
         sm_max_mhz = (clocks or {}).get("sm_max_mhz") or 1965.0
         peak_tflops = props.multi_processor_count * FP32_LANES_PER_SM * 2 * sm_max_mhz * 1e6 / 1e12
-        # algorithmic flops per pair*channel credited to each kernel: forward 4 (s and p.v), dq kernel 6 (s, t, dq),
-        # dk/dv kernel 4 (dk, dv; its recomputation of s and t is not credited) -- 14 in total = 4 forward + 10 backward
-        kernels = {"forward": (ms_fwd, 4.0), "backward_dq": (ms_dq, 6.0), "backward_dkdv": (ms_dkdv, 4.0)}
-        dominant = max(kernels, key=lambda n: kernels[n][0])
-        dom_ms, dom_flops_per_unit = kernels[dominant]
-        achieved = dom_flops_per_unit * units / (dom_ms * 1e-3) / 1e12
-        traffic = NCU_DRAM_BYTES_PER_LAUNCH.get((wl.name, dominant))
         peak_measured = sna.sna_measure_fp32_fma_peak()   # pure-FMA loop on this device, TFLOP/s
+        hbm_gbs, hbm_source = hbm_peak_gbs()
+        # algorithmic flops per pair*channel credited to each kernel: forward 4 (s and p.v), dq kernel 6 (s, t, dq),
+        # dk/dv kernel 4 (dk, dv; its recomputation of s and t is not credited) -- 14 in total = 4 forward + 10 backward.
+        # Every kernel's roofline time is the slower of those flops at the FP32 FMA peak and its compulsory bytes at the
+        # measured HBM copy bandwidth.
+        roofs = kernel_rooflines(wl, units, peak_tflops)
+        times = {"forward": ms_fwd, "backward_dq": ms_dq, "backward_dkdv": ms_dkdv}
+        dominant = max(times, key=times.get)
+        dom = roofs[dominant]
+        if dom["bound"] == "alu":
+            achieved, peak, unit = dom["flops_per_unit"] * units / (times[dominant] * 1e-3) / 1e12, peak_tflops, "TFLOP/s"
+            peak_note = (f"peak = SMs x 128 FP32 lanes x 2 x max SM clock (derived; the pure-FMA probe measured "
+                         f"{peak_measured:.1f} TFLOP/s on this device)")
+        else:
+            achieved, peak, unit = dom["bytes"] / (times[dominant] * 1e-3) / 1e9, hbm_gbs, "GB/s"
+            peak_note = f"peak = copy bandwidth ({hbm_source})"
         ms_step = ms_total_max / args.steps
-        roof_fwd_ms = 4.0 * units / (peak_tflops * 1e12) * 1e3
-        roof_bwd_ms = 10.0 * units / (peak_tflops * 1e12) * 1e3
+        roof_ms = sum(r["roofline_ms"] for r in roofs.values())
         result = {
             "metric": METRIC, "value": world * units / (ms_step * 1e-3), "unit": UNIT, "n_gpus": world,
             "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": ms_step, "higher_is_better": True,
@@ -287,31 +415,61 @@ def run_ours(args, wl):
             "config": workload_config(wl, world),
             "ms_forward": ms_fwd, "ms_backward": ms_dq + ms_dkdv, "ms_backward_dq": ms_dq, "ms_backward_dkdv": ms_dkdv,
             "pairs_per_step": pairs,
-            "roofline_step": {"bound": "alu", "roofline_ms": roof_fwd_ms + roof_bwd_ms, "frac": (roof_fwd_ms + roof_bwd_ms) / ms_step,
+            "roofline_step": {"bound": "alu" if all(r["bound"] == "alu" for r in roofs.values()) else "mixed",
+                              "roofline_ms": roof_ms, "frac": roof_ms / ms_step,
                               "peak_derived_tflops": peak_tflops, "peak_fma_measured_tflops": peak_measured,
-                              "frac_of_measured_peak": (roof_fwd_ms + roof_bwd_ms) * (peak_tflops / peak_measured) / ms_step,
-                              "note": "algorithmic flops (4C fwd + 10C bwd per pair) at the FP32 FMA peak of measured-max clock"},
-            "roofline": {"bound": "alu", "kernel": dominant, "achieved": achieved, "peak": peak_tflops, "unit": "TFLOP/s",
-                         "frac": achieved / peak_tflops, "traffic": traffic,
-                         "note": f"{dom_flops_per_unit:g} flops per pair*channel credited; peak = SMs x 128 FP32 lanes x 2 x max SM clock "
-                                 "(of derived peak; a pure-FMA loop measured 127.7 of 128 FMA/clk/SM); contractions run on tensor cores "
-                                 "as 3xTF32 MMAs; traffic = ncu dram bytes read+written per launch (profiles/)"},
+                              "frac_of_measured_peak": roof_ms * (peak_tflops / peak_measured) / ms_step,
+                              "hbm_gbs": hbm_gbs, "hbm_source": hbm_source,
+                              "note": "per kernel the slower of its algorithmic flops (4C fwd + 10C bwd per pair) at the FP32 FMA "
+                                      "peak and its compulsory bytes at the HBM copy bandwidth, summed over the three kernels"},
+            "roofline": {"bound": dom["bound"], "kernel": dominant, "achieved": achieved, "peak": peak, "unit": unit,
+                         "frac": achieved / peak, "traffic": NCU_DRAM_BYTES_PER_LAUNCH.get((wl.name, dominant)),
+                         "note": f"{dom['flops_per_unit']:g} flops per pair*channel credited, {dom['bytes'] / 1e6:.0f} MB compulsory; "
+                                 f"{peak_note}; the contractions run on tensor cores (TF32 main term + stacked BF16 corrections, "
+                                 "tcgen05 for whole-ring windows); traffic = recorded ncu DRAM bytes read+written per launch, "
+                                 "null when this workload has no capture"},
             "e2e": {"value": world * units / (ms_e2e_step_max * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
                     "d2h_bytes_per_step": d2h, "ms_per_step": ms_e2e_step_max},
             "gpu_launches": launches_per_step * args.steps,
             "clocks": clocks,
         }
+        if world == 1 and not args.no_extras:
+            # reduced-precision variant on the same workload, and the other benchmark configurations (10 steps each)
+            step_prec = prob.step       # restore the fp32 results afterwards for the accuracy check
+            t = time_steps(torch, prob, 10, 3, prob.step_tf32, flush)
+            result["variants"] = {"tf32": {"ms_forward": t["ms_forward"], "ms_backward": t["ms_backward_dkdv"],
+                                           "ms_per_step": t["ms_per_step"], "frac": roof_ms / t["ms_per_step"],
+                                           "note": "sna_forward_tf32 + sna_backward_tf32: one TF32 product per contraction, "
+                                                   "tolerance 5e-3 instead of 1e-5 / 1e-4; not the headline"}}
+            step_prec()
+            torch.cuda.synchronize()
+            result["workloads"] = {wl.name: {"ms_forward": ms_fwd, "ms_backward_dq": ms_dq, "ms_backward_dkdv": ms_dkdv,
+                                             "ms_per_step": ms_step, "roofline_ms": roof_ms, "roofline_frac": roof_ms / ms_step,
+                                             "l2": l2_policy(wl)}}
+            big_flush = torch.zeros(64 * 1024 * 1024, dtype=torch.float32, device="cuda")
+            for name in sorted(WORKLOADS):
+                if name == wl.name:
+                    continue
+                other = WORKLOADS[name]
+                po = Problem(sna, torch, other)
+                t = time_steps(torch, po, 10, 3, None, None if input_bytes(other) > L2_BYTES else big_flush)
+                r_ms = sum(r["roofline_ms"] for r in kernel_rooflines(other, po.units, peak_tflops).values())
+                t.update({"roofline_ms": r_ms, "roofline_frac": r_ms / t["ms_per_step"], "l2": l2_policy(other)})
+                result["workloads"][name] = t
+                po.close()
+                del po
+                torch.cuda.empty_cache()
         if not args.no_cpu_baseline and world == 1:
             from oracle import sna_oracle as orc
             g = orc.geometry(wl.nlat_in, wl.nlon_in, wl.nlat_out, wl.nlon_out, wl.grid_in, wl.grid_out, wl.theta_cutoff)
             n_slices = min(wl.N, 4)
-            arrays = [h.numpy() for h in host]
-            t = oracle_sample_step(orc, g, wl, *arrays, n_slices)
-            result["cpu_baseline"] = {"value": g.nnz * wl.nlon_out * n_slices * C / t, "unit": UNIT, "cores": orc.num_threads(),
-                                      "kind": "oracle", "seconds": t,
+            seconds, acc = accuracy_against_oracle(orc, g, prob, n_slices)
+            result["cpu_baseline"] = {"value": g.nnz * wl.nlon_out * n_slices * C / seconds, "unit": UNIT, "cores": orc.num_threads(),
+                                      "kind": "oracle", "seconds": seconds,
                                       "sample": f"{n_slices} of {wl.N} batch*head slices, forward+backward, fp64"}
+            result["accuracy"] = {"slices": n_slices, "gate": "normalised_max_error <= 1e-5 (out), 1e-4 (dq, dk, dv)", **acc}
         print(json.dumps(result))
-    plan.close()
+    prob.close()
     if dist is not None:
         dist.destroy_process_group()
 

@@ -177,6 +177,23 @@ sna_status_t sna_backward_dkdv(const sna_plan_t* plan, const float* q, const flo
                                int B, int H, int C, void* cuda_stream);
 
 /*
+ * Reduced-precision variant of the forward and backward pass.  The paper lists "neither reduced precision nor tensor
+ * core" support as a limitation of its kernels (Sec. 5, Limitations); here every contraction of
+ * Eq. s2_attention_discrete_detailed and App. B.4 is taken as ONE TF32 tensor-core product (operands rounded to 11
+ * significand bits, fp32 accumulation, fp32 softmax) instead of the error-compensated products of the default path.
+ * Same arguments, layouts and semantics as sna_forward_ex / sna_backward_ex.  Accuracy: normalised maximum error
+ * max|x - ref| / max|ref| per tensor below 5e-3 against an fp64 evaluation (measured ~1e-3); about 1.5x faster.
+ * Needs C in {16, 32, 64} and nlon_out >= 32 (SNA_ERR_UNSUPPORTED otherwise).
+ */
+sna_status_t sna_forward_tf32(const sna_plan_t* plan, const float* q, const float* k, const float* v, float* out,
+                              float* lse, int B, int H, int C, void* cuda_stream);
+sna_status_t sna_backward_tf32(const sna_plan_t* plan, const float* q, const float* k, const float* v,
+                               const float* dout, const float* out, const float* lse,
+                               float* dq, float* dk, float* dv,
+                               void* workspace, size_t workspace_bytes,
+                               int B, int H, int C, void* cuda_stream);
+
+/*
  * Backward pass for callers that must not allocate device memory.  (The paper has no counterpart; this is a
  * packaging variant of sna_backward.)
  *

@@ -225,7 +225,10 @@ static sna_status_t plan_create(int nlat_in, int nlon_in, int nlat_out, int nlon
     d.tb_stream = (const int4*)at(22); d.tb_chunk_ptr = at(23); d.tb_grp_order = at(24);
     d.t_dense_ptr = at(25); d.t_dense_lat = at(26); d.t_dense_rows = at(27);
     d.n_t_dense_rows = (int)t_dense.rows.size();
+    // opt in to the kernels' dynamic shared-memory sizes on this device (once here instead of on every launch)
     e = sna::dense2_prepare_device();
+    if (e == cudaSuccess) e = sna::dense_prepare_device();
+    if (e == cudaSuccess) e = sna::mma_prepare_device();
     if (e != cudaSuccess) { sna_plan_destroy(plan); return cuda_fail(e, "cudaFuncSetAttribute"); }
     *plan_out = plan;
     return SNA_OK;
@@ -461,6 +464,45 @@ sna_status_t sna_backward(const sna_plan_t* plan, const float* q, const float* k
         ws = plan->ws;
     }
     return sna_backward_ex(plan, q, k, v, dout, nullptr, nullptr, dq, dk, dv, ws, need, B, H, C, cuda_stream);
+}
+
+sna_status_t sna_forward_tf32(const sna_plan_t* plan, const float* q, const float* k, const float* v, float* out,
+                              float* lse, int B, int H, int C, void* cuda_stream) {
+    sna_status_t st = check_problem(plan, B, H, C);
+    if (st != SNA_OK) return st;
+    if (!q || !k || !v || !out) { set_error("q, k, v and out must not be NULL"); return SNA_ERR_INVALID_ARG; }
+    if (!all_aligned(q, k, v, out) || (reinterpret_cast<uintptr_t>(lse) & 3u)) { set_error("device pointers must be 16-byte aligned"); return SNA_ERR_INVALID_ARG; }
+    if (!sna::mma_path_supported(plan->dev, C)) { set_error("the reduced-precision variant needs C in {16, 32, 64} and nlon_out >= 32"); return SNA_ERR_UNSUPPORTED; }
+    cudaError_t e = sna::launch_forward_mma_lp(plan->dev, q, k, v, out, lse, B * H, C, (cudaStream_t)cuda_stream);
+    if (e != cudaSuccess) return cuda_fail(e, "forward launch");
+    return SNA_OK;
+}
+
+sna_status_t sna_backward_tf32(const sna_plan_t* plan, const float* q, const float* k, const float* v,
+                               const float* dout, const float* out, const float* lse, float* dq, float* dk, float* dv,
+                               void* workspace, size_t workspace_bytes, int B, int H, int C, void* cuda_stream) {
+    sna_status_t st = check_problem(plan, B, H, C);
+    if (st != SNA_OK) return st;
+    if (!q || !k || !v || !dout || !dq || !dk || !dv) { set_error("q, k, v, dout, dq, dk and dv must not be NULL"); return SNA_ERR_INVALID_ARG; }
+    if (!all_aligned(q, k, v, dout, dq, dk, dv, out) || (reinterpret_cast<uintptr_t>(lse) & 3u)) { set_error("device pointers must be 16-byte aligned"); return SNA_ERR_INVALID_ARG; }
+    if (workspace == nullptr || (reinterpret_cast<uintptr_t>(workspace) & 255u)) { set_error("workspace must be non-NULL and 256-byte aligned"); return SNA_ERR_INVALID_ARG; }
+    if (workspace_bytes < sna_workspace_bytes(plan, B, H, C)) { set_error("workspace too small: %zu < %zu bytes", workspace_bytes, sna_workspace_bytes(plan, B, H, C)); return SNA_ERR_WORKSPACE; }
+    if (!sna::mma_path_supported(plan->dev, C)) { set_error("the reduced-precision variant needs C in {16, 32, 64} and nlon_out >= 32"); return SNA_ERR_UNSUPPORTED; }
+    cudaStream_t stream = (cudaStream_t)cuda_stream;
+    const int N = B * H;
+    float* ws_lse = (float*)workspace;
+    float* ws_D = ws_lse + stats_elems(plan, B, H);
+    cudaError_t e;
+    if (lse == nullptr || out == nullptr) {   // recompute the forward pass: lse into the workspace, out into the dq buffer
+        e = sna::launch_forward_mma_lp(plan->dev, q, k, v, dq, ws_lse, N, C, stream);
+        if (e != cudaSuccess) return cuda_fail(e, "statistics launch");
+        lse = ws_lse;
+        out = dq;
+    }
+    e = sna::launch_backward_dq_mma_lp(plan->dev, q, k, v, dout, out, lse, dq, ws_D, N, C, stream);
+    if (e == cudaSuccess) e = sna::launch_backward_dkdv_mma_lp(plan->dev, q, k, v, dout, lse, ws_D, dk, dv, N, C, stream);
+    if (e != cudaSuccess) return cuda_fail(e, "backward launch");
+    return SNA_OK;
 }
 
 }  // extern "C"

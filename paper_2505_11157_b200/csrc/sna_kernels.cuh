@@ -49,12 +49,21 @@ struct DevPlan {
 };
 
 // Tensor-core kernels (C = 16, 32 or 64, nlon_out >= 32); same contracts as the generic launchers.
+cudaError_t mma_prepare_device();   // once per device: opt in to the kernels' shared-memory sizes
 bool mma_path_supported(const DevPlan& p, int C);
+// Reduced-precision variant of the three kernels: every product is one TF32 MMA (relative product error ~2^-11).
+cudaError_t launch_forward_mma_lp(const DevPlan& p, const float* q, const float* k, const float* v, float* out, float* lse,
+                                  int N, int C, cudaStream_t stream);
+cudaError_t launch_backward_dq_mma_lp(const DevPlan& p, const float* q, const float* k, const float* v, const float* dout,
+                                      const float* out, const float* lse, float* dq, float* Dws, int N, int C, cudaStream_t stream);
+cudaError_t launch_backward_dkdv_mma_lp(const DevPlan& p, const float* q, const float* k, const float* v, const float* dout,
+                                        const float* lse, const float* Dws, float* dk, float* dv, int N, int C, cudaStream_t stream);
 cudaError_t launch_forward_mma(const DevPlan& p, const float* q, const float* k, const float* v, float* out, float* lse,
                                int N, int C, cudaStream_t stream);
 // Dense (tcgen05) forward over the whole-ring windows only: writes the partial result (normalised out, lse) of the
 // output latitudes in p.dense_rows; launch_forward_mma_band then continues from it with the banded windows.
 // Both need lse != null.  dense_path_supported tells whether the pair may be used for this problem.
+cudaError_t dense_prepare_device();   // once per device: opt in to the kernels' shared-memory size
 bool dense_path_supported(const DevPlan& p, int C);
 cudaError_t launch_forward_dense(const DevPlan& p, const float* q, const float* k, const float* v, float* out, float* lse,
                                  int N, int C, cudaStream_t stream);

@@ -779,6 +779,13 @@ backward_dkdv_dense_kernel(DevPlan p, const float* __restrict__ q, const float* 
 }
 }  // namespace
 
+cudaError_t dense_prepare_device() {
+    cudaError_t e = cudaFuncSetAttribute(forward_dense_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)DENSE_SMEM);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(backward_dq_dense_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)DENSE_SMEM);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(backward_dkdv_dense_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)DENSE_SMEM);
+    return e;
+}
+
 bool dense_path_supported(const DevPlan& p, int C) {
     return C == DC && p.dense_ptr != nullptr && p.n_dense_rows > 0 && p.fwdb_stream != nullptr && mma_path_supported(p, C);
 }
@@ -790,8 +797,6 @@ cudaError_t launch_forward_dense(const DevPlan& p, const float* q, const float* 
     const long long blocks = (long long)blocks_per_row * p.n_dense_rows * N;
     if (blocks <= 0) return cudaSuccess;
     if (blocks > 0x7fffffffLL) return cudaErrorInvalidValue;
-    cudaError_t e = cudaFuncSetAttribute(forward_dense_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)DENSE_SMEM);
-    if (e != cudaSuccess) return e;
     forward_dense_kernel<<<(unsigned)blocks, DM, DENSE_SMEM, stream>>>(p, q, k, v, out, lse, N, LOG2E_D / sqrtf((float)C), blocks_per_row);
     return cudaGetLastError();
 }
@@ -803,8 +808,6 @@ cudaError_t launch_backward_dq_dense(const DevPlan& p, const float* q, const flo
     const long long blocks = (long long)blocks_per_row * p.n_dense_rows * N;
     if (blocks <= 0) return cudaSuccess;
     if (blocks > 0x7fffffffLL) return cudaErrorInvalidValue;
-    cudaError_t e = cudaFuncSetAttribute(backward_dq_dense_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)DENSE_SMEM);
-    if (e != cudaSuccess) return e;
     backward_dq_dense_kernel<<<(unsigned)blocks, DM, DENSE_SMEM, stream>>>(p, q, k, v, dout, out, lse, dq, N, 1.0f / sqrtf((float)C), blocks_per_row);
     return cudaGetLastError();
 }
@@ -816,8 +819,6 @@ cudaError_t launch_backward_dkdv_dense(const DevPlan& p, const float* q, const f
     const long long blocks = (long long)blocks_per_row * p.n_t_dense_rows * N;
     if (blocks <= 0) return cudaSuccess;
     if (blocks > 0x7fffffffLL) return cudaErrorInvalidValue;
-    cudaError_t e = cudaFuncSetAttribute(backward_dkdv_dense_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)DENSE_SMEM);
-    if (e != cudaSuccess) return e;
     backward_dkdv_dense_kernel<<<(unsigned)blocks, DM, DENSE_SMEM, stream>>>(p, q, k, v, dout, lse, Dws, dk, dv, N, 1.0f / sqrtf((float)C), blocks_per_row);
     return cudaGetLastError();
 }

@@ -194,7 +194,7 @@ struct FwdView {
 // ---------------------------------------------------------------------------------------------------------
 // forward
 // ---------------------------------------------------------------------------------------------------------
-template <int C>
+template <int C, bool LP>
 __global__ void __launch_bounds__(THREADS, 4)
 forward_mma_kernel(DevPlan p, FwdView fv, const float* __restrict__ q, const float* __restrict__ k, const float* __restrict__ v,
                    float* out, float* lse, int N, float scale_log2, int tiles_per_row, long long total_tasks) {
@@ -249,7 +249,8 @@ forward_mma_kernel(DevPlan p, FwdView fv, const float* __restrict__ q, const flo
             float kr[2][CPT];
             lds_row<CPT>(st.a, g, t, kr[0]);
             lds_row<CPT>(st.a, 8 + g, t, kr[1]);
-            rows_dot_points3<CPT>(s, qh, ql, kr);   // scores at full precision (three TF32 MMAs per product)
+            if constexpr (LP) rows_dot_points1<CPT>(s, qh, kr);
+            else rows_dot_points3<CPT>(s, qh, ql, kr);   // scores at full precision (three TF32 MMAs per product)
         }
         float vr[2][2][KS];
 #pragma unroll
@@ -292,7 +293,8 @@ forward_mma_kernel(DevPlan p, FwdView fv, const float* __restrict__ q, const flo
         l0 = fmaf(l0, corr0, ps0);
         l1 = fmaf(l1, corr1, ps1);
         float pv[KS][4];
-        scores_times_points2<KS, true>(pv, s, vr);
+        if constexpr (LP) scores_times_points1<KS>(pv, s, vr);
+        else scores_times_points2<KS, true>(pv, s, vr);
 #pragma unroll
         for (int nt = 0; nt < KS; ++nt) {
             o[nt][0] = fmaf(o[nt][0], corr0, pv[nt][0]); o[nt][1] = fmaf(o[nt][1], corr0, pv[nt][1]);
@@ -323,7 +325,7 @@ forward_mma_kernel(DevPlan p, FwdView fv, const float* __restrict__ q, const flo
 // backward, dq:  dq_i = scale * sum_j p_ij (t_ij - D_i) k_j,  D_i = dout_i . out_i  (App. B.4)
 // `out` and `dq` may be the same buffer: a warp reads its own 16 rows of `out` before it writes them as dq.
 // ---------------------------------------------------------------------------------------------------------
-template <int C>
+template <int C, bool LP>
 __global__ void __launch_bounds__(THREADS, 3)
 backward_dq_mma_kernel(DevPlan p, FwdView fv, const float* __restrict__ q, const float* __restrict__ k, const float* __restrict__ v,
                        const float* __restrict__ dout, const float* out, const float* __restrict__ lse,
@@ -377,10 +379,10 @@ backward_dq_mma_kernel(DevPlan p, FwdView fv, const float* __restrict__ q, const
             float xr[2][CPT];
             lds_row<CPT>(st.a, g, t, xr[0]);
             lds_row<CPT>(st.a, 8 + g, t, xr[1]);
-            rows_dot_points2<CPT>(s, qh, ql, xr);
+            if constexpr (LP) rows_dot_points1<CPT>(s, qh, xr); else rows_dot_points2<CPT>(s, qh, ql, xr);
             lds_row<CPT>(st.b, g, t, xr[0]);
             lds_row<CPT>(st.b, 8 + g, t, xr[1]);
-            rows_dot_points2<CPT>(tt, yh, yl, xr);
+            if constexpr (LP) rows_dot_points1<CPT>(tt, yh, xr); else rows_dot_points2<CPT>(tt, yh, yl, xr);
         }
         float kr[2][2][KS];
 #pragma unroll
@@ -400,7 +402,7 @@ backward_dq_mma_kernel(DevPlan p, FwdView fv, const float* __restrict__ q, const
             s[tl][3] = p11 * (tt[tl][3] - D1);
         }
         float part[KS][4];
-        scores_times_points2<KS>(part, s, kr);
+        if constexpr (LP) scores_times_points1<KS>(part, s, kr); else scores_times_points2<KS>(part, s, kr);
 #pragma unroll
         for (int nt = 0; nt < KS; ++nt) {
             acc[nt][0] += part[nt][0]; acc[nt][1] += part[nt][1]; acc[nt][2] += part[nt][2]; acc[nt][3] += part[nt][3];
@@ -438,7 +440,7 @@ backward_dq_mma_kernel(DevPlan p, FwdView fv, const float* __restrict__ q, const
 // Tile rows are the input columns c = ps*(u0+i) + r, i < 8, of the two rings of an input ring group; stream
 // columns are output points.
 // ---------------------------------------------------------------------------------------------------------
-template <int C>
+template <int C, bool LP>
 __global__ void __launch_bounds__(THREADS, 2)
 backward_dkdv_mma_kernel(DevPlan p, FwdView tv, const float* __restrict__ q, const float* __restrict__ k, const float* __restrict__ v,
                          const float* __restrict__ dout, const float* __restrict__ lse, const float* __restrict__ Dws,
@@ -492,10 +494,10 @@ backward_dkdv_mma_kernel(DevPlan p, FwdView tv, const float* __restrict__ q, con
             float xr[2][CPT];
             lds_row<CPT>(st.a, g, t, xr[0]);
             lds_row<CPT>(st.a, 8 + g, t, xr[1]);
-            rows_dot_points2<CPT>(s, kh, kl, xr);
+            if constexpr (LP) rows_dot_points1<CPT>(s, kh, xr); else rows_dot_points2<CPT>(s, kh, kl, xr);
             lds_row<CPT>(st.b, g, t, xr[0]);
             lds_row<CPT>(st.b, 8 + g, t, xr[1]);
-            rows_dot_points2<CPT>(tt, vh, vl, xr);
+            if constexpr (LP) rows_dot_points1<CPT>(tt, vh, xr); else rows_dot_points2<CPT>(tt, vh, vl, xr);
         }
         float qr[2][2][KS], yr[2][2][KS];
         float pr[2][4];
@@ -520,10 +522,10 @@ backward_dkdv_mma_kernel(DevPlan p, FwdView tv, const float* __restrict__ q, con
             s[tl][3] = pr[tl][3] * (tt[tl][3] - Dd.y);
         }
         float part[KS][4];
-        scores_times_points2<KS>(part, pr, yr);
+        if constexpr (LP) scores_times_points1<KS>(part, pr, yr); else scores_times_points2<KS>(part, pr, yr);
 #pragma unroll
         for (int nt = 0; nt < KS; ++nt) { gv[nt][0] += part[nt][0]; gv[nt][1] += part[nt][1]; gv[nt][2] += part[nt][2]; gv[nt][3] += part[nt][3]; }
-        scores_times_points2<KS>(part, s, qr);
+        if constexpr (LP) scores_times_points1<KS>(part, s, qr); else scores_times_points2<KS>(part, s, qr);
 #pragma unroll
         for (int nt = 0; nt < KS; ++nt) { gk[nt][0] += part[nt][0]; gk[nt][1] += part[nt][1]; gk[nt][2] += part[nt][2]; gk[nt][3] += part[nt][3]; }
     });
@@ -568,11 +570,18 @@ backward_dkdv_mma_kernel(DevPlan p, FwdView tv, const float* __restrict__ q, con
 template <int C>
 constexpr size_t smem_bytes() { return sizeof(Stage<C>) * 2 * WARPS; }
 
-// Dynamic shared memory above 48 KB needs an opt-in per kernel; it is requested on every launch (a cheap
-// host-side call) so that it holds on whichever device is current.
+// Dynamic shared memory above 48 KB needs an opt-in per kernel and device; mma_prepare_device does it once per plan
+// creation for every instantiation.
 template <typename K>
 cudaError_t prepare_kernel(K kernel, size_t bytes) {
     return bytes > 48 * 1024 ? cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes) : cudaSuccess;
+}
+template <int C, bool LP>
+cudaError_t prepare_instantiation() {
+    cudaError_t e = prepare_kernel(forward_mma_kernel<C, LP>, smem_bytes<C>());
+    if (e == cudaSuccess) e = prepare_kernel(backward_dq_mma_kernel<C, LP>, smem_bytes<C>());
+    if (e == cudaSuccess) e = prepare_kernel(backward_dkdv_mma_kernel<C, LP>, smem_bytes<C>());
+    return e;
 }
 
 template <typename F>
@@ -587,13 +596,23 @@ cudaError_t dispatch_c(int C, F&& f) {
 
 }  // namespace
 
+cudaError_t mma_prepare_device() {
+    cudaError_t e = prepare_instantiation<16, false>();
+    if (e == cudaSuccess) e = prepare_instantiation<32, false>();
+    if (e == cudaSuccess) e = prepare_instantiation<64, false>();
+    if (e == cudaSuccess) e = prepare_instantiation<16, true>();
+    if (e == cudaSuccess) e = prepare_instantiation<32, true>();
+    if (e == cudaSuccess) e = prepare_instantiation<64, true>();
+    return e;
+}
+
 bool mma_path_supported(const DevPlan& p, int C) {
     return p.fwd_stream != nullptr && (C == 16 || C == 32 || C == 64) && p.nlon_out >= 32 && p.nlon_out < 32768 &&
            (long long)p.nlat_in * p.nlon_in * C < (1LL << 32) && (long long)p.nlat_out * p.nlon_out * C < (1LL << 32);
 }
 
 static cudaError_t launch_forward_view(const DevPlan& p, const FwdView& fv, const float* q, const float* k, const float* v, float* out,
-                                       float* lse, int N, int C, cudaStream_t stream) {
+                                       float* lse, int N, int C, cudaStream_t stream, bool lp = false) {
     const float scale_log2 = LOG2E / sqrtf((float)C);
     const int tiles = (p.nlon_out + TILE_LON - 1) / TILE_LON;
     const long long tasks = (long long)tiles * ((p.nlat_out + TILE_LAT - 1) / TILE_LAT) * N;
@@ -601,9 +620,8 @@ static cudaError_t launch_forward_view(const DevPlan& p, const FwdView& fv, cons
     if (blocks > 0x7fffffffLL) return cudaErrorInvalidValue;
     return dispatch_c(C, [&](auto c) {
         constexpr int CC = decltype(c)::value;
-        cudaError_t e = prepare_kernel(forward_mma_kernel<CC>, smem_bytes<CC>());
-        if (e != cudaSuccess) return e;
-        forward_mma_kernel<CC><<<(unsigned)blocks, THREADS, smem_bytes<CC>(), stream>>>(p, fv, q, k, v, out, lse, N, scale_log2, tiles, tasks);
+        if (lp) forward_mma_kernel<CC, true><<<(unsigned)blocks, THREADS, smem_bytes<CC>(), stream>>>(p, fv, q, k, v, out, lse, N, scale_log2, tiles, tasks);
+        else forward_mma_kernel<CC, false><<<(unsigned)blocks, THREADS, smem_bytes<CC>(), stream>>>(p, fv, q, k, v, out, lse, N, scale_log2, tiles, tasks);
         return cudaGetLastError();
     });
 }
@@ -621,7 +639,7 @@ cudaError_t launch_forward_mma_band(const DevPlan& p, const float* q, const floa
 }
 
 static cudaError_t launch_backward_dq_view(const DevPlan& p, const FwdView& fv, const float* q, const float* k, const float* v, const float* dout,
-                                           const float* out, const float* lse, float* dq, float* Dws, int N, int C, cudaStream_t stream) {
+                                           const float* out, const float* lse, float* dq, float* Dws, int N, int C, cudaStream_t stream, bool lp = false) {
     const float scale = 1.0f / sqrtf((float)C);
     const int tiles = (p.nlon_out + TILE_LON - 1) / TILE_LON;
     const long long tasks = (long long)tiles * ((p.nlat_out + TILE_LAT - 1) / TILE_LAT) * N;
@@ -629,9 +647,8 @@ static cudaError_t launch_backward_dq_view(const DevPlan& p, const FwdView& fv, 
     if (blocks > 0x7fffffffLL) return cudaErrorInvalidValue;
     return dispatch_c(C, [&](auto c) {
         constexpr int CC = decltype(c)::value;
-        cudaError_t e = prepare_kernel(backward_dq_mma_kernel<CC>, smem_bytes<CC>());
-        if (e != cudaSuccess) return e;
-        backward_dq_mma_kernel<CC><<<(unsigned)blocks, THREADS, smem_bytes<CC>(), stream>>>(p, fv, q, k, v, dout, out, lse, dq, Dws, N, scale, tiles, tasks);
+        if (lp) backward_dq_mma_kernel<CC, true><<<(unsigned)blocks, THREADS, smem_bytes<CC>(), stream>>>(p, fv, q, k, v, dout, out, lse, dq, Dws, N, scale, tiles, tasks);
+        else backward_dq_mma_kernel<CC, false><<<(unsigned)blocks, THREADS, smem_bytes<CC>(), stream>>>(p, fv, q, k, v, dout, out, lse, dq, Dws, N, scale, tiles, tasks);
         return cudaGetLastError();
     });
 }
@@ -649,7 +666,7 @@ cudaError_t launch_backward_dq_mma_band(const DevPlan& p, const float* q, const 
 }
 
 static cudaError_t launch_backward_dkdv_view(const DevPlan& p, const FwdView& tv, const float* q, const float* k, const float* v, const float* dout,
-                                             const float* lse, const float* Dws, float* dk, float* dv, int N, int C, cudaStream_t stream) {
+                                             const float* lse, const float* Dws, float* dk, float* dv, int N, int C, cudaStream_t stream, bool lp = false) {
     const float scale = 1.0f / sqrtf((float)C);
     const int tiles = p.t_consecutive ? (p.nlon_in + TILE_LON - 1) / TILE_LON : p.ps * ((p.nlon_out + TILE_LON - 1) / TILE_LON);
     const long long tasks = (long long)tiles * ((p.nlat_in + TILE_LAT - 1) / TILE_LAT) * N;
@@ -657,9 +674,8 @@ static cudaError_t launch_backward_dkdv_view(const DevPlan& p, const FwdView& tv
     if (blocks > 0x7fffffffLL) return cudaErrorInvalidValue;
     return dispatch_c(C, [&](auto c) {
         constexpr int CC = decltype(c)::value;
-        cudaError_t e = prepare_kernel(backward_dkdv_mma_kernel<CC>, smem_bytes<CC>());
-        if (e != cudaSuccess) return e;
-        backward_dkdv_mma_kernel<CC><<<(unsigned)blocks, THREADS, smem_bytes<CC>(), stream>>>(p, tv, q, k, v, dout, lse, Dws, dk, dv, N, scale, tiles, tasks);
+        if (lp) backward_dkdv_mma_kernel<CC, true><<<(unsigned)blocks, THREADS, smem_bytes<CC>(), stream>>>(p, tv, q, k, v, dout, lse, Dws, dk, dv, N, scale, tiles, tasks);
+        else backward_dkdv_mma_kernel<CC, false><<<(unsigned)blocks, THREADS, smem_bytes<CC>(), stream>>>(p, tv, q, k, v, dout, lse, Dws, dk, dv, N, scale, tiles, tasks);
         return cudaGetLastError();
     });
 }
@@ -674,6 +690,23 @@ cudaError_t launch_backward_dkdv_mma_band(const DevPlan& p, const float* q, cons
                                           const float* lse, const float* Dws, float* dk, float* dv, int N, int C, cudaStream_t stream) {
     const FwdView tv{p.tb_stream, p.tb_chunk_ptr, p.tb_grp_order, p.t_dense_ptr};
     return launch_backward_dkdv_view(p, tv, q, k, v, dout, lse, Dws, dk, dv, N, C, stream);
+}
+
+// Reduced-precision variant: the same kernels with every product taken as a single TF32 MMA (full streams, no dense split).
+cudaError_t launch_forward_mma_lp(const DevPlan& p, const float* q, const float* k, const float* v, float* out, float* lse,
+                                  int N, int C, cudaStream_t stream) {
+    const FwdView fv{p.fwd_stream, p.fwd_chunk_ptr, p.grp_order, nullptr};
+    return launch_forward_view(p, fv, q, k, v, out, lse, N, C, stream, true);
+}
+cudaError_t launch_backward_dq_mma_lp(const DevPlan& p, const float* q, const float* k, const float* v, const float* dout,
+                                      const float* out, const float* lse, float* dq, float* Dws, int N, int C, cudaStream_t stream) {
+    const FwdView fv{p.fwd_stream, p.fwd_chunk_ptr, p.grp_order, nullptr};
+    return launch_backward_dq_view(p, fv, q, k, v, dout, out, lse, dq, Dws, N, C, stream, true);
+}
+cudaError_t launch_backward_dkdv_mma_lp(const DevPlan& p, const float* q, const float* k, const float* v, const float* dout,
+                                        const float* lse, const float* Dws, float* dk, float* dv, int N, int C, cudaStream_t stream) {
+    const FwdView tv{p.t_stream, p.t_chunk_ptr, p.t_grp_order, nullptr};
+    return launch_backward_dkdv_view(p, tv, q, k, v, dout, lse, Dws, dk, dv, N, C, stream, true);
 }
 
 }  // namespace sna

@@ -221,6 +221,34 @@ __device__ __forceinline__ void scores_times_points2(float (&d)[KS][4], const fl
     for (int nt = 0; nt < KS; ++nt) mma_acc(d[nt], wm[1], xm[1][0][nt], xm[1][1][nt]);
 }
 
+// ---------------------------------------------------------------------------------------------------------
+// One-MMA products for the reduced-precision variant: both operands are used as plain TF32 (the tensor core reads the
+// top 19 bits of the fp32 words), fp32 accumulation.  Relative error of a product ~2^-11.
+// ---------------------------------------------------------------------------------------------------------
+template <int CPT>
+__device__ __forceinline__ void rows_dot_points1(float (&d)[2][4], const uint32_t (&ah)[CPT / 2][4], const float (&x)[2][CPT]) {
+    mma_zero(d[0], ah[0], __float_as_uint(x[0][0]), __float_as_uint(x[0][1]));
+    mma_zero(d[1], ah[0], __float_as_uint(x[1][0]), __float_as_uint(x[1][1]));
+#pragma unroll
+    for (int ks = 1; ks < CPT / 2; ++ks) {
+        mma_acc(d[0], ah[ks], __float_as_uint(x[0][2 * ks]), __float_as_uint(x[0][2 * ks + 1]));
+        mma_acc(d[1], ah[ks], __float_as_uint(x[1][2 * ks]), __float_as_uint(x[1][2 * ks + 1]));
+    }
+}
+template <int KS>
+__device__ __forceinline__ void scores_times_points1(float (&d)[KS][4], const float (&w)[2][4], const float (&x)[2][2][KS]) {
+    uint32_t wm[2][4];
+#pragma unroll
+    for (int tl = 0; tl < 2; ++tl) {
+        wm[tl][0] = __float_as_uint(w[tl][0]); wm[tl][1] = __float_as_uint(w[tl][2]);   // TF32 A quad: (g,2t) (g+8,2t) (g,2t+1) (g+8,2t+1)
+        wm[tl][2] = __float_as_uint(w[tl][1]); wm[tl][3] = __float_as_uint(w[tl][3]);
+    }
+#pragma unroll
+    for (int nt = 0; nt < KS; ++nt) mma_zero(d[nt], wm[0], __float_as_uint(x[0][0][nt]), __float_as_uint(x[0][1][nt]));
+#pragma unroll
+    for (int nt = 0; nt < KS; ++nt) mma_acc(d[nt], wm[1], __float_as_uint(x[1][0][nt]), __float_as_uint(x[1][1][nt]));
+}
+
 template <int CPT>
 __device__ __forceinline__ void store_row(float* p, const float (&x)[CPT]) {
 #pragma unroll

@@ -57,6 +57,8 @@ _SIGNATURES = {
     "sna_backward_ex": (_i, [_vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _sz, _i, _i, _i, _vp]),
     "sna_backward_dq": (_i, [_vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _i, _i, _i, _vp]),
     "sna_backward_dkdv": (_i, [_vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _i, _i, _i, _vp]),
+    "sna_forward_tf32": (_i, [_vp, _vp, _vp, _vp, _vp, _vp, _i, _i, _i, _vp]),
+    "sna_backward_tf32": (_i, [_vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _sz, _i, _i, _i, _vp]),
     "sna_backward_static": (_i, [_vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _i, _i, _i, _vp]),
     "sna_measure_fp32_fma_peak": (_i, [ctypes.POINTER(ctypes.c_double)]),
     "sna_status_string": (ctypes.c_char_p, [_i]),
@@ -165,6 +167,17 @@ def sna_backward_dq(plan, q, k, v, dout, out, lse, dq, D, B, H, C, stream=None):
 def sna_backward_dkdv(plan, q, k, v, dout, lse, D, dk, dv, B, H, C, stream=None):
     _check(_lib.sna_backward_dkdv(plan, _ptr(q), _ptr(k), _ptr(v), _ptr(dout), _ptr(lse), _ptr(D), _ptr(dk), _ptr(dv),
                                   B, H, C, _stream(stream)))
+
+
+def sna_forward_tf32(plan, q, k, v, out, lse, B, H, C, stream=None):
+    """Reduced-precision forward pass (one TF32 product per contraction; normalised error below 5e-3)."""
+    _check(_lib.sna_forward_tf32(plan, _ptr(q), _ptr(k), _ptr(v), _ptr(out), _ptr(lse), B, H, C, _stream(stream)))
+
+
+def sna_backward_tf32(plan, q, k, v, dout, out, lse, dq, dk, dv, workspace, workspace_bytes, B, H, C, stream=None):
+    """Reduced-precision backward pass; arguments as sna_backward_ex."""
+    _check(_lib.sna_backward_tf32(plan, _ptr(q), _ptr(k), _ptr(v), _ptr(dout), _ptr(out), _ptr(lse), _ptr(dq), _ptr(dk),
+                                  _ptr(dv), _ptr(workspace), workspace_bytes, B, H, C, _stream(stream)))
 
 
 SNA_STATIC_SCRATCH_MAX_POINTS = 1 << 20
@@ -284,27 +297,39 @@ class Plan:
     def workspace_bytes(self, B, H, C) -> int:
         return sna_workspace_bytes(self.handle, B, H, C)
 
-    def forward(self, q, k, v, out=None, lse=None, return_lse=False, stream=None):
+    def forward(self, q, k, v, out=None, lse=None, return_lse=False, stream=None, precision="fp32"):
+        """precision: "fp32" (default, error-compensated products) or "tf32" (reduced-precision variant)."""
         import torch
         B, H, C = self._bhc(q, k)
         self._validate(q, k=k, v=v, out=out, lse=lse)
+        if precision not in ("fp32", "tf32"):
+            raise ValueError("precision must be 'fp32' or 'tf32'")
         if out is None:
             out = torch.empty_like(q)
         if return_lse and lse is None:
             lse = torch.empty(q.shape[:-1], dtype=torch.float32, device=q.device)
-        sna_forward_ex(self.handle, q, k, v, out, lse, B, H, C, stream)
+        (sna_forward_ex if precision == "fp32" else sna_forward_tf32)(self.handle, q, k, v, out, lse, B, H, C, stream)
         return (out, lse) if return_lse else out
 
-    def backward(self, q, k, v, dout, out=None, lse=None, dq=None, dk=None, dv=None, workspace=None, stream=None):
+    def backward(self, q, k, v, dout, out=None, lse=None, dq=None, dk=None, dv=None, workspace=None, stream=None,
+                 precision="fp32"):
         import torch
         B, H, C = self._bhc(q, k)
+        if precision not in ("fp32", "tf32"):
+            raise ValueError("precision must be 'fp32' or 'tf32'")
         self._validate(q, k=k, v=v, dout=dout, out=out, lse=lse, dq=dq, dk=dk, dv=dv)
         if workspace is not None and (not workspace.is_cuda or workspace.device != q.device or not workspace.is_contiguous()):
             raise ValueError("workspace must be a contiguous CUDA tensor on the device of q")
         dq = torch.empty_like(q) if dq is None else dq
         dk = torch.empty_like(k) if dk is None else dk
         dv = torch.empty_like(k) if dv is None else dv
-        if workspace is None and out is None and lse is None:
+        if precision == "tf32":
+            need = self.workspace_bytes(B, H, C)
+            if workspace is None:
+                workspace = torch.empty(need, dtype=torch.uint8, device=q.device)
+            sna_backward_tf32(self.handle, q, k, v, dout, out, lse, dq, dk, dv, workspace,
+                              workspace.numel() * workspace.element_size(), B, H, C, stream)
+        elif workspace is None and out is None and lse is None:
             sna_backward(self.handle, q, k, v, dout, dq, dk, dv, B, H, C, stream)
         else:
             need = self.workspace_bytes(B, H, C)

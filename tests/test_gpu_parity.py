@@ -171,6 +171,42 @@ def test_extreme_score_magnitudes(q_scale, v_scale):
     assert nerr(dv.reshape(rdv.shape), rdv) <= BWD_TOL
 
 
+LP_TOL = 5e-3   # stated tolerance of the reduced-precision variant (single TF32 product per contraction)
+
+
+@pytest.mark.parametrize("wl", [SMALL[0], SMALL[2], SMALL[3], SMALL[15], SMALL[7], SMALL[10], SMALL[24], WORKLOADS["c2"]], ids=lambda w: w.name)
+def test_reduced_precision_variant_against_oracle(wl):
+    """sna_forward_tf32 / sna_backward_tf32: same operator, one TF32 product per contraction; its own, looser gate.  It must
+    also be measurably less accurate than the default path (otherwise it is not the variant it claims to be)."""
+    g = _geometry(wl)
+    q, k, v, dout = make_inputs(wl)
+    with _plan(wl) as plan:
+        qd, kd, vd, dd = _dev(q, k, v, dout)
+        out, lse = plan.forward(qd, kd, vd, return_lse=True, precision="tf32")
+        dq, dk, dv = plan.backward(qd, kd, vd, dd, out=out, lse=lse, precision="tf32")
+        dq2, dk2, dv2 = plan.backward(qd, kd, vd, dd, precision="tf32")          # recomputed statistics
+        torch.cuda.synchronize()
+        sna.sna_plan_check(plan.handle)
+    ref_out = orc.forward(g, q, k, v)
+    rdq, rdk, rdv = orc.backward(g, q, k, v, dout)
+    e_out = nerr(out.cpu().numpy().reshape(ref_out.shape), ref_out)
+    assert 1e-5 < e_out <= LP_TOL
+    for x, x2, r in ((dq, dq2, rdq), (dk, dk2, rdk), (dv, dv2, rdv)):
+        assert nerr(x.cpu().numpy().reshape(r.shape), r) <= LP_TOL
+        assert nerr(x2.cpu().numpy().reshape(r.shape), r) <= LP_TOL
+
+
+def test_reduced_precision_variant_refuses_unsupported_shapes():
+    wl = SMALL[5]      # C = 4: no tensor-core path
+    q, k, v, dout = make_inputs(wl)
+    with _plan(wl) as plan:
+        qd, kd, vd = _dev(q, k, v)
+        with pytest.raises(sna.SnaError) as e:
+            plan.forward(qd, kd, vd, precision="tf32")
+        assert e.value.status == sna.SNA_ERR_UNSUPPORTED
+    torch.cuda.synchronize()
+
+
 def test_global_limit_against_dense_oracle():
     wl = small_workload("global", 16, 32, 16, 32, EQ, EQ, math.pi, 1, 2, 32, 30)
     g = _geometry(wl)
