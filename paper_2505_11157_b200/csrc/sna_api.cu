@@ -137,7 +137,11 @@ static sna_status_t plan_create(int nlat_in, int nlon_in, int nlat_out, int nlon
     sna::Stream fwd_stream, t_stream, fwdb_stream, tb_stream;
     sna::DenseLists dense, t_dense;
     std::vector<int32_t> grp_order, t_grp_order, grpb_order, tb_grp_order;
+#ifdef SNA_PROF
+    const int32_t zero_status[512] = {};   // room for the per-role profile of a -DSNA_PROF build
+#else
     const int32_t zero_status[64] = {};
+#endif
     bool t_consecutive = false;
     try {
         sna::build_forward_stream(hp, fwd_stream);
@@ -375,9 +379,11 @@ sna_status_t sna_backward_dq(const sna_plan_t* plan, const float* q, const float
     cudaError_t e;
     // The dense dq kernel pays off when whole-ring windows are a large share of the work (measured: 1.5x on the
     // global limit, -3 % at a 25 % share), so it is used from a 35 % share on.
-    if (out != nullptr && out != dq && plan->dev.dense_fraction >= 0.35f && sna::dense_path_supported(plan->dev, C)) {
+    if (out != nullptr && out != dq && plan->dev.dense_fraction >= 0.10f && sna::dense_path_supported(plan->dev, C)) {
         // whole-ring windows on the tcgen05 kernel (its part of dq is written first), the banded rest is added by the band kernel
-        e = sna::launch_backward_dq_dense(plan->dev, q, k, v, dout, out, lse, dq, B * H, C, (cudaStream_t)cuda_stream);
+        e = sna::dense2_path_supported(plan->dev, C)
+                ? sna::launch_backward_dq_dense2(plan->dev, q, k, v, dout, out, lse, dq, nullptr, B * H, C, (cudaStream_t)cuda_stream)
+                : sna::launch_backward_dq_dense(plan->dev, q, k, v, dout, out, lse, dq, B * H, C, (cudaStream_t)cuda_stream);
         if (e == cudaSuccess) e = sna::launch_backward_dq_mma_band(plan->dev, q, k, v, dout, out, lse, dq, D, B * H, C, (cudaStream_t)cuda_stream);
     } else if (out != nullptr && sna::mma_path_supported(plan->dev, C)) {
         e = sna::launch_backward_dq_mma(plan->dev, q, k, v, dout, out, lse, dq, D, B * H, C, (cudaStream_t)cuda_stream);
@@ -396,9 +402,11 @@ sna_status_t sna_backward_dkdv(const sna_plan_t* plan, const float* q, const flo
     if (!q || !k || !v || !dout || !lse || !D || !dk || !dv) { set_error("q, k, v, dout, lse, D, dk and dv must not be NULL"); return SNA_ERR_INVALID_ARG; }
     if (!all_aligned(q, k, v, dout, dk, dv) || ((reinterpret_cast<uintptr_t>(lse) | reinterpret_cast<uintptr_t>(D)) & 3u)) { set_error("device pointers must be 16-byte aligned"); return SNA_ERR_INVALID_ARG; }
     cudaError_t e;
-    if (plan->dev.dense_fraction >= 0.35f && plan->dev.n_t_dense_rows > 0 && sna::dense_path_supported(plan->dev, C)) {
+    if (plan->dev.dense_fraction >= 0.10f && plan->dev.n_t_dense_rows > 0 && sna::dense_path_supported(plan->dev, C)) {
         // whole-ring partners on the tcgen05 kernel (its part of dk, dv is written first), the band kernel adds the rest
-        e = sna::launch_backward_dkdv_dense(plan->dev, q, k, v, dout, lse, D, dk, dv, B * H, C, (cudaStream_t)cuda_stream);
+        e = sna::dense2_path_supported(plan->dev, C)
+                ? sna::launch_backward_dkdv_dense2(plan->dev, q, k, v, dout, lse, D, dk, dv, B * H, C, (cudaStream_t)cuda_stream)
+                : sna::launch_backward_dkdv_dense(plan->dev, q, k, v, dout, lse, D, dk, dv, B * H, C, (cudaStream_t)cuda_stream);
         if (e == cudaSuccess) e = sna::launch_backward_dkdv_mma_band(plan->dev, q, k, v, dout, lse, D, dk, dv, B * H, C, (cudaStream_t)cuda_stream);
     } else if (sna::mma_path_supported(plan->dev, C)) {
         e = sna::launch_backward_dkdv_mma(plan->dev, q, k, v, dout, lse, D, dk, dv, B * H, C, (cudaStream_t)cuda_stream);
@@ -558,3 +566,11 @@ extern "C" sna_status_t sna_backward_static(const sna_plan_t* plan, const float*
                            sizeof(float) * 2 * (size_t)SNA_STATIC_SCRATCH_MAX_POINTS, B, H, C, cuda_stream);
 }
 
+
+#ifdef SNA_PROF
+// Profiling builds only: copies the per-role cycle counters that a -DSNA_PROF kernel left in the plan's status area.
+extern "C" int sna_debug_read(const sna_plan_t* plan, long long* out, int count) {
+    cudaDeviceSynchronize();
+    return (int)cudaMemcpy(out, plan->dev.dev_status + 2, (size_t)count * 8, cudaMemcpyDeviceToHost);
+}
+#endif

@@ -72,6 +72,12 @@ cudaError_t dense2_prepare_device();   // once per device: opt in to the kernel'
 bool dense2_path_supported(const DevPlan& p, int C);
 cudaError_t launch_forward_dense2(const DevPlan& p, const float* q, const float* k, const float* v, float* out, float* lse,
                                   int N, int C, cudaStream_t stream);
+// Pipelined dense dq kernel; same contract as launch_backward_dq_dense, and it also writes D (Dws may be null).
+cudaError_t launch_backward_dq_dense2(const DevPlan& p, const float* q, const float* k, const float* v, const float* dout,
+                                      const float* out, const float* lse, float* dq, float* Dws, int N, int C, cudaStream_t stream);
+// Pipelined dense dk/dv kernel; same contract as launch_backward_dkdv_dense.
+cudaError_t launch_backward_dkdv_dense2(const DevPlan& p, const float* q, const float* k, const float* v, const float* dout,
+                                        const float* lse, const float* Dws, float* dk, float* dv, int N, int C, cudaStream_t stream);
 // The same split for the dq stage: the dense kernel writes the whole-ring part of dq (out and dq must be different
 // buffers), the band kernel adds its banded part to it.
 cudaError_t launch_backward_dq_dense(const DevPlan& p, const float* q, const float* k, const float* v, const float* dout,

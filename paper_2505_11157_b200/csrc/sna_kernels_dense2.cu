@@ -29,6 +29,19 @@
 
 #include <cstdint>
 
+// Optional per-role wait accounting (build with -DSNA_PROF; not part of the product build): every role of block 0 writes
+// its total cycles and the cycles spent in up to three kinds of waits to the plan's status area.
+#ifdef SNA_PROF
+#define PROF_DECL long long prof_w[3] = {0, 0, 0}; const long long prof_t0 = clock64();
+#define PROF_WAIT(i, stmt) { const long long t0_ = clock64(); stmt; prof_w[i] += clock64() - t0_; }
+#define PROF_DUMP(status, warp, lane, blocks) if ((lane) == 0 && blockIdx.x == 0) { long long* d_ = reinterpret_cast<long long*>((status) + 2) + (warp) * 5; \
+    d_[0] = clock64() - prof_t0; d_[1] = prof_w[0]; d_[2] = prof_w[1]; d_[3] = prof_w[2]; d_[4] = (blocks); }
+#else
+#define PROF_DECL
+#define PROF_WAIT(i, stmt) stmt
+#define PROF_DUMP(status, warp, lane, blocks)
+#endif
+
 namespace sna {
 namespace {
 
@@ -108,6 +121,11 @@ __device__ __forceinline__ void tm_ld16_issue(uint32_t (&r)[16], uint32_t addr) 
 __device__ __forceinline__ void tm_st16(uint32_t addr, const uint32_t (&r)[16]) {
     asm volatile("tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16};"
         :: "r"(addr), "r"(r[0]),"r"(r[1]),"r"(r[2]),"r"(r[3]),"r"(r[4]),"r"(r[5]),"r"(r[6]),"r"(r[7]),"r"(r[8]),"r"(r[9]),"r"(r[10]),"r"(r[11]),"r"(r[12]),"r"(r[13]),"r"(r[14]),"r"(r[15]) : "memory");
+}
+__device__ __forceinline__ void tm_st32(uint32_t addr, const uint32_t (&r)[32]) {
+    asm volatile("tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31,%32};"
+        :: "r"(addr), "r"(r[0]),"r"(r[1]),"r"(r[2]),"r"(r[3]),"r"(r[4]),"r"(r[5]),"r"(r[6]),"r"(r[7]),"r"(r[8]),"r"(r[9]),"r"(r[10]),"r"(r[11]),"r"(r[12]),"r"(r[13]),"r"(r[14]),"r"(r[15]),
+           "r"(r[16]),"r"(r[17]),"r"(r[18]),"r"(r[19]),"r"(r[20]),"r"(r[21]),"r"(r[22]),"r"(r[23]),"r"(r[24]),"r"(r[25]),"r"(r[26]),"r"(r[27]),"r"(r[28]),"r"(r[29]),"r"(r[30]),"r"(r[31]) : "memory");
 }
 __device__ __forceinline__ int sw_off(int row, int c4) { return row * 128 + ((c4 ^ (row & 7)) << 4); }
 
@@ -410,6 +428,631 @@ forward_dense2_kernel(DevPlan p, const __grid_constant__ CUtensorMap map_q, cons
     if (warp == 0) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tm), "r"(T_COLS));
 }
 
+// ---------------------------------------------------------------------------------------------------------
+// Pipelined dense part of the dq stage (App. B.4) for the whole input rings of an output ring:
+//   p = exp2(s + log2 omega - lse),  ds = p (t - D),  dq += scale * dS K,   s = q.k (log2 domain),  t = dout.v.
+// Same cast as the forward kernel, with blocks of 64 columns.  The tile's own operands (q, dout and their lo parts) live
+// in TMEM for the whole kernel, so the two first GEMMs (S = Q K^T and T = dY V^T, one issuing thread each) read only
+// the k / v blocks from shared memory.  Two groups of 128 threads turn (S, T) into dS (written over S, its top 19 bits
+// are the hi part) and dS_lo (over T), each for one half of the block's columns; four threads issue dq_part = dS K over
+// two 8-column steps each, into their own accumulators; the row's two threads add their parts in a fixed order and the
+// two halves are merged at the end.  S and T are double-buffered, so the GEMMs of block j+1 overlap the element-wise
+// work of block j and dS K of block j-1.
+// ---------------------------------------------------------------------------------------------------------
+constexpr int BNQ = 64;                          // columns per block
+constexpr int TILE_Q = BNQ * 128;                // 8 KB: 64 points x 128 bytes
+// per stage: k raw, k lo, v raw, v lo, k^T hi, k^T lo
+constexpr int QST = 6 * TILE_Q;
+constexpr int FOLDQ = 4;                         // dS K accumulates in TMEM over this many blocks before it is folded into registers
+constexpr int NSQ = 4;                           // shared-memory stages (TMA runs three blocks ahead of the GEMMs)
+constexpr size_t DQ2_SMEM = NSQ * QST + 1024;
+constexpr int TQ_AQ = 0, TQ_AQL = 32, TQ_AY = 64, TQ_AYL = 96, TQ_BUF = 128 /* + 128 b: S | T */, TQ_ACC = 384 /* + 32 part */;
+enum { Q_KFULL = 0, Q_VFULL = 4, Q_KCONV = 8, Q_VCONV = 12, Q_KSFREE = 16, Q_VFREE = 20, Q_KTFREE = 24 /* all [stage] */,
+       Q_STFULL = 28 /* [buffer] */, Q_DSREADY = 30 /* [group] */, Q_G2DONE = 32 /* [group][buffer] */, Q_AREADY = 36, Q_COUNT = 37 };
+
+__global__ void __launch_bounds__(THREADS2, 1)
+backward_dq_dense2_kernel(DevPlan p, const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_v,
+                          const float* __restrict__ q, const float* __restrict__ dout, const float* __restrict__ out,
+                          const float* __restrict__ lse, float* __restrict__ dq, float* __restrict__ Dws, int N, float scale,
+                          int tiles_per_row) {
+    extern __shared__ unsigned char dense2_raw[];
+    unsigned char* base = (unsigned char*)(((uintptr_t)dense2_raw + 1023) & ~(uintptr_t)1023);
+    __shared__ unsigned long long bars[Q_COUNT];
+    __shared__ uint32_t tmem_base_s;
+    __shared__ int fail_s;
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int tile = blockIdx.x % tiles_per_row;
+    const int rest = blockIdx.x / tiles_per_row;
+    const int n = rest % N;
+    const int h = p.dense_rows[rest / N];
+    const int w0 = tile * M2;
+    const int nblk = (p.nlon_in + BNQ - 1) / BNQ;
+    const int e_begin = p.dense_ptr[h], e_end = p.dense_ptr[h + 1];
+    const int total = (e_end - e_begin) * nblk;
+    const float scale_log2 = scale * LOG2E_2;
+
+    if (tid == 0) {
+        for (int s = 0; s < NSQ; ++s) {
+            mb_init(s32(&bars[Q_KFULL + s]), 1);
+            mb_init(s32(&bars[Q_VFULL + s]), 1);
+            mb_init(s32(&bars[Q_KCONV + s]), 128);
+            mb_init(s32(&bars[Q_VCONV + s]), 128);
+            mb_init(s32(&bars[Q_KSFREE + s]), 1);
+            mb_init(s32(&bars[Q_VFREE + s]), 1);
+            mb_init(s32(&bars[Q_KTFREE + s]), 4);
+        }
+        for (int s = 0; s < 2; ++s) {
+            mb_init(s32(&bars[Q_STFULL + s]), 2);
+            mb_init(s32(&bars[Q_DSREADY + s]), 128);
+            mb_init(s32(&bars[Q_G2DONE + s]), 2);
+            mb_init(s32(&bars[Q_G2DONE + 2 + s]), 2);
+        }
+        mb_init(s32(&bars[Q_AREADY]), 128);
+        fail_s = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 0) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(s32(&tmem_base_s)), "r"(T_COLS));
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::);
+    }
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    const uint32_t tm = tmem_base_s;
+    const uint32_t sbase = s32(base);
+    bool ok = true;
+    PROF_DECL
+
+    if (warp < 8) {
+        asm volatile("setmaxnreg.inc.sync.aligned.u32 152;");
+        // ------------------------------------------------------------------ element-wise: thread (grp, r) owns tile row r for
+        // the columns [32 grp, 32 grp + 32) of every block
+        const int grp = warp >> 2, r = tid & 127;
+        const uint32_t lanebits = (uint32_t)((warp & 3) * 32) << 16;
+        const int w = w0 + r;
+        const bool row_ok = w < p.nlon_out;
+        const size_t opt = (size_t)(n * p.nlat_out + h) * p.nlon_out + min(w, p.nlon_out - 1);
+        float D = 0.f;
+        if (grp == 0) {
+            // this row's q and dout into TMEM (A operands of the first GEMMs): raw words as hi parts, lo = x - trunc19(x)
+            uint32_t xq[32], xy[32];
+            const float4* qs = reinterpret_cast<const float4*>(q + opt * C2);
+            const float4* ys = reinterpret_cast<const float4*>(dout + opt * C2);
+            const float4* os = reinterpret_cast<const float4*>(out + opt * C2);
+#pragma unroll
+            for (int c4 = 0; c4 < C2 / 4; ++c4) {
+                const float4 a = __ldg(qs + c4), b = __ldg(ys + c4), o4 = __ldg(os + c4);
+                xq[4 * c4] = __float_as_uint(a.x); xq[4 * c4 + 1] = __float_as_uint(a.y); xq[4 * c4 + 2] = __float_as_uint(a.z); xq[4 * c4 + 3] = __float_as_uint(a.w);
+                xy[4 * c4] = __float_as_uint(b.x); xy[4 * c4 + 1] = __float_as_uint(b.y); xy[4 * c4 + 2] = __float_as_uint(b.z); xy[4 * c4 + 3] = __float_as_uint(b.w);
+                D = fmaf(b.x, o4.x, fmaf(b.y, o4.y, fmaf(b.z, o4.z, fmaf(b.w, o4.w, D))));
+            }
+            tm_st32(tm + TQ_AQ + lanebits, xq);
+            tm_st32(tm + TQ_AY + lanebits, xy);
+#pragma unroll
+            for (int j = 0; j < 32; ++j) {
+                const float a = __uint_as_float(xq[j]), b = __uint_as_float(xy[j]);
+                xq[j] = __float_as_uint(a - trunc19f(a));
+                xy[j] = __float_as_uint(b - trunc19f(b));
+            }
+            tm_st32(tm + TQ_AQL + lanebits, xq);
+            tm_st32(tm + TQ_AYL + lanebits, xy);
+            asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
+            asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+            mb_arrive(s32(&bars[Q_AREADY]));
+            if (Dws != nullptr && row_ok) Dws[opt] = D;
+        } else {
+            const float4* ys = reinterpret_cast<const float4*>(dout + opt * C2);
+            const float4* os = reinterpret_cast<const float4*>(out + opt * C2);
+#pragma unroll
+            for (int c4 = 0; c4 < C2 / 4; ++c4) {
+                const float4 b = __ldg(ys + c4), o4 = __ldg(os + c4);
+                D = fmaf(b.x, o4.x, fmaf(b.y, o4.y, fmaf(b.z, o4.z, fmaf(b.w, o4.w, D))));
+            }
+        }
+        const float nl = -__ldg(lse + opt) * LOG2E_2;
+        constexpr int GC = BNQ / 2;                       // columns per thread and block
+        float acc[C2];
+#pragma unroll
+        for (int i = 0; i < C2; ++i) acc[i] = 0.f;
+        for (int it = 0; it <= total && ok; ++it) {
+            if (it < total) {
+                const int b = it & 1, u = it >> 1;
+                const int hp = p.dense_lat[e_begin + it / nblk];
+                const float nbias = p.log2_omega[hp] + nl;
+                const int nvalid = p.nlon_in - (it % nblk) * BNQ - grp * GC;     // columns of this thread's half that exist
+                PROF_WAIT(0, ok = mb_wait(s32(&bars[Q_STFULL + b]), u & 1, ok) && ok);
+                asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                const uint32_t tS = tm + TQ_BUF + 128 * b + grp * GC + lanebits, tT = tS + BNQ;
+                uint32_t sv[32], tv[32];
+                tm_ld32_issue(sv, tS);
+                tm_ld32_issue(tv, tT);
+                tm_ld_wait();
+#pragma unroll
+                for (int j = 0; j < 32; ++j) {
+                    float pj = ex2f(fmaf(__uint_as_float(sv[j]), scale_log2, nbias));
+                    if (nvalid < GC && j >= nvalid) pj = 0.f;
+                    const float ds = pj * (__uint_as_float(tv[j]) - D);
+                    sv[j] = __float_as_uint(ds);                       // dS over S
+                    tv[j] = __float_as_uint(ds - trunc19f(ds));        // dS_lo over T
+                }
+                tm_st32(tS, sv);
+                tm_st32(tT, tv);
+            }
+            if (it > 0 && (it % FOLDQ == 0 || it == total)) {
+                // fold dS K of the blocks since the last fold (this half's two parts, fixed order): the tensor core has
+                // accumulated them in TMEM (chains of at most 6 * FOLDQ products); this also frees the accumulators
+                const int bp = (it - 1) & 1, up = (it - 1) >> 1;
+                PROF_WAIT(1, ok = mb_wait(s32(&bars[Q_G2DONE + 2 * grp + bp]), up & 1, ok) && ok);
+                asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                uint32_t oa[32], ob[32];
+                tm_ld32_issue(oa, tm + TQ_ACC + grp * 64 + lanebits);
+                tm_ld32_issue(ob, tm + TQ_ACC + grp * 64 + 32 + lanebits);
+                tm_ld_wait();
+#pragma unroll
+                for (int j = 0; j < C2; ++j) acc[j] += __uint_as_float(oa[j]) + __uint_as_float(ob[j]);
+            }
+            if (it < total) {
+                asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
+                asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+                mb_arrive(s32(&bars[Q_DSREADY + grp]));
+            }
+        }
+        // merge the two column halves of every row through shared memory (the staging tiles are dead by now)
+        float* xs = reinterpret_cast<float*>(base);
+        if (grp == 1) {
+#pragma unroll
+            for (int j = 0; j < C2; ++j) xs[j * 128 + r] = acc[j];
+        }
+        asm volatile("bar.sync 1, 256;" ::: "memory");
+        if (grp == 0 && ok && row_ok) {
+            float4* dst = reinterpret_cast<float4*>(dq + opt * C2);
+#pragma unroll
+            for (int c4 = 0; c4 < C2 / 4; ++c4) {
+                float rr[4];
+#pragma unroll
+                for (int i = 0; i < 4; ++i) rr[i] = (acc[4 * c4 + i] + xs[(4 * c4 + i) * 128 + r]) * scale;
+                dst[c4] = make_float4(rr[0], rr[1], rr[2], rr[3]);
+            }
+        }
+    } else if (warp < 12) {
+        asm volatile("setmaxnreg.dec.sync.aligned.u32 48;");
+        if (warp == 8 && lane == 0) {
+            // -------------------------------------------------------------- TMA producer
+            for (int it = 0; it < total && ok; ++it) {
+                const int s = it % NSQ, u = it / NSQ;
+                const int hp = p.dense_lat[e_begin + it / nblk];
+                const int c0 = (it % nblk) * BNQ;
+                if (u > 0) {   // the stage is free once both first GEMMs and all four dS K issuers of block it-NSQ are done
+                    PROF_WAIT(0, ok = mb_wait(s32(&bars[Q_KSFREE + s]), (u - 1) & 1, ok));
+                    PROF_WAIT(1, ok = mb_wait(s32(&bars[Q_VFREE + s]), (u - 1) & 1, ok) && ok);
+                    PROF_WAIT(2, ok = mb_wait(s32(&bars[Q_KTFREE + s]), (u - 1) & 1, ok) && ok);
+                }
+                mb_expect(s32(&bars[Q_KFULL + s]), TILE_Q);
+                tma_tile(sbase + s * QST, &map_k, c0, n * p.nlat_in + hp, s32(&bars[Q_KFULL + s]));
+                mb_expect(s32(&bars[Q_VFULL + s]), TILE_Q);
+                tma_tile(sbase + s * QST + 2 * TILE_Q, &map_v, c0, n * p.nlat_in + hp, s32(&bars[Q_VFULL + s]));
+            }
+        }
+        if ((warp == 9 || warp == 10) && lane == 0) {
+            // -------------------------------------------------------------- S = Q K^T (warp 9) and T = dY V^T (warp 10)
+            const bool isT = warp == 10;
+            ok = mb_wait(s32(&bars[Q_AREADY]), 0, ok);
+            const uint32_t idS = idesc_tf32(BNQ);
+            const uint32_t tA = tm + (isT ? TQ_AY : TQ_AQ), tAl = tm + (isT ? TQ_AYL : TQ_AQL);
+            for (int it = 0; it < total && ok; ++it) {
+                const int s = it % NSQ, us = it / NSQ, b = it & 1, u = it >> 1;
+                PROF_WAIT(0, ok = mb_wait(s32(&bars[(isT ? Q_VFULL : Q_KFULL) + s]), us & 1, ok));
+                PROF_WAIT(1, ok = mb_wait(s32(&bars[(isT ? Q_VCONV : Q_KCONV) + s]), us & 1, ok) && ok);
+                if (u > 0) {   // dS / dS_lo of block it-2 (in this buffer) have been consumed by all four dS K issuers
+                    PROF_WAIT(2, ok = mb_wait(s32(&bars[Q_G2DONE + b]), (u - 1) & 1, ok) && ok);
+                    PROF_WAIT(2, ok = mb_wait(s32(&bars[Q_G2DONE + 2 + b]), (u - 1) & 1, ok) && ok);
+                }
+                asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                const uint32_t tile0 = sbase + s * QST + (isT ? 2 * TILE_Q : 0);
+                const uint64_t db = desc_k(tile0), dbl = desc_k(tile0 + TILE_Q);
+                const uint32_t tD = tm + TQ_BUF + 128 * b + (isT ? BNQ : 0);
+#pragma unroll
+                for (int ks = 0; ks < C2 / 8; ++ks) mma_ts(tD, tAl + ks * 8, db + 2 * ks, idS, ks > 0);
+#pragma unroll
+                for (int ks = 0; ks < C2 / 8; ++ks) mma_ts(tD, tA + ks * 8, dbl + 2 * ks, idS, 1);
+#pragma unroll
+                for (int ks = 0; ks < C2 / 8; ++ks) mma_ts(tD, tA + ks * 8, db + 2 * ks, idS, 1);
+                mma_commit(s32(&bars[Q_STFULL + b]));
+                mma_commit(s32(&bars[(isT ? Q_VFREE : Q_KSFREE) + s]));
+            }
+        }
+    } else if (warp < 16) {
+        asm volatile("setmaxnreg.dec.sync.aligned.u32 48;");
+        // ------------------------------------------------------------------ dq_part = dS K over two 8-column steps
+        if (lane == 0) {
+            const int part = warp - 12, grp = part >> 1;
+            const uint32_t idO = idesc_tf32(C2);
+            const uint32_t tO = tm + TQ_ACC + part * 32;
+            for (int it = 0; it < total && ok; ++it) {
+                const int s = it % NSQ, us = it / NSQ, b = it & 1;
+                PROF_WAIT(0, ok = mb_wait(s32(&bars[Q_KCONV + s]), us & 1, ok));
+                PROF_WAIT(1, ok = mb_wait(s32(&bars[Q_DSREADY + grp]), it & 1, ok) && ok);
+                asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                const uint32_t tS = tm + TQ_BUF + 128 * b, tT = tS + BNQ;
+                const uint32_t kt = sbase + s * QST + 4 * TILE_Q;
+#pragma unroll
+                for (int k8 = 0; k8 < 2; ++k8) {
+                    const int ks = part * 2 + k8;                                   // 8-column step within the block
+                    const uint32_t off = (uint32_t)(ks >> 2) * (C2 * 128) + (uint32_t)(ks & 3) * 32;
+                    const uint64_t dkh = desc_k(kt + off), dkl = desc_k(kt + TILE_Q + off);
+                    mma_ts(tO, tT + ks * 8, dkh, idO, (k8 > 0) || (it % FOLDQ != 0));
+                    mma_ts(tO, tS + ks * 8, dkl, idO, 1);
+                    mma_ts(tO, tS + ks * 8, dkh, idO, 1);
+                }
+                mma_commit(s32(&bars[Q_G2DONE + 2 * grp + b]));
+                mma_commit(s32(&bars[Q_KTFREE + s]));
+            }
+        }
+    } else {
+        asm volatile("setmaxnreg.dec.sync.aligned.u32 80;");
+        // ------------------------------------------------------------------ converters (warps 16-19, 128 threads)
+        const int ct = tid - 512, cw = ct >> 5;
+        auto lo4 = [](const float4& x) { return make_float4(x.x - trunc19f(x.x), x.y - trunc19f(x.y), x.z - trunc19f(x.z), x.w - trunc19f(x.w)); };
+        for (int it = 0; it < total && ok; ++it) {
+            const int s = it % NSQ, u = it / NSQ;
+            unsigned char* st = base + s * QST;
+            // k_lo (same swizzled position as the raw element) and k transposed: warp cw takes the 16 columns [16 cw, 16 cw + 16),
+            // lane = channel
+            PROF_WAIT(0, ok = mb_wait(s32(&bars[Q_KFULL + s]), u & 1, ok));
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                const int off = (j * 128 + ct) * 16;
+                *reinterpret_cast<float4*>(st + TILE_Q + off) = lo4(*reinterpret_cast<const float4*>(st + off));
+            }
+            {
+                unsigned char* kth = st + 4 * TILE_Q + (cw >> 1) * (C2 * 128);
+#pragma unroll
+                for (int c8 = 0; c8 < 4; ++c8) {
+                    float hi[4], lo[4];
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) {
+                        const int col = cw * 16 + c8 * 4 + i;
+                        const float x = *reinterpret_cast<const float*>(st + sw_off(col, lane >> 2) + (lane & 3) * 4);
+                        hi[i] = trunc19f(x);
+                        lo[i] = x - hi[i];
+                    }
+                    const int chunk = (cw & 1) * 4 + c8;
+                    *reinterpret_cast<float4*>(kth + sw_off(lane, chunk)) = make_float4(hi[0], hi[1], hi[2], hi[3]);
+                    *reinterpret_cast<float4*>(kth + TILE_Q + sw_off(lane, chunk)) = make_float4(lo[0], lo[1], lo[2], lo[3]);
+                }
+            }
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+            mb_arrive(s32(&bars[Q_KCONV + s]));
+            // v_lo
+            PROF_WAIT(1, ok = mb_wait(s32(&bars[Q_VFULL + s]), u & 1, ok) && ok);
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                const int off = (j * 128 + ct) * 16;
+                *reinterpret_cast<float4*>(st + 3 * TILE_Q + off) = lo4(*reinterpret_cast<const float4*>(st + 2 * TILE_Q + off));
+            }
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+            mb_arrive(s32(&bars[Q_VCONV + s]));
+        }
+    }
+    if (!ok) atomicExch(&fail_s, 1);
+    PROF_DUMP(p.dev_status, warp, lane, total)
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    if (fail_s && tid == 0) atomicExch(p.dev_status, 1);
+    if (warp == 0) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tm), "r"(T_COLS));
+}
+
+// ---------------------------------------------------------------------------------------------------------
+// Pipelined dense part of the dk/dv stage (App. B.4), transposed roles: a block owns 128 consecutive input columns of
+// an input ring (tile row = input point j, its k and v rows and their lo parts live in TMEM) and walks, in blocks of 64,
+// the output points i of the output rings that attend to this input ring as a whole:
+//   S^T = K Q^T, T^T = V dY^T (one issuing thread each);  p = exp2(s + log2 omega_j - lse_i),  ds = p (t - D_i);
+//   dV += P dY,  dK += scale * dS Q   (A operands P, dS from TMEM; B operands: q and dout blocks transposed by the converters).
+// Two groups of 128 threads do the element-wise work for one half of the block's columns each and write P over S^T, dS
+// over T^T and the two lo parts beside them; four threads issue the second GEMMs (dV or dK, one column half each) into
+// their own accumulators, which collect FOLDK blocks in TMEM before the row's threads fold them into registers.  TMEM
+// holds only one (S^T, T^T) buffer here (128 columns of fixed operands + 256 of S, T, P_lo, dS_lo + 128 of accumulators), so
+// the first GEMMs of block j+1 wait for the second GEMMs of block j; TMA and the converters run three blocks ahead.
+// ---------------------------------------------------------------------------------------------------------
+constexpr int BNK = 64;                          // partner points per block
+constexpr int TILE_K = BNK * 128;                // 8 KB
+constexpr int FOLDK = 4;
+constexpr int NSK = 3;                           // shared-memory stages
+// per stage: q raw, q lo, y raw, y lo, q^T hi, q^T lo, y^T hi, y^T lo, then log2 omega - lse*log2e and D of the 64 partner points
+constexpr int KST = 8 * TILE_K + 1024;
+constexpr size_t DKDV2_SMEM = NSK * KST + 1024;
+constexpr int TK_AK = 0, TK_AKL = 32, TK_AV = 64, TK_AVL = 96, TK_S = 128, TK_T = 192, TK_PLO = 256, TK_DSLO = 320, TK_ACC = 384 /* + 32 part */;
+enum { K_QFULL = 0, K_YFULL = 3, K_QCONV = 6, K_YCONV = 9, K_FREE = 12 /* all [stage] */, K_STFULL = 15, K_READY = 16 /* [group] */,
+       K_G2DONE = 18 /* [group] */, K_AREADY = 20, K_COUNT = 21 };
+
+__global__ void __launch_bounds__(THREADS2, 1)
+backward_dkdv_dense2_kernel(DevPlan p, const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_y,
+                            const float* __restrict__ k, const float* __restrict__ v, const float* __restrict__ lse,
+                            const float* __restrict__ Dws, float* __restrict__ dk, float* __restrict__ dv, int N, float scale,
+                            int tiles_per_row) {
+    extern __shared__ unsigned char dense2_raw[];
+    unsigned char* base = (unsigned char*)(((uintptr_t)dense2_raw + 1023) & ~(uintptr_t)1023);
+    __shared__ unsigned long long bars[K_COUNT];
+    __shared__ uint32_t tmem_base_s;
+    __shared__ int fail_s;
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int tile = blockIdx.x % tiles_per_row;
+    const int rest = blockIdx.x / tiles_per_row;
+    const int n = rest % N;
+    const int hp = p.t_dense_rows[rest / N];
+    const int c0 = tile * M2;
+    const int nblk = (p.nlon_out + BNK - 1) / BNK;
+    const int e_begin = p.t_dense_ptr[hp], e_end = p.t_dense_ptr[hp + 1];
+    const int total = (e_end - e_begin) * nblk;
+    const float scale_log2 = scale * LOG2E_2;
+
+    if (tid == 0) {
+        for (int s = 0; s < NSK; ++s) {
+            mb_init(s32(&bars[K_QFULL + s]), 1);
+            mb_init(s32(&bars[K_YFULL + s]), 1);
+            mb_init(s32(&bars[K_QCONV + s]), 128);
+            mb_init(s32(&bars[K_YCONV + s]), 128);
+            mb_init(s32(&bars[K_FREE + s]), 6);         // both first GEMMs and the four second-GEMM issuers
+        }
+        mb_init(s32(&bars[K_STFULL]), 2);
+        for (int g = 0; g < 2; ++g) {
+            mb_init(s32(&bars[K_READY + g]), 128);
+            mb_init(s32(&bars[K_G2DONE + g]), 2);
+        }
+        mb_init(s32(&bars[K_AREADY]), 128);
+        fail_s = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 0) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(s32(&tmem_base_s)), "r"(T_COLS));
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::);
+    }
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    const uint32_t tm = tmem_base_s;
+    const uint32_t sbase = s32(base);
+    bool ok = true;
+    PROF_DECL
+
+    if (warp < 8) {
+        // register budget of the block: 640 threads x 96 at launch; a warpgroup can only grow by what the others give back:
+        // 256 x 160 + 256 x 40 + 128 x 72 = 60416 <= 61440
+        asm volatile("setmaxnreg.inc.sync.aligned.u32 160;");
+        // ------------------------------------------------------------------ element-wise: thread (grp, r) owns tile row r (an
+        // input point) for the partner columns [32 grp, 32 grp + 32) of every block
+        const int grp = warp >> 2, r = tid & 127;
+        const uint32_t lanebits = (uint32_t)((warp & 3) * 32) << 16;
+        const int c = c0 + r;
+        const bool row_ok = c < p.nlon_in;
+        const size_t ipt = (size_t)(n * p.nlat_in + hp) * p.nlon_in + min(c, p.nlon_in - 1);
+        if (grp == 0) {
+            // this row's k and v into TMEM (A operands of the first GEMMs): raw words as hi parts, lo = x - trunc19(x)
+            uint32_t xk[32], xv[32];
+            const float4* ks = reinterpret_cast<const float4*>(k + ipt * C2);
+            const float4* vs = reinterpret_cast<const float4*>(v + ipt * C2);
+#pragma unroll
+            for (int c4 = 0; c4 < C2 / 4; ++c4) {
+                const float4 a = __ldg(ks + c4), b = __ldg(vs + c4);
+                xk[4 * c4] = __float_as_uint(a.x); xk[4 * c4 + 1] = __float_as_uint(a.y); xk[4 * c4 + 2] = __float_as_uint(a.z); xk[4 * c4 + 3] = __float_as_uint(a.w);
+                xv[4 * c4] = __float_as_uint(b.x); xv[4 * c4 + 1] = __float_as_uint(b.y); xv[4 * c4 + 2] = __float_as_uint(b.z); xv[4 * c4 + 3] = __float_as_uint(b.w);
+            }
+            tm_st32(tm + TK_AK + lanebits, xk);
+            tm_st32(tm + TK_AV + lanebits, xv);
+#pragma unroll
+            for (int j = 0; j < 32; ++j) {
+                const float a = __uint_as_float(xk[j]), b = __uint_as_float(xv[j]);
+                xk[j] = __float_as_uint(a - trunc19f(a));
+                xv[j] = __float_as_uint(b - trunc19f(b));
+            }
+            tm_st32(tm + TK_AKL + lanebits, xk);
+            tm_st32(tm + TK_AVL + lanebits, xv);
+            asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
+            asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+            mb_arrive(s32(&bars[K_AREADY]));
+        }
+        constexpr int GC = BNK / 2;                       // columns per thread and block
+        float gk[C2], gv[C2];
+#pragma unroll
+        for (int i = 0; i < C2; ++i) { gk[i] = 0.f; gv[i] = 0.f; }
+        for (int it = 0; it <= total && ok; ++it) {
+            if (it > 0 && (it % FOLDK == 0 || it == total)) {
+                // fold the second GEMMs of the blocks since the last fold; this also frees the accumulators
+                PROF_WAIT(1, ok = mb_wait(s32(&bars[K_G2DONE + grp]), (it - 1) & 1, ok) && ok);
+                asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                uint32_t oa[32], ob[32];
+                tm_ld32_issue(oa, tm + TK_ACC + grp * 32 + lanebits);          // dV, this column half
+                tm_ld32_issue(ob, tm + TK_ACC + 64 + grp * 32 + lanebits);     // dK, this column half
+                tm_ld_wait();
+#pragma unroll
+                for (int j = 0; j < C2; ++j) { gv[j] += __uint_as_float(oa[j]); gk[j] += __uint_as_float(ob[j]); }
+            }
+            if (it < total) {
+                const int s = it % NSK;
+                const int nvalid = p.nlon_out - (it % nblk) * BNK - grp * GC;     // partner columns of this thread's half that exist
+                PROF_WAIT(0, ok = mb_wait(s32(&bars[K_STFULL]), it & 1, ok) && ok);     // implies QCONV of this stage (the S issuer waited for it)
+                asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                const float* nlc = reinterpret_cast<const float*>(base + s * KST + 8 * TILE_K) + grp * GC;
+                const float* Dc = nlc + BNK;
+                const uint32_t tS = tm + TK_S + grp * GC + lanebits, tT = tm + TK_T + grp * GC + lanebits;
+                const uint32_t tPl = tm + TK_PLO + grp * GC + lanebits, tDl = tm + TK_DSLO + grp * GC + lanebits;
+#pragma unroll
+                for (int hf = 0; hf < 2; ++hf) {
+                    uint32_t sv[16], tv[16], pl[16], dl[16];
+                    tm_ld16_issue(sv, tS + hf * 16);
+                    tm_ld16_issue(tv, tT + hf * 16);
+                    tm_ld_wait();
+#pragma unroll
+                    for (int j = 0; j < 16; ++j) {
+                        const int col = hf * 16 + j;
+                        float pj = ex2f(fmaf(__uint_as_float(sv[j]), scale_log2, nlc[col]));
+                        if (nvalid < GC && col >= nvalid) pj = 0.f;
+                        const float ds = pj * (__uint_as_float(tv[j]) - Dc[col]);
+                        sv[j] = __float_as_uint(pj);
+                        tv[j] = __float_as_uint(ds);
+                        pl[j] = __float_as_uint(pj - trunc19f(pj));
+                        dl[j] = __float_as_uint(ds - trunc19f(ds));
+                    }
+                    tm_st16(tS + hf * 16, sv);
+                    tm_st16(tT + hf * 16, tv);
+                    tm_st16(tPl + hf * 16, pl);
+                    tm_st16(tDl + hf * 16, dl);
+                }
+                asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
+                asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+                mb_arrive(s32(&bars[K_READY + grp]));
+            }
+        }
+        // merge the two column halves of every row through shared memory (the staging tiles are dead by now)
+        float* xs = reinterpret_cast<float*>(base);
+        if (grp == 1) {
+#pragma unroll
+            for (int j = 0; j < C2; ++j) { xs[j * 128 + r] = gk[j]; xs[(C2 + j) * 128 + r] = gv[j]; }
+        }
+        asm volatile("bar.sync 1, 256;" ::: "memory");
+        if (grp == 0 && ok && row_ok) {
+            float4* dkp = reinterpret_cast<float4*>(dk + ipt * C2);
+            float4* dvp = reinterpret_cast<float4*>(dv + ipt * C2);
+#pragma unroll
+            for (int c4 = 0; c4 < C2 / 4; ++c4) {
+                float a[4], b[4];
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    a[i] = (gk[4 * c4 + i] + xs[(4 * c4 + i) * 128 + r]) * scale;
+                    b[i] = gv[4 * c4 + i] + xs[(C2 + 4 * c4 + i) * 128 + r];
+                }
+                dkp[c4] = make_float4(a[0], a[1], a[2], a[3]);
+                dvp[c4] = make_float4(b[0], b[1], b[2], b[3]);
+            }
+        }
+    } else if (warp < 12) {
+        asm volatile("setmaxnreg.dec.sync.aligned.u32 40;");
+        if (warp == 8 && lane == 0) {
+            // -------------------------------------------------------------- TMA producer: q and dout blocks of the partner rings
+            for (int it = 0; it < total && ok; ++it) {
+                const int s = it % NSK, u = it / NSK;
+                const int h = p.t_dense_lat[e_begin + it / nblk];
+                const int w0 = (it % nblk) * BNK;
+                if (u > 0) PROF_WAIT(0, ok = mb_wait(s32(&bars[K_FREE + s]), (u - 1) & 1, ok));
+                mb_expect(s32(&bars[K_QFULL + s]), TILE_K);
+                tma_tile(sbase + s * KST, &map_q, w0, n * p.nlat_out + h, s32(&bars[K_QFULL + s]));
+                mb_expect(s32(&bars[K_YFULL + s]), TILE_K);
+                tma_tile(sbase + s * KST + 2 * TILE_K, &map_y, w0, n * p.nlat_out + h, s32(&bars[K_YFULL + s]));
+            }
+        }
+        if ((warp == 9 || warp == 10) && lane == 0) {
+            // -------------------------------------------------------------- S^T = K Q^T (warp 9) and T^T = V dY^T (warp 10)
+            const bool isT = warp == 10;
+            ok = mb_wait(s32(&bars[K_AREADY]), 0, ok);
+            const uint32_t idS = idesc_tf32(BNK);
+            const uint32_t tA = tm + (isT ? TK_AV : TK_AK), tAl = tm + (isT ? TK_AVL : TK_AKL);
+            for (int it = 0; it < total && ok; ++it) {
+                const int s = it % NSK, us = it / NSK;
+                PROF_WAIT(0, ok = mb_wait(s32(&bars[(isT ? K_YFULL : K_QFULL) + s]), us & 1, ok));
+                PROF_WAIT(1, ok = mb_wait(s32(&bars[(isT ? K_YCONV : K_QCONV) + s]), us & 1, ok) && ok);
+                if (it > 0) {   // the single (S^T, T^T) buffer is free once all four second-GEMM issuers of block it-1 are done
+                    PROF_WAIT(2, ok = mb_wait(s32(&bars[K_G2DONE]), (it - 1) & 1, ok) && ok);
+                    PROF_WAIT(2, ok = mb_wait(s32(&bars[K_G2DONE + 1]), (it - 1) & 1, ok) && ok);
+                }
+                asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                const uint32_t tile0 = sbase + s * KST + (isT ? 2 * TILE_K : 0);
+                const uint64_t db = desc_k(tile0), dbl = desc_k(tile0 + TILE_K);
+                const uint32_t tD = tm + (isT ? TK_T : TK_S);
+#pragma unroll
+                for (int ks = 0; ks < C2 / 8; ++ks) mma_ts(tD, tAl + ks * 8, db + 2 * ks, idS, ks > 0);
+#pragma unroll
+                for (int ks = 0; ks < C2 / 8; ++ks) mma_ts(tD, tA + ks * 8, dbl + 2 * ks, idS, 1);
+#pragma unroll
+                for (int ks = 0; ks < C2 / 8; ++ks) mma_ts(tD, tA + ks * 8, db + 2 * ks, idS, 1);
+                mma_commit(s32(&bars[K_STFULL]));
+                mma_commit(s32(&bars[K_FREE + s]));
+            }
+        }
+    } else if (warp < 16) {
+        asm volatile("setmaxnreg.dec.sync.aligned.u32 40;");
+        // ------------------------------------------------------------------ second GEMMs: part = (kind, column half)
+        if (lane == 0) {
+            const int part = warp - 12, kind = part >> 1, grp = part & 1;      // kind 0: dV = P dY, kind 1: dK = dS Q
+            const uint32_t idO = idesc_tf32(C2);
+            const uint32_t tO = tm + TK_ACC + part * 32;
+            const uint32_t tA = tm + (kind ? TK_T : TK_S), tAl = tm + (kind ? TK_DSLO : TK_PLO);
+            for (int it = 0; it < total && ok; ++it) {
+                const int s = it % NSK, us = it / NSK;
+                PROF_WAIT(0, ok = mb_wait(s32(&bars[(kind ? K_QCONV : K_YCONV) + s]), us & 1, ok));
+                PROF_WAIT(1, ok = mb_wait(s32(&bars[K_READY + grp]), it & 1, ok) && ok);
+                asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                const uint32_t bt = sbase + s * KST + (kind ? 4 : 6) * TILE_K;          // q^T (dK) or y^T (dV) tiles
+#pragma unroll
+                for (int k8 = 0; k8 < 4; ++k8) {
+                    const int ks = grp * 4 + k8;                                    // 8-column step within the block
+                    const uint32_t off = (uint32_t)(ks >> 2) * (C2 * 128) + (uint32_t)(ks & 3) * 32;
+                    const uint64_t dh = desc_k(bt + off), dl = desc_k(bt + TILE_K + off);
+                    mma_ts(tO, tAl + ks * 8, dh, idO, (k8 > 0) || (it % FOLDK != 0));
+                    mma_ts(tO, tA + ks * 8, dl, idO, 1);
+                    mma_ts(tO, tA + ks * 8, dh, idO, 1);
+                }
+                mma_commit(s32(&bars[K_G2DONE + grp]));
+                mma_commit(s32(&bars[K_FREE + s]));
+            }
+        }
+    } else {
+        asm volatile("setmaxnreg.dec.sync.aligned.u32 72;");
+        // ------------------------------------------------------------------ converters (warps 16-19, 128 threads)
+        const int ct = tid - 512, cw = ct >> 5;
+        auto lo4 = [](const float4& x) { return make_float4(x.x - trunc19f(x.x), x.y - trunc19f(x.y), x.z - trunc19f(x.z), x.w - trunc19f(x.w)); };
+        // lo tile (same swizzled positions) and transposed hi / lo tiles of one raw tile: warp cw takes the 16 columns
+        // [16 cw, 16 cw + 16), lane = channel
+        auto convert = [&](unsigned char* raw, unsigned char* lo, unsigned char* th) {
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                const int off = (j * 128 + ct) * 16;
+                *reinterpret_cast<float4*>(lo + off) = lo4(*reinterpret_cast<const float4*>(raw + off));
+            }
+            unsigned char* t = th + (cw >> 1) * (C2 * 128);
+#pragma unroll
+            for (int c8 = 0; c8 < 4; ++c8) {
+                float hi[4], lw[4];
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    const int col = cw * 16 + c8 * 4 + i;
+                    const float x = *reinterpret_cast<const float*>(raw + sw_off(col, lane >> 2) + (lane & 3) * 4);
+                    hi[i] = trunc19f(x);
+                    lw[i] = x - hi[i];
+                }
+                const int chunk = (cw & 1) * 4 + c8;
+                *reinterpret_cast<float4*>(t + sw_off(lane, chunk)) = make_float4(hi[0], hi[1], hi[2], hi[3]);
+                *reinterpret_cast<float4*>(t + TILE_K + sw_off(lane, chunk)) = make_float4(lw[0], lw[1], lw[2], lw[3]);
+            }
+        };
+        for (int it = 0; it < total && ok; ++it) {
+            const int s = it % NSK, u = it / NSK;
+            unsigned char* st = base + s * KST;
+            const int h = p.t_dense_lat[e_begin + it / nblk];
+            const int w0 = (it % nblk) * BNK;
+            PROF_WAIT(0, ok = mb_wait(s32(&bars[K_QFULL + s]), u & 1, ok));       // also: the stage (and its statistics arrays) is free
+            if (ct < BNK) {
+                const size_t o = (size_t)(n * p.nlat_out + h) * p.nlon_out + min(w0 + ct, p.nlon_out - 1);
+                float* nlc = reinterpret_cast<float*>(st + 8 * TILE_K);
+                nlc[ct] = fmaf(-__ldg(lse + o), LOG2E_2, p.log2_omega[hp]);   // log2 omega_j - lse_i in the log2 domain
+                nlc[BNK + ct] = __ldg(Dws + o);
+            }
+            convert(st, st + TILE_K, st + 4 * TILE_K);
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+            mb_arrive(s32(&bars[K_QCONV + s]));
+            PROF_WAIT(1, ok = mb_wait(s32(&bars[K_YFULL + s]), u & 1, ok) && ok);
+            convert(st + 2 * TILE_K, st + 3 * TILE_K, st + 6 * TILE_K);
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+            mb_arrive(s32(&bars[K_YCONV + s]));
+        }
+    }
+    if (!ok) atomicExch(&fail_s, 1);
+    PROF_DUMP(p.dev_status, warp, lane, total)
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    if (fail_s && tid == 0) atomicExch(p.dev_status, 1);
+    if (warp == 0) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tm), "r"(T_COLS));
+}
+
 using EncodeFn2 = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
                                const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
                                CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
@@ -424,13 +1067,13 @@ EncodeFn2 encode_fn2() {
     }();
     return fn;
 }
-// Tensor map over a channels-last array [slices * rings][nlon][32] with boxes of 128 points x 32 channels.
-cudaError_t make_map2(CUtensorMap* map, const float* base, int rings_total, int nlon) {
+// Tensor map over a channels-last array [slices * rings][nlon][32] with boxes of box_rows points x 32 channels.
+cudaError_t make_map2(CUtensorMap* map, const float* base, int rings_total, int nlon, int box_rows = BN2) {
     EncodeFn2 fn = encode_fn2();
     if (fn == nullptr) return cudaErrorNotSupported;
     const cuuint64_t dims[3] = {(cuuint64_t)C2, (cuuint64_t)nlon, (cuuint64_t)rings_total};
     const cuuint64_t strides[2] = {(cuuint64_t)C2 * 4, (cuuint64_t)nlon * C2 * 4};
-    const cuuint32_t box[3] = {(cuuint32_t)C2, (cuuint32_t)BN2, 1};
+    const cuuint32_t box[3] = {(cuuint32_t)C2, (cuuint32_t)box_rows, 1};
     const cuuint32_t estr[3] = {1, 1, 1};
     const CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, const_cast<float*>(base), dims, strides, box, estr,
                           CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
@@ -441,11 +1084,44 @@ cudaError_t make_map2(CUtensorMap* map, const float* base, int rings_total, int 
 }  // namespace
 
 cudaError_t dense2_prepare_device() {
-    return cudaFuncSetAttribute(forward_dense2_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)DENSE2_SMEM);
+    cudaError_t e = cudaFuncSetAttribute(forward_dense2_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)DENSE2_SMEM);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(backward_dq_dense2_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)DQ2_SMEM);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(backward_dkdv_dense2_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)DKDV2_SMEM);
+    return e;
 }
 
 bool dense2_path_supported(const DevPlan& p, int C) {
     return dense_path_supported(p, C) && encode_fn2() != nullptr;
+}
+
+cudaError_t launch_backward_dq_dense2(const DevPlan& p, const float* q, const float* k, const float* v, const float* dout,
+                                      const float* out, const float* lse, float* dq, float* Dws, int N, int C, cudaStream_t stream) {
+    if (C != C2 || out == nullptr || lse == nullptr || out == dq) return cudaErrorInvalidValue;
+    const int tiles_per_row = (p.nlon_out + M2 - 1) / M2;
+    const long long blocks = (long long)tiles_per_row * p.n_dense_rows * N;
+    if (blocks <= 0) return cudaSuccess;
+    if (blocks > 0x7fffffffLL) return cudaErrorInvalidValue;
+    CUtensorMap mk, mv;
+    cudaError_t e = make_map2(&mk, k, N * p.nlat_in, p.nlon_in, BNQ);
+    if (e == cudaSuccess) e = make_map2(&mv, v, N * p.nlat_in, p.nlon_in, BNQ);
+    if (e != cudaSuccess) return e;
+    backward_dq_dense2_kernel<<<(unsigned)blocks, THREADS2, DQ2_SMEM, stream>>>(p, mk, mv, q, dout, out, lse, dq, Dws, N, 1.0f / sqrtf((float)C), tiles_per_row);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_backward_dkdv_dense2(const DevPlan& p, const float* q, const float* k, const float* v, const float* dout,
+                                        const float* lse, const float* Dws, float* dk, float* dv, int N, int C, cudaStream_t stream) {
+    if (C != C2) return cudaErrorInvalidValue;
+    const int tiles_per_row = (p.nlon_in + M2 - 1) / M2;
+    const long long blocks = (long long)tiles_per_row * p.n_t_dense_rows * N;
+    if (blocks <= 0) return cudaSuccess;
+    if (blocks > 0x7fffffffLL) return cudaErrorInvalidValue;
+    CUtensorMap mq, my;
+    cudaError_t e = make_map2(&mq, q, N * p.nlat_out, p.nlon_out, BNK);
+    if (e == cudaSuccess) e = make_map2(&my, dout, N * p.nlat_out, p.nlon_out, BNK);
+    if (e != cudaSuccess) return e;
+    backward_dkdv_dense2_kernel<<<(unsigned)blocks, THREADS2, DKDV2_SMEM, stream>>>(p, mq, my, k, v, lse, Dws, dk, dv, N, 1.0f / sqrtf((float)C), tiles_per_row);
+    return cudaGetLastError();
 }
 
 cudaError_t launch_forward_dense2(const DevPlan& p, const float* q, const float* k, const float* v, float* out, float* lse,
