@@ -82,6 +82,17 @@ sna_status_t sna_plan_create(int nlat_in, int nlon_in, int nlat_out, int nlon_ou
                              sna_grid_t grid_in, sna_grid_t grid_out, double theta_cutoff,
                              sna_plan_t** plan_out);
 
+/*
+ * Plan for GLOBAL spherical attention (Eq. s2_attention_discrete; App. B.1-B.2): every output point attends to every
+ * input point, i.e. softmax attention over the whole input grid with the additive bias log omega_j.  Equivalent to
+ * sna_plan_create with theta_cutoff >= pi, but no per-pair structure is built or stored: the plan holds only the grids,
+ * the quadrature weights and the per-ring lists the dense tensor-core kernels walk.  All compute calls accept it; with
+ * C = 32 they run entirely on the dense tcgen05 kernels (the forward pass then needs an lse buffer, and the backward
+ * pass runs fastest with out and lse from sna_forward_ex); other shapes use the generic kernels.
+ */
+sna_status_t sna_plan_create_global(int nlat_in, int nlon_in, int nlat_out, int nlon_out,
+                                    sna_grid_t grid_in, sna_grid_t grid_out, sna_plan_t** plan_out);
+
 /* Same construction, but nothing is copied to a GPU and no CUDA call is made: the plan serves the
  * introspection calls below only (compute calls on it return SNA_ERR_INVALID_ARG).  For inspecting or
  * validating tables on a machine without a GPU. */

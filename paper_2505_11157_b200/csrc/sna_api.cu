@@ -43,6 +43,7 @@ struct sna_plan {
     sna::HostPlan host;
     sna::DevPlan dev{};
     int device = 0;
+    bool is_global = false;            // created by sna_plan_create_global: no column streams, dense kernels only
     void* dev_blob = nullptr;          // one allocation holding every device table
     mutable std::mutex ws_mutex;
     mutable void* ws = nullptr;        // workspace grown on demand by sna_backward
@@ -101,7 +102,8 @@ const char* sna_status_string(sna_status_t s) {
 const char* sna_last_error_message(void) { return g_last_error; }
 
 static sna_status_t plan_create(int nlat_in, int nlon_in, int nlat_out, int nlon_out, sna_grid_t grid_in,
-                                sna_grid_t grid_out, double theta_cutoff, bool upload, sna_plan_t** plan_out) {
+                                sna_grid_t grid_out, double theta_cutoff, bool upload, sna_plan_t** plan_out,
+                                bool global = false) {
     if (plan_out == nullptr) { set_error("plan_out is NULL"); return SNA_ERR_INVALID_ARG; }
     sna_plan* plan = new (std::nothrow) sna_plan();
     if (plan == nullptr) { set_error("out of host memory"); return SNA_ERR_ALLOC; }
@@ -143,10 +145,28 @@ static sna_status_t plan_create(int nlat_in, int nlon_in, int nlat_out, int nlon
     const int32_t zero_status[64] = {};
 #endif
     bool t_consecutive = false;
+    plan->is_global = global;
     try {
+        sna::build_dense_lists(hp, dense);
+        sna::build_transposed_dense_lists(hp, t_dense);
+        // rows with the most whole rings first: the dense kernels run one block per SM, so the long tiles must not start last
+        std::stable_sort(dense.rows.begin(), dense.rows.end(), [&](int a, int b) { return dense.ptr[a + 1] - dense.ptr[a] > dense.ptr[b + 1] - dense.ptr[b]; });
+        std::stable_sort(t_dense.rows.begin(), t_dense.rows.end(), [&](int a, int b) { return t_dense.ptr[a + 1] - t_dense.ptr[a] > t_dense.ptr[b + 1] - t_dense.ptr[b]; });
+        if (global) {
+            // every window is a whole ring: the dense kernels do all the work, so the column streams (which would list
+            // every pair of the dense problem) are not built; they stay empty and the band kernels are never launched
+            const size_t g_out = (hp.nlat_out + sna::TILE_LAT - 1) / sna::TILE_LAT, g_in = (hp.nlat_in + sna::TILE_LAT - 1) / sna::TILE_LAT;
+            fwd_stream.chunk_ptr.assign(g_out + 1, 0);
+            fwdb_stream.chunk_ptr.assign(g_out + 1, 0);
+            t_stream.chunk_ptr.assign(g_in + 1, 0);
+            tb_stream.chunk_ptr.assign(g_in + 1, 0);
+            t_consecutive = true;
+            grp_order.resize(g_out);
+            std::iota(grp_order.begin(), grp_order.end(), 0);
+            grpb_order = grp_order;
+        } else {
         sna::build_forward_stream(hp, fwd_stream);
         t_consecutive = sna::build_transposed_stream(hp, t_stream);
-        sna::build_dense_lists(hp, dense);
         sna::build_forward_stream(hp, fwdb_stream, /*include_whole=*/false);
         grpb_order.resize(fwdb_stream.chunk_ptr.size() - 1);
         std::iota(grpb_order.begin(), grpb_order.end(), 0);
@@ -159,8 +179,8 @@ static sna_status_t plan_create(int nlat_in, int nlon_in, int nlat_out, int nlon
         std::stable_sort(grp_order.begin(), grp_order.end(), [&](int a, int b) {
             return fwd_stream.chunk_ptr[a + 1] - fwd_stream.chunk_ptr[a] > fwd_stream.chunk_ptr[b + 1] - fwd_stream.chunk_ptr[b];
         });
-        sna::build_transposed_dense_lists(hp, t_dense);
         sna::build_transposed_stream(hp, tb_stream, /*include_whole=*/false);
+        }
         const int rows_per_group = t_consecutive ? 1 : hp.ps;
         tb_grp_order.resize((tb_stream.chunk_ptr.size() - 1) / rows_per_group);
         std::iota(tb_grp_order.begin(), tb_grp_order.end(), 0);
@@ -223,8 +243,9 @@ static sna_status_t plan_create(int nlat_in, int nlon_in, int nlat_out, int nlon
     {
         size_t whole = 0;
         for (const sna::StreamEntry& en : fwd_stream.entries) whole += en.base < 0;
-        d.dense_fraction = fwd_stream.entries.empty() ? 0.f : (float)whole / (float)fwd_stream.entries.size();
+        d.dense_fraction = global ? 1.f : fwd_stream.entries.empty() ? 0.f : (float)whole / (float)fwd_stream.entries.size();
     }
+    d.is_global = global ? 1 : 0;
     d.dev_status = (int*)((char*)plan->dev_blob + pieces[21].offset);
     d.tb_stream = (const int4*)at(22); d.tb_chunk_ptr = at(23); d.tb_grp_order = at(24);
     d.t_dense_ptr = at(25); d.t_dense_lat = at(26); d.t_dense_rows = at(27);
@@ -241,6 +262,12 @@ static sna_status_t plan_create(int nlat_in, int nlon_in, int nlat_out, int nlon
 sna_status_t sna_plan_create(int nlat_in, int nlon_in, int nlat_out, int nlon_out, sna_grid_t grid_in,
                              sna_grid_t grid_out, double theta_cutoff, sna_plan_t** plan_out) {
     return plan_create(nlat_in, nlon_in, nlat_out, nlon_out, grid_in, grid_out, theta_cutoff, true, plan_out);
+}
+
+sna_status_t sna_plan_create_global(int nlat_in, int nlon_in, int nlat_out, int nlon_out, sna_grid_t grid_in,
+                                    sna_grid_t grid_out, sna_plan_t** plan_out) {
+    // theta_cutoff = pi selects every input point for every output point; no distance is evaluated
+    return plan_create(nlat_in, nlon_in, nlat_out, nlon_out, grid_in, grid_out, 3.14159265358979323846, true, plan_out, true);
 }
 
 sna_status_t sna_plan_create_host_only(int nlat_in, int nlon_in, int nlat_out, int nlon_out, sna_grid_t grid_in,
@@ -339,6 +366,7 @@ size_t sna_workspace_bytes(const sna_plan_t* plan, int B, int H, int C) {
 
 int sna_forward_kernel_count(const sna_plan_t* plan, int C, int with_lse) {
     if (plan == nullptr || plan->dev_blob == nullptr || !supported_C(C)) return 0;
+    if (plan->is_global) return 1;
     return (with_lse && sna::dense_path_supported(plan->dev, C)) ? 2 : 1;
 }
 
@@ -349,7 +377,12 @@ sna_status_t sna_forward_ex(const sna_plan_t* plan, const float* q, const float*
     if (!q || !k || !v || !out) { set_error("q, k, v and out must not be NULL"); return SNA_ERR_INVALID_ARG; }
     if (!all_aligned(q, k, v, out) || (reinterpret_cast<uintptr_t>(lse) & 3u)) { set_error("device pointers must be 16-byte aligned"); return SNA_ERR_INVALID_ARG; }
     cudaError_t e;
-    if (lse != nullptr && sna::dense_path_supported(plan->dev, C)) {
+    if (plan->is_global) {
+        // global attention: the dense kernel alone produces the final out and lse
+        e = (lse != nullptr && sna::dense2_global_supported(plan->dev, C))
+                ? sna::launch_forward_dense2(plan->dev, q, k, v, out, lse, B * H, C, (cudaStream_t)cuda_stream)
+                : sna::launch_forward_generic(plan->dev, q, k, v, out, lse, B * H, C, (cudaStream_t)cuda_stream);
+    } else if (lse != nullptr && sna::dense_path_supported(plan->dev, C)) {
         // whole-ring windows on the tcgen05 kernel (its partial result travels in out / lse), the rest on the band kernel
         e = sna::dense2_path_supported(plan->dev, C)
                 ? sna::launch_forward_dense2(plan->dev, q, k, v, out, lse, B * H, C, (cudaStream_t)cuda_stream)
@@ -377,9 +410,13 @@ sna_status_t sna_backward_dq(const sna_plan_t* plan, const float* q, const float
     if (!q || !k || !v || !dout || !lse || !dq || !D) { set_error("q, k, v, dout, lse, dq and D must not be NULL"); return SNA_ERR_INVALID_ARG; }
     if (!all_aligned(q, k, v, dout, dq, out) || ((reinterpret_cast<uintptr_t>(lse) | reinterpret_cast<uintptr_t>(D)) & 3u)) { set_error("device pointers must be 16-byte aligned"); return SNA_ERR_INVALID_ARG; }
     cudaError_t e;
-    // The dense dq kernel pays off when whole-ring windows are a large share of the work (measured: 1.5x on the
-    // global limit, -3 % at a 25 % share), so it is used from a 35 % share on.
-    if (out != nullptr && out != dq && plan->dev.dense_fraction >= 0.10f && sna::dense_path_supported(plan->dev, C)) {
+    // The dense dq kernel takes the whole-ring windows when they are at least a tenth of the work (measured on the
+    // benchmark configurations: -8 % on the dq stage at a 22 % share, -6 % at 13 %).
+    if (plan->is_global) {
+        e = (out != nullptr && out != dq && sna::dense2_global_supported(plan->dev, C))
+                ? sna::launch_backward_dq_dense2(plan->dev, q, k, v, dout, out, lse, dq, D, B * H, C, (cudaStream_t)cuda_stream)
+                : sna::launch_backward_dq_generic(plan->dev, q, k, v, dout, out, lse, dq, D, B * H, C, (cudaStream_t)cuda_stream);
+    } else if (out != nullptr && out != dq && plan->dev.dense_fraction >= 0.10f && sna::dense_path_supported(plan->dev, C)) {
         // whole-ring windows on the tcgen05 kernel (its part of dq is written first), the banded rest is added by the band kernel
         e = sna::dense2_path_supported(plan->dev, C)
                 ? sna::launch_backward_dq_dense2(plan->dev, q, k, v, dout, out, lse, dq, nullptr, B * H, C, (cudaStream_t)cuda_stream)
@@ -402,7 +439,11 @@ sna_status_t sna_backward_dkdv(const sna_plan_t* plan, const float* q, const flo
     if (!q || !k || !v || !dout || !lse || !D || !dk || !dv) { set_error("q, k, v, dout, lse, D, dk and dv must not be NULL"); return SNA_ERR_INVALID_ARG; }
     if (!all_aligned(q, k, v, dout, dk, dv) || ((reinterpret_cast<uintptr_t>(lse) | reinterpret_cast<uintptr_t>(D)) & 3u)) { set_error("device pointers must be 16-byte aligned"); return SNA_ERR_INVALID_ARG; }
     cudaError_t e;
-    if (plan->dev.dense_fraction >= 0.10f && plan->dev.n_t_dense_rows > 0 && sna::dense_path_supported(plan->dev, C)) {
+    if (plan->is_global) {
+        e = sna::dense2_global_supported(plan->dev, C)
+                ? sna::launch_backward_dkdv_dense2(plan->dev, q, k, v, dout, lse, D, dk, dv, B * H, C, (cudaStream_t)cuda_stream)
+                : sna::launch_backward_dkdv_generic(plan->dev, q, k, v, dout, lse, D, dk, dv, B * H, C, (cudaStream_t)cuda_stream);
+    } else if (plan->dev.dense_fraction >= 0.10f && plan->dev.n_t_dense_rows > 0 && sna::dense_path_supported(plan->dev, C)) {
         // whole-ring partners on the tcgen05 kernel (its part of dk, dv is written first), the band kernel adds the rest
         e = sna::dense2_path_supported(plan->dev, C)
                 ? sna::launch_backward_dkdv_dense2(plan->dev, q, k, v, dout, lse, D, dk, dv, B * H, C, (cudaStream_t)cuda_stream)
@@ -431,7 +472,23 @@ sna_status_t sna_backward_ex(const sna_plan_t* plan, const float* q, const float
     float* ws_lse = (float*)workspace;
     float* ws_D = ws_lse + stats_elems(plan, B, H);
     cudaError_t e;
-    if (sna::mma_path_supported(plan->dev, C)) {
+    if (plan->is_global) {
+        if (lse == nullptr || out == nullptr) {
+            // recompute the forward pass.  The dense dq kernel may not read out from the dq buffer, so out goes into
+            // the dk buffer (written only after the dq stage) when that is large enough; otherwise only the
+            // statistics are recomputed and the generic dq kernel runs.
+            const bool fits = (long long)plan->host.nlat_in * plan->host.nlon_in >= (long long)plan->host.nlat_out * plan->host.nlon_out;
+            if (fits && sna::dense2_global_supported(plan->dev, C)) {
+                e = sna::launch_forward_dense2(plan->dev, q, k, v, dk, ws_lse, N, C, stream);
+                out = dk;
+            } else {
+                e = sna::launch_forward_generic(plan->dev, q, k, v, nullptr, ws_lse, N, C, stream);
+                out = nullptr;
+            }
+            if (e != cudaSuccess) return cuda_fail(e, "statistics launch");
+            lse = ws_lse;
+        }
+    } else if (sna::mma_path_supported(plan->dev, C)) {
         if (lse == nullptr || out == nullptr) {
             // recompute the forward pass: lse into the workspace, out into the dq buffer, which the dq stage
             // reads row by row before it overwrites the same rows with dq

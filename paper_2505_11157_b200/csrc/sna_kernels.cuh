@@ -46,6 +46,7 @@ struct DevPlan {
     const int32_t* t_chunk_ptr;     // [groups of input latitudes * ps + 1]
     const int32_t* t_grp_order;     // groups of input latitudes, longest stream first
     int t_consecutive;              // 1: transposed tiles are 8 consecutive input columns; 0: split by residue mod ps
+    int is_global;                  // 1: every window is a whole ring and no column stream exists (dense kernels or generic kernels only)
 };
 
 // Tensor-core kernels (C = 16, 32 or 64, nlon_out >= 32); same contracts as the generic launchers.
@@ -70,6 +71,7 @@ cudaError_t launch_forward_dense(const DevPlan& p, const float* q, const float* 
 // Pipelined version of the dense forward kernel (TMA loads, warp-specialised, see sna_kernels_dense2.cu); same contract.
 cudaError_t dense2_prepare_device();   // once per device: opt in to the kernel's shared-memory size
 bool dense2_path_supported(const DevPlan& p, int C);
+bool dense2_global_supported(const DevPlan& p, int C);   // the dense kernels can serve a global plan on their own
 cudaError_t launch_forward_dense2(const DevPlan& p, const float* q, const float* k, const float* v, float* out, float* lse,
                                   int N, int C, cudaStream_t stream);
 // Pipelined dense dq kernel; same contract as launch_backward_dq_dense, and it also writes D (Dws may be null).

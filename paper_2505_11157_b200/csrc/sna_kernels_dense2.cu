@@ -1094,6 +1094,11 @@ bool dense2_path_supported(const DevPlan& p, int C) {
     return dense_path_supported(p, C) && encode_fn2() != nullptr;
 }
 
+bool dense2_global_supported(const DevPlan& p, int C) {
+    return C == C2 && p.is_global && p.n_dense_rows > 0 && p.n_t_dense_rows > 0 && encode_fn2() != nullptr &&
+           (long long)p.nlat_in * p.nlon_in * C < (1LL << 32) && (long long)p.nlat_out * p.nlon_out * C < (1LL << 32);
+}
+
 cudaError_t launch_backward_dq_dense2(const DevPlan& p, const float* q, const float* k, const float* v, const float* dout,
                                       const float* out, const float* lse, float* dq, float* Dws, int N, int C, cudaStream_t stream) {
     if (C != C2 || out == nullptr || lse == nullptr || out == dq) return cudaErrorInvalidValue;

@@ -607,7 +607,7 @@ cudaError_t mma_prepare_device() {
 }
 
 bool mma_path_supported(const DevPlan& p, int C) {
-    return p.fwd_stream != nullptr && (C == 16 || C == 32 || C == 64) && p.nlon_out >= 32 && p.nlon_out < 32768 &&
+    return p.fwd_stream != nullptr && !p.is_global && (C == 16 || C == 32 || C == 64) && p.nlon_out >= 32 && p.nlon_out < 32768 &&
            (long long)p.nlat_in * p.nlon_in * C < (1LL << 32) && (long long)p.nlat_out * p.nlon_out * C < (1LL << 32);
 }
 

@@ -42,6 +42,7 @@ _vp, _i, _d, _sz = ctypes.c_void_p, ctypes.c_int, ctypes.c_double, ctypes.c_size
 _SIGNATURES = {
     "sna_plan_create": (_i, [_i, _i, _i, _i, _i, _i, _d, ctypes.POINTER(_vp)]),
     "sna_plan_create_host_only": (_i, [_i, _i, _i, _i, _i, _i, _d, ctypes.POINTER(_vp)]),
+    "sna_plan_create_global": (_i, [_i, _i, _i, _i, _i, _i, ctypes.POINTER(_vp)]),
     "sna_plan_destroy": (_i, [_vp]),
     "sna_plan_check": (_i, [_vp]),
     "sna_plan_get_nnz": (_i, [_vp, ctypes.POINTER(ctypes.c_int64)]),
@@ -111,6 +112,13 @@ def sna_plan_create(nlat_in, nlon_in, nlat_out, nlon_out, grid_in, grid_out, the
     handle = _vp()
     fn = _lib.sna_plan_create_host_only if host_only else _lib.sna_plan_create
     _check(fn(nlat_in, nlon_in, nlat_out, nlon_out, grid_in, grid_out, float(theta_cutoff), ctypes.byref(handle)))
+    return handle.value
+
+
+def sna_plan_create_global(nlat_in, nlon_in, nlat_out, nlon_out, grid_in, grid_out) -> int:
+    """Plan for global spherical attention (every output point attends to every input point)."""
+    handle = _vp()
+    _check(_lib.sna_plan_create_global(nlat_in, nlon_in, nlat_out, nlon_out, grid_in, grid_out, ctypes.byref(handle)))
     return handle.value
 
 
@@ -204,12 +212,15 @@ class Plan:
     """Owns one ``sna_plan_t``.  Shapes follow the header: q/out [B,H,nlat_out,nlon_out,C], k/v [B,H,nlat_in,nlon_in,C]."""
 
     def __init__(self, nlat_in, nlon_in, nlat_out, nlon_out, grid_in=SNA_GRID_EQUIANGULAR,
-                 grid_out=SNA_GRID_EQUIANGULAR, theta_cutoff=0.1, host_only=False):
+                 grid_out=SNA_GRID_EQUIANGULAR, theta_cutoff=0.1, host_only=False, global_attention=False):
         self.nlat_in, self.nlon_in, self.nlat_out, self.nlon_out = nlat_in, nlon_in, nlat_out, nlon_out
         self.grid_in, self.grid_out, self.theta_cutoff = grid_in, grid_out, float(theta_cutoff)
         self.host_only = host_only
         self.handle = None
-        self.handle = sna_plan_create(nlat_in, nlon_in, nlat_out, nlon_out, grid_in, grid_out, theta_cutoff, host_only)
+        if global_attention:
+            self.handle = sna_plan_create_global(nlat_in, nlon_in, nlat_out, nlon_out, grid_in, grid_out)
+        else:
+            self.handle = sna_plan_create(nlat_in, nlon_in, nlat_out, nlon_out, grid_in, grid_out, theta_cutoff, host_only)
         self.ps = nlon_in // nlon_out
 
     def close(self):

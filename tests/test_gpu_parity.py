@@ -218,6 +218,29 @@ def test_global_limit_against_dense_oracle():
     assert nerr(out.reshape(ref.shape), ref) <= FWD_TOL
 
 
+@pytest.mark.parametrize("shape", [(16, 32, 16, 32, EQ, EQ, 1, 2, 32), (33, 160, 17, 80, EQ, GL, 1, 2, 32),
+                                   (40, 200, 40, 200, GL, GL, 2, 1, 32), (12, 24, 12, 24, EQ, EQ, 1, 2, 16)],
+                         ids=["16x32", "33x160_down2", "40x200_gl", "C16_generic"])
+@pytest.mark.parametrize("reuse", [True, False], ids=["saved_state", "recompute"])
+def test_global_plan_against_oracle(shape, reuse):
+    """sna_plan_create_global: forward against the dense definition written out, backward against the
+    neighbourhood oracle with the cutoff at pi (whose forward the same dense definition pins on CPU)."""
+    nlat_in, nlon_in, nlat_out, nlon_out, grid_in, grid_out, B, H, C = shape
+    wl = small_workload("global_plan", nlat_in, nlon_in, nlat_out, nlon_out, grid_in, grid_out, math.pi, B, H, C, 31)
+    g = _geometry(wl)
+    q, k, v, dout = make_inputs(wl)
+    with sna.Plan(nlat_in, nlon_in, nlat_out, nlon_out, grid_in, grid_out, global_attention=True) as plan:
+        out, lse, dq, dk, dv = _run_gpu(plan, q, k, v, dout, reuse)
+        assert sna.sna_forward_kernel_count(plan.handle, C, True) == 1
+    ref = orc.dense_forward(np.repeat(g.omega, wl.nlon_in), q.reshape(wl.N, -1, wl.C), k.reshape(wl.N, -1, wl.C),
+                            v.reshape(wl.N, -1, wl.C))
+    assert nerr(out.reshape(ref.shape), ref) <= FWD_TOL
+    ref_out, ref_lse = orc.forward(g, q, k, v, return_lse=True)
+    assert np.max(np.abs(lse.reshape(ref_lse.shape) - ref_lse)) <= 1e-4
+    for name, x, r in zip(("dq", "dk", "dv"), (dq, dk, dv), orc.backward(g, q, k, v, dout)):
+        assert nerr(x.reshape(r.shape), r) <= BWD_TOL, name
+
+
 def test_results_are_reproducible_bit_for_bit():
     wl = SMALL[2]
     q, k, v, dout = make_inputs(wl)
