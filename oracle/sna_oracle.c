@@ -21,6 +21,11 @@
  *
  * Readings taken where the paper is silent (all listed again in the design notes):
  *   - equiangular grid includes both poles, theta_h = pi*h/(nlat-1), Clenshaw-Curtis weights;
+ *   - the grid App. A.1 itself prints (theta_i = pi*i/nlat, i = 0..nlat-1: north pole in, south pole out, point
+ *     weights 2 pi^2/(nlat nlon) sin(theta_i)) is the third grid, "equiangular trapezoid": its weights are the
+ *     composite trapezoid rule in theta and sum to 4 pi only approximately; its pole ring has weight zero, so
+ *     those points are members of a disc but contribute nothing, and an output point whose whole disc has
+ *     weight zero has no defined result (0/0) and is reported as an empty neighborhood;
  *   - "Gaussian grid" = Gauss-Legendre nodes in cos(theta), ordered north to south;
  *   - point weight w_{h'} = (latitude weight) * 2*pi/nlon_in, so the weights sum to 4*pi;
  *   - different resolutions: input column = (w' + w*ps) mod nlon_in with ps = nlon_in/nlon_out;
@@ -54,6 +59,7 @@
 
 #define GRID_EQUIANGULAR 0
 #define GRID_LEGENDRE_GAUSS 1
+#define GRID_EQUIANGULAR_TRAPEZOID 2
 
 static const double PI = 3.14159265358979323846264338327950288;
 
@@ -102,6 +108,10 @@ int sna_oracle_colatitudes(int grid, int nlat, double *theta) {
         for (int h = 0; h < nlat; ++h) theta[h] = PI * h / (nlat - 1);
         return ORACLE_OK;
     }
+    if (grid == GRID_EQUIANGULAR_TRAPEZOID) {   /* Eq. (latlon_grid) */
+        for (int h = 0; h < nlat; ++h) theta[h] = PI * h / nlat;
+        return ORACLE_OK;
+    }
     if (grid == GRID_LEGENDRE_GAUSS) {
         double *x = (double *)malloc(sizeof(double) * nlat * 2);
         if (!x) return ORACLE_ERR_INVALID;
@@ -113,7 +123,8 @@ int sna_oracle_colatitudes(int grid, int nlat, double *theta) {
     return ORACLE_ERR_INVALID;
 }
 
-/* Latitude quadrature weights for int_{-1}^{1} f(cos theta) d(cos theta); they sum to 2. */
+/* Latitude quadrature weights for int_{-1}^{1} f(cos theta) d(cos theta); they sum to 2 (the trapezoid
+ * grid's to (pi/nlat) cot(pi/(2 nlat)) = 2 - pi^2/(6 nlat^2) + ...). */
 int sna_oracle_latitude_weights(int grid, int nlat, double *wlat) {
     if (nlat < 2 || !wlat) return ORACLE_ERR_INVALID;
     if (grid == GRID_EQUIANGULAR) {
@@ -129,6 +140,11 @@ int sna_oracle_latitude_weights(int grid, int nlat, double *wlat) {
             double c = (h == 0 || h == n) ? 1.0 : 2.0;
             wlat[h] = c / n * s;
         }
+        return ORACLE_OK;
+    }
+    if (grid == GRID_EQUIANGULAR_TRAPEZOID) {
+        /* Eq. (latlon_quad_weights): q_ij = 2 pi^2/(nlat nlon) sin(theta_i) = wlat_i * 2 pi/nlon. */
+        for (int h = 0; h < nlat; ++h) wlat[h] = PI / nlat * sin(PI * h / nlat);
         return ORACLE_OK;
     }
     if (grid == GRID_LEGENDRE_GAUSS) {
@@ -161,16 +177,18 @@ int sna_oracle_neighborhood(int grid_in, int nlat_in, int nlon_in, int grid_out,
     if (nlat_in < 2 || nlat_out < 2 || nlon_in < 1 || !(theta_cutoff > 0.0) || !nnz_out) return ORACLE_ERR_INVALID;
     double *th_in = (double *)malloc(sizeof(double) * nlat_in);
     double *th_out = (double *)malloc(sizeof(double) * nlat_out);
+    double *w_in = (double *)malloc(sizeof(double) * nlat_in);
     int rc = sna_oracle_colatitudes(grid_in, nlat_in, th_in);
     if (!rc) rc = sna_oracle_colatitudes(grid_out, nlat_out, th_out);
-    if (rc) { free(th_in); free(th_out); return rc; }
+    if (!rc) rc = sna_oracle_latitude_weights(grid_in, nlat_in, w_in);
+    if (rc) { free(th_in); free(th_out); free(w_in); return rc; }
     const int everything = theta_cutoff >= PI;
     int64_t n = 0;
     int status = ORACLE_OK;
     for (int h = 0; h < nlat_out; ++h) {
         if (row_ptr) row_ptr[h] = n;
         const double xo[3] = { sin(th_out[h]), 0.0, cos(th_out[h]) };
-        int64_t row_start = n;
+        int64_t weighted = 0;   /* members with a non-zero quadrature weight */
         for (int hp = 0; hp < nlat_in; ++hp) {
             for (int wp = 0; wp < nlon_in; ++wp) {
                 int member;
@@ -190,14 +208,15 @@ int sna_oracle_neighborhood(int grid_in, int nlat_in, int nlon_in, int grid_out,
                 if (member) {
                     if (n < capacity && lat_in && lon_off) { lat_in[n] = hp; lon_off[n] = wp; }
                     ++n;
+                    if (w_in[hp] > 0.0) ++weighted;
                 }
             }
         }
-        if (n == row_start && status == ORACLE_OK) status = ORACLE_ERR_EMPTY_NEIGHBORHOOD;
+        if (weighted == 0 && status == ORACLE_OK) status = ORACLE_ERR_EMPTY_NEIGHBORHOOD;
     }
     if (row_ptr) row_ptr[nlat_out] = n;
     *nnz_out = n;
-    free(th_in); free(th_out);
+    free(th_in); free(th_out); free(w_in);
     if (status) return status;
     if (capacity > 0 && n > capacity) return ORACLE_ERR_CAPACITY;
     return ORACLE_OK;

@@ -23,6 +23,7 @@ _LIB = os.path.join(_HERE, "libsna_oracle.so")
 
 EQUIANGULAR = 0
 LEGENDRE_GAUSS = 1
+EQUIANGULAR_TRAPEZOID = 2   # the grid App. A.1 prints: theta_i = pi i / nlat, weights ~ sin(theta_i), pole ring weight 0
 
 _ERRORS = {1: "invalid argument", 2: "ambiguous tie on the disc boundary", 3: "empty neighborhood",
            4: "capacity too small"}

@@ -14,7 +14,7 @@ import torch
 
 from oracle import sna_oracle as orc
 
-EQ, GL = orc.EQUIANGULAR, orc.LEGENDRE_GAUSS
+EQ, GL, TZ = orc.EQUIANGULAR, orc.LEGENDRE_GAUSS, orc.EQUIANGULAR_TRAPEZOID
 
 
 def _rand(g, N, C, seed, dtype=np.float64):
@@ -31,6 +31,8 @@ GEOMS = {
     "eq_down": (17, 32, 9, 16, EQ, EQ, 0.5),
     "gl_same": (10, 20, 10, 20, GL, GL, 0.7),
     "gl_to_eq_down3": (12, 24, 7, 8, GL, EQ, 0.8),
+    "tz_same": (12, 24, 12, 24, TZ, TZ, 0.6),
+    "tz_down": (16, 32, 8, 16, TZ, TZ, 0.5),
 }
 
 
@@ -122,7 +124,7 @@ def _sdpa(q, k, v, omega_pt):
                                                             attn_mask=mask), (q_t, k_t, v_t)
 
 
-@pytest.mark.parametrize("args", [(8, 16, 8, 16, EQ, EQ), (9, 12, 5, 6, EQ, GL), (6, 12, 6, 12, GL, GL)])
+@pytest.mark.parametrize("args", [(8, 16, 8, 16, EQ, EQ), (9, 12, 5, 6, EQ, GL), (6, 12, 6, 12, GL, GL), (8, 16, 8, 16, TZ, TZ)])
 def test_global_limit_matches_library_dense_attention(args):
     g = orc.geometry(*args, math.pi)
     N, C = 2, 8
@@ -142,6 +144,31 @@ def test_global_limit_matches_library_dense_attention(args):
     assert np.allclose(dv.reshape(N, -1, C), vt.grad.numpy(), rtol=0, atol=1e-12)
 
 
+def test_zero_weight_pole_ring_contributes_nothing():
+    # on the grid of Eq. (latlon_grid) the pole ring has quadrature weight sin(0) = 0: its points are inside the
+    # discs near the pole but neither their keys nor their values can reach any output, and they get no gradient
+    g = orc.geometry(10, 20, 10, 20, TZ, TZ, 0.7)
+    assert g.omega[0] == 0.0 and np.any(g.lat_in == 0)
+    q, k, v, dout = _rand(g, 2, 6, 21)
+    out = orc.forward(g, q, k, v)
+    k2, v2 = k.copy(), v.copy()
+    k2[:, 0] += 3.0
+    v2[:, 0] = 100.0
+    # (not bit-equal: a pole-ring score may set the running maximum, which moves the rounding)
+    assert np.allclose(orc.forward(g, q, k2, v2), out, rtol=0, atol=1e-13)
+    dq, dk, dv = orc.backward(g, q, k, v, dout)
+    assert not dk[:, 0].any() and not dv[:, 0].any()
+    assert dk[:, 1].any() and dv[:, 1].any() and np.isfinite(dq).all()
+
+
+def test_a_disc_of_total_weight_zero_is_reported():
+    # the disc of the pole output point holds only the (zero-weight) pole ring: Eq. (s2_attention_discrete_detailed) is 0/0
+    with pytest.raises(orc.OracleError) as e:
+        orc.geometry(16, 32, 16, 32, TZ, TZ, 0.05)
+    assert e.value.code == 3
+    orc.geometry(16, 32, 16, 32, TZ, TZ, 0.25)      # one more ring inside: defined again
+
+
 def test_lse_definition(geom):
     q, k, v, _ = _rand(geom, 1, 4, 9)
     out, lse = orc.forward(geom, q, k, v, return_lse=True)
@@ -153,7 +180,8 @@ def test_lse_definition(geom):
     assert abs(lse[0, h, w] - math.log(np.sum(np.exp(s) * geom.omega[lat]))) < 1e-13
 
 
-@pytest.mark.parametrize("args", [(6, 12, 6, 12, EQ, EQ, 0.9), (8, 16, 4, 8, EQ, EQ, 0.9), (5, 10, 5, 10, GL, GL, 1.0)])
+@pytest.mark.parametrize("args", [(6, 12, 6, 12, EQ, EQ, 0.9), (8, 16, 4, 8, EQ, EQ, 0.9), (5, 10, 5, 10, GL, GL, 1.0),
+                                  (6, 12, 6, 12, TZ, TZ, 0.9)])
 def test_backward_matches_central_finite_differences(args):
     g = orc.geometry(*args)
     N, C = 1, 4

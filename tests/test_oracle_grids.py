@@ -6,7 +6,7 @@ import pytest
 
 from oracle import sna_oracle as orc
 
-EQ, GL = orc.EQUIANGULAR, orc.LEGENDRE_GAUSS
+EQ, GL, TZ = orc.EQUIANGULAR, orc.LEGENDRE_GAUSS, orc.EQUIANGULAR_TRAPEZOID
 
 
 def test_equiangular_colatitudes_include_both_poles():
@@ -78,6 +78,41 @@ def test_quadrature_integrates_a_smooth_function():
         z = np.cos(th)[:, None] * np.ones_like(phi)[None, :]
         total = np.sum((1 + z + x * x) * om[:, None])
         assert abs(total - (4 * math.pi + 4 * math.pi / 3)) < 1e-12
+
+
+def test_trapezoid_grid_has_the_north_pole_but_not_the_south_pole():
+    # Eq. (latlon_grid): theta_i = pi i / nlat for i = 0 .. nlat-1
+    th = orc.colatitudes(TZ, 6)
+    assert th[0] == 0.0 and abs(th[-1] - (math.pi - math.pi / 6)) < 1e-15
+    assert np.allclose(np.diff(th), math.pi / 6, rtol=0, atol=1e-15)
+
+
+def test_trapezoid_weights_values_from_the_printed_formula():
+    # Eq. (latlon_quad_weights) by hand for nlat = 4, nlon = 8: 2 pi^2/32 * sin(0, pi/4, pi/2, 3pi/4)
+    om = orc.quad_weights(TZ, 4, 8)
+    unit = 2 * math.pi ** 2 / 32
+    assert om[0] == 0.0
+    assert np.allclose(om, [0.0, unit * math.sqrt(0.5), unit, unit * math.sqrt(0.5)], rtol=1e-15, atol=0)
+
+
+@pytest.mark.parametrize("nlat", [2, 5, 64, 361])
+def test_trapezoid_weights_are_the_library_trapezoid_rule_in_theta(nlat):
+    # int_0^pi f(theta) sin(theta) dtheta by the composite trapezoid rule on nlat intervals: the integrand
+    # vanishes at both ends, so the rule needs no south-pole node and equals the weighted sum over the grid
+    from scipy.integrate import trapezoid
+    w, th = orc.latitude_weights(TZ, nlat), orc.colatitudes(TZ, nlat)
+    nodes = np.linspace(0.0, math.pi, nlat + 1)
+    for f in (lambda t: np.ones_like(t), lambda t: np.cos(t) ** 2, lambda t: np.exp(0.3 * t)):
+        assert abs(np.sum(w * f(th)) - trapezoid(f(nodes) * np.sin(nodes), nodes)) < 1e-13
+
+
+@pytest.mark.parametrize("nlat, nlon", [(4, 8), (33, 64), (361, 720)])
+def test_trapezoid_point_weights_sum_only_approximately_to_sphere_area(nlat, nlon):
+    # closed form: sum_i sin(pi i/n) = cot(pi/(2n)), so the total is (2 pi^2/n) cot(pi/(2n)) = 4 pi (1 - pi^2/(12 n^2) + ...)
+    total = np.sum(orc.quad_weights(TZ, nlat, nlon)) * nlon
+    assert abs(total - 2 * math.pi ** 2 / nlat / math.tan(math.pi / (2 * nlat))) < 1e-12
+    lead = 4 * math.pi * math.pi ** 2 / (12 * nlat ** 2)          # x cot x = 1 - x^2/3 - x^4/45 - ... at x = pi/(2n)
+    assert lead < 4 * math.pi - total < lead * 1.02
 
 
 def test_invalid_arguments():
