@@ -60,7 +60,14 @@ typedef enum {
     SNA_GRID_EQUIANGULAR = 0,
     /* "Gaussian grid" (Sec. 3.3): theta_h = arccos(x_h), x_h the roots of the Legendre polynomial P_nlat in
      * descending order (north to south), Gauss-Legendre weights. */
-    SNA_GRID_LEGENDRE_GAUSS = 1
+    SNA_GRID_LEGENDRE_GAUSS = 1,
+    /* The equiangular grid exactly as App. A.1 prints it (Eq. latlon_grid, Eq. latlon_quad_weights):
+     * theta_h = pi*h/nlat, h = 0..nlat-1 (north pole a ring, south pole not), point weights
+     * 2 pi^2/(nlat nlon) sin(theta_h): the trapezoid rule in theta, summing to 4 pi only approximately.  The pole
+     * ring has weight zero: its points are listed by the table queries but contribute to no output, and their
+     * dk / dv are zero.  A theta_cutoff so small that the pole output point sees only the pole ring leaves that
+     * output undefined (0/0) and is refused with SNA_ERR_EMPTY_NEIGHBORHOOD. */
+    SNA_GRID_EQUIANGULAR_TRAPEZOID = 2
 } sna_grid_t;
 
 /*

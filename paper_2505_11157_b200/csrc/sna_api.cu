@@ -43,6 +43,7 @@ struct sna_plan {
     sna::HostPlan host;
     sna::DevPlan dev{};
     int device = 0;
+    std::vector<int> zero_rings;       // input rings of quadrature weight zero (no kernel of a global plan visits them)
     bool is_global = false;            // created by sna_plan_create_global: no column streams, dense kernels only
     void* dev_blob = nullptr;          // one allocation holding every device table
     mutable std::mutex ws_mutex;
@@ -122,8 +123,12 @@ static sna_status_t plan_create(int nlat_in, int nlon_in, int nlat_out, int nlon
         return ps == sna::PLAN_INVALID ? SNA_ERR_INVALID_ARG : ps == sna::PLAN_UNSUPPORTED ? SNA_ERR_UNSUPPORTED
              : ps == sna::PLAN_EMPTY ? SNA_ERR_EMPTY_NEIGHBORHOOD : SNA_ERR_AMBIGUOUS_TIE;
     }
-    const sna::HostPlan& hp = plan->host;
     if (!upload) { *plan_out = plan; return SNA_OK; }
+    // the kernels walk the table without rings of weight zero; plan->host keeps every member for the table queries
+    sna::HostPlan weighted;
+    const bool dropped = sna::drop_zero_weight_rings(plan->host, weighted);
+    const sna::HostPlan& hp = dropped ? weighted : plan->host;
+    for (int h = 0; h < hp.nlat_in; ++h) if (!(hp.omega[h] > 0.0)) plan->zero_rings.push_back(h);
     // heavy-first orders
     std::vector<int32_t> row_order(hp.nlat_out), t_row_order(hp.nlat_in);
     std::iota(row_order.begin(), row_order.end(), 0);
@@ -440,7 +445,16 @@ sna_status_t sna_backward_dkdv(const sna_plan_t* plan, const float* q, const flo
     if (!all_aligned(q, k, v, dout, dk, dv) || ((reinterpret_cast<uintptr_t>(lse) | reinterpret_cast<uintptr_t>(D)) & 3u)) { set_error("device pointers must be 16-byte aligned"); return SNA_ERR_INVALID_ARG; }
     cudaError_t e;
     if (plan->is_global) {
-        e = sna::dense2_global_supported(plan->dev, C)
+        // the dense kernel writes only the rings some window refers to; rings of weight zero get their (zero) gradient here
+        const bool dense = sna::dense2_global_supported(plan->dev, C);
+        const size_t ring_bytes = (size_t)plan->host.nlon_in * C * sizeof(float), pitch = ring_bytes * plan->host.nlat_in;
+        for (size_t i = 0; dense && i < plan->zero_rings.size(); ++i) {
+            const size_t off = ring_bytes * plan->zero_rings[i];
+            e = cudaMemset2DAsync((char*)dk + off, pitch, 0, ring_bytes, (size_t)B * H, (cudaStream_t)cuda_stream);
+            if (e == cudaSuccess) e = cudaMemset2DAsync((char*)dv + off, pitch, 0, ring_bytes, (size_t)B * H, (cudaStream_t)cuda_stream);
+            if (e != cudaSuccess) return cuda_fail(e, "clearing the gradients of zero-weight rings");
+        }
+        e = dense
                 ? sna::launch_backward_dkdv_dense2(plan->dev, q, k, v, dout, lse, D, dk, dv, B * H, C, (cudaStream_t)cuda_stream)
                 : sna::launch_backward_dkdv_generic(plan->dev, q, k, v, dout, lse, D, dk, dv, B * H, C, (cudaStream_t)cuda_stream);
     } else if (plan->dev.dense_fraction >= 0.10f && plan->dev.n_t_dense_rows > 0 && sna::dense_path_supported(plan->dev, C)) {

@@ -90,6 +90,17 @@ bool make_grid(int grid, int nlat, std::vector<double>& theta, std::vector<doubl
         for (int h = 0; h < nlat; ++h) theta[h] = std::acos(x[h]);
         return true;
     }
+    if (grid == 2) {
+        // the grid as App. A.1 prints it (Eq. latlon_grid, Eq. latlon_quad_weights): north pole in, south pole out,
+        // trapezoid weights (pi/nlat) sin(theta) in latitude; the pole ring's weight is exactly zero
+        theta.resize(nlat);
+        wlat.resize(nlat);
+        for (int h = 0; h < nlat; ++h) {
+            theta[h] = (double)(PI_L * h / nlat);
+            wlat[h] = h == 0 ? 0.0 : (double)(PI_L / nlat * sinl(PI_L * h / nlat));
+        }
+        return true;
+    }
     return false;
 }
 
@@ -171,6 +182,9 @@ PlanStatus build_plan(int nlat_in, int nlon_in, int nlat_out, int nlon_out, int 
         }
         P.row_ptr[h + 1] = (int32_t)P.windows.size();
         if (P.row_ptr[h + 1] == P.row_ptr[h] && !ambiguous) { why = "an output latitude has no input point within theta_cutoff"; return PLAN_EMPTY; }
+        bool weighted = false;
+        for (int i = P.row_ptr[h]; i < P.row_ptr[h + 1]; ++i) weighted = weighted || P.omega[P.windows[i].lat] > 0.0;
+        if (!weighted && !ambiguous) { why = "every input point within theta_cutoff of an output latitude has quadrature weight zero"; return PLAN_EMPTY; }
         P.nnz += P.row_nnz[h];
     }
     if (ambiguous) { why = "a grid point lies within 1e-8 rad of the disc boundary without being on it"; return PLAN_AMBIGUOUS; }
@@ -185,6 +199,39 @@ PlanStatus build_plan(int nlat_in, int nlon_in, int nlat_out, int nlon_out, int 
         P.t_row_ptr[hp + 1] = (int32_t)P.t_windows.size();
     }
     return PLAN_OK;
+}
+
+bool drop_zero_weight_rings(const HostPlan& full, HostPlan& out) {
+    bool any = false;
+    for (double w : full.omega) any = any || !(w > 0.0);
+    if (!any) return false;
+    out = full;
+    out.windows.clear();
+    out.t_windows.clear();
+    out.nnz = 0;
+    for (int h = 0; h < full.nlat_out; ++h) {
+        out.row_ptr[h] = (int32_t)out.windows.size();
+        out.row_nnz[h] = 0;
+        for (int i = full.row_ptr[h]; i < full.row_ptr[h + 1]; ++i) {
+            const RingWindow& w = full.windows[i];
+            if (!(full.omega[w.lat] > 0.0)) continue;
+            out.windows.push_back(w);
+            out.row_nnz[h] += full.window_count(w);
+        }
+        out.nnz += out.row_nnz[h];
+    }
+    out.row_ptr[full.nlat_out] = (int32_t)out.windows.size();
+    for (int hp = 0; hp < full.nlat_in; ++hp) {
+        out.t_row_ptr[hp] = (int32_t)out.t_windows.size();
+        out.t_row_nnz[hp] = 0;
+        if (!(full.omega[hp] > 0.0)) continue;
+        for (int i = full.t_row_ptr[hp]; i < full.t_row_ptr[hp + 1]; ++i) {
+            out.t_windows.push_back(full.t_windows[i]);
+            out.t_row_nnz[hp] += full.window_count(full.t_windows[i]);
+        }
+    }
+    out.t_row_ptr[full.nlat_in] = (int32_t)out.t_windows.size();
+    return true;
 }
 
 namespace {

@@ -33,6 +33,12 @@ struct HostPlan {
     int window_count(const RingWindow& w) const { return w.m < 0 ? nlon_in : 2 * w.m + 1; }
 };
 
+// The table the kernels walk: `full` without the input rings of quadrature weight zero (the pole ring of the
+// trapezoid grid).  Such points are members of discs but add nothing to any sum, and their own gradients are zero,
+// which the kernels produce for any input ring no window refers to.  Returns false (out untouched) if no ring has
+// weight zero.
+bool drop_zero_weight_rings(const HostPlan& full, HostPlan& out);
+
 // Column streams for the tensor-core kernels.  A warp owns a tile of 16 points: TILE_LON = 8 consecutive
 // longitudes on each of TILE_LAT = 2 adjacent rings (a "ring group"); tile row i is ring i / 8 of the group,
 // longitude first + i % 8.  Two adjacent rings see almost the same partner points, and 8-wide rows waste fewer

@@ -21,6 +21,7 @@ LIB_PATH = os.path.join(_PKG, "libsna.so")
 
 SNA_GRID_EQUIANGULAR = 0
 SNA_GRID_LEGENDRE_GAUSS = 1
+SNA_GRID_EQUIANGULAR_TRAPEZOID = 2
 
 SNA_OK = 0
 SNA_ERR_INVALID_ARG = 1

@@ -13,7 +13,7 @@ from paper_2505_11157_b200 import sna
 from paper_2505_11157_b200.synthetic import WORKLOADS
 
 ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
-EQ, GL = 0, 1
+EQ, GL, TZ = 0, 1, 2
 
 
 def _declared_functions():
@@ -49,6 +49,9 @@ CASES = {
     "odd_nlon": (10, 15, 10, 15, EQ, EQ, 0.8),
     "tiny": (4, 8, 4, 8, EQ, EQ, 1.1),
     "wide": (16, 32, 16, 32, EQ, EQ, 2.5),
+    "trapezoid": (24, 48, 24, 48, TZ, TZ, 0.4),
+    "trapezoid_down2_from_gl": (24, 48, 12, 24, GL, TZ, 0.6),
+    "trapezoid_global": (8, 16, 8, 16, TZ, TZ, math.pi),
 }
 
 
@@ -66,7 +69,10 @@ def test_planner_matches_oracle_bit_for_bit(name):
         assert np.allclose(ti, orc.colatitudes(args[4], args[0]), rtol=0, atol=2e-15)
         assert np.allclose(to, orc.colatitudes(args[5], args[2]), rtol=0, atol=2e-15)
         assert np.allclose(p.quad_weights(), g.omega, rtol=1e-13, atol=0)
-        assert abs(p.quad_weights().sum() * args[1] - 4 * math.pi) < 1e-12
+        if args[4] != TZ:
+            assert abs(p.quad_weights().sum() * args[1] - 4 * math.pi) < 1e-12
+        else:
+            assert p.quad_weights()[0] == 0.0
         # transposed table, rebuilt here from the oracle's table
         ps = args[1] // args[3]
         t_ptr, t_lat, t_off = p.table_transposed()
@@ -97,6 +103,7 @@ def test_headline_table_sizes():
     ((8, 16, 8, 16, EQ, EQ, 0.0), sna.SNA_ERR_INVALID_ARG),
     ((8, 16, 8, 16, EQ, EQ, float("nan")), sna.SNA_ERR_INVALID_ARG),
     ((5, 8, 16, 8, EQ, GL, 0.02), sna.SNA_ERR_EMPTY_NEIGHBORHOOD),
+    ((16, 32, 16, 32, TZ, TZ, 0.05), sna.SNA_ERR_EMPTY_NEIGHBORHOOD),   # the pole's disc holds only the zero-weight pole ring
     ((17, 32, 17, 32, EQ, EQ, 2 * math.pi / 16 + 1e-10), sna.SNA_ERR_AMBIGUOUS_TIE),
 ])
 def test_plan_errors(args, status):

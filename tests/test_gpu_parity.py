@@ -15,7 +15,7 @@ from paper_2505_11157_b200.synthetic import WORKLOADS, make_inputs, sample_point
 
 pytestmark = pytest.mark.gpu
 
-EQ, GL = 0, 1
+EQ, GL, TZ = 0, 1, 2
 FWD_TOL, BWD_TOL = 1e-5, 1e-4
 
 
@@ -81,6 +81,13 @@ SMALL = [
     small_workload("eq_c12", 12, 24, 12, 24, EQ, EQ, 0.6, 1, 2, 12, 37),
     small_workload("gl_down2_c24", 17, 64, 9, 32, GL, GL, 0.5, 2, 1, 24, 38),
     small_workload("eq_c48", 10, 40, 10, 40, EQ, EQ, 0.7, 1, 1, 48, 39),
+    # the grid as the paper prints it: pole ring of quadrature weight zero (inside discs, contributes nothing, dk = dv = 0)
+    small_workload("trapezoid_c32", 24, 48, 24, 48, TZ, TZ, 0.45, 1, 2, 32, 43),
+    small_workload("trapezoid_down2_c32", 32, 128, 16, 64, TZ, TZ, 0.5, 1, 2, 32, 44),
+    small_workload("trapezoid_polar_heavy_c32", 16, 64, 16, 64, TZ, TZ, 1.2, 1, 2, 32, 45),   # dense and banded windows mixed
+    small_workload("trapezoid_c16", 12, 32, 12, 32, TZ, TZ, 0.6, 1, 2, 16, 46),
+    small_workload("trapezoid_c12_generic", 12, 24, 12, 24, TZ, GL, 0.6, 1, 2, 12, 47),
+    small_workload("trapezoid_global_c32", 12, 64, 12, 64, TZ, TZ, math.pi, 1, 2, 32, 48),
 ]
 
 
@@ -219,8 +226,9 @@ def test_global_limit_against_dense_oracle():
 
 
 @pytest.mark.parametrize("shape", [(16, 32, 16, 32, EQ, EQ, 1, 2, 32), (33, 160, 17, 80, EQ, GL, 1, 2, 32),
-                                   (40, 200, 40, 200, GL, GL, 2, 1, 32), (12, 24, 12, 24, EQ, EQ, 1, 2, 16)],
-                         ids=["16x32", "33x160_down2", "40x200_gl", "C16_generic"])
+                                   (40, 200, 40, 200, GL, GL, 2, 1, 32), (12, 24, 12, 24, EQ, EQ, 1, 2, 16),
+                                   (20, 72, 20, 72, TZ, TZ, 1, 3, 32), (12, 24, 12, 24, TZ, EQ, 1, 2, 8)],
+                         ids=["16x32", "33x160_down2", "40x200_gl", "C16_generic", "trapezoid", "trapezoid_C8_generic"])
 @pytest.mark.parametrize("reuse", [True, False], ids=["saved_state", "recompute"])
 def test_global_plan_against_oracle(shape, reuse):
     """sna_plan_create_global: forward against the dense definition written out, backward against the
@@ -239,6 +247,8 @@ def test_global_plan_against_oracle(shape, reuse):
     assert np.max(np.abs(lse.reshape(ref_lse.shape) - ref_lse)) <= 1e-4
     for name, x, r in zip(("dq", "dk", "dv"), (dq, dk, dv), orc.backward(g, q, k, v, dout)):
         assert nerr(x.reshape(r.shape), r) <= BWD_TOL, name
+    if grid_in == TZ:       # the zero-weight pole ring: exact zeros, not small numbers
+        assert not dk.reshape(wl.N, nlat_in, -1)[:, 0].any() and not dv.reshape(wl.N, nlat_in, -1)[:, 0].any()
 
 
 def test_results_are_reproducible_bit_for_bit():
