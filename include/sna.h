@@ -112,8 +112,16 @@ sna_status_t sna_plan_destroy(sna_plan_t* plan);
 
 /* Waits for the plan's device to finish and reports whether any kernel launched through this plan gave up on one of
  * its bounded waits (SNA_ERR_CUDA; its outputs would be incomplete).  Kernels never spin without limit; this is the
- * way to find out that a limit was hit.  Not expected to happen. */
+ * way to find out that a limit was hit.  Not expected to happen.  A failure is reported once: the call that returns
+ * SNA_ERR_CUDA also clears the record, so outputs written since the previous check must be recomputed. */
 sna_status_t sna_plan_check(const sna_plan_t* plan);
+
+/* Test aid for that failure path.  Launches, on the given stream, one tiny kernel in which a single thread waits on a
+ * barrier that nothing ever arrives on, using the same bounded wait routine as the tensor-core kernels but limited to
+ * `polls` polls (1..100000; each poll suspends for at most about 2 microseconds).  The wait runs out, the kernel
+ * records that in the plan's status word and returns normally: no trap, no fault, the context stays usable.  The next
+ * sna_plan_check reports SNA_ERR_CUDA once and clears the word; compute calls on the plan work before and after. */
+sna_status_t sna_debug_exercise_bounded_wait(const sna_plan_t* plan, int polls, void* cuda_stream);
 
 /* ---- introspection into caller-owned HOST buffers ------------------------------------------------------ */
 

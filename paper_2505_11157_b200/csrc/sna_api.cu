@@ -298,7 +298,23 @@ sna_status_t sna_plan_check(const sna_plan_t* plan) {
     int status = 0;
     e = cudaMemcpy(&status, plan->dev.dev_status, sizeof(int), cudaMemcpyDeviceToHost);
     if (e != cudaSuccess) return cuda_fail(e, "cudaMemcpy of the device status word");
-    if (status != 0) { set_error("a kernel gave up on a bounded wait; its outputs are incomplete"); return SNA_ERR_CUDA; }
+    if (status != 0) {
+        // reported once: the word is cleared so that the plan can be used (and checked) again
+        e = cudaMemset(plan->dev.dev_status, 0, sizeof(int));
+        if (e != cudaSuccess) return cuda_fail(e, "cudaMemset of the device status word");
+        set_error("a kernel gave up on a bounded wait; its outputs are incomplete");
+        return SNA_ERR_CUDA;
+    }
+    return SNA_OK;
+}
+
+sna_status_t sna_debug_exercise_bounded_wait(const sna_plan_t* plan, int polls, void* cuda_stream) {
+    if (!plan || plan->dev_blob == nullptr) { set_error("needs a plan that lives on a GPU"); return SNA_ERR_INVALID_ARG; }
+    if (polls < 1 || polls > 100000) { set_error("polls must be between 1 and 100000"); return SNA_ERR_INVALID_ARG; }
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev != plan->device) { set_error("the plan's device is not current"); return SNA_ERR_INVALID_ARG; }
+    cudaError_t e = sna::launch_bounded_wait_probe(plan->dev, polls, (cudaStream_t)cuda_stream);
+    if (e != cudaSuccess) return cuda_fail(e, "probe launch");
     return SNA_OK;
 }
 

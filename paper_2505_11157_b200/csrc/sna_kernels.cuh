@@ -71,6 +71,7 @@ cudaError_t launch_forward_dense(const DevPlan& p, const float* q, const float* 
 // Pipelined version of the dense forward kernel (TMA loads, warp-specialised, see sna_kernels_dense2.cu); same contract.
 cudaError_t dense2_prepare_device();   // once per device: opt in to the kernel's shared-memory size
 bool dense2_path_supported(const DevPlan& p, int C);
+cudaError_t launch_bounded_wait_probe(const DevPlan& p, int polls, cudaStream_t stream);
 bool dense2_global_supported(const DevPlan& p, int C);   // the dense kernels can serve a global plan on their own
 cudaError_t launch_forward_dense2(const DevPlan& p, const float* q, const float* k, const float* v, float* out, float* lse,
                                   int N, int C, cudaStream_t stream);

@@ -77,13 +77,15 @@ __device__ __forceinline__ void mb_arrive(uint32_t bar) { asm volatile("mbarrier
 __device__ __forceinline__ void mb_expect(uint32_t bar, uint32_t bytes) { asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory"); }
 // Bounded wait.  try_wait suspends the thread in hardware for up to the hinted time, so a waiting warp takes few issue
 // slots from the warps that share its scheduler.  Once a wait has run out (`healthy` false) later waits give up at once.
-__device__ __forceinline__ bool mb_wait(uint32_t bar, uint32_t parity, bool healthy) {
+__device__ __forceinline__ bool mb_wait_polls(uint32_t bar, uint32_t parity, int limit) {
     uint32_t done = 0;
-    const int limit = healthy ? WAIT2 : 4;
     for (int it = 0; it < limit && !done; ++it)
         asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\tselp.u32 %0, 1, 0, p;\n\t}\n"
                      : "=r"(done) : "r"(bar), "r"(parity), "r"(2000u) : "memory");
     return done != 0;
+}
+__device__ __forceinline__ bool mb_wait(uint32_t bar, uint32_t parity, bool healthy) {
+    return mb_wait_polls(bar, parity, healthy ? WAIT2 : 4);
 }
 __device__ __forceinline__ void tma_tile(uint32_t dst, const CUtensorMap* map, int col, int ring, uint32_t bar) {
     asm volatile("cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];"
@@ -1088,6 +1090,24 @@ cudaError_t dense2_prepare_device() {
     if (e == cudaSuccess) e = cudaFuncSetAttribute(backward_dq_dense2_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)DQ2_SMEM);
     if (e == cudaSuccess) e = cudaFuncSetAttribute(backward_dkdv_dense2_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)DKDV2_SMEM);
     return e;
+}
+
+// The give-up path of the bounded waits, exercised without disturbing any real kernel: one thread waits, with the
+// production wait routine but only `polls` polls, on an mbarrier that nothing ever arrives on, then records the failure
+// in the plan's status word exactly as the dense kernels do, and returns normally.
+__global__ void bounded_wait_probe_kernel(int* dev_status, int polls) {
+    __shared__ __align__(8) uint64_t bar;
+    if (threadIdx.x == 0) {
+        mb_init(s32(&bar), 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        const bool ok = mb_wait_polls(s32(&bar), 0, polls);
+        if (!ok) atomicExch(dev_status, 1);
+    }
+}
+
+cudaError_t launch_bounded_wait_probe(const DevPlan& p, int polls, cudaStream_t stream) {
+    bounded_wait_probe_kernel<<<1, 32, 0, stream>>>(p.dev_status, polls);
+    return cudaGetLastError();
 }
 
 bool dense2_path_supported(const DevPlan& p, int C) {

@@ -43,6 +43,7 @@ _vp, _i, _d, _sz = ctypes.c_void_p, ctypes.c_int, ctypes.c_double, ctypes.c_size
 _SIGNATURES = {
     "sna_plan_create": (_i, [_i, _i, _i, _i, _i, _i, _d, ctypes.POINTER(_vp)]),
     "sna_plan_create_host_only": (_i, [_i, _i, _i, _i, _i, _i, _d, ctypes.POINTER(_vp)]),
+    "sna_debug_exercise_bounded_wait": (_i, [_vp, _i, _vp]),
     "sna_plan_create_global": (_i, [_i, _i, _i, _i, _i, _i, ctypes.POINTER(_vp)]),
     "sna_plan_destroy": (_i, [_vp]),
     "sna_plan_check": (_i, [_vp]),
@@ -121,6 +122,11 @@ def sna_plan_create_global(nlat_in, nlon_in, nlat_out, nlon_out, grid_in, grid_o
     handle = _vp()
     _check(_lib.sna_plan_create_global(nlat_in, nlon_in, nlat_out, nlon_out, grid_in, grid_out, ctypes.byref(handle)))
     return handle.value
+
+
+def sna_debug_exercise_bounded_wait(plan: int, polls: int = 1000, stream=None) -> None:
+    """Test aid: make one bounded wait run out on the GPU so that ``sna_plan_check`` has a failure to report."""
+    _check(_lib.sna_debug_exercise_bounded_wait(plan, polls, _stream(stream)))
 
 
 def sna_plan_create_host_only(nlat_in, nlon_in, nlat_out, nlon_out, grid_in, grid_out, theta_cutoff) -> int:

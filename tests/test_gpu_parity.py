@@ -251,6 +251,28 @@ def test_global_plan_against_oracle(shape, reuse):
         assert not dk.reshape(wl.N, nlat_in, -1)[:, 0].any() and not dv.reshape(wl.N, nlat_in, -1)[:, 0].any()
 
 
+def test_a_bounded_wait_that_runs_out_is_reported_once_and_the_plan_stays_usable():
+    """The failure path of the bounded waits, without faulting or hanging anything: a probe kernel waits 1000 polls
+    on a barrier nobody arrives on, gives up, records it; the check reports it once; compute calls still work."""
+    wl = SMALL[0]
+    g = _geometry(wl)
+    q, k, v, dout = make_inputs(wl)
+    ref = orc.forward(g, q, k, v)
+    with _plan(wl) as plan:
+        sna.sna_plan_check(plan.handle)                          # clean to begin with
+        sna.sna_debug_exercise_bounded_wait(plan.handle, 1000)
+        with pytest.raises(sna.SnaError) as e:
+            sna.sna_plan_check(plan.handle)
+        assert e.value.status == sna.SNA_ERR_CUDA and "bounded wait" in str(e.value)
+        sna.sna_plan_check(plan.handle)                          # reported once, then clear again
+        out = plan.forward(*_dev(q, k, v))
+        torch.cuda.synchronize()
+        sna.sna_plan_check(plan.handle)
+        assert nerr(out.cpu().numpy().reshape(ref.shape), ref) <= FWD_TOL
+        with pytest.raises(sna.SnaError):
+            sna.sna_debug_exercise_bounded_wait(plan.handle, 0)  # refused on the host
+
+
 def test_results_are_reproducible_bit_for_bit():
     wl = SMALL[2]
     q, k, v, dout = make_inputs(wl)
