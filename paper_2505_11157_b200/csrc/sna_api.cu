@@ -102,6 +102,11 @@ const char* sna_status_string(sna_status_t s) {
 
 const char* sna_last_error_message(void) { return g_last_error; }
 
+// Measured on the benchmark configurations (fwd+bwd, against whole rings only): 128 gives -4 % at 361x720, -1.5 % at
+// 128x256 and -0.7 % on the 2:1 down-sampling case; 96 and below lose, because a masked 128-row block uses at most
+// W / (ps * 127 + W) of its entries.
+constexpr int DENSE_MIN_WIDTH = 128;
+
 static sna_status_t plan_create(int nlat_in, int nlon_in, int nlat_out, int nlon_out, sna_grid_t grid_in,
                                 sna_grid_t grid_out, double theta_cutoff, bool upload, sna_plan_t** plan_out,
                                 bool global = false) {
@@ -151,9 +156,12 @@ static sna_status_t plan_create(int nlat_in, int nlon_in, int nlat_out, int nlon
 #endif
     bool t_consecutive = false;
     plan->is_global = global;
+    // Windows at least this many input columns wide (and whole rings) run on the dense tcgen05 kernels, as masked blocks;
+    // narrower ones stay on the band kernels, whose 8-column tiles waste less on a slanted band.
+    const int dense_min_width = DENSE_MIN_WIDTH;
     try {
-        sna::build_dense_lists(hp, dense);
-        sna::build_transposed_dense_lists(hp, t_dense);
+        sna::build_dense_lists(hp, dense, dense_min_width);
+        sna::build_transposed_dense_lists(hp, t_dense, dense_min_width);
         // rows with the most whole rings first: the dense kernels run one block per SM, so the long tiles must not start last
         std::stable_sort(dense.rows.begin(), dense.rows.end(), [&](int a, int b) { return dense.ptr[a + 1] - dense.ptr[a] > dense.ptr[b + 1] - dense.ptr[b]; });
         std::stable_sort(t_dense.rows.begin(), t_dense.rows.end(), [&](int a, int b) { return t_dense.ptr[a + 1] - t_dense.ptr[a] > t_dense.ptr[b + 1] - t_dense.ptr[b]; });
@@ -172,7 +180,7 @@ static sna_status_t plan_create(int nlat_in, int nlon_in, int nlat_out, int nlon
         } else {
         sna::build_forward_stream(hp, fwd_stream);
         t_consecutive = sna::build_transposed_stream(hp, t_stream);
-        sna::build_forward_stream(hp, fwdb_stream, /*include_whole=*/false);
+        sna::build_forward_stream(hp, fwdb_stream, dense_min_width);
         grpb_order.resize(fwdb_stream.chunk_ptr.size() - 1);
         std::iota(grpb_order.begin(), grpb_order.end(), 0);
         std::stable_sort(grpb_order.begin(), grpb_order.end(), [&](int a, int b) {
@@ -184,7 +192,7 @@ static sna_status_t plan_create(int nlat_in, int nlon_in, int nlat_out, int nlon
         std::stable_sort(grp_order.begin(), grp_order.end(), [&](int a, int b) {
             return fwd_stream.chunk_ptr[a + 1] - fwd_stream.chunk_ptr[a] > fwd_stream.chunk_ptr[b + 1] - fwd_stream.chunk_ptr[b];
         });
-        sna::build_transposed_stream(hp, tb_stream, /*include_whole=*/false);
+        sna::build_transposed_stream(hp, tb_stream, dense_min_width);
         }
         const int rows_per_group = t_consecutive ? 1 : hp.ps;
         tb_grp_order.resize((tb_stream.chunk_ptr.size() - 1) / rows_per_group);
@@ -220,7 +228,8 @@ static sna_status_t plan_create(int nlat_in, int nlon_in, int nlat_out, int nlon
         {dense.lat.data(), dense.lat.size() * 4, 0}, {dense.rows.data(), dense.rows.size() * 4, 0}, {zero_status, sizeof(zero_status), 0},
         {tb_stream.entries.data(), tb_stream.entries.size() * 16, 0}, {tb_stream.chunk_ptr.data(), tb_stream.chunk_ptr.size() * 4, 0},
         {tb_grp_order.data(), tb_grp_order.size() * 4, 0}, {t_dense.ptr.data(), t_dense.ptr.size() * 4, 0},
-        {t_dense.lat.data(), t_dense.lat.size() * 4, 0}, {t_dense.rows.data(), t_dense.rows.size() * 4, 0}};
+        {t_dense.lat.data(), t_dense.lat.size() * 4, 0}, {t_dense.rows.data(), t_dense.rows.size() * 4, 0},
+        {dense.m.data(), dense.m.size() * 4, 0}, {t_dense.m.data(), t_dense.m.size() * 4, 0}};
     size_t total = 0;
     for (Piece& p : pieces) { p.offset = total; total += round256(p.bytes); }
     cudaError_t e = cudaGetDevice(&plan->device);
@@ -245,19 +254,15 @@ static sna_status_t plan_create(int nlat_in, int nlon_in, int nlat_out, int nlon
     d.fwdb_stream = (const int4*)at(15); d.fwdb_chunk_ptr = at(16); d.grpb_order = at(17);
     d.dense_ptr = at(18); d.dense_lat = at(19); d.dense_rows = at(20);
     d.n_dense_rows = (int)dense.rows.size();
-    {
-        size_t whole = 0;
-        for (const sna::StreamEntry& en : fwd_stream.entries) whole += en.base < 0;
-        d.dense_fraction = global ? 1.f : fwd_stream.entries.empty() ? 0.f : (float)whole / (float)fwd_stream.entries.size();
-    }
+    d.dense_fraction = hp.nnz > 0 ? (float)((double)dense.pairs / (double)hp.nnz) : 0.f;
     d.is_global = global ? 1 : 0;
     d.dev_status = (int*)((char*)plan->dev_blob + pieces[21].offset);
     d.tb_stream = (const int4*)at(22); d.tb_chunk_ptr = at(23); d.tb_grp_order = at(24);
     d.t_dense_ptr = at(25); d.t_dense_lat = at(26); d.t_dense_rows = at(27);
     d.n_t_dense_rows = (int)t_dense.rows.size();
+    d.dense_m = at(28); d.t_dense_m = at(29);
     // opt in to the kernels' dynamic shared-memory sizes on this device (once here instead of on every launch)
     e = sna::dense2_prepare_device();
-    if (e == cudaSuccess) e = sna::dense_prepare_device();
     if (e == cudaSuccess) e = sna::mma_prepare_device();
     if (e != cudaSuccess) { sna_plan_destroy(plan); return cuda_fail(e, "cudaFuncSetAttribute"); }
     *plan_out = plan;
@@ -388,7 +393,7 @@ size_t sna_workspace_bytes(const sna_plan_t* plan, int B, int H, int C) {
 int sna_forward_kernel_count(const sna_plan_t* plan, int C, int with_lse) {
     if (plan == nullptr || plan->dev_blob == nullptr || !supported_C(C)) return 0;
     if (plan->is_global) return 1;
-    return (with_lse && sna::dense_path_supported(plan->dev, C)) ? 2 : 1;
+    return (with_lse && sna::dense2_path_supported(plan->dev, C)) ? 2 : 1;
 }
 
 sna_status_t sna_forward_ex(const sna_plan_t* plan, const float* q, const float* k, const float* v, float* out,
@@ -403,11 +408,9 @@ sna_status_t sna_forward_ex(const sna_plan_t* plan, const float* q, const float*
         e = (lse != nullptr && sna::dense2_global_supported(plan->dev, C))
                 ? sna::launch_forward_dense2(plan->dev, q, k, v, out, lse, B * H, C, (cudaStream_t)cuda_stream)
                 : sna::launch_forward_generic(plan->dev, q, k, v, out, lse, B * H, C, (cudaStream_t)cuda_stream);
-    } else if (lse != nullptr && sna::dense_path_supported(plan->dev, C)) {
+    } else if (lse != nullptr && sna::dense2_path_supported(plan->dev, C)) {
         // whole-ring windows on the tcgen05 kernel (its partial result travels in out / lse), the rest on the band kernel
-        e = sna::dense2_path_supported(plan->dev, C)
-                ? sna::launch_forward_dense2(plan->dev, q, k, v, out, lse, B * H, C, (cudaStream_t)cuda_stream)
-                : sna::launch_forward_dense(plan->dev, q, k, v, out, lse, B * H, C, (cudaStream_t)cuda_stream);
+        e = sna::launch_forward_dense2(plan->dev, q, k, v, out, lse, B * H, C, (cudaStream_t)cuda_stream);
         if (e == cudaSuccess) e = sna::launch_forward_mma_band(plan->dev, q, k, v, out, lse, B * H, C, (cudaStream_t)cuda_stream);
     } else if (sna::mma_path_supported(plan->dev, C)) {
         e = sna::launch_forward_mma(plan->dev, q, k, v, out, lse, B * H, C, (cudaStream_t)cuda_stream);
@@ -437,11 +440,9 @@ sna_status_t sna_backward_dq(const sna_plan_t* plan, const float* q, const float
         e = (out != nullptr && out != dq && sna::dense2_global_supported(plan->dev, C))
                 ? sna::launch_backward_dq_dense2(plan->dev, q, k, v, dout, out, lse, dq, D, B * H, C, (cudaStream_t)cuda_stream)
                 : sna::launch_backward_dq_generic(plan->dev, q, k, v, dout, out, lse, dq, D, B * H, C, (cudaStream_t)cuda_stream);
-    } else if (out != nullptr && out != dq && plan->dev.dense_fraction >= 0.10f && sna::dense_path_supported(plan->dev, C)) {
+    } else if (out != nullptr && out != dq && plan->dev.dense_fraction >= 0.10f && sna::dense2_path_supported(plan->dev, C)) {
         // whole-ring windows on the tcgen05 kernel (its part of dq is written first), the banded rest is added by the band kernel
-        e = sna::dense2_path_supported(plan->dev, C)
-                ? sna::launch_backward_dq_dense2(plan->dev, q, k, v, dout, out, lse, dq, nullptr, B * H, C, (cudaStream_t)cuda_stream)
-                : sna::launch_backward_dq_dense(plan->dev, q, k, v, dout, out, lse, dq, B * H, C, (cudaStream_t)cuda_stream);
+        e = sna::launch_backward_dq_dense2(plan->dev, q, k, v, dout, out, lse, dq, nullptr, B * H, C, (cudaStream_t)cuda_stream);
         if (e == cudaSuccess) e = sna::launch_backward_dq_mma_band(plan->dev, q, k, v, dout, out, lse, dq, D, B * H, C, (cudaStream_t)cuda_stream);
     } else if (out != nullptr && sna::mma_path_supported(plan->dev, C)) {
         e = sna::launch_backward_dq_mma(plan->dev, q, k, v, dout, out, lse, dq, D, B * H, C, (cudaStream_t)cuda_stream);
@@ -473,11 +474,9 @@ sna_status_t sna_backward_dkdv(const sna_plan_t* plan, const float* q, const flo
         e = dense
                 ? sna::launch_backward_dkdv_dense2(plan->dev, q, k, v, dout, lse, D, dk, dv, B * H, C, (cudaStream_t)cuda_stream)
                 : sna::launch_backward_dkdv_generic(plan->dev, q, k, v, dout, lse, D, dk, dv, B * H, C, (cudaStream_t)cuda_stream);
-    } else if (plan->dev.dense_fraction >= 0.10f && plan->dev.n_t_dense_rows > 0 && sna::dense_path_supported(plan->dev, C)) {
+    } else if (plan->dev.dense_fraction >= 0.10f && plan->dev.n_t_dense_rows > 0 && sna::dense2_path_supported(plan->dev, C)) {
         // whole-ring partners on the tcgen05 kernel (its part of dk, dv is written first), the band kernel adds the rest
-        e = sna::dense2_path_supported(plan->dev, C)
-                ? sna::launch_backward_dkdv_dense2(plan->dev, q, k, v, dout, lse, D, dk, dv, B * H, C, (cudaStream_t)cuda_stream)
-                : sna::launch_backward_dkdv_dense(plan->dev, q, k, v, dout, lse, D, dk, dv, B * H, C, (cudaStream_t)cuda_stream);
+        e = sna::launch_backward_dkdv_dense2(plan->dev, q, k, v, dout, lse, D, dk, dv, B * H, C, (cudaStream_t)cuda_stream);
         if (e == cudaSuccess) e = sna::launch_backward_dkdv_mma_band(plan->dev, q, k, v, dout, lse, D, dk, dv, B * H, C, (cudaStream_t)cuda_stream);
     } else if (sna::mma_path_supported(plan->dev, C)) {
         e = sna::launch_backward_dkdv_mma(plan->dev, q, k, v, dout, lse, D, dk, dv, B * H, C, (cudaStream_t)cuda_stream);

@@ -27,8 +27,9 @@ struct DevPlan {
     const int4* fwdb_stream;
     const int32_t* fwdb_chunk_ptr;
     const int32_t* grpb_order;
-    const int32_t* dense_ptr;       // [nlat_out+1] whole-ring windows per output latitude
+    const int32_t* dense_ptr;       // [nlat_out+1] the dense kernels' windows per output latitude
     const int32_t* dense_lat;       // their input rings
+    const int32_t* dense_m;         // their half widths in input columns, -1 = whole ring
     const int32_t* dense_rows;      // output latitudes with at least one whole-ring window
     int n_dense_rows;
     // the same for the transposed side (dk/dv): band-only transposed stream and, per input latitude, the output rings
@@ -38,9 +39,10 @@ struct DevPlan {
     const int32_t* tb_grp_order;
     const int32_t* t_dense_ptr;     // [nlat_in+1]
     const int32_t* t_dense_lat;     // output rings
+    const int32_t* t_dense_m;       // half widths in input columns, -1 = whole ring
     const int32_t* t_dense_rows;    // input latitudes with at least one such output ring
     int n_t_dense_rows;
-    float dense_fraction;           // share of the full forward stream's columns that belong to whole-ring windows
+    float dense_fraction;           // share of the table's entries that the dense kernels' windows cover
     int* dev_status;                // set to non-zero by a kernel whose bounded wait ran out
     const int4* t_stream;
     const int32_t* t_chunk_ptr;     // [groups of input latitudes * ps + 1]
@@ -61,34 +63,26 @@ cudaError_t launch_backward_dkdv_mma_lp(const DevPlan& p, const float* q, const 
                                         const float* lse, const float* Dws, float* dk, float* dv, int N, int C, cudaStream_t stream);
 cudaError_t launch_forward_mma(const DevPlan& p, const float* q, const float* k, const float* v, float* out, float* lse,
                                int N, int C, cudaStream_t stream);
-// Dense (tcgen05) forward over the whole-ring windows only: writes the partial result (normalised out, lse) of the
-// output latitudes in p.dense_rows; launch_forward_mma_band then continues from it with the banded windows.
-// Both need lse != null.  dense_path_supported tells whether the pair may be used for this problem.
-cudaError_t dense_prepare_device();   // once per device: opt in to the kernels' shared-memory size
-bool dense_path_supported(const DevPlan& p, int C);
-cudaError_t launch_forward_dense(const DevPlan& p, const float* q, const float* k, const float* v, float* out, float* lse,
-                                 int N, int C, cudaStream_t stream);
-// Pipelined version of the dense forward kernel (TMA loads, warp-specialised, see sna_kernels_dense2.cu); same contract.
-cudaError_t dense2_prepare_device();   // once per device: opt in to the kernel's shared-memory size
+// Dense (tcgen05) kernels (sna_kernels_dense2.cu: TMA loads, warp-specialised, operands and accumulators in TMEM) for
+// the windows in the plan's dense lists: whole input rings, and wide banded windows as masked blocks.  The forward kernel
+// writes the partial result (normalised out, lse) of the output latitudes in p.dense_rows and launch_forward_mma_band
+// continues from it with the narrower windows; both need lse != null.  dense2_path_supported tells whether the pair may
+// be used for this problem.
+cudaError_t dense2_prepare_device();   // once per device: opt in to the kernels' shared-memory sizes
 bool dense2_path_supported(const DevPlan& p, int C);
 cudaError_t launch_bounded_wait_probe(const DevPlan& p, int polls, cudaStream_t stream);
 bool dense2_global_supported(const DevPlan& p, int C);   // the dense kernels can serve a global plan on their own
 cudaError_t launch_forward_dense2(const DevPlan& p, const float* q, const float* k, const float* v, float* out, float* lse,
                                   int N, int C, cudaStream_t stream);
-// Pipelined dense dq kernel; same contract as launch_backward_dq_dense, and it also writes D (Dws may be null).
+// The same split for the dq stage: the dense kernel writes its part of dq (out and dq must be different buffers) and,
+// if Dws != null, D; the band kernel adds the narrower windows' part.
 cudaError_t launch_backward_dq_dense2(const DevPlan& p, const float* q, const float* k, const float* v, const float* dout,
                                       const float* out, const float* lse, float* dq, float* Dws, int N, int C, cudaStream_t stream);
-// Pipelined dense dk/dv kernel; same contract as launch_backward_dkdv_dense.
+// And for dk/dv: the dense kernel writes its part for the input latitudes in p.t_dense_rows, the band kernel adds the rest.
 cudaError_t launch_backward_dkdv_dense2(const DevPlan& p, const float* q, const float* k, const float* v, const float* dout,
                                         const float* lse, const float* Dws, float* dk, float* dv, int N, int C, cudaStream_t stream);
-// The same split for the dq stage: the dense kernel writes the whole-ring part of dq (out and dq must be different
-// buffers), the band kernel adds its banded part to it.
-cudaError_t launch_backward_dq_dense(const DevPlan& p, const float* q, const float* k, const float* v, const float* dout,
-                                     const float* out, const float* lse, float* dq, int N, int C, cudaStream_t stream);
 cudaError_t launch_backward_dq_mma_band(const DevPlan& p, const float* q, const float* k, const float* v, const float* dout,
                                         const float* out, const float* lse, float* dq, float* Dws, int N, int C, cudaStream_t stream);
-cudaError_t launch_backward_dkdv_dense(const DevPlan& p, const float* q, const float* k, const float* v, const float* dout,
-                                       const float* lse, const float* Dws, float* dk, float* dv, int N, int C, cudaStream_t stream);
 cudaError_t launch_backward_dkdv_mma_band(const DevPlan& p, const float* q, const float* k, const float* v, const float* dout,
                                           const float* lse, const float* Dws, float* dk, float* dv, int N, int C, cudaStream_t stream);
 cudaError_t launch_forward_mma_band(const DevPlan& p, const float* q, const float* k, const float* v, float* out, float* lse,

@@ -1,10 +1,12 @@
-// Pipelined dense forward kernel for whole-ring windows on tcgen05 / TMEM (sm_100a, C = 32).
+// Dense kernels on tcgen05 / TMEM (sm_100a, C = 32) for whole-ring and wide windows.
 //
 // Near the poles, and in the global limit theta_cutoff = pi, an output ring attends to EVERY point of an input ring:
 // that part of Eq. (s2_attention_discrete_detailed) is a dense attention block with the additive bias log omega of
-// App. B.2.  One thread block owns 128 consecutive output longitudes of one ring (the M = 128 rows of the MMA) and walks
-// the ring's whole input rings in blocks of 128 columns.  Unlike the serial kernel in sna_kernels_dense.cu the work of a
-// block is spread over specialised warps that run concurrently, coupled only by mbarriers:
+// App. B.2.  A little further from the poles the windows are still hundreds of columns wide; they run here too, as the
+// blocks of the ring that the tile's windows touch, with the entries outside each row's own window masked (TileWalk).
+// One thread block owns 128 consecutive output longitudes of one ring (the M = 128 rows of the MMA) and walks its list of
+// partner rings in blocks of 128 columns.  The work of a block is spread over specialised warps that run concurrently,
+// coupled only by mbarriers:
 //
 //   warp 8 (one thread)  TMA: raw k and v tiles of the next blocks, 128 points x 128 bytes, 128-byte swizzle
 //   warps 16-19          convert: k_lo = k - trunc19(k) (same layout as the raw tile), and v transposed and split into
@@ -131,6 +133,67 @@ __device__ __forceinline__ void tm_st32(uint32_t addr, const uint32_t (&r)[32]) 
 }
 __device__ __forceinline__ int sw_off(int row, int c4) { return row * 128 + ((c4 ^ (row & 7)) << 4); }
 
+__device__ __forceinline__ int fdiv(int a, int b) { const int q = a / b; return (a % b != 0 && ((a < 0) != (b < 0))) ? q - 1 : q; }
+__device__ __forceinline__ int cdiv(int a, int b) { return -fdiv(-a, b); }
+
+// Walks the blocks of partner points a tile needs.  The tile's list names partner rings, each with a window half width m
+// in input columns (m < 0: the whole ring).  Partner points of a ring are addressed by an unwrapped index u (the point
+// u mod period): the tile's rows together need u in [cdiv(a_lo - m, d), fdiv(a_hi + m, d)], where [a_lo, a_hi] are the
+// centres of the first and last existing row and d converts input columns to partner points.  That range is cut where it
+// crosses the ring's seam and each piece is covered by blocks of `step` points from its start, so a block never wraps:
+// points of a block beyond the end of its piece (`seg_end`) either do not exist (TMA fills zeros) or belong to no row's
+// window, and the element-wise code masks them.  Every role of a kernel walks the same sequence.
+constexpr int M_WHOLE = 1 << 28;
+// which turn of the ring the unwrapped index u lies in; the walks stay within (-period, 2 period) because a banded
+// window is narrower than the ring
+__device__ __forceinline__ int turn_of(int u, int period) { return (u >= period ? 1 : 0) - (u < 0 ? 1 : 0); }
+struct TileWalk {
+    const int32_t* lat;
+    const int32_t* hw;
+    int e, e_end, period, step, a_lo, a_hi, d;
+    int ring, m, u, seg_end, uhi;        // current block: unwrapped start u, last wanted point of its piece seg_end
+    __device__ __forceinline__ void load_entry() {
+        if (e >= e_end) return;
+        ring = lat[e];
+        const int mm = hw[e];
+        if (mm < 0) { m = M_WHOLE; u = 0; uhi = period - 1; }
+        else if (d == 1) { m = mm; u = a_lo - mm; uhi = a_hi + mm; }
+        else { m = mm; u = cdiv(a_lo - mm, d); uhi = fdiv(a_hi + mm, d); }
+        seg_end = min(uhi, (turn_of(u, period) + 1) * period - 1);
+    }
+    __device__ __forceinline__ TileWalk(const int32_t* lat_, const int32_t* hw_, int e_begin, int e_end_, int period_, int step_,
+                                        int a_lo_, int a_hi_, int d_)
+        : lat(lat_), hw(hw_), e(e_begin), e_end(e_end_), period(period_), step(step_), a_lo(a_lo_), a_hi(a_hi_), d(d_),
+          ring(0), m(0), u(0), seg_end(-1), uhi(-1) { load_entry(); }
+    __device__ __forceinline__ int col() const { return u - turn_of(u, period) * period; }     // actual first point of the block
+    __device__ __forceinline__ void advance() {
+        u += step;
+        if (u > seg_end) {
+            u = seg_end + 1;                                  // a multiple of the period unless the ring is done
+            if (u > uhi) { ++e; load_entry(); }
+            else seg_end = min(uhi, u + period - 1);
+        }
+    }
+};
+// Number of blocks a TileWalk with the same arguments visits; called by one whole warp (entries spread over its lanes).
+__device__ __forceinline__ int tile_block_count(const int32_t* lat, const int32_t* hw, int e_begin, int e_end, int period, int step,
+                                                int a_lo, int a_hi, int d, int lane) {
+    int cnt = 0;
+    for (int e = e_begin + lane; e < e_end; e += 32) {
+        const int mm = hw[e];
+        int u = mm < 0 ? 0 : cdiv(a_lo - mm, d);
+        const int uhi = mm < 0 ? period - 1 : fdiv(a_hi + mm, d);
+        while (u <= uhi) {
+            const int se = min(uhi, (turn_of(u, period) + 1) * period - 1);
+            cnt += (se - u + step) / step;
+            u = se + 1;
+        }
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) cnt += __shfl_xor_sync(0xffffffffu, cnt, o);
+    return cnt;
+}
+
 __global__ void __launch_bounds__(THREADS2, 1)
 forward_dense2_kernel(DevPlan p, const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
                       const __grid_constant__ CUtensorMap map_v, float* __restrict__ out, float* __restrict__ lse, int N,
@@ -146,9 +209,14 @@ forward_dense2_kernel(DevPlan p, const __grid_constant__ CUtensorMap map_q, cons
     const int n = rest % N;
     const int h = p.dense_rows[rest / N];
     const int w0 = tile * M2;
-    const int nblk = (p.nlon_in + BN2 - 1) / BN2;
     const int e_begin = p.dense_ptr[h], e_end = p.dense_ptr[h + 1];
-    const int total = (e_end - e_begin) * nblk;
+    // the walk over this tile's blocks: centres of its first and last existing row, in input columns
+    const int a_lo = p.ps * w0, a_hi = p.ps * (min(w0 + M2, p.nlon_out) - 1);
+    __shared__ int total_s;
+    if (warp == 1) {
+        const int cnt = tile_block_count(p.dense_lat, p.dense_m, e_begin, e_end, p.nlon_in, BN2, a_lo, a_hi, 1, lane);
+        if (lane == 0) total_s = cnt;
+    }
 
     if (tid == 0) {
         for (int s = 0; s < 2; ++s) {
@@ -176,6 +244,7 @@ forward_dense2_kernel(DevPlan p, const __grid_constant__ CUtensorMap map_q, cons
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     const uint32_t tm = tmem_base_s;
     const uint32_t sbase = s32(base);
+    const int total = total_s;
     bool ok = true;
 
     if (warp < 8) {
@@ -191,6 +260,8 @@ forward_dense2_kernel(DevPlan p, const __grid_constant__ CUtensorMap map_q, cons
 #pragma unroll
         for (int i = 0; i < C2; ++i) o[i] = 0.f;
         float corr_prev = 1.f;
+        const int ctr = p.ps * w;                          // this row's window centre, in input columns
+        TileWalk wk(p.dense_lat, p.dense_m, e_begin, e_end, p.nlon_in, BN2, a_lo, a_hi, 1);
         for (int it = 0; it <= total && ok; ++it) {
             float corr = 1.f;
             if (it > 0) {
@@ -208,9 +279,13 @@ forward_dense2_kernel(DevPlan p, const __grid_constant__ CUtensorMap map_q, cons
             }
             if (it < total) {
                 const int b = it & 1, u = it >> 1;
-                const int hp = p.dense_lat[e_begin + it / nblk];
-                const float bias = p.log2_omega[hp];
-                const int nvalid = p.nlon_in - (it % nblk) * BN2 - half * HC;     // columns of this thread's half that exist
+                const float bias = p.log2_omega[wk.ring];
+                // the columns [jl, jh] of this thread's half that exist and lie in this row's window
+                int jl = max(0, ctr - wk.m - wk.u) - half * HC, jh = min(wk.seg_end - wk.u, ctr + wk.m - wk.u) - half * HC;
+                if (!row_ok || jh < jl || jh < 0 || jl >= HC) { jl = HC; jh = HC; }     // none
+                const uint32_t span = (uint32_t)(jh - jl);
+                const bool full = __all_sync(0xffffffffu, jl <= 0 && jh >= HC - 1);     // no masking anywhere in this warp
+                wk.advance();
                 ok = mb_wait(s32(&bars[B_SFULL + b]), u & 1, ok) && ok;
                 asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
                 const uint32_t tS = tm + (b ? T_S1 : T_S0) + half * HC + lanebits;
@@ -221,14 +296,14 @@ forward_dense2_kernel(DevPlan p, const __grid_constant__ CUtensorMap map_q, cons
                     tm_ld32_issue(sa, tS);
                     tm_ld32_issue(sb, tS + 32);
                     tm_ld_wait();
-                    if (nvalid >= HC) {
+                    if (full) {
 #pragma unroll
                         for (int j = 0; j < 32; ++j) mxr[j & 3] = fmaxf(mxr[j & 3], fmaxf(__uint_as_float(sa[j]), __uint_as_float(sb[j])));
                     } else {
 #pragma unroll
                         for (int j = 0; j < 32; ++j) {
-                            if (j < nvalid) mxr[j & 3] = fmaxf(mxr[j & 3], __uint_as_float(sa[j]));
-                            if (32 + j < nvalid) mxr[j & 3] = fmaxf(mxr[j & 3], __uint_as_float(sb[j]));
+                            if ((uint32_t)(j - jl) <= span) mxr[j & 3] = fmaxf(mxr[j & 3], __uint_as_float(sa[j]));
+                            if ((uint32_t)(32 + j - jl) <= span) mxr[j & 3] = fmaxf(mxr[j & 3], __uint_as_float(sb[j]));
                         }
                     }
                 }
@@ -247,7 +322,7 @@ forward_dense2_kernel(DevPlan p, const __grid_constant__ CUtensorMap map_q, cons
 #pragma unroll
                     for (int j = 0; j < 16; ++j) {
                         float pj = ex2f(fmaf(__uint_as_float(x[j]), scale_log2, nb));
-                        if (nvalid < HC && c0 + j >= nvalid) pj = 0.f;
+                        if (!full && (uint32_t)(c0 + j - jl) > span) pj = 0.f;
                         ps[j & 3] += pj;
                         x[j] = __float_as_uint(pj);
                         lo[j] = __float_as_uint(pj - trunc19f(pj));
@@ -284,7 +359,7 @@ forward_dense2_kernel(DevPlan p, const __grid_constant__ CUtensorMap map_q, cons
         if (half == 0 && ok && row_ok) {
             const float m1 = xs[C2 * 128 + r], l1 = xs[(C2 + 1) * 128 + r];
             const float mm = fmaxf(m, m1);
-            const float c0 = ex2f(m - mm), c1 = ex2f(m1 - mm);      // mm is finite: half 0 always has valid columns
+            const float c0 = ex2f(m - mm), c1 = ex2f(m1 - mm);      // mm is finite: every existing row has a column in its window
             const float lt = l * c0 + l1 * c1;
             const size_t opt = (size_t)(n * p.nlat_out + h) * p.nlon_out + w;
             const float inv = 1.f / lt;
@@ -304,10 +379,11 @@ forward_dense2_kernel(DevPlan p, const __grid_constant__ CUtensorMap map_q, cons
         if (warp == 8 && lane == 0) {
             mb_expect(s32(&bars[B_QFULL]), TILE_B);
             tma_tile(sbase + OFF_Q, &map_q, w0, n * p.nlat_out + h, s32(&bars[B_QFULL]));
-            for (int it = 0; it < total && ok; ++it) {
+            TileWalk wk(p.dense_lat, p.dense_m, e_begin, e_end, p.nlon_in, BN2, a_lo, a_hi, 1);
+            for (int it = 0; it < total && ok; ++it, wk.advance()) {
                 const int s = it & 1, u = it >> 1;
-                const int hp = p.dense_lat[e_begin + it / nblk];
-                const int c0 = (it % nblk) * BN2;
+                const int hp = wk.ring;
+                const int c0 = wk.col();
                 if (u > 0) {
                     ok = mb_wait(s32(&bars[B_KFREE + s]), (u - 1) & 1, ok);
                     ok = mb_wait(s32(&bars[B_VRAWFREE + s]), (u - 1) & 1, ok) && ok;
@@ -468,9 +544,13 @@ backward_dq_dense2_kernel(DevPlan p, const __grid_constant__ CUtensorMap map_k, 
     const int n = rest % N;
     const int h = p.dense_rows[rest / N];
     const int w0 = tile * M2;
-    const int nblk = (p.nlon_in + BNQ - 1) / BNQ;
     const int e_begin = p.dense_ptr[h], e_end = p.dense_ptr[h + 1];
-    const int total = (e_end - e_begin) * nblk;
+    const int a_lo = p.ps * w0, a_hi = p.ps * (min(w0 + M2, p.nlon_out) - 1);     // see the forward kernel
+    __shared__ int total_s;
+    if (warp == 1) {
+        const int cnt = tile_block_count(p.dense_lat, p.dense_m, e_begin, e_end, p.nlon_in, BNQ, a_lo, a_hi, 1, lane);
+        if (lane == 0) total_s = cnt;
+    }
     const float scale_log2 = scale * LOG2E_2;
 
     if (tid == 0) {
@@ -502,6 +582,7 @@ backward_dq_dense2_kernel(DevPlan p, const __grid_constant__ CUtensorMap map_k, 
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     const uint32_t tm = tmem_base_s;
     const uint32_t sbase = s32(base);
+    const int total = total_s;
     bool ok = true;
     PROF_DECL
 
@@ -556,12 +637,18 @@ backward_dq_dense2_kernel(DevPlan p, const __grid_constant__ CUtensorMap map_k, 
         float acc[C2];
 #pragma unroll
         for (int i = 0; i < C2; ++i) acc[i] = 0.f;
+        const int ctr = p.ps * w;                          // this row's window centre, in input columns
+        TileWalk wk(p.dense_lat, p.dense_m, e_begin, e_end, p.nlon_in, BNQ, a_lo, a_hi, 1);
         for (int it = 0; it <= total && ok; ++it) {
             if (it < total) {
                 const int b = it & 1, u = it >> 1;
-                const int hp = p.dense_lat[e_begin + it / nblk];
-                const float nbias = p.log2_omega[hp] + nl;
-                const int nvalid = p.nlon_in - (it % nblk) * BNQ - grp * GC;     // columns of this thread's half that exist
+                const float nbias = p.log2_omega[wk.ring] + nl;
+                // the columns [jl, jh] of this thread's half that exist and lie in this row's window
+                int jl = max(0, ctr - wk.m - wk.u) - grp * GC, jh = min(wk.seg_end - wk.u, ctr + wk.m - wk.u) - grp * GC;
+                if (!row_ok || jh < jl || jh < 0 || jl >= GC) { jl = GC; jh = GC; }     // none
+                const uint32_t span = (uint32_t)(jh - jl);
+                const bool full = __all_sync(0xffffffffu, jl <= 0 && jh >= GC - 1);     // no masking anywhere in this warp
+                wk.advance();
                 PROF_WAIT(0, ok = mb_wait(s32(&bars[Q_STFULL + b]), u & 1, ok) && ok);
                 asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
                 const uint32_t tS = tm + TQ_BUF + 128 * b + grp * GC + lanebits, tT = tS + BNQ;
@@ -572,7 +659,7 @@ backward_dq_dense2_kernel(DevPlan p, const __grid_constant__ CUtensorMap map_k, 
 #pragma unroll
                 for (int j = 0; j < 32; ++j) {
                     float pj = ex2f(fmaf(__uint_as_float(sv[j]), scale_log2, nbias));
-                    if (nvalid < GC && j >= nvalid) pj = 0.f;
+                    if (!full && (uint32_t)(j - jl) > span) pj = 0.f;
                     const float ds = pj * (__uint_as_float(tv[j]) - D);
                     sv[j] = __float_as_uint(ds);                       // dS over S
                     tv[j] = __float_as_uint(ds - trunc19f(ds));        // dS_lo over T
@@ -620,10 +707,11 @@ backward_dq_dense2_kernel(DevPlan p, const __grid_constant__ CUtensorMap map_k, 
         asm volatile("setmaxnreg.dec.sync.aligned.u32 48;");
         if (warp == 8 && lane == 0) {
             // -------------------------------------------------------------- TMA producer
-            for (int it = 0; it < total && ok; ++it) {
+            TileWalk wk(p.dense_lat, p.dense_m, e_begin, e_end, p.nlon_in, BNQ, a_lo, a_hi, 1);
+            for (int it = 0; it < total && ok; ++it, wk.advance()) {
                 const int s = it % NSQ, u = it / NSQ;
-                const int hp = p.dense_lat[e_begin + it / nblk];
-                const int c0 = (it % nblk) * BNQ;
+                const int hp = wk.ring;
+                const int c0 = wk.col();
                 if (u > 0) {   // the stage is free once both first GEMMs and all four dS K issuers of block it-NSQ are done
                     PROF_WAIT(0, ok = mb_wait(s32(&bars[Q_KSFREE + s]), (u - 1) & 1, ok));
                     PROF_WAIT(1, ok = mb_wait(s32(&bars[Q_VFREE + s]), (u - 1) & 1, ok) && ok);
@@ -783,9 +871,15 @@ backward_dkdv_dense2_kernel(DevPlan p, const __grid_constant__ CUtensorMap map_q
     const int n = rest % N;
     const int hp = p.t_dense_rows[rest / N];
     const int c0 = tile * M2;
-    const int nblk = (p.nlon_out + BNK - 1) / BNK;
     const int e_begin = p.t_dense_ptr[hp], e_end = p.t_dense_ptr[hp + 1];
-    const int total = (e_end - e_begin) * nblk;
+    // the walk over this tile's blocks of output points: rows are the input columns [a_lo, a_hi]; output point w is a
+    // partner of column c iff |ps w - c| <= m, so the walk runs over w with d = ps
+    const int a_lo = c0, a_hi = min(c0 + M2, p.nlon_in) - 1;
+    __shared__ int total_s;
+    if (warp == 1) {
+        const int cnt = tile_block_count(p.t_dense_lat, p.t_dense_m, e_begin, e_end, p.nlon_out, BNK, a_lo, a_hi, p.ps, lane);
+        if (lane == 0) total_s = cnt;
+    }
     const float scale_log2 = scale * LOG2E_2;
 
     if (tid == 0) {
@@ -814,6 +908,7 @@ backward_dkdv_dense2_kernel(DevPlan p, const __grid_constant__ CUtensorMap map_q
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     const uint32_t tm = tmem_base_s;
     const uint32_t sbase = s32(base);
+    const int total = total_s;
     bool ok = true;
     PROF_DECL
 
@@ -857,6 +952,8 @@ backward_dkdv_dense2_kernel(DevPlan p, const __grid_constant__ CUtensorMap map_q
         float gk[C2], gv[C2];
 #pragma unroll
         for (int i = 0; i < C2; ++i) { gk[i] = 0.f; gv[i] = 0.f; }
+        TileWalk wk(p.t_dense_lat, p.t_dense_m, e_begin, e_end, p.nlon_out, BNK, a_lo, a_hi, p.ps);
+        const int ps_shift = (p.ps & (p.ps - 1)) == 0 ? 31 - __clz(p.ps) : -1;      // ps a power of two: divide by shifting
         for (int it = 0; it <= total && ok; ++it) {
             if (it > 0 && (it % FOLDK == 0 || it == total)) {
                 // fold the second GEMMs of the blocks since the last fold; this also frees the accumulators
@@ -871,7 +968,14 @@ backward_dkdv_dense2_kernel(DevPlan p, const __grid_constant__ CUtensorMap map_q
             }
             if (it < total) {
                 const int s = it % NSK;
-                const int nvalid = p.nlon_out - (it % nblk) * BNK - grp * GC;     // partner columns of this thread's half that exist
+                // the partner columns [jl, jh] of this thread's half that exist and have this row's input point in their window
+                const int wl = ps_shift >= 0 ? -((wk.m - c) >> ps_shift) : cdiv(c - wk.m, p.ps);      // ceil((c - m) / ps)
+                const int wh = ps_shift >= 0 ? (c + wk.m) >> ps_shift : fdiv(c + wk.m, p.ps);         // floor((c + m) / ps)
+                int jl = max(0, wl - wk.u) - grp * GC, jh = min(wk.seg_end - wk.u, wh - wk.u) - grp * GC;
+                if (!row_ok || jh < jl || jh < 0 || jl >= GC) { jl = GC; jh = GC; }     // none
+                const uint32_t span = (uint32_t)(jh - jl);
+                const bool full = __all_sync(0xffffffffu, jl <= 0 && jh >= GC - 1);     // no masking anywhere in this warp
+                wk.advance();
                 PROF_WAIT(0, ok = mb_wait(s32(&bars[K_STFULL]), it & 1, ok) && ok);     // implies QCONV of this stage (the S issuer waited for it)
                 asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
                 const float* nlc = reinterpret_cast<const float*>(base + s * KST + 8 * TILE_K) + grp * GC;
@@ -888,7 +992,7 @@ backward_dkdv_dense2_kernel(DevPlan p, const __grid_constant__ CUtensorMap map_q
                     for (int j = 0; j < 16; ++j) {
                         const int col = hf * 16 + j;
                         float pj = ex2f(fmaf(__uint_as_float(sv[j]), scale_log2, nlc[col]));
-                        if (nvalid < GC && col >= nvalid) pj = 0.f;
+                        if (!full && (uint32_t)(col - jl) > span) pj = 0.f;
                         const float ds = pj * (__uint_as_float(tv[j]) - Dc[col]);
                         sv[j] = __float_as_uint(pj);
                         tv[j] = __float_as_uint(ds);
@@ -931,10 +1035,11 @@ backward_dkdv_dense2_kernel(DevPlan p, const __grid_constant__ CUtensorMap map_q
         asm volatile("setmaxnreg.dec.sync.aligned.u32 40;");
         if (warp == 8 && lane == 0) {
             // -------------------------------------------------------------- TMA producer: q and dout blocks of the partner rings
-            for (int it = 0; it < total && ok; ++it) {
+            TileWalk wk(p.t_dense_lat, p.t_dense_m, e_begin, e_end, p.nlon_out, BNK, a_lo, a_hi, p.ps);
+            for (int it = 0; it < total && ok; ++it, wk.advance()) {
                 const int s = it % NSK, u = it / NSK;
-                const int h = p.t_dense_lat[e_begin + it / nblk];
-                const int w0 = (it % nblk) * BNK;
+                const int h = wk.ring;
+                const int w0 = wk.col();
                 if (u > 0) PROF_WAIT(0, ok = mb_wait(s32(&bars[K_FREE + s]), (u - 1) & 1, ok));
                 mb_expect(s32(&bars[K_QFULL + s]), TILE_K);
                 tma_tile(sbase + s * KST, &map_q, w0, n * p.nlat_out + h, s32(&bars[K_QFULL + s]));
@@ -1026,11 +1131,12 @@ backward_dkdv_dense2_kernel(DevPlan p, const __grid_constant__ CUtensorMap map_q
                 *reinterpret_cast<float4*>(t + TILE_K + sw_off(lane, chunk)) = make_float4(lw[0], lw[1], lw[2], lw[3]);
             }
         };
-        for (int it = 0; it < total && ok; ++it) {
+        TileWalk wk(p.t_dense_lat, p.t_dense_m, e_begin, e_end, p.nlon_out, BNK, a_lo, a_hi, p.ps);
+        for (int it = 0; it < total && ok; ++it, wk.advance()) {
             const int s = it % NSK, u = it / NSK;
             unsigned char* st = base + s * KST;
-            const int h = p.t_dense_lat[e_begin + it / nblk];
-            const int w0 = (it % nblk) * BNK;
+            const int h = wk.ring;
+            const int w0 = wk.col();
             PROF_WAIT(0, ok = mb_wait(s32(&bars[K_QFULL + s]), u & 1, ok));       // also: the stage (and its statistics arrays) is free
             if (ct < BNK) {
                 const size_t o = (size_t)(n * p.nlat_out + h) * p.nlon_out + min(w0 + ct, p.nlon_out - 1);
@@ -1111,7 +1217,8 @@ cudaError_t launch_bounded_wait_probe(const DevPlan& p, int polls, cudaStream_t 
 }
 
 bool dense2_path_supported(const DevPlan& p, int C) {
-    return dense_path_supported(p, C) && encode_fn2() != nullptr;
+    return C == C2 && p.dense_ptr != nullptr && p.n_dense_rows > 0 && p.fwdb_stream != nullptr && mma_path_supported(p, C) &&
+           encode_fn2() != nullptr;
 }
 
 bool dense2_global_supported(const DevPlan& p, int C) {

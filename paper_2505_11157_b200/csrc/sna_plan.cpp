@@ -303,31 +303,37 @@ void merge_group(const std::vector<int32_t>& ptr, const std::vector<RingWindow>&
 
 }  // namespace
 
-void build_dense_lists(const HostPlan& P, DenseLists& D) {
+void build_dense_lists(const HostPlan& P, DenseLists& D, int dense_min_width) {
+    D = DenseLists();
     D.ptr.assign(P.nlat_out + 1, 0);
-    D.lat.clear();
-    D.rows.clear();
     for (int h = 0; h < P.nlat_out; ++h) {
-        for (int e = P.row_ptr[h]; e < P.row_ptr[h + 1]; ++e)
-            if (P.windows[e].m < 0) D.lat.push_back(P.windows[e].lat);
+        for (int e = P.row_ptr[h]; e < P.row_ptr[h + 1]; ++e) {
+            if (!served_by_dense(P.windows[e], dense_min_width)) continue;
+            D.lat.push_back(P.windows[e].lat);
+            D.m.push_back(P.windows[e].m);
+            D.pairs += P.window_count(P.windows[e]);
+        }
         D.ptr[h + 1] = (int32_t)D.lat.size();
         if (D.ptr[h + 1] > D.ptr[h]) D.rows.push_back(h);
     }
 }
 
-void build_transposed_dense_lists(const HostPlan& P, DenseLists& D) {
+void build_transposed_dense_lists(const HostPlan& P, DenseLists& D, int dense_min_width) {
+    D = DenseLists();
     D.ptr.assign(P.nlat_in + 1, 0);
-    D.lat.clear();
-    D.rows.clear();
     for (int hp = 0; hp < P.nlat_in; ++hp) {
-        for (int e = P.t_row_ptr[hp]; e < P.t_row_ptr[hp + 1]; ++e)
-            if (P.t_windows[e].m < 0) D.lat.push_back(P.t_windows[e].lat);
+        for (int e = P.t_row_ptr[hp]; e < P.t_row_ptr[hp + 1]; ++e) {
+            if (!served_by_dense(P.t_windows[e], dense_min_width)) continue;
+            D.lat.push_back(P.t_windows[e].lat);
+            D.m.push_back(P.t_windows[e].m);
+            D.pairs += P.window_count(P.t_windows[e]);
+        }
         D.ptr[hp + 1] = (int32_t)D.lat.size();
         if (D.ptr[hp + 1] > D.ptr[hp]) D.rows.push_back(hp);
     }
 }
 
-void build_forward_stream(const HostPlan& P, Stream& S, bool include_whole) {
+void build_forward_stream(const HostPlan& P, Stream& S, int dense_min_width) {
     const int groups = (P.nlat_out + TILE_LAT - 1) / TILE_LAT;
     S.chunk_ptr.assign(groups + 1, 0);
     S.entries.clear();
@@ -339,7 +345,7 @@ void build_forward_stream(const HostPlan& P, Stream& S, bool include_whole) {
                 GroupRange rg[TILE_LAT];
                 for (int k = 0; k < TILE_LAT; ++k) {
                     if (m[k] == -2) continue;
-                    if (m[k] < 0 && !include_whole) continue;   // served by the dense kernel
+                    if (served_by_dense(RingWindow{lat, m[k]}, dense_min_width)) continue;
                     rg[k].present = true;
                     if (m[k] < 0) rg[k].whole = true;
                     else { rg[k].lo = ceil_div(-m[k] - r, P.ps); rg[k].hi = floor_div(m[k] - r, P.ps); }
@@ -352,7 +358,7 @@ void build_forward_stream(const HostPlan& P, Stream& S, bool include_whole) {
     }
 }
 
-bool build_transposed_stream(const HostPlan& P, Stream& S, bool include_whole) {
+bool build_transposed_stream(const HostPlan& P, Stream& S, int dense_min_width) {
     const int groups = (P.nlat_in + TILE_LAT - 1) / TILE_LAT;
     S.entries.clear();
     if (TILE_LON % P.ps == 0) {
@@ -367,7 +373,8 @@ bool build_transposed_stream(const HostPlan& P, Stream& S, bool include_whole) {
                 int lo = INT32_MAX, hi = INT32_MIN;
                 for (int k = 0; k < TILE_LAT; ++k) {
                     if (m[k] == -2) continue;
-                    if (m[k] < 0) { if (include_whole) whole_rows |= ((1u << TILE_LON) - 1u) << (k * TILE_LON); continue; }
+                    if (served_by_dense(RingWindow{lat, m[k]}, dense_min_width)) continue;
+                    if (m[k] < 0) { whole_rows |= ((1u << TILE_LON) - 1u) << (k * TILE_LON); continue; }
                     lo = std::min(lo, ceil_div(-m[k], P.ps));
                     hi = std::max(hi, floor_div(TILE_LON - 1 + m[k], P.ps));
                 }
@@ -377,7 +384,7 @@ bool build_transposed_stream(const HostPlan& P, Stream& S, bool include_whole) {
                 for (int e_rel = lo; e_rel <= hi; ++e_rel) {
                     uint32_t mask = 0;
                     for (int k = 0; k < TILE_LAT; ++k) {
-                        if (m[k] < 0) continue;   // absent (-2) or whole (-1, handled above)
+                        if (m[k] < 0 || served_by_dense(RingWindow{lat, m[k]}, dense_min_width)) continue;   // absent, whole (above) or dense
                         for (int i = 0; i < TILE_LON; ++i)
                             if (e_rel >= ceil_div(i - m[k], P.ps) && e_rel <= floor_div(i + m[k], P.ps)) mask |= 1u << (k * TILE_LON + i);
                     }
@@ -399,7 +406,7 @@ bool build_transposed_stream(const HostPlan& P, Stream& S, bool include_whole) {
                 GroupRange rg[TILE_LAT];
                 for (int k = 0; k < TILE_LAT; ++k) {
                     if (m[k] == -2) continue;
-                    if (m[k] < 0 && !include_whole) continue;   // served by the dense kernel
+                    if (served_by_dense(RingWindow{lat, m[k]}, dense_min_width)) continue;
                     rg[k].present = true;
                     if (m[k] < 0) rg[k].whole = true;
                     else { rg[k].lo = ceil_div(r - m[k], P.ps); rg[k].hi = floor_div(r + m[k], P.ps); }

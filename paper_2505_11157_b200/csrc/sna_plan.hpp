@@ -65,21 +65,29 @@ struct Stream {
 
 // Forward stream: one row per group of output latitudes (ceil(nlat_out / TILE_LAT) rows); partners are input
 // points, flat index base + u*ps.
-// With include_whole = false the columns of windows that cover a whole input ring are left out: those are
-// served by the dense kernel (see DenseLists), and the stream only carries the banded windows.
-void build_forward_stream(const HostPlan& plan, Stream& out, bool include_whole = true);
+// With dense_min_width > 0 the columns of the windows that served_by_dense() accepts are left out: those are served
+// by the dense kernels (see DenseLists), and the stream only carries the narrower windows.
+void build_forward_stream(const HostPlan& plan, Stream& out, int dense_min_width = 0);
 
-// Whole-ring windows per output latitude, for the dense (tcgen05) forward kernel: ring h attends to every point
-// of the input rings lat[ptr[h]] .. lat[ptr[h+1]-1].
+// Which windows the dense (tcgen05) kernels take: whole rings, and banded windows of at least dense_min_width input
+// columns (they run as masked blocks there).  dense_min_width = nlon_in + 1 selects the whole rings only.
+inline bool served_by_dense(const RingWindow& w, int dense_min_width) {
+    return dense_min_width > 0 && (w.m < 0 || 2 * w.m + 1 >= dense_min_width);
+}
+
+// The dense kernels' windows per output latitude: ring h attends to the input rings lat[ptr[h]] .. lat[ptr[h+1]-1],
+// to all of ring lat[e] if m[e] < 0, else to the columns within m[e] of its own.
 struct DenseLists {
     std::vector<int32_t> ptr;    // [nlat_out+1]
     std::vector<int32_t> lat;    // input rings
-    std::vector<int32_t> rows;   // output latitudes that have at least one whole-ring window
+    std::vector<int32_t> m;      // window half widths in input columns, -1 = whole ring
+    std::vector<int32_t> rows;   // output latitudes that have at least one such window
+    int64_t pairs = 0;           // table entries covered, per output longitude / input column
 };
-void build_dense_lists(const HostPlan& plan, DenseLists& out);
-// The transposed lists for the dense dk/dv kernel: input ring h' is attended to as a whole by the output rings
-// lat[ptr[h']] .. lat[ptr[h'+1]-1]; rows = input latitudes with at least one such output ring.
-void build_transposed_dense_lists(const HostPlan& plan, DenseLists& out);
+void build_dense_lists(const HostPlan& plan, DenseLists& out, int dense_min_width);
+// The transposed lists for the dense dk/dv kernel: input ring h' is attended to through such a window by the output
+// rings lat[ptr[h']] .. lat[ptr[h'+1]-1]; rows = input latitudes with at least one such output ring.
+void build_transposed_dense_lists(const HostPlan& plan, DenseLists& out, int dense_min_width);
 // Transposed stream for dk/dv; partners are output points (h, w).  Two layouts:
 //  - consecutive (when ps divides 8): one stream row per group of input latitudes; tile rows are 8 consecutive
 //    input columns c = c0 + i%8 (c0 a multiple of 8) and the partner index is c0/ps + e_rel.  Neighbouring
@@ -88,7 +96,7 @@ void build_transposed_dense_lists(const HostPlan& plan, DenseLists& out);
 //  - by residue (any other ps): one stream row per (group, residue r); tile rows are c = ps*(u0+i%8) + r and
 //    the partner index is u0 + e_rel.
 // Returns true for the consecutive layout.
-bool build_transposed_stream(const HostPlan& plan, Stream& out, bool include_whole = true);
+bool build_transposed_stream(const HostPlan& plan, Stream& out, int dense_min_width = 0);
 
 // Builds the plan.  On failure returns a status and fills `why`.
 PlanStatus build_plan(int nlat_in, int nlon_in, int nlat_out, int nlon_out, int grid_in, int grid_out,

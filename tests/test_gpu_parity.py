@@ -88,6 +88,11 @@ SMALL = [
     small_workload("trapezoid_c16", 12, 32, 12, 32, TZ, TZ, 0.6, 1, 2, 16, 46),
     small_workload("trapezoid_c12_generic", 12, 24, 12, 24, TZ, GL, 0.6, 1, 2, 12, 47),
     small_workload("trapezoid_global_c32", 12, 64, 12, 64, TZ, TZ, math.pi, 1, 2, 32, 48),
+    # windows of 128 columns and more that are not whole rings: masked blocks on the dense kernels, pieces across the seam
+    small_workload("wide_windows_c32", 24, 320, 24, 320, EQ, EQ, 0.55, 1, 1, 32, 49),
+    small_workload("wide_windows_down2_c32", 33, 384, 17, 192, EQ, EQ, 0.5, 1, 2, 32, 50),
+    small_workload("wide_windows_down4_gl_c32", 20, 640, 10, 160, GL, GL, 0.6, 1, 1, 32, 51),
+    small_workload("wide_windows_trapezoid_c32", 20, 300, 20, 300, TZ, TZ, 0.6, 2, 1, 32, 52),   # 300: ragged tiles and blocks
 ]
 
 
