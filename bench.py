@@ -215,10 +215,11 @@ def max_over_ranks(values, dist, device):
 class Problem:
     """Device tensors and the plan of one workload, plus one step (forward, dq, dk/dv) through the C ABI."""
 
-    def __init__(self, sna, torch, wl, keep_host=False):
+    def __init__(self, sna, torch, wl, keep_host=False, global_plan=False):
         from paper_2505_11157_b200.synthetic import make_inputs
         self.sna, self.torch, self.wl = sna, torch, wl
-        self.plan = sna.Plan(wl.nlat_in, wl.nlon_in, wl.nlat_out, wl.nlon_out, wl.grid_in, wl.grid_out, wl.theta_cutoff)
+        self.plan = sna.Plan(wl.nlat_in, wl.nlon_in, wl.nlat_out, wl.nlon_out, wl.grid_in, wl.grid_out, wl.theta_cutoff,
+                             global_attention=global_plan)
         self.pairs = self.plan.nnz * wl.nlon_out * wl.N
         self.units = self.pairs * wl.C                  # neighbor-pair-channels per step (forward and backward)
         host = [torch.from_numpy(a) for a in make_inputs(wl)]
@@ -441,6 +442,30 @@ def run_ours(args, wl):
                                            "ms_per_step": t["ms_per_step"], "frac": roof_ms / t["ms_per_step"],
                                            "note": "sna_forward_tf32 + sna_backward_tf32: one TF32 product per contraction, "
                                                    "tolerance 5e-3 instead of 1e-5 / 1e-4; not the headline"}}
+            # channels-first entry points on the same workload: the layout changes (HBM-bound transposes) run inside the calls
+            cf = lambda x: x.permute(0, 1, 4, 2, 3).reshape(x.shape[0], -1, x.shape[2], x.shape[3]).contiguous()
+            cf_in = [cf(x) for x in (prob.q, prob.k, prob.v, prob.dout)]
+            cf_out = [torch.empty_like(cf_in[0]), torch.empty_like(cf_in[0]), torch.empty_like(cf_in[1]), torch.empty_like(cf_in[1])]
+            state = torch.empty(sna.sna_cf_state_bytes(prob.plan.handle, wl.B, wl.H, C), dtype=torch.uint8, device="cuda")
+            scratch = torch.empty(sna.sna_cf_scratch_bytes(prob.plan.handle, wl.B, wl.H, C), dtype=torch.uint8, device="cuda")
+
+            def step_cf(marks=None):
+                sna.sna_forward_cf(prob.plan.handle, cf_in[0], cf_in[1], cf_in[2], cf_out[0], state, state.numel(), wl.B, wl.H, C, prob.stream)
+                if marks is not None:
+                    marks[1].record(prob.stream)
+                    marks[2].record(prob.stream)
+                sna.sna_backward_cf(prob.plan.handle, cf_in[3], state, state.numel(), scratch, scratch.numel(), cf_out[1], cf_out[2],
+                                    cf_out[3], wl.B, wl.H, C, prob.stream)
+
+            t = time_steps(torch, prob, 10, 3, step_cf, flush)
+            moved = 2 * 4 * sum(x.numel() for x in cf_in + cf_out)
+            result["variants"]["channels_first"] = {
+                "ms_forward": t["ms_forward"], "ms_backward": t["ms_backward_dkdv"], "ms_per_step": t["ms_per_step"],
+                "layout_bytes_per_step": moved, "layout_ms_at_hbm_peak": moved / (hbm_gbs * 1e6),
+                "note": "sna_forward_cf + sna_backward_cf on [B, H*C, nlat, nlon] tensors: eight tiled transposes per step around "
+                        "the same kernels (each element read once and written once)"}
+            del cf_in, cf_out, state, scratch
+            torch.cuda.empty_cache()
             step_prec()
             torch.cuda.synchronize()
             result["workloads"] = {wl.name: {"ms_forward": ms_fwd, "ms_backward_dq": ms_dq, "ms_backward_dkdv": ms_dkdv,
@@ -459,6 +484,17 @@ def run_ours(args, wl):
                 po.close()
                 del po
                 torch.cuda.empty_cache()
+            # the global limit once more through the plan that never builds per-pair structure (dense kernels only)
+            c5 = WORKLOADS["c5"]
+            pg = Problem(sna, torch, c5, global_plan=True)
+            t = time_steps(torch, pg, 10, 3, None, big_flush)
+            r_ms = sum(r["roofline_ms"] for r in kernel_rooflines(c5, pg.units, peak_tflops).values())
+            t.update({"roofline_ms": r_ms, "roofline_frac": r_ms / t["ms_per_step"], "l2": l2_policy(c5),
+                      "note": "c5 through sna_plan_create_global"})
+            result["workloads"]["c5_global_plan"] = t
+            pg.close()
+            del pg
+            torch.cuda.empty_cache()
         if not args.no_cpu_baseline and world == 1:
             from oracle import sna_oracle as orc
             g = orc.geometry(wl.nlat_in, wl.nlon_in, wl.nlat_out, wl.nlon_out, wl.grid_in, wl.grid_out, wl.theta_cutoff)

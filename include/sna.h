@@ -203,6 +203,28 @@ sna_status_t sna_backward_dkdv(const sna_plan_t* plan, const float* q, const flo
                                int B, int H, int C, void* cuda_stream);
 
 /*
+ * Channels-first entry points.  The paper states its tensors as B x C x H x W (App. B.3); with heads, tensor x_cf
+ * has the layout [B][H*C][nlat][nlon], i.e. channel c of head h of batch b is the plane (b*H + h)*C + c, while every
+ * other call of this header takes channels-last arrays [B][H][nlat][nlon][C].  These two calls change the layout on the
+ * GPU (tiled transposes, HBM-bound: each element read once and written once) around sna_forward_ex / sna_backward_ex:
+ *
+ *   sna_forward_cf   q_cf, k_cf, v_cf -> out_cf; leaves the channels-last q, k, v, out and lse in `state` (device,
+ *                    sna_cf_state_bytes, 256-byte aligned, caller-owned) for the backward pass;
+ *   sna_backward_cf  dout_cf and that state -> dq_cf, dk_cf, dv_cf; `scratch` (device, sna_cf_scratch_bytes, 256-byte
+ *                    aligned) is private to the call until its work on the stream has finished.
+ *
+ * B*H must not exceed 65535.  Neither call allocates.  Errors as for sna_forward_ex / sna_backward_ex, plus
+ * SNA_ERR_WORKSPACE for a state or scratch buffer that is too small.  The size queries return 0 for invalid arguments.
+ */
+size_t sna_cf_state_bytes(const sna_plan_t* plan, int B, int H, int C);
+size_t sna_cf_scratch_bytes(const sna_plan_t* plan, int B, int H, int C);
+sna_status_t sna_forward_cf(const sna_plan_t* plan, const float* q_cf, const float* k_cf, const float* v_cf, float* out_cf,
+                            void* state, size_t state_bytes, int B, int H, int C, void* cuda_stream);
+sna_status_t sna_backward_cf(const sna_plan_t* plan, const float* dout_cf, const void* state, size_t state_bytes,
+                             void* scratch, size_t scratch_bytes, float* dq_cf, float* dk_cf, float* dv_cf,
+                             int B, int H, int C, void* cuda_stream);
+
+/*
  * Reduced-precision variant of the forward and backward pass.  The paper lists "neither reduced precision nor tensor
  * core" support as a limitation of its kernels (Sec. 5, Limitations); here every contraction of
  * Eq. s2_attention_discrete_detailed and App. B.4 is taken as ONE TF32 tensor-core product (operands rounded to 11

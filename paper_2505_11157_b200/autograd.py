@@ -32,3 +32,24 @@ class _SphericalNeighborhoodAttention(torch.autograd.Function):
 def spherical_neighborhood_attention(plan: "sna.Plan", q: torch.Tensor, k: torch.Tensor, v: torch.Tensor) -> torch.Tensor:
     """out = NAttn_{S^2}[q, k, v] on the grids and cutoff of ``plan`` (differentiable in q, k, v)."""
     return _SphericalNeighborhoodAttention.apply(plan, q, k, v)
+
+
+class _SphericalNeighborhoodAttentionCF(torch.autograd.Function):
+    @staticmethod
+    def forward(ctx, plan: "sna.Plan", heads: int, q, k, v):
+        if q.dtype != torch.float32 or k.dtype != torch.float32 or v.dtype != torch.float32:
+            raise ValueError("spherical_neighborhood_attention_cf computes in float32: cast q, k, v first")
+        out, state = plan.forward_cf(q.contiguous(), k.contiguous(), v.contiguous(), heads)
+        ctx.plan, ctx.heads, ctx.state = plan, heads, state
+        return out
+
+    @staticmethod
+    def backward(ctx, dout):
+        dq, dk, dv = ctx.plan.backward_cf(dout.contiguous().float(), ctx.state, ctx.heads)
+        return None, None, dq, dk, dv
+
+
+def spherical_neighborhood_attention_cf(plan: "sna.Plan", q: torch.Tensor, k: torch.Tensor, v: torch.Tensor, heads: int = 1) -> torch.Tensor:
+    """The same operator on channels-first tensors [B, heads*C, nlat, nlon], as a 2D convolutional network carries
+    them; the layout change runs on the GPU inside the call (differentiable in q, k, v)."""
+    return _SphericalNeighborhoodAttentionCF.apply(plan, heads, q, k, v)

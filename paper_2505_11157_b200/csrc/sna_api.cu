@@ -560,6 +560,95 @@ sna_status_t sna_backward(const sna_plan_t* plan, const float* q, const float* k
     return sna_backward_ex(plan, q, k, v, dout, nullptr, nullptr, dq, dk, dv, ws, need, B, H, C, cuda_stream);
 }
 
+// ---- channels-first entry points --------------------------------------------------------------------------
+namespace {
+struct CfState { float *q, *k, *v, *out, *lse; };
+size_t in_elems(const sna_plan_t* plan, int B, int H, int C) { return (size_t)B * H * plan->host.nlat_in * plan->host.nlon_in * C; }
+size_t out_elems(const sna_plan_t* plan, int B, int H, int C) { return stats_elems(plan, B, H) * C; }
+CfState carve_state(const sna_plan_t* plan, void* state, int B, int H, int C) {
+    char* p = (char*)state;
+    CfState s;
+    s.q = (float*)p;   p += round256(out_elems(plan, B, H, C) * sizeof(float));
+    s.k = (float*)p;   p += round256(in_elems(plan, B, H, C) * sizeof(float));
+    s.v = (float*)p;   p += round256(in_elems(plan, B, H, C) * sizeof(float));
+    s.out = (float*)p; p += round256(out_elems(plan, B, H, C) * sizeof(float));
+    s.lse = (float*)p;
+    return s;
+}
+}  // namespace
+
+size_t sna_cf_state_bytes(const sna_plan_t* plan, int B, int H, int C) {
+    if (!plan || B <= 0 || H <= 0 || !supported_C(C)) return 0;
+    return 2 * round256(out_elems(plan, B, H, C) * sizeof(float)) + 2 * round256(in_elems(plan, B, H, C) * sizeof(float)) +
+           round256(stats_elems(plan, B, H) * sizeof(float));
+}
+
+size_t sna_cf_scratch_bytes(const sna_plan_t* plan, int B, int H, int C) {
+    if (!plan || B <= 0 || H <= 0 || !supported_C(C)) return 0;
+    return 2 * round256(out_elems(plan, B, H, C) * sizeof(float)) + 2 * round256(in_elems(plan, B, H, C) * sizeof(float)) +
+           sna_workspace_bytes(plan, B, H, C);
+}
+
+sna_status_t sna_forward_cf(const sna_plan_t* plan, const float* q_cf, const float* k_cf, const float* v_cf, float* out_cf,
+                            void* state, size_t state_bytes, int B, int H, int C, void* cuda_stream) {
+    sna_status_t st = check_problem(plan, B, H, C);
+    if (st != SNA_OK) return st;
+    if (!q_cf || !k_cf || !v_cf || !out_cf) { set_error("q, k, v and out must not be NULL"); return SNA_ERR_INVALID_ARG; }
+    if (!all_aligned(q_cf, k_cf, v_cf, out_cf)) { set_error("device pointers must be 16-byte aligned"); return SNA_ERR_INVALID_ARG; }
+    if (state == nullptr || (reinterpret_cast<uintptr_t>(state) & 255u)) { set_error("state must be non-NULL and 256-byte aligned"); return SNA_ERR_INVALID_ARG; }
+    if (state_bytes < sna_cf_state_bytes(plan, B, H, C)) { set_error("state too small: %zu < %zu bytes", state_bytes, sna_cf_state_bytes(plan, B, H, C)); return SNA_ERR_WORKSPACE; }
+    if ((long long)B * H > 65535) { set_error("the channels-first entry points take at most 65535 batch*head slices"); return SNA_ERR_UNSUPPORTED; }
+    cudaStream_t stream = (cudaStream_t)cuda_stream;
+    const CfState s = carve_state(plan, state, B, H, C);
+    const long long p_in = (long long)plan->host.nlat_in * plan->host.nlon_in, p_out = (long long)plan->host.nlat_out * plan->host.nlon_out;
+    cudaError_t e = sna::launch_cf_to_cl(q_cf, s.q, B * H, C, p_out, stream);
+    if (e == cudaSuccess) e = sna::launch_cf_to_cl(k_cf, s.k, B * H, C, p_in, stream);
+    if (e == cudaSuccess) e = sna::launch_cf_to_cl(v_cf, s.v, B * H, C, p_in, stream);
+    if (e != cudaSuccess) return cuda_fail(e, "layout launch");
+    st = sna_forward_ex(plan, s.q, s.k, s.v, s.out, s.lse, B, H, C, cuda_stream);
+    if (st != SNA_OK) return st;
+    e = sna::launch_cl_to_cf(s.out, out_cf, B * H, C, p_out, stream);
+    if (e != cudaSuccess) return cuda_fail(e, "layout launch");
+    return SNA_OK;
+}
+
+sna_status_t sna_backward_cf(const sna_plan_t* plan, const float* dout_cf, const void* state, size_t state_bytes,
+                             void* scratch, size_t scratch_bytes, float* dq_cf, float* dk_cf, float* dv_cf,
+                             int B, int H, int C, void* cuda_stream) {
+    sna_status_t st = check_problem(plan, B, H, C);
+    if (st != SNA_OK) return st;
+    if (!dout_cf || !dq_cf || !dk_cf || !dv_cf) { set_error("dout, dq, dk and dv must not be NULL"); return SNA_ERR_INVALID_ARG; }
+    if (!all_aligned(dout_cf, dq_cf, dk_cf, dv_cf)) { set_error("device pointers must be 16-byte aligned"); return SNA_ERR_INVALID_ARG; }
+    if (state == nullptr || (reinterpret_cast<uintptr_t>(state) & 255u) || scratch == nullptr || (reinterpret_cast<uintptr_t>(scratch) & 255u)) {
+        set_error("state and scratch must be non-NULL and 256-byte aligned");
+        return SNA_ERR_INVALID_ARG;
+    }
+    if (state_bytes < sna_cf_state_bytes(plan, B, H, C) || scratch_bytes < sna_cf_scratch_bytes(plan, B, H, C)) {
+        set_error("state or scratch too small: %zu / %zu bytes given, %zu / %zu needed", state_bytes, scratch_bytes,
+                  sna_cf_state_bytes(plan, B, H, C), sna_cf_scratch_bytes(plan, B, H, C));
+        return SNA_ERR_WORKSPACE;
+    }
+    if ((long long)B * H > 65535) { set_error("the channels-first entry points take at most 65535 batch*head slices"); return SNA_ERR_UNSUPPORTED; }
+    cudaStream_t stream = (cudaStream_t)cuda_stream;
+    const CfState s = carve_state(plan, const_cast<void*>(state), B, H, C);
+    char* p = (char*)scratch;
+    float* dout = (float*)p; p += round256(out_elems(plan, B, H, C) * sizeof(float));
+    float* dq = (float*)p;   p += round256(out_elems(plan, B, H, C) * sizeof(float));
+    float* dk = (float*)p;   p += round256(in_elems(plan, B, H, C) * sizeof(float));
+    float* dv = (float*)p;   p += round256(in_elems(plan, B, H, C) * sizeof(float));
+    void* ws = p;
+    const long long p_in = (long long)plan->host.nlat_in * plan->host.nlon_in, p_out = (long long)plan->host.nlat_out * plan->host.nlon_out;
+    cudaError_t e = sna::launch_cf_to_cl(dout_cf, dout, B * H, C, p_out, stream);
+    if (e != cudaSuccess) return cuda_fail(e, "layout launch");
+    st = sna_backward_ex(plan, s.q, s.k, s.v, dout, s.out, s.lse, dq, dk, dv, ws, sna_workspace_bytes(plan, B, H, C), B, H, C, cuda_stream);
+    if (st != SNA_OK) return st;
+    e = sna::launch_cl_to_cf(dq, dq_cf, B * H, C, p_out, stream);
+    if (e == cudaSuccess) e = sna::launch_cl_to_cf(dk, dk_cf, B * H, C, p_in, stream);
+    if (e == cudaSuccess) e = sna::launch_cl_to_cf(dv, dv_cf, B * H, C, p_in, stream);
+    if (e != cudaSuccess) return cuda_fail(e, "layout launch");
+    return SNA_OK;
+}
+
 sna_status_t sna_forward_tf32(const sna_plan_t* plan, const float* q, const float* k, const float* v, float* out,
                               float* lse, int B, int H, int C, void* cuda_stream) {
     sna_status_t st = check_problem(plan, B, H, C);

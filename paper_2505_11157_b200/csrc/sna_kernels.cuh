@@ -93,6 +93,10 @@ cudaError_t launch_backward_dq_mma(const DevPlan& p, const float* q, const float
 cudaError_t launch_backward_dkdv_mma(const DevPlan& p, const float* q, const float* k, const float* v, const float* dout,
                                      const float* lse, const float* Dws, float* dk, float* dv, int N, int C, cudaStream_t stream);
 
+// Layout changes (sna_kernels_layout.cu): [slices][C][P] channels first <-> [slices][P][C] channels last, slices <= 65535.
+cudaError_t launch_cf_to_cl(const float* src, float* dst, int slices, int C, long long P, cudaStream_t stream);
+cudaError_t launch_cl_to_cf(const float* src, float* dst, int slices, int C, long long P, cudaStream_t stream);
+
 // Generic kernels (any supported C): C/4 lanes cooperate on one grid point.
 // forward: out and/or lse may be null (lse-only pass = softmax statistics).
 cudaError_t launch_forward_generic(const DevPlan& p, const float* q, const float* k, const float* v, float* out,

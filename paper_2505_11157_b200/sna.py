@@ -60,6 +60,10 @@ _SIGNATURES = {
     "sna_backward_ex": (_i, [_vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _sz, _i, _i, _i, _vp]),
     "sna_backward_dq": (_i, [_vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _i, _i, _i, _vp]),
     "sna_backward_dkdv": (_i, [_vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _i, _i, _i, _vp]),
+    "sna_cf_state_bytes": (_sz, [_vp, _i, _i, _i]),
+    "sna_cf_scratch_bytes": (_sz, [_vp, _i, _i, _i]),
+    "sna_forward_cf": (_i, [_vp, _vp, _vp, _vp, _vp, _vp, _sz, _i, _i, _i, _vp]),
+    "sna_backward_cf": (_i, [_vp, _vp, _vp, _sz, _vp, _sz, _vp, _vp, _vp, _i, _i, _i, _vp]),
     "sna_forward_tf32": (_i, [_vp, _vp, _vp, _vp, _vp, _vp, _i, _i, _i, _vp]),
     "sna_backward_tf32": (_i, [_vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _sz, _i, _i, _i, _vp]),
     "sna_backward_static": (_i, [_vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _i, _i, _i, _vp]),
@@ -215,6 +219,24 @@ def sna_measure_fp32_fma_peak() -> float:
 
 # ---- convenience wrapper -----------------------------------------------------------------------------------
 
+def sna_cf_state_bytes(plan: int, B: int, H: int, C: int) -> int:
+    return int(_lib.sna_cf_state_bytes(plan, B, H, C))
+
+
+def sna_cf_scratch_bytes(plan: int, B: int, H: int, C: int) -> int:
+    return int(_lib.sna_cf_scratch_bytes(plan, B, H, C))
+
+
+def sna_forward_cf(plan, q_cf, k_cf, v_cf, out_cf, state, state_bytes, B, H, C, stream=None) -> None:
+    _check(_lib.sna_forward_cf(plan, _ptr(q_cf), _ptr(k_cf), _ptr(v_cf), _ptr(out_cf), _ptr(state), state_bytes, B, H, C,
+                               _stream(stream)))
+
+
+def sna_backward_cf(plan, dout_cf, state, state_bytes, scratch, scratch_bytes, dq_cf, dk_cf, dv_cf, B, H, C, stream=None) -> None:
+    _check(_lib.sna_backward_cf(plan, _ptr(dout_cf), _ptr(state), state_bytes, _ptr(scratch), scratch_bytes,
+                                _ptr(dq_cf), _ptr(dk_cf), _ptr(dv_cf), B, H, C, _stream(stream)))
+
+
 class Plan:
     """Owns one ``sna_plan_t``.  Shapes follow the header: q/out [B,H,nlat_out,nlon_out,C], k/v [B,H,nlat_in,nlon_in,C]."""
 
@@ -328,6 +350,61 @@ class Plan:
             lse = torch.empty(q.shape[:-1], dtype=torch.float32, device=q.device)
         (sna_forward_ex if precision == "fp32" else sna_forward_tf32)(self.handle, q, k, v, out, lse, B, H, C, stream)
         return (out, lse) if return_lse else out
+
+    def _validate_cf(self, heads, **tensors):
+        """Channels-first tensors [B, heads*C, nlat, nlon]: out-grid (q, out, dout, dq) or in-grid (k, v, dk, dv)."""
+        import torch
+        q = tensors["q"] if "q" in tensors else tensors["dout"]
+        if not isinstance(q, torch.Tensor) or q.dim() != 4 or heads < 1 or q.shape[1] % heads != 0:
+            raise ValueError("channels-first tensors must be [B, heads*C, nlat, nlon]")
+        B, HC = q.shape[0], q.shape[1]
+        out_shape, in_shape = (B, HC, self.nlat_out, self.nlon_out), (B, HC, self.nlat_in, self.nlon_in)
+        expected = {"q": out_shape, "out": out_shape, "dout": out_shape, "dq": out_shape,
+                    "k": in_shape, "v": in_shape, "dk": in_shape, "dv": in_shape}
+        for name, t in tensors.items():
+            if t is None:
+                continue
+            if not isinstance(t, torch.Tensor) or t.dtype != torch.float32:
+                raise ValueError(f"{name} must be a float32 torch.Tensor")
+            if tuple(t.shape) != expected[name]:
+                raise ValueError(f"{name} has shape {tuple(t.shape)}, expected {expected[name]}")
+            if not t.is_contiguous():
+                raise ValueError(f"{name} must be contiguous")
+            if not t.is_cuda or t.device != q.device:
+                raise ValueError(f"{name} must be a CUDA tensor on the device of the first tensor ({q.device})")
+        return B, heads, HC // heads
+
+    def forward_cf(self, q, k, v, heads, out=None, state=None, stream=None):
+        """Channels-first forward: q [B, heads*C, nlat_out, nlon_out], k, v [B, heads*C, nlat_in, nlon_in].
+        Returns (out, state); pass the state to backward_cf."""
+        import torch
+        B, H, C = self._validate_cf(heads, q=q, k=k, v=v, out=out)
+        need = sna_cf_state_bytes(self.handle, B, H, C)
+        if state is None:
+            state = torch.empty(need, dtype=torch.uint8, device=q.device)
+        elif not state.is_cuda or state.device != q.device or not state.is_contiguous():
+            raise ValueError("state must be a contiguous CUDA tensor on the device of q")
+        out = torch.empty_like(q) if out is None else out
+        sna_forward_cf(self.handle, q, k, v, out, state, state.numel() * state.element_size(), B, H, C, stream)
+        return out, state
+
+    def backward_cf(self, dout, state, heads, dq=None, dk=None, dv=None, scratch=None, stream=None):
+        """Channels-first backward from the state forward_cf left: returns (dq, dk, dv), channels first."""
+        import torch
+        B, H, C = self._validate_cf(heads, dout=dout, dq=dq, dk=dk, dv=dv)
+        need = sna_cf_scratch_bytes(self.handle, B, H, C)
+        if scratch is None:
+            scratch = torch.empty(need, dtype=torch.uint8, device=dout.device)
+        for name, t in (("state", state), ("scratch", scratch)):
+            if not isinstance(t, torch.Tensor) or not t.is_cuda or t.device != dout.device or not t.is_contiguous():
+                raise ValueError(f"{name} must be a contiguous CUDA tensor on the device of dout")
+        in_shape = (B, H * C, self.nlat_in, self.nlon_in)
+        dq = torch.empty_like(dout) if dq is None else dq
+        dk = torch.empty(in_shape, dtype=torch.float32, device=dout.device) if dk is None else dk
+        dv = torch.empty(in_shape, dtype=torch.float32, device=dout.device) if dv is None else dv
+        sna_backward_cf(self.handle, dout, state, state.numel() * state.element_size(), scratch,
+                        scratch.numel() * scratch.element_size(), dq, dk, dv, B, H, C, stream)
+        return dq, dk, dv
 
     def backward(self, q, k, v, dout, out=None, lse=None, dq=None, dk=None, dv=None, workspace=None, stream=None,
                  precision="fp32"):

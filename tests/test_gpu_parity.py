@@ -278,6 +278,59 @@ def test_a_bounded_wait_that_runs_out_is_reported_once_and_the_plan_stays_usable
             sna.sna_debug_exercise_bounded_wait(plan.handle, 0)  # refused on the host
 
 
+@pytest.mark.parametrize("wl", [SMALL[0], SMALL[2], SMALL[4], SMALL[26], WORKLOADS["c1"]], ids=lambda w: w.name)
+def test_channels_first_entry_points_against_oracle(wl):
+    """sna_forward_cf / sna_backward_cf: tensors [B, H*C, nlat, nlon]; the oracle sees the same values channels last."""
+    g = _geometry(wl)
+    q, k, v, dout = make_inputs(wl)                               # [B, H, nlat, nlon, C]
+
+    def to_cf(x):
+        B, H, nlat, nlon, C = x.shape
+        return np.ascontiguousarray(x.transpose(0, 1, 4, 2, 3).reshape(B, H * C, nlat, nlon))
+
+    def to_cl(x, like):
+        B, H, nlat, nlon, C = like.shape
+        return x.reshape(B, H, C, nlat, nlon).transpose(0, 1, 3, 4, 2)
+
+    with _plan(wl) as plan:
+        out, state = plan.forward_cf(*_dev(to_cf(q), to_cf(k), to_cf(v)), heads=wl.H)
+        dq, dk, dv = plan.backward_cf(_dev(to_cf(dout))[0], state, heads=wl.H)
+        torch.cuda.synchronize()
+        sna.sna_plan_check(plan.handle)
+    ref_out = orc.forward(g, q, k, v)
+    rdq, rdk, rdv = orc.backward(g, q, k, v, dout)
+    assert nerr(to_cl(out.cpu().numpy(), q).reshape(ref_out.shape), ref_out) <= FWD_TOL
+    assert nerr(to_cl(dq.cpu().numpy(), q).reshape(rdq.shape), rdq) <= BWD_TOL
+    assert nerr(to_cl(dk.cpu().numpy(), k).reshape(rdk.shape), rdk) <= BWD_TOL
+    assert nerr(to_cl(dv.cpu().numpy(), k).reshape(rdv.shape), rdv) <= BWD_TOL
+
+
+def test_channels_first_autograd_wrapper_and_buffer_checks():
+    from paper_2505_11157_b200.autograd import spherical_neighborhood_attention_cf
+    wl = SMALL[0]
+    g = _geometry(wl)
+    q, k, v, dout = make_inputs(wl)
+    cf = lambda x: torch.from_numpy(np.ascontiguousarray(x.transpose(0, 1, 4, 2, 3).reshape(x.shape[0], -1, x.shape[2], x.shape[3]))).cuda()
+    with _plan(wl) as plan:
+        qt, kt, vt = (cf(x).requires_grad_(True) for x in (q, k, v))
+        out = spherical_neighborhood_attention_cf(plan, qt, kt, vt, heads=wl.H)
+        out.backward(cf(dout))
+        torch.cuda.synchronize()
+        rdq, rdk, rdv = orc.backward(g, q, k, v, dout)
+        back = lambda t, like: t.detach().cpu().numpy().reshape(like.shape[0], like.shape[1], like.shape[4], like.shape[2], like.shape[3]).transpose(0, 1, 3, 4, 2)
+        assert nerr(back(qt.grad, q).reshape(rdq.shape), rdq) <= BWD_TOL
+        assert nerr(back(kt.grad, k).reshape(rdk.shape), rdk) <= BWD_TOL
+        assert nerr(back(vt.grad, k).reshape(rdv.shape), rdv) <= BWD_TOL
+        # a state buffer that is too small is refused on the host
+        small = torch.empty(256, dtype=torch.uint8, device="cuda")
+        with pytest.raises(sna.SnaError) as e:
+            plan.forward_cf(cf(q), cf(k), cf(v), heads=wl.H, state=small)
+        assert e.value.status == sna.SNA_ERR_WORKSPACE
+        with pytest.raises(ValueError):
+            plan.forward_cf(cf(q), cf(k), cf(v), heads=5)     # channel count not divisible by the heads
+    torch.cuda.synchronize()
+
+
 def test_results_are_reproducible_bit_for_bit():
     wl = SMALL[2]
     q, k, v, dout = make_inputs(wl)
