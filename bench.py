@@ -33,12 +33,13 @@ if ROOT not in sys.path:
 
 import numpy as np  # noqa: E402
 
-# Recorded constants: dram__bytes_read.sum + dram__bytes_write.sum per launch from an ncu capture of the band kernels on
-# workload c3 (bench.py cannot run ncu itself; the value is reported as `roofline.traffic` for that workload only).
+# Recorded constants: dram__bytes_read.sum + dram__bytes_write.sum per stage (its dense kernel + its band kernel) from an
+# ncu capture on workload c3 (bench.py cannot run ncu itself; the value is reported as `roofline.traffic` for that
+# workload only).
 NCU_DRAM_BYTES_PER_LAUNCH = {
-    ("c3", "forward"): 816768768 + 63346432,
-    ("c3", "backward_dq"): 980778752 + 66266112,
-    ("c3", "backward_dkdv"): 715740160 + 502913024,
+    ("c3", "forward"): (46338304 + 934144) + (810467584 + 61794560),
+    ("c3", "backward_dq"): (58616832 + 2412544) + (973628928 + 63840000),
+    ("c3", "backward_dkdv"): (49178368 + 7201024) + (760083968 + 501852160),
 }
 HBM_GBS_FALLBACK = 6650.0          # used only if MEASURED_PEAKS.json is absent
 L2_BYTES = 126 * 1024 * 1024
@@ -427,8 +428,8 @@ def run_ours(args, wl):
                          "frac": achieved / peak, "traffic": NCU_DRAM_BYTES_PER_LAUNCH.get((wl.name, dominant)),
                          "note": f"{dom['flops_per_unit']:g} flops per pair*channel credited, {dom['bytes'] / 1e6:.0f} MB compulsory; "
                                  f"{peak_note}; the contractions run on tensor cores (TF32 main term + stacked BF16 corrections, "
-                                 "tcgen05 for whole-ring windows); traffic = recorded ncu DRAM bytes read+written per launch, "
-                                 "null when this workload has no capture"},
+                                 "tcgen05 for whole-ring and wide windows); traffic = recorded ncu DRAM bytes read+written per "
+                                 "stage (dense + band kernel), null when this workload has no capture"},
             "e2e": {"value": world * units / (ms_e2e_step_max * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
                     "d2h_bytes_per_step": d2h, "ms_per_step": ms_e2e_step_max},
             "gpu_launches": launches_per_step * args.steps,
