@@ -278,7 +278,7 @@ def test_a_bounded_wait_that_runs_out_is_reported_once_and_the_plan_stays_usable
             sna.sna_debug_exercise_bounded_wait(plan.handle, 0)  # refused on the host
 
 
-@pytest.mark.parametrize("wl", [SMALL[0], SMALL[2], SMALL[4], SMALL[26], WORKLOADS["c1"]], ids=lambda w: w.name)
+@pytest.mark.parametrize("wl", [SMALL[0], SMALL[2], SMALL[4], SMALL[6], SMALL[8], SMALL[26], WORKLOADS["c1"]], ids=lambda w: w.name)
 def test_channels_first_entry_points_against_oracle(wl):
     """sna_forward_cf / sna_backward_cf: tensors [B, H*C, nlat, nlon]; the oracle sees the same values channels last."""
     g = _geometry(wl)
