@@ -284,7 +284,8 @@ def time_steps(torch, prob, steps, warmup, step_fn=None, flush=None):
 
 def accuracy_against_oracle(orc, g, prob, n_slices):
     """Errors of the GPU results of the first n_slices batch*head slices against the oracle: the gated measure
-    max|x-o| / max|o| per tensor, and the element-wise relative error with denominator max(|o|, 1e-3 max|o|)."""
+    max|x-o| / max|o| per tensor, the element-wise relative error with denominator max(|o|, 1e-3 max|o|), and the
+    per-point relative error ||x_i - o_i|| / max(||o_i||, 1e-3 max_i ||o_i||) over the channel vectors."""
     wl = prob.wl
     arrays = [h.numpy() for h in prob.host]
     sl = lambda a, nlat, nlon: a.reshape(wl.N, nlat, nlon, wl.C)[:n_slices]
@@ -299,8 +300,10 @@ def accuracy_against_oracle(orc, g, prob, n_slices):
     for name, x, r in zip(("out", "dq", "dk", "dv"), got, refs):
         x = x.reshape((wl.N,) + r.shape[1:])[:n_slices].cpu().numpy().astype(np.float64)
         scale = np.max(np.abs(r))
+        norms = np.linalg.norm(r, axis=-1)
         acc[name] = {"normalised_max_error": float(np.max(np.abs(x - r)) / scale),
-                     "floor_relative_max_error": float(np.max(np.abs(x - r) / np.maximum(np.abs(r), 1e-3 * scale)))}
+                     "floor_relative_max_error": float(np.max(np.abs(x - r) / np.maximum(np.abs(r), 1e-3 * scale))),
+                     "per_point_relative_max_error": float(np.max(np.linalg.norm(x - r, axis=-1) / np.maximum(norms, 1e-3 * norms.max())))}
     return seconds, acc
 
 
