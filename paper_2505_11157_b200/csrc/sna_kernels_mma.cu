@@ -195,7 +195,7 @@ struct FwdView {
 // forward
 // ---------------------------------------------------------------------------------------------------------
 template <int C, bool LP>
-__global__ void __launch_bounds__(THREADS, 4)
+__global__ void __launch_bounds__(THREADS, C == 64 ? 2 : 4)
 forward_mma_kernel(DevPlan p, FwdView fv, const float* __restrict__ q, const float* __restrict__ k, const float* __restrict__ v,
                    float* out, float* lse, int N, float scale_log2, int tiles_per_row, long long total_tasks) {
     constexpr int CPT = C / 4, KS = C / 8;
@@ -326,7 +326,7 @@ forward_mma_kernel(DevPlan p, FwdView fv, const float* __restrict__ q, const flo
 // `out` and `dq` may be the same buffer: a warp reads its own 16 rows of `out` before it writes them as dq.
 // ---------------------------------------------------------------------------------------------------------
 template <int C, bool LP>
-__global__ void __launch_bounds__(THREADS, 3)
+__global__ void __launch_bounds__(THREADS, C == 64 ? 2 : 3)
 backward_dq_mma_kernel(DevPlan p, FwdView fv, const float* __restrict__ q, const float* __restrict__ k, const float* __restrict__ v,
                        const float* __restrict__ dout, const float* out, const float* __restrict__ lse,
                        float* dq, float* __restrict__ Dws, int N, float scale, int tiles_per_row, long long total_tasks) {
