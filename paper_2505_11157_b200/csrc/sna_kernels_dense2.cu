@@ -834,26 +834,29 @@ backward_dq_dense2_kernel(DevPlan p, const __grid_constant__ CUtensorMap map_k, 
 
 // ---------------------------------------------------------------------------------------------------------
 // Pipelined dense part of the dk/dv stage (App. B.4), transposed roles: a block owns 128 consecutive input columns of
-// an input ring (tile row = input point j, its k and v rows and their lo parts live in TMEM) and walks, in blocks of 64,
-// the output points i of the output rings that attend to this input ring as a whole:
+// an input ring (tile row = input point j, its k and v rows and their lo parts live in TMEM) and walks, in blocks of 32,
+// the output points i of the output rings that attend to this input ring:
 //   S^T = K Q^T, T^T = V dY^T (one issuing thread each);  p = exp2(s + log2 omega_j - lse_i),  ds = p (t - D_i);
 //   dV += P dY,  dK += scale * dS Q   (A operands P, dS from TMEM; B operands: q and dout blocks transposed by the converters).
 // Two groups of 128 threads do the element-wise work for one half of the block's columns each and write P over S^T, dS
 // over T^T and the two lo parts beside them; four threads issue the second GEMMs (dV or dK, one column half each) into
-// their own accumulators, which collect FOLDK blocks in TMEM before the row's threads fold them into registers.  TMEM
-// holds only one (S^T, T^T) buffer here (128 columns of fixed operands + 256 of S, T, P_lo, dS_lo + 128 of accumulators), so
-// the first GEMMs of block j+1 wait for the second GEMMs of block j; TMA and the converters run three blocks ahead.
+// their own accumulators, which collect FOLDK blocks in TMEM before the row's threads fold them into registers.  TMEM:
+// 128 columns of fixed operands, two buffers of 128 (S^T, T^T, P_lo, dS_lo of 32 columns each) and 128 of accumulators.
+// With two buffers the first GEMMs of block j+1 run while the element-wise threads work on block j and the second
+// GEMMs on block j-1 (blocks of 64 points leave room for one buffer only, which serialised the three phases); TMA and
+// the converters run up to four blocks ahead.
 // ---------------------------------------------------------------------------------------------------------
-constexpr int BNK = 64;                          // partner points per block
-constexpr int TILE_K = BNK * 128;                // 8 KB
-constexpr int FOLDK = 4;
-constexpr int NSK = 3;                           // shared-memory stages
+constexpr int BNK = 32;                          // partner points per block
+constexpr int TILE_K = BNK * 128;                // 4 KB
+constexpr int FOLDK = 8;
+constexpr int NSK = 5;                           // shared-memory stages
 // per stage: q raw, q lo, y raw, y lo, q^T hi, q^T lo, y^T hi, y^T lo, then log2 omega - lse*log2e and D of the 64 partner points
 constexpr int KST = 8 * TILE_K + 1024;
 constexpr size_t DKDV2_SMEM = NSK * KST + 1024;
-constexpr int TK_AK = 0, TK_AKL = 32, TK_AV = 64, TK_AVL = 96, TK_S = 128, TK_T = 192, TK_PLO = 256, TK_DSLO = 320, TK_ACC = 384 /* + 32 part */;
-enum { K_QFULL = 0, K_YFULL = 3, K_QCONV = 6, K_YCONV = 9, K_FREE = 12 /* all [stage] */, K_STFULL = 15, K_READY = 16 /* [group] */,
-       K_G2DONE = 18 /* [group] */, K_AREADY = 20, K_COUNT = 21 };
+constexpr int TK_AK = 0, TK_AKL = 32, TK_AV = 64, TK_AVL = 96, TK_BUF = 128 /* + 128 b: S | T | P_lo | dS_lo, 32 columns each */, TK_ACC = 384 /* + 32 part */;
+constexpr int TK_S = 0, TK_T = 32, TK_PLO = 64, TK_DSLO = 96;      // offsets inside a buffer
+enum { K_QFULL = 0, K_YFULL = NSK, K_QCONV = 2 * NSK, K_YCONV = 3 * NSK, K_FREE = 4 * NSK /* all [stage] */, K_STFULL = 5 * NSK /* [buffer] */,
+       K_READY = 5 * NSK + 2 /* [group] */, K_G2DONE = 5 * NSK + 4 /* [group][buffer] */, K_AREADY = 5 * NSK + 8, K_COUNT = 5 * NSK + 9 };
 
 __global__ void __launch_bounds__(THREADS2, 1)
 backward_dkdv_dense2_kernel(DevPlan p, const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_y,
@@ -890,10 +893,11 @@ backward_dkdv_dense2_kernel(DevPlan p, const __grid_constant__ CUtensorMap map_q
             mb_init(s32(&bars[K_YCONV + s]), 128);
             mb_init(s32(&bars[K_FREE + s]), 6);         // both first GEMMs and the four second-GEMM issuers
         }
-        mb_init(s32(&bars[K_STFULL]), 2);
         for (int g = 0; g < 2; ++g) {
+            mb_init(s32(&bars[K_STFULL + g]), 2);            // buffer g: both first GEMMs
             mb_init(s32(&bars[K_READY + g]), 128);
-            mb_init(s32(&bars[K_G2DONE + g]), 2);
+            mb_init(s32(&bars[K_G2DONE + 2 * g]), 2);        // group g, buffer 0: its dV and dK issuers
+            mb_init(s32(&bars[K_G2DONE + 2 * g + 1]), 2);    // group g, buffer 1
         }
         mb_init(s32(&bars[K_AREADY]), 128);
         fail_s = 0;
@@ -917,7 +921,7 @@ backward_dkdv_dense2_kernel(DevPlan p, const __grid_constant__ CUtensorMap map_q
         // 256 x 160 + 256 x 40 + 128 x 72 = 60416 <= 61440
         asm volatile("setmaxnreg.inc.sync.aligned.u32 160;");
         // ------------------------------------------------------------------ element-wise: thread (grp, r) owns tile row r (an
-        // input point) for the partner columns [32 grp, 32 grp + 32) of every block
+        // input point) for the partner columns [16 grp, 16 grp + 16) of every block
         const int grp = warp >> 2, r = tid & 127;
         const uint32_t lanebits = (uint32_t)((warp & 3) * 32) << 16;
         const int c = c0 + r;
@@ -957,7 +961,7 @@ backward_dkdv_dense2_kernel(DevPlan p, const __grid_constant__ CUtensorMap map_q
         for (int it = 0; it <= total && ok; ++it) {
             if (it > 0 && (it % FOLDK == 0 || it == total)) {
                 // fold the second GEMMs of the blocks since the last fold; this also frees the accumulators
-                PROF_WAIT(1, ok = mb_wait(s32(&bars[K_G2DONE + grp]), (it - 1) & 1, ok) && ok);
+                PROF_WAIT(1, ok = mb_wait(s32(&bars[K_G2DONE + 2 * grp + ((it - 1) & 1)]), ((it - 1) >> 1) & 1, ok) && ok);
                 asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
                 uint32_t oa[32], ob[32];
                 tm_ld32_issue(oa, tm + TK_ACC + grp * 32 + lanebits);          // dV, this column half
@@ -967,7 +971,7 @@ backward_dkdv_dense2_kernel(DevPlan p, const __grid_constant__ CUtensorMap map_q
                 for (int j = 0; j < C2; ++j) { gv[j] += __uint_as_float(oa[j]); gk[j] += __uint_as_float(ob[j]); }
             }
             if (it < total) {
-                const int s = it % NSK;
+                const int s = it % NSK, b = it & 1;
                 // the partner columns [jl, jh] of this thread's half that exist and have this row's input point in their window
                 const int wl = ps_shift >= 0 ? -((wk.m - c) >> ps_shift) : cdiv(c - wk.m, p.ps);      // ceil((c - m) / ps)
                 const int wh = ps_shift >= 0 ? (c + wk.m) >> ps_shift : fdiv(c + wk.m, p.ps);         // floor((c + m) / ps)
@@ -976,24 +980,32 @@ backward_dkdv_dense2_kernel(DevPlan p, const __grid_constant__ CUtensorMap map_q
                 const uint32_t span = (uint32_t)(jh - jl);
                 const bool full = __all_sync(0xffffffffu, jl <= 0 && jh >= GC - 1);     // no masking anywhere in this warp
                 wk.advance();
-                PROF_WAIT(0, ok = mb_wait(s32(&bars[K_STFULL]), it & 1, ok) && ok);     // implies QCONV of this stage (the S issuer waited for it)
+                PROF_WAIT(0, ok = mb_wait(s32(&bars[K_STFULL + b]), (it >> 1) & 1, ok) && ok);     // implies QCONV of this stage (the S issuer waited for it)
                 asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
                 const float* nlc = reinterpret_cast<const float*>(base + s * KST + 8 * TILE_K) + grp * GC;
                 const float* Dc = nlc + BNK;
-                const uint32_t tS = tm + TK_S + grp * GC + lanebits, tT = tm + TK_T + grp * GC + lanebits;
-                const uint32_t tPl = tm + TK_PLO + grp * GC + lanebits, tDl = tm + TK_DSLO + grp * GC + lanebits;
-#pragma unroll
-                for (int hf = 0; hf < 2; ++hf) {
+                const uint32_t tB = tm + TK_BUF + 128 * b + grp * GC + lanebits;
+                const uint32_t tS = tB + TK_S, tT = tB + TK_T, tPl = tB + TK_PLO, tDl = tB + TK_DSLO;
+                {
+                    constexpr int hf = 0;
                     uint32_t sv[16], tv[16], pl[16], dl[16];
                     tm_ld16_issue(sv, tS + hf * 16);
                     tm_ld16_issue(tv, tT + hf * 16);
+                    // the per-column statistics of this thread's 16 columns, as 16-byte loads while the TMEM loads are in flight
+                    float nlv[16], Dv[16];
+#pragma unroll
+                    for (int q4 = 0; q4 < 4; ++q4) {
+                        const float4 a = reinterpret_cast<const float4*>(nlc)[q4], d4 = reinterpret_cast<const float4*>(Dc)[q4];
+                        nlv[4 * q4] = a.x; nlv[4 * q4 + 1] = a.y; nlv[4 * q4 + 2] = a.z; nlv[4 * q4 + 3] = a.w;
+                        Dv[4 * q4] = d4.x; Dv[4 * q4 + 1] = d4.y; Dv[4 * q4 + 2] = d4.z; Dv[4 * q4 + 3] = d4.w;
+                    }
                     tm_ld_wait();
 #pragma unroll
                     for (int j = 0; j < 16; ++j) {
                         const int col = hf * 16 + j;
-                        float pj = ex2f(fmaf(__uint_as_float(sv[j]), scale_log2, nlc[col]));
+                        float pj = ex2f(fmaf(__uint_as_float(sv[j]), scale_log2, nlv[j]));
                         if (!full && (uint32_t)(col - jl) > span) pj = 0.f;
-                        const float ds = pj * (__uint_as_float(tv[j]) - Dc[col]);
+                        const float ds = pj * (__uint_as_float(tv[j]) - Dv[j]);
                         sv[j] = __float_as_uint(pj);
                         tv[j] = __float_as_uint(ds);
                         pl[j] = __float_as_uint(pj - trunc19f(pj));
@@ -1054,24 +1066,24 @@ backward_dkdv_dense2_kernel(DevPlan p, const __grid_constant__ CUtensorMap map_q
             const uint32_t idS = idesc_tf32(BNK);
             const uint32_t tA = tm + (isT ? TK_AV : TK_AK), tAl = tm + (isT ? TK_AVL : TK_AKL);
             for (int it = 0; it < total && ok; ++it) {
-                const int s = it % NSK, us = it / NSK;
+                const int s = it % NSK, us = it / NSK, b = it & 1, u = it >> 1;
                 PROF_WAIT(0, ok = mb_wait(s32(&bars[(isT ? K_YFULL : K_QFULL) + s]), us & 1, ok));
                 PROF_WAIT(1, ok = mb_wait(s32(&bars[(isT ? K_YCONV : K_QCONV) + s]), us & 1, ok) && ok);
-                if (it > 0) {   // the single (S^T, T^T) buffer is free once all four second-GEMM issuers of block it-1 are done
-                    PROF_WAIT(2, ok = mb_wait(s32(&bars[K_G2DONE]), (it - 1) & 1, ok) && ok);
-                    PROF_WAIT(2, ok = mb_wait(s32(&bars[K_G2DONE + 1]), (it - 1) & 1, ok) && ok);
+                if (u > 0) {   // this (S^T, T^T, P_lo, dS_lo) buffer is free once all four second-GEMM issuers of block it-2 are done
+                    PROF_WAIT(2, ok = mb_wait(s32(&bars[K_G2DONE + b]), (u - 1) & 1, ok) && ok);
+                    PROF_WAIT(2, ok = mb_wait(s32(&bars[K_G2DONE + 2 + b]), (u - 1) & 1, ok) && ok);
                 }
                 asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
                 const uint32_t tile0 = sbase + s * KST + (isT ? 2 * TILE_K : 0);
                 const uint64_t db = desc_k(tile0), dbl = desc_k(tile0 + TILE_K);
-                const uint32_t tD = tm + (isT ? TK_T : TK_S);
+                const uint32_t tD = tm + TK_BUF + 128 * b + (isT ? TK_T : TK_S);
 #pragma unroll
                 for (int ks = 0; ks < C2 / 8; ++ks) mma_ts(tD, tAl + ks * 8, db + 2 * ks, idS, ks > 0);
 #pragma unroll
                 for (int ks = 0; ks < C2 / 8; ++ks) mma_ts(tD, tA + ks * 8, dbl + 2 * ks, idS, 1);
 #pragma unroll
                 for (int ks = 0; ks < C2 / 8; ++ks) mma_ts(tD, tA + ks * 8, db + 2 * ks, idS, 1);
-                mma_commit(s32(&bars[K_STFULL]));
+                mma_commit(s32(&bars[K_STFULL + b]));
                 mma_commit(s32(&bars[K_FREE + s]));
             }
         }
@@ -1082,23 +1094,23 @@ backward_dkdv_dense2_kernel(DevPlan p, const __grid_constant__ CUtensorMap map_q
             const int part = warp - 12, kind = part >> 1, grp = part & 1;      // kind 0: dV = P dY, kind 1: dK = dS Q
             const uint32_t idO = idesc_tf32(C2);
             const uint32_t tO = tm + TK_ACC + part * 32;
-            const uint32_t tA = tm + (kind ? TK_T : TK_S), tAl = tm + (kind ? TK_DSLO : TK_PLO);
             for (int it = 0; it < total && ok; ++it) {
-                const int s = it % NSK, us = it / NSK;
+                const int s = it % NSK, us = it / NSK, b = it & 1;
+                const uint32_t tA = tm + TK_BUF + 128 * b + (kind ? TK_T : TK_S), tAl = tm + TK_BUF + 128 * b + (kind ? TK_DSLO : TK_PLO);
                 PROF_WAIT(0, ok = mb_wait(s32(&bars[(kind ? K_QCONV : K_YCONV) + s]), us & 1, ok));
                 PROF_WAIT(1, ok = mb_wait(s32(&bars[K_READY + grp]), it & 1, ok) && ok);
                 asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
                 const uint32_t bt = sbase + s * KST + (kind ? 4 : 6) * TILE_K;          // q^T (dK) or y^T (dV) tiles
 #pragma unroll
-                for (int k8 = 0; k8 < 4; ++k8) {
-                    const int ks = grp * 4 + k8;                                    // 8-column step within the block
-                    const uint32_t off = (uint32_t)(ks >> 2) * (C2 * 128) + (uint32_t)(ks & 3) * 32;
+                for (int k8 = 0; k8 < 2; ++k8) {
+                    const int ks = grp * 2 + k8;                                    // 8-column step within the block
+                    const uint32_t off = (uint32_t)ks * 32;                         // the block is one K block of 32 points
                     const uint64_t dh = desc_k(bt + off), dl = desc_k(bt + TILE_K + off);
                     mma_ts(tO, tAl + ks * 8, dh, idO, (k8 > 0) || (it % FOLDK != 0));
                     mma_ts(tO, tA + ks * 8, dl, idO, 1);
                     mma_ts(tO, tA + ks * 8, dh, idO, 1);
                 }
-                mma_commit(s32(&bars[K_G2DONE + grp]));
+                mma_commit(s32(&bars[K_G2DONE + 2 * grp + b]));
                 mma_commit(s32(&bars[K_FREE + s]));
             }
         }
@@ -1107,28 +1119,27 @@ backward_dkdv_dense2_kernel(DevPlan p, const __grid_constant__ CUtensorMap map_q
         // ------------------------------------------------------------------ converters (warps 16-19, 128 threads)
         const int ct = tid - 512, cw = ct >> 5;
         auto lo4 = [](const float4& x) { return make_float4(x.x - trunc19f(x.x), x.y - trunc19f(x.y), x.z - trunc19f(x.z), x.w - trunc19f(x.w)); };
-        // lo tile (same swizzled positions) and transposed hi / lo tiles of one raw tile: warp cw takes the 16 columns
-        // [16 cw, 16 cw + 16), lane = channel
+        // lo tile (same swizzled positions) and transposed hi / lo tiles of one raw tile (one K block of 32 points: row =
+        // channel, 128 bytes of points): warp cw takes the 8 columns [8 cw, 8 cw + 8), lane = channel
         auto convert = [&](unsigned char* raw, unsigned char* lo, unsigned char* th) {
 #pragma unroll
-            for (int j = 0; j < 4; ++j) {
+            for (int j = 0; j < TILE_K / (128 * 16); ++j) {
                 const int off = (j * 128 + ct) * 16;
                 *reinterpret_cast<float4*>(lo + off) = lo4(*reinterpret_cast<const float4*>(raw + off));
             }
-            unsigned char* t = th + (cw >> 1) * (C2 * 128);
 #pragma unroll
-            for (int c8 = 0; c8 < 4; ++c8) {
+            for (int c8 = 0; c8 < 2; ++c8) {
                 float hi[4], lw[4];
 #pragma unroll
                 for (int i = 0; i < 4; ++i) {
-                    const int col = cw * 16 + c8 * 4 + i;
+                    const int col = cw * 8 + c8 * 4 + i;
                     const float x = *reinterpret_cast<const float*>(raw + sw_off(col, lane >> 2) + (lane & 3) * 4);
                     hi[i] = trunc19f(x);
                     lw[i] = x - hi[i];
                 }
-                const int chunk = (cw & 1) * 4 + c8;
-                *reinterpret_cast<float4*>(t + sw_off(lane, chunk)) = make_float4(hi[0], hi[1], hi[2], hi[3]);
-                *reinterpret_cast<float4*>(t + TILE_K + sw_off(lane, chunk)) = make_float4(lw[0], lw[1], lw[2], lw[3]);
+                const int chunk = cw * 2 + c8;
+                *reinterpret_cast<float4*>(th + sw_off(lane, chunk)) = make_float4(hi[0], hi[1], hi[2], hi[3]);
+                *reinterpret_cast<float4*>(th + TILE_K + sw_off(lane, chunk)) = make_float4(lw[0], lw[1], lw[2], lw[3]);
             }
         };
         TileWalk wk(p.t_dense_lat, p.t_dense_m, e_begin, e_end, p.nlon_out, BNK, a_lo, a_hi, p.ps);
