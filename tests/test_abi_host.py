@@ -88,6 +88,35 @@ def test_planner_matches_oracle_bit_for_bit(name):
             assert got == exp, row
 
 
+def test_planner_matches_oracle_on_random_problems():
+    """Sixty seeded random problems (all three grids, ps in 1..4, arbitrary latitude counts and cutoffs): the planner's
+    table, or its refusal, must be the oracle's."""
+    rng = np.random.default_rng(2505)
+    status_of = {2: sna.SNA_ERR_AMBIGUOUS_TIE, 3: sna.SNA_ERR_EMPTY_NEIGHBORHOOD}
+    compared = refused = 0
+    for _ in range(60):
+        ps = int(rng.integers(1, 5))
+        nlon_out = int(rng.integers(3, 40))
+        nlat_in, nlat_out = int(rng.integers(2, 40)), int(rng.integers(2, 40))
+        gi, go = int(rng.integers(0, 3)), int(rng.integers(0, 3))
+        theta = float(rng.uniform(0.02, 1.0)) if rng.random() < 0.8 else float(rng.uniform(1.0, 3.3))
+        args = (nlat_in, nlon_out * ps, nlat_out, nlon_out, gi, go, theta)
+        try:
+            g = orc.geometry(*args)
+        except orc.OracleError as e:
+            with pytest.raises(sna.SnaError) as pe:
+                sna.Plan(*args, host_only=True)
+            assert pe.value.status == status_of[e.code], args
+            refused += 1
+            continue
+        with sna.Plan(*args, host_only=True) as p:
+            row_ptr, lat, off = p.table()
+            assert np.array_equal(row_ptr, g.row_ptr) and np.array_equal(lat, g.lat_in) and np.array_equal(off, g.lon_off), args
+            assert np.allclose(p.quad_weights(), g.omega, rtol=1e-13, atol=0), args
+        compared += 1
+    assert compared >= 30 and refused >= 1
+
+
 def test_headline_table_sizes():
     for name, nnz in (("c3", 53800), ("c4", 98995)):
         wl = WORKLOADS[name]

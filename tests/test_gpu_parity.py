@@ -351,6 +351,41 @@ def test_channels_first_autograd_wrapper_and_buffer_checks():
     torch.cuda.synchronize()
 
 
+def _random_problems(count, seed):
+    """Seeded random problems that the oracle accepts; wide rings so that banded, wide and whole-ring windows all occur."""
+    rng = np.random.default_rng(seed)
+    found = []
+    while len(found) < count:
+        ps = int(rng.choice([1, 1, 2, 2, 3, 4]))
+        nlon_out = int(rng.integers(32, 200 // ps + 33))
+        nlat_in, nlat_out = int(rng.integers(6, 25)), int(rng.integers(6, 25))
+        gi, go = int(rng.integers(0, 3)), int(rng.integers(0, 3))
+        theta = float(rng.uniform(0.25, 1.3))
+        C = int(rng.choice([32, 32, 32, 16, 64, 8]))
+        wl = small_workload(f"random{len(found)}", nlat_in, nlon_out * ps, nlat_out, nlon_out, gi, go, theta, 1, int(rng.integers(1, 3)), C,
+                            100 + len(found))
+        try:
+            _geometry(wl)
+        except orc.OracleError:
+            continue
+        found.append(wl)
+    return found
+
+
+@pytest.mark.parametrize("wl", _random_problems(12, 11157), ids=lambda w: f"{w.name}_{w.nlat_in}x{w.nlon_in}_to_{w.nlat_out}x{w.nlon_out}_C{w.C}")
+def test_random_problems_full_comparison(wl):
+    g = _geometry(wl)
+    q, k, v, dout = make_inputs(wl)
+    with _plan(wl) as plan:
+        out, lse, dq, dk, dv = _run_gpu(plan, q, k, v, dout, True)
+    ref_out = orc.forward(g, q, k, v)
+    rdq, rdk, rdv = orc.backward(g, q, k, v, dout)
+    assert nerr(out.reshape(ref_out.shape), ref_out) <= FWD_TOL
+    for name, x, r in zip(("dq", "dk", "dv"), (dq, dk, dv), (rdq, rdk, rdv)):
+        assert nerr(x.reshape(r.shape), r) <= BWD_TOL, name
+    assert perr(out, ref_out) <= PT_FWD_TOL
+
+
 def test_results_are_reproducible_bit_for_bit():
     wl = SMALL[2]
     q, k, v, dout = make_inputs(wl)
