@@ -37,9 +37,9 @@ import numpy as np  # noqa: E402
 # ncu capture on workload c3 (bench.py cannot run ncu itself; the value is reported as `roofline.traffic` for that
 # workload only).
 NCU_DRAM_BYTES_PER_LAUNCH = {
-    ("c3", "forward"): (46338304 + 934144) + (810467584 + 61794560),
-    ("c3", "backward_dq"): (58616832 + 2412544) + (973628928 + 63840000),
-    ("c3", "backward_dkdv"): (49178368 + 7201024) + (760083968 + 501852160),
+    ("c3", "forward"): (44229120 + 1959168) + (794043136 + 64422144),
+    ("c3", "backward_dq"): (56711424 + 2130688) + (965255936 + 63726080),
+    ("c3", "backward_dkdv"): (49354752 + 9662976) + (762001152 + 503494912),
 }
 HBM_GBS_FALLBACK = 6650.0          # used only if MEASURED_PEAKS.json is absent
 L2_BYTES = 126 * 1024 * 1024
