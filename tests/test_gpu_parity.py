@@ -386,6 +386,36 @@ def test_random_problems_full_comparison(wl):
     assert perr(out, ref_out) <= PT_FWD_TOL
 
 
+def test_multi_head_module_matches_oracle_composition():
+    """The nn.Module wrapper: pointwise projections (library GEMMs) around the channels-first operator.  Reference:
+    the same projections in fp64 numpy around the oracle; gradients of the projection weights through autograd."""
+    from paper_2505_11157_b200.module import SphericalNeighborhoodAttention
+    nlat_in, nlon_in, nlat_out, nlon_out, heads, hd, cin = 17, 48, 9, 24, 2, 16, 12
+    g = orc.geometry(nlat_in, nlon_in, nlat_out, nlon_out, EQ, EQ, 0.6)
+    torch.manual_seed(5)
+    with sna.Plan(nlat_in, nlon_in, nlat_out, nlon_out, EQ, EQ, 0.6) as plan:
+        layer = SphericalNeighborhoodAttention(plan, cin, heads, hd).cuda()
+        prev = torch.backends.cudnn.allow_tf32, torch.backends.cuda.matmul.allow_tf32
+        torch.backends.cudnn.allow_tf32 = torch.backends.cuda.matmul.allow_tf32 = False
+        try:
+            xq = torch.randn(2, cin, nlat_out, nlon_out, device="cuda", requires_grad=True)
+            xkv = torch.randn(2, cin, nlat_in, nlon_in, device="cuda", requires_grad=True)
+            y = layer(xq, xkv)
+            y.square().sum().backward()
+            torch.cuda.synchronize()
+        finally:
+            torch.backends.cudnn.allow_tf32, torch.backends.cuda.matmul.allow_tf32 = prev
+    f64 = lambda t: t.detach().cpu().double().numpy()
+    proj = lambda x, w, b: np.einsum("oi,bihw->bohw", f64(w)[:, :, 0, 0], x) + f64(b)[None, :, None, None]
+    heads_last = lambda t: t.reshape(t.shape[0], heads, hd, t.shape[2], t.shape[3]).transpose(0, 1, 3, 4, 2)   # [B, H, lat, lon, C]
+    q, k, v = (heads_last(proj(f64(x), w, b)) for x, w, b in ((xq, layer.wq, layer.bq), (xkv, layer.wk, layer.bk), (xkv, layer.wv, layer.bv)))
+    att = orc.forward(g, q, k, v).reshape(2, heads, nlat_out, nlon_out, hd).transpose(0, 1, 4, 2, 3).reshape(2, heads * hd, nlat_out, nlon_out)
+    ref = proj(att, layer.wo, layer.bo)
+    assert nerr(f64(y), ref) <= 2e-5
+    assert all(p.grad is not None and torch.isfinite(p.grad).all() for p in layer.parameters())
+    assert xq.grad is not None and xkv.grad is not None and float(xkv.grad.abs().max()) > 0
+
+
 def test_results_are_reproducible_bit_for_bit():
     wl = SMALL[2]
     q, k, v, dout = make_inputs(wl)
