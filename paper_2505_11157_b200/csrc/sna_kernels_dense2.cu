@@ -108,6 +108,47 @@ __device__ __forceinline__ void mma_ts(uint32_t d, uint32_t a_tmem, uint64_t b, 
     asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\ttcgen05.mma.cta_group::1.kind::tf32 [%0], [%1], %2, %3, {%5, %5, %5, %5}, p;\n\t}\n"
                  ::"r"(d), "r"(a_tmem), "l"(b), "r"(idesc), "r"(acc), "r"(0u));
 }
+// byte offset of the 16-byte chunk c4 of row `row` in a K-major tile with 128-byte swizzle
+__device__ __forceinline__ int sw_off(int row, int c4) { return row * 128 + ((c4 ^ (row & 7)) << 4); }
+// BF16 UMMA (K = 16 per instruction) for the two correction terms of a product at once: the 16 k-slots of a step hold
+// [a_lo(8) | a_hi(8)] on the A side against [b_hi(8) ; b_lo(8)] on the B side, so one instruction adds a_lo*b_hi + a_hi*b_lo
+// for 8 contraction indices.  The corrections are ~2^-11 of the product, so BF16's 8 bits leave ~2^-19 relative error:
+// used by the backward kernels (gate 1e-4); the forward scores keep three TF32 products.  A step is 32 bytes, like a TF32 step.
+__device__ __forceinline__ uint32_t idesc_bf16(int n) {
+    return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(M2 >> 4) << 24);
+}
+__device__ __forceinline__ void mma_ts16(uint32_t d, uint32_t a_tmem, uint64_t b, uint32_t idesc, uint32_t acc) {
+    asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\ttcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, {%5, %5, %5, %5}, p;\n\t}\n"
+                 ::"r"(d), "r"(a_tmem), "l"(b), "r"(idesc), "r"(acc), "r"(0u));
+}
+// {low half = bf16(x0), high half = bf16(x1)}, round to nearest
+__device__ __forceinline__ uint32_t bf16x2(float x0, float x1) {
+    uint32_t r;
+    asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(x1), "f"(x0));
+    return r;
+}
+// Stacked A operand in TMEM: per group of 8 channels, 4 words of lo pairs then 4 words of hi pairs (src: the 32 raw words).
+__device__ __forceinline__ void pack_a16(const uint32_t (&src)[32], uint32_t (&dst)[32]) {
+#pragma unroll
+    for (int gq = 0; gq < 4; ++gq) {
+        float hi[8], lo[8];
+#pragma unroll
+        for (int i = 0; i < 8; ++i) { hi[i] = trunc19f(__uint_as_float(src[gq * 8 + i])); lo[i] = __uint_as_float(src[gq * 8 + i]) - hi[i]; }
+#pragma unroll
+        for (int i = 0; i < 4; ++i) { dst[gq * 8 + i] = bf16x2(lo[2 * i], lo[2 * i + 1]); dst[gq * 8 + 4 + i] = bf16x2(hi[2 * i], hi[2 * i + 1]); }
+    }
+}
+// Stacked B tile beside a raw K-major tile: for point `row` and channel group `grp` (8 channels = the raw chunks 2 grp and
+// 2 grp + 1) the chunk 2 grp receives the 8 hi parts and the chunk 2 grp + 1 the 8 lo parts, as BF16.
+__device__ __forceinline__ void stack_b16(const unsigned char* raw, unsigned char* dst, int row, int grp) {
+    const float4 a = *reinterpret_cast<const float4*>(raw + sw_off(row, 2 * grp)), b = *reinterpret_cast<const float4*>(raw + sw_off(row, 2 * grp + 1));
+    const float x[8] = {a.x, a.y, a.z, a.w, b.x, b.y, b.z, b.w};
+    float hi[8], lo[8];
+#pragma unroll
+    for (int i = 0; i < 8; ++i) { hi[i] = trunc19f(x[i]); lo[i] = x[i] - hi[i]; }
+    *reinterpret_cast<uint4*>(dst + sw_off(row, 2 * grp)) = make_uint4(bf16x2(hi[0], hi[1]), bf16x2(hi[2], hi[3]), bf16x2(hi[4], hi[5]), bf16x2(hi[6], hi[7]));
+    *reinterpret_cast<uint4*>(dst + sw_off(row, 2 * grp + 1)) = make_uint4(bf16x2(lo[0], lo[1]), bf16x2(lo[2], lo[3]), bf16x2(lo[4], lo[5]), bf16x2(lo[6], lo[7]));
+}
 __device__ __forceinline__ void mma_commit(uint32_t bar) {
     asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
 }
@@ -131,7 +172,6 @@ __device__ __forceinline__ void tm_st32(uint32_t addr, const uint32_t (&r)[32]) 
         :: "r"(addr), "r"(r[0]),"r"(r[1]),"r"(r[2]),"r"(r[3]),"r"(r[4]),"r"(r[5]),"r"(r[6]),"r"(r[7]),"r"(r[8]),"r"(r[9]),"r"(r[10]),"r"(r[11]),"r"(r[12]),"r"(r[13]),"r"(r[14]),"r"(r[15]),
            "r"(r[16]),"r"(r[17]),"r"(r[18]),"r"(r[19]),"r"(r[20]),"r"(r[21]),"r"(r[22]),"r"(r[23]),"r"(r[24]),"r"(r[25]),"r"(r[26]),"r"(r[27]),"r"(r[28]),"r"(r[29]),"r"(r[30]),"r"(r[31]) : "memory");
 }
-__device__ __forceinline__ int sw_off(int row, int c4) { return row * 128 + ((c4 ^ (row & 7)) << 4); }
 
 __device__ __forceinline__ int fdiv(int a, int b) { const int q = a / b; return (a % b != 0 && ((a < 0) != (b < 0))) ? q - 1 : q; }
 __device__ __forceinline__ int cdiv(int a, int b) { return -fdiv(-a, b); }
@@ -611,14 +651,13 @@ backward_dq_dense2_kernel(DevPlan p, const __grid_constant__ CUtensorMap map_k, 
             }
             tm_st32(tm + TQ_AQ + lanebits, xq);
             tm_st32(tm + TQ_AY + lanebits, xy);
-#pragma unroll
-            for (int j = 0; j < 32; ++j) {
-                const float a = __uint_as_float(xq[j]), b = __uint_as_float(xy[j]);
-                xq[j] = __float_as_uint(a - trunc19f(a));
-                xy[j] = __float_as_uint(b - trunc19f(b));
+            {   // the stacked BF16 operands of the correction UMMAs
+                uint32_t pk[32];
+                pack_a16(xq, pk);
+                tm_st32(tm + TQ_AQL + lanebits, pk);
+                pack_a16(xy, pk);
+                tm_st32(tm + TQ_AYL + lanebits, pk);
             }
-            tm_st32(tm + TQ_AQL + lanebits, xq);
-            tm_st32(tm + TQ_AYL + lanebits, xy);
             asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
             asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
             mb_arrive(s32(&bars[Q_AREADY]));
@@ -727,7 +766,7 @@ backward_dq_dense2_kernel(DevPlan p, const __grid_constant__ CUtensorMap map_k, 
             // -------------------------------------------------------------- S = Q K^T (warp 9) and T = dY V^T (warp 10)
             const bool isT = warp == 10;
             ok = mb_wait(s32(&bars[Q_AREADY]), 0, ok);
-            const uint32_t idS = idesc_tf32(BNQ);
+            const uint32_t idS = idesc_tf32(BNQ), idS16 = idesc_bf16(BNQ);
             const uint32_t tA = tm + (isT ? TQ_AY : TQ_AQ), tAl = tm + (isT ? TQ_AYL : TQ_AQL);
             for (int it = 0; it < total && ok; ++it) {
                 const int s = it % NSQ, us = it / NSQ, b = it & 1, u = it >> 1;
@@ -742,9 +781,7 @@ backward_dq_dense2_kernel(DevPlan p, const __grid_constant__ CUtensorMap map_k, 
                 const uint64_t db = desc_k(tile0), dbl = desc_k(tile0 + TILE_Q);
                 const uint32_t tD = tm + TQ_BUF + 128 * b + (isT ? BNQ : 0);
 #pragma unroll
-                for (int ks = 0; ks < C2 / 8; ++ks) mma_ts(tD, tAl + ks * 8, db + 2 * ks, idS, ks > 0);
-#pragma unroll
-                for (int ks = 0; ks < C2 / 8; ++ks) mma_ts(tD, tA + ks * 8, dbl + 2 * ks, idS, 1);
+                for (int ks = 0; ks < C2 / 8; ++ks) mma_ts16(tD, tAl + ks * 8, dbl + 2 * ks, idS16, ks > 0);     // a_lo b_hi + a_hi b_lo
 #pragma unroll
                 for (int ks = 0; ks < C2 / 8; ++ks) mma_ts(tD, tA + ks * 8, db + 2 * ks, idS, 1);
                 mma_commit(s32(&bars[Q_STFULL + b]));
@@ -782,7 +819,6 @@ backward_dq_dense2_kernel(DevPlan p, const __grid_constant__ CUtensorMap map_k, 
         asm volatile("setmaxnreg.dec.sync.aligned.u32 80;");
         // ------------------------------------------------------------------ converters (warps 16-19, 128 threads)
         const int ct = tid - 512, cw = ct >> 5;
-        auto lo4 = [](const float4& x) { return make_float4(x.x - trunc19f(x.x), x.y - trunc19f(x.y), x.z - trunc19f(x.z), x.w - trunc19f(x.w)); };
         for (int it = 0; it < total && ok; ++it) {
             const int s = it % NSQ, u = it / NSQ;
             unsigned char* st = base + s * QST;
@@ -790,10 +826,7 @@ backward_dq_dense2_kernel(DevPlan p, const __grid_constant__ CUtensorMap map_k, 
             // lane = channel
             PROF_WAIT(0, ok = mb_wait(s32(&bars[Q_KFULL + s]), u & 1, ok));
 #pragma unroll
-            for (int j = 0; j < 4; ++j) {
-                const int off = (j * 128 + ct) * 16;
-                *reinterpret_cast<float4*>(st + TILE_Q + off) = lo4(*reinterpret_cast<const float4*>(st + off));
-            }
+            for (int j = 0; j < BNQ * 4 / 128; ++j) stack_b16(st, st + TILE_Q, (j * 128 + ct) >> 2, ct & 3);
             {
                 unsigned char* kth = st + 4 * TILE_Q + (cw >> 1) * (C2 * 128);
 #pragma unroll
@@ -816,10 +849,7 @@ backward_dq_dense2_kernel(DevPlan p, const __grid_constant__ CUtensorMap map_k, 
             // v_lo
             PROF_WAIT(1, ok = mb_wait(s32(&bars[Q_VFULL + s]), u & 1, ok) && ok);
 #pragma unroll
-            for (int j = 0; j < 4; ++j) {
-                const int off = (j * 128 + ct) * 16;
-                *reinterpret_cast<float4*>(st + 3 * TILE_Q + off) = lo4(*reinterpret_cast<const float4*>(st + 2 * TILE_Q + off));
-            }
+            for (int j = 0; j < BNQ * 4 / 128; ++j) stack_b16(st + 2 * TILE_Q, st + 3 * TILE_Q, (j * 128 + ct) >> 2, ct & 3);
             asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
             mb_arrive(s32(&bars[Q_VCONV + s]));
         }
@@ -940,14 +970,13 @@ backward_dkdv_dense2_kernel(DevPlan p, const __grid_constant__ CUtensorMap map_q
             }
             tm_st32(tm + TK_AK + lanebits, xk);
             tm_st32(tm + TK_AV + lanebits, xv);
-#pragma unroll
-            for (int j = 0; j < 32; ++j) {
-                const float a = __uint_as_float(xk[j]), b = __uint_as_float(xv[j]);
-                xk[j] = __float_as_uint(a - trunc19f(a));
-                xv[j] = __float_as_uint(b - trunc19f(b));
+            {   // the stacked BF16 operands of the correction UMMAs
+                uint32_t pk[32];
+                pack_a16(xk, pk);
+                tm_st32(tm + TK_AKL + lanebits, pk);
+                pack_a16(xv, pk);
+                tm_st32(tm + TK_AVL + lanebits, pk);
             }
-            tm_st32(tm + TK_AKL + lanebits, xk);
-            tm_st32(tm + TK_AVL + lanebits, xv);
             asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
             asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
             mb_arrive(s32(&bars[K_AREADY]));
@@ -1063,7 +1092,7 @@ backward_dkdv_dense2_kernel(DevPlan p, const __grid_constant__ CUtensorMap map_q
             // -------------------------------------------------------------- S^T = K Q^T (warp 9) and T^T = V dY^T (warp 10)
             const bool isT = warp == 10;
             ok = mb_wait(s32(&bars[K_AREADY]), 0, ok);
-            const uint32_t idS = idesc_tf32(BNK);
+            const uint32_t idS = idesc_tf32(BNK), idS16 = idesc_bf16(BNK);
             const uint32_t tA = tm + (isT ? TK_AV : TK_AK), tAl = tm + (isT ? TK_AVL : TK_AKL);
             for (int it = 0; it < total && ok; ++it) {
                 const int s = it % NSK, us = it / NSK, b = it & 1, u = it >> 1;
@@ -1078,9 +1107,7 @@ backward_dkdv_dense2_kernel(DevPlan p, const __grid_constant__ CUtensorMap map_q
                 const uint64_t db = desc_k(tile0), dbl = desc_k(tile0 + TILE_K);
                 const uint32_t tD = tm + TK_BUF + 128 * b + (isT ? TK_T : TK_S);
 #pragma unroll
-                for (int ks = 0; ks < C2 / 8; ++ks) mma_ts(tD, tAl + ks * 8, db + 2 * ks, idS, ks > 0);
-#pragma unroll
-                for (int ks = 0; ks < C2 / 8; ++ks) mma_ts(tD, tA + ks * 8, dbl + 2 * ks, idS, 1);
+                for (int ks = 0; ks < C2 / 8; ++ks) mma_ts16(tD, tAl + ks * 8, dbl + 2 * ks, idS16, ks > 0);     // a_lo b_hi + a_hi b_lo
 #pragma unroll
                 for (int ks = 0; ks < C2 / 8; ++ks) mma_ts(tD, tA + ks * 8, db + 2 * ks, idS, 1);
                 mma_commit(s32(&bars[K_STFULL + b]));
@@ -1118,15 +1145,11 @@ backward_dkdv_dense2_kernel(DevPlan p, const __grid_constant__ CUtensorMap map_q
         asm volatile("setmaxnreg.dec.sync.aligned.u32 72;");
         // ------------------------------------------------------------------ converters (warps 16-19, 128 threads)
         const int ct = tid - 512, cw = ct >> 5;
-        auto lo4 = [](const float4& x) { return make_float4(x.x - trunc19f(x.x), x.y - trunc19f(x.y), x.z - trunc19f(x.z), x.w - trunc19f(x.w)); };
         // lo tile (same swizzled positions) and transposed hi / lo tiles of one raw tile (one K block of 32 points: row =
         // channel, 128 bytes of points): warp cw takes the 8 columns [8 cw, 8 cw + 8), lane = channel
         auto convert = [&](unsigned char* raw, unsigned char* lo, unsigned char* th) {
 #pragma unroll
-            for (int j = 0; j < TILE_K / (128 * 16); ++j) {
-                const int off = (j * 128 + ct) * 16;
-                *reinterpret_cast<float4*>(lo + off) = lo4(*reinterpret_cast<const float4*>(raw + off));
-            }
+            for (int j = 0; j < BNK * 4 / 128; ++j) stack_b16(raw, lo, (j * 128 + ct) >> 2, ct & 3);
 #pragma unroll
             for (int c8 = 0; c8 < 2; ++c8) {
                 float hi[4], lw[4];
