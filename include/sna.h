@@ -152,7 +152,7 @@ sna_status_t sna_forward(const sna_plan_t* plan, const float* q, const float* k,
                          int B, int H, int C, void* cuda_stream);
 
 /* Number of GPU kernels sna_forward_ex launches for this plan and channel count (with_lse != 0: an lse buffer is
- * passed).  1, or 2 when the whole-ring windows take the dense tensor-core kernel first.  0 for invalid arguments. */
+ * passed).  1, or 2 when whole-ring and wide windows take the dense tensor-core kernel first.  0 for invalid arguments. */
 int sna_forward_kernel_count(const sna_plan_t* plan, int C, int with_lse);
 
 /* Forward pass that also stores lse[n,h,w] = log(sum_j exp(s_j) omega_j) (device, may be NULL), which the

@@ -162,7 +162,7 @@ static sna_status_t plan_create(int nlat_in, int nlon_in, int nlat_out, int nlon
     try {
         sna::build_dense_lists(hp, dense, dense_min_width);
         sna::build_transposed_dense_lists(hp, t_dense, dense_min_width);
-        // rows with the most whole rings first: the dense kernels run one block per SM, so the long tiles must not start last
+        // rows with the longest lists first: the dense kernels run one block per SM, so the long tiles must not start last
         std::stable_sort(dense.rows.begin(), dense.rows.end(), [&](int a, int b) { return dense.ptr[a + 1] - dense.ptr[a] > dense.ptr[b + 1] - dense.ptr[b]; });
         std::stable_sort(t_dense.rows.begin(), t_dense.rows.end(), [&](int a, int b) { return t_dense.ptr[a + 1] - t_dense.ptr[a] > t_dense.ptr[b + 1] - t_dense.ptr[b]; });
         if (global) {
@@ -409,7 +409,7 @@ sna_status_t sna_forward_ex(const sna_plan_t* plan, const float* q, const float*
                 ? sna::launch_forward_dense2(plan->dev, q, k, v, out, lse, B * H, C, (cudaStream_t)cuda_stream)
                 : sna::launch_forward_generic(plan->dev, q, k, v, out, lse, B * H, C, (cudaStream_t)cuda_stream);
     } else if (lse != nullptr && sna::dense2_path_supported(plan->dev, C)) {
-        // whole-ring windows on the tcgen05 kernel (its partial result travels in out / lse), the rest on the band kernel
+        // whole-ring and wide windows on the tcgen05 kernel (its partial result travels in out / lse), the rest on the band kernel
         e = sna::launch_forward_dense2(plan->dev, q, k, v, out, lse, B * H, C, (cudaStream_t)cuda_stream);
         if (e == cudaSuccess) e = sna::launch_forward_mma_band(plan->dev, q, k, v, out, lse, B * H, C, (cudaStream_t)cuda_stream);
     } else if (sna::mma_path_supported(plan->dev, C)) {
@@ -434,14 +434,14 @@ sna_status_t sna_backward_dq(const sna_plan_t* plan, const float* q, const float
     if (!q || !k || !v || !dout || !lse || !dq || !D) { set_error("q, k, v, dout, lse, dq and D must not be NULL"); return SNA_ERR_INVALID_ARG; }
     if (!all_aligned(q, k, v, dout, dq, out) || ((reinterpret_cast<uintptr_t>(lse) | reinterpret_cast<uintptr_t>(D)) & 3u)) { set_error("device pointers must be 16-byte aligned"); return SNA_ERR_INVALID_ARG; }
     cudaError_t e;
-    // The dense dq kernel takes the whole-ring windows when they are at least a tenth of the work (measured on the
+    // The dense dq kernel takes the whole-ring and wide windows when they are at least a tenth of the work (measured on the
     // benchmark configurations: -8 % on the dq stage at a 22 % share, -6 % at 13 %).
     if (plan->is_global) {
         e = (out != nullptr && out != dq && sna::dense2_global_supported(plan->dev, C))
                 ? sna::launch_backward_dq_dense2(plan->dev, q, k, v, dout, out, lse, dq, D, B * H, C, (cudaStream_t)cuda_stream)
                 : sna::launch_backward_dq_generic(plan->dev, q, k, v, dout, out, lse, dq, D, B * H, C, (cudaStream_t)cuda_stream);
     } else if (out != nullptr && out != dq && plan->dev.dense_fraction >= 0.10f && sna::dense2_path_supported(plan->dev, C)) {
-        // whole-ring windows on the tcgen05 kernel (its part of dq is written first), the banded rest is added by the band kernel
+        // whole-ring and wide windows on the tcgen05 kernel (its part of dq is written first), the rest is added by the band kernel
         e = sna::launch_backward_dq_dense2(plan->dev, q, k, v, dout, out, lse, dq, nullptr, B * H, C, (cudaStream_t)cuda_stream);
         if (e == cudaSuccess) e = sna::launch_backward_dq_mma_band(plan->dev, q, k, v, dout, out, lse, dq, D, B * H, C, (cudaStream_t)cuda_stream);
     } else if (out != nullptr && sna::mma_path_supported(plan->dev, C)) {
@@ -475,7 +475,7 @@ sna_status_t sna_backward_dkdv(const sna_plan_t* plan, const float* q, const flo
                 ? sna::launch_backward_dkdv_dense2(plan->dev, q, k, v, dout, lse, D, dk, dv, B * H, C, (cudaStream_t)cuda_stream)
                 : sna::launch_backward_dkdv_generic(plan->dev, q, k, v, dout, lse, D, dk, dv, B * H, C, (cudaStream_t)cuda_stream);
     } else if (plan->dev.dense_fraction >= 0.10f && plan->dev.n_t_dense_rows > 0 && sna::dense2_path_supported(plan->dev, C)) {
-        // whole-ring partners on the tcgen05 kernel (its part of dk, dv is written first), the band kernel adds the rest
+        // whole-ring and wide windows on the tcgen05 kernel (its part of dk, dv is written first), the band kernel adds the rest
         e = sna::launch_backward_dkdv_dense2(plan->dev, q, k, v, dout, lse, D, dk, dv, B * H, C, (cudaStream_t)cuda_stream);
         if (e == cudaSuccess) e = sna::launch_backward_dkdv_mma_band(plan->dev, q, k, v, dout, lse, D, dk, dv, B * H, C, (cudaStream_t)cuda_stream);
     } else if (sna::mma_path_supported(plan->dev, C)) {

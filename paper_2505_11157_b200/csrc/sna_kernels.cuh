@@ -23,14 +23,14 @@ struct DevPlan {
     const int4* fwd_stream;         // 16 entries per chunk: {base|abs flag, e | mask<<16, bias, aux}
     const int32_t* fwd_chunk_ptr;   // [groups of output latitudes + 1]
     const int32_t* grp_order;       // groups of output latitudes, longest stream first
-    // band-only forward stream (whole-ring windows left to the dense kernel) and the dense kernel's lists
+    // band-only forward stream (whole-ring and wide windows left to the dense kernel) and the dense kernel's lists
     const int4* fwdb_stream;
     const int32_t* fwdb_chunk_ptr;
     const int32_t* grpb_order;
     const int32_t* dense_ptr;       // [nlat_out+1] the dense kernels' windows per output latitude
     const int32_t* dense_lat;       // their input rings
     const int32_t* dense_m;         // their half widths in input columns, -1 = whole ring
-    const int32_t* dense_rows;      // output latitudes with at least one whole-ring window
+    const int32_t* dense_rows;      // output latitudes with at least one such window
     int n_dense_rows;
     // the same for the transposed side (dk/dv): band-only transposed stream and, per input latitude, the output rings
     // that attend to it as a whole

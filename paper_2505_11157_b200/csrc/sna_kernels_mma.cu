@@ -183,7 +183,7 @@ __device__ __forceinline__ bool decode_task(int N, int tiles_per_row, long long 
 
 
 // The column stream a forward launch walks: the full one, or the band-only one when the dense kernel has already
-// produced the whole-ring part (dense_ptr != null: rows with whole-ring windows start from that partial result).
+// produced its part (dense_ptr != null: rows with windows on the dense kernel start from that partial result).
 struct FwdView {
     const int4* stream;
     const int32_t* chunk_ptr;
@@ -415,7 +415,7 @@ backward_dq_mma_kernel(DevPlan p, FwdView fv, const float* __restrict__ q, const
         r1v[nt] = acc[nt][2] * scale; r1v[KS + nt] = acc[nt][3] * scale;
     }
     if (fv.dense_ptr != nullptr) {
-        // the dense kernel has already written the whole-ring part of dq for rows that have such windows: add it
+        // the dense kernel has already written its part of dq for rows that have windows there: add it
         const int ha = hg * TILE_LAT, hb = min(hg * TILE_LAT + 1, p.nlat_out - 1);
         if (fv.dense_ptr[ha + 1] > fv.dense_ptr[ha]) {
             float r[CPT];
@@ -537,7 +537,7 @@ backward_dkdv_mma_kernel(DevPlan p, FwdView tv, const float* __restrict__ q, con
         b0[nt] = gv[nt][0]; b0[KS + nt] = gv[nt][1]; b1[nt] = gv[nt][2]; b1[KS + nt] = gv[nt][3];
     }
     if (tv.dense_ptr != nullptr) {
-        // the dense kernel has already written the whole-ring part of dk, dv for input rings that have such partners
+        // the dense kernel has already written its part of dk, dv for input rings that have windows there
         if (tv.dense_ptr[hp0 + 1] > tv.dense_ptr[hp0]) {
             float r[CPT];
             load_row<CPT>(dk + pt0 * C + t * CPT, r);
