@@ -30,6 +30,7 @@
 #include "sna_kernels.cuh"
 
 #include <cstdint>
+#include <type_traits>
 
 // Optional per-role wait accounting (build with -DSNA_PROF; not part of the product build): every role of block 0 writes
 // its total cycles and the cycles spent in up to three kinds of waits to the plan's status area.
@@ -234,6 +235,10 @@ __device__ __forceinline__ int tile_block_count(const int32_t* lat, const int32_
     return cnt;
 }
 
+// SPLIT: two instantiations of the second softmax pass, with and without the per-element window test, chosen per block.
+// It pays when (nearly) every block is unmasked - plans whose windows are all whole rings: -4 % - and costs 2 % where
+// masked and unmasked blocks alternate (the unrolled pass is long), so the launcher sets it for all-whole plans only.
+template <bool SPLIT>
 __global__ void __launch_bounds__(THREADS2, 1)
 forward_dense2_kernel(DevPlan p, const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
                       const __grid_constant__ CUtensorMap map_v, float* __restrict__ out, float* __restrict__ lse, int N,
@@ -356,30 +361,34 @@ forward_dense2_kernel(DevPlan p, const __grid_constant__ CUtensorMap map_q, cons
                 const float nb = bias - msafe;
                 // pass 2: P over S (its top 19 bits are the hi part) and P_lo = P - trunc19(P) beside it
                 float ps[4] = {0.f, 0.f, 0.f, 0.f};
-                uint32_t bufa[16], bufb[16];
-                auto softmax16 = [&](uint32_t (&x)[16], int c0) {
-                    uint32_t lo[16];
+                auto pass2 = [&](auto unmasked) {
+                    constexpr bool UNMASKED = decltype(unmasked)::value;
+                    uint32_t bufa[16], bufb[16];
+                    auto softmax16 = [&](uint32_t (&x)[16], int c0) {
+                        uint32_t lo[16];
 #pragma unroll
-                    for (int j = 0; j < 16; ++j) {
-                        float pj = ex2f(fmaf(__uint_as_float(x[j]), scale_log2, nb));
-                        if (!full && (uint32_t)(c0 + j - jl) > span) pj = 0.f;
-                        ps[j & 3] += pj;
-                        x[j] = __float_as_uint(pj);
-                        lo[j] = __float_as_uint(pj - trunc19f(pj));
+                        for (int j = 0; j < 16; ++j) {
+                            float pj = ex2f(fmaf(__uint_as_float(x[j]), scale_log2, nb));
+                            if (!UNMASKED && !full && (uint32_t)(c0 + j - jl) > span) pj = 0.f;
+                            ps[j & 3] += pj;
+                            x[j] = __float_as_uint(pj);
+                            lo[j] = __float_as_uint(pj - trunc19f(pj));
+                        }
+                        tm_st16(tS + c0, x);
+                        tm_st16(tm + T_PLO + half * HC + lanebits + c0, lo);
+                    };
+                    tm_ld16_issue(bufa, tS);
+#pragma unroll
+                    for (int c0 = 0; c0 < HC; c0 += 32) {
+                        tm_ld_wait();
+                        tm_ld16_issue(bufb, tS + c0 + 16);            // in flight while the first 16 columns are processed
+                        softmax16(bufa, c0);
+                        tm_ld_wait();
+                        if (c0 + 32 < HC) tm_ld16_issue(bufa, tS + c0 + 32);
+                        softmax16(bufb, c0 + 16);
                     }
-                    tm_st16(tS + c0, x);
-                    tm_st16(tm + T_PLO + half * HC + lanebits + c0, lo);
                 };
-                tm_ld16_issue(bufa, tS);
-#pragma unroll
-                for (int c0 = 0; c0 < HC; c0 += 32) {
-                    tm_ld_wait();
-                    tm_ld16_issue(bufb, tS + c0 + 16);            // in flight while the first 16 columns are processed
-                    softmax16(bufa, c0);
-                    tm_ld_wait();
-                    if (c0 + 32 < HC) tm_ld16_issue(bufa, tS + c0 + 32);
-                    softmax16(bufb, c0 + 16);
-                }
+                if (SPLIT && full) pass2(std::true_type{}); else pass2(std::false_type{});
                 l = fmaf(l, corr, (ps[0] + ps[1]) + (ps[2] + ps[3]));
                 asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
                 asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
@@ -695,14 +704,19 @@ backward_dq_dense2_kernel(DevPlan p, const __grid_constant__ CUtensorMap map_k, 
                 tm_ld32_issue(sv, tS);
                 tm_ld32_issue(tv, tT);
                 tm_ld_wait();
+                // (two instantiations: blocks in which no row of the warp is masked skip the per-element range test)
+                auto elementwise = [&](auto unmasked) {
+                    constexpr bool UNMASKED = decltype(unmasked)::value;
 #pragma unroll
-                for (int j = 0; j < 32; ++j) {
-                    float pj = ex2f(fmaf(__uint_as_float(sv[j]), scale_log2, nbias));
-                    if (!full && (uint32_t)(j - jl) > span) pj = 0.f;
-                    const float ds = pj * (__uint_as_float(tv[j]) - D);
-                    sv[j] = __float_as_uint(ds);                       // dS over S
-                    tv[j] = __float_as_uint(ds - trunc19f(ds));        // dS_lo over T
-                }
+                    for (int j = 0; j < 32; ++j) {
+                        float pj = ex2f(fmaf(__uint_as_float(sv[j]), scale_log2, nbias));
+                        if (!UNMASKED && (uint32_t)(j - jl) > span) pj = 0.f;
+                        const float ds = pj * (__uint_as_float(tv[j]) - D);
+                        sv[j] = __float_as_uint(ds);                       // dS over S
+                        tv[j] = __float_as_uint(ds - trunc19f(ds));        // dS_lo over T
+                    }
+                };
+                if (full) elementwise(std::true_type{}); else elementwise(std::false_type{});
                 tm_st32(tS, sv);
                 tm_st32(tT, tv);
             }
@@ -1029,17 +1043,22 @@ backward_dkdv_dense2_kernel(DevPlan p, const __grid_constant__ CUtensorMap map_q
                         Dv[4 * q4] = d4.x; Dv[4 * q4 + 1] = d4.y; Dv[4 * q4 + 2] = d4.z; Dv[4 * q4 + 3] = d4.w;
                     }
                     tm_ld_wait();
+                    // (two instantiations: blocks in which no row of the warp is masked skip the per-element range test)
+                    auto elementwise = [&](auto unmasked) {
+                        constexpr bool UNMASKED = decltype(unmasked)::value;
 #pragma unroll
-                    for (int j = 0; j < 16; ++j) {
-                        const int col = hf * 16 + j;
-                        float pj = ex2f(fmaf(__uint_as_float(sv[j]), scale_log2, nlv[j]));
-                        if (!full && (uint32_t)(col - jl) > span) pj = 0.f;
-                        const float ds = pj * (__uint_as_float(tv[j]) - Dv[j]);
-                        sv[j] = __float_as_uint(pj);
-                        tv[j] = __float_as_uint(ds);
-                        pl[j] = __float_as_uint(pj - trunc19f(pj));
-                        dl[j] = __float_as_uint(ds - trunc19f(ds));
-                    }
+                        for (int j = 0; j < 16; ++j) {
+                            const int col = hf * 16 + j;
+                            float pj = ex2f(fmaf(__uint_as_float(sv[j]), scale_log2, nlv[j]));
+                            if (!UNMASKED && (uint32_t)(col - jl) > span) pj = 0.f;
+                            const float ds = pj * (__uint_as_float(tv[j]) - Dv[j]);
+                            sv[j] = __float_as_uint(pj);
+                            tv[j] = __float_as_uint(ds);
+                            pl[j] = __float_as_uint(pj - trunc19f(pj));
+                            dl[j] = __float_as_uint(ds - trunc19f(ds));
+                        }
+                    };
+                    if (full) elementwise(std::true_type{}); else elementwise(std::false_type{});
                     tm_st16(tS + hf * 16, sv);
                     tm_st16(tT + hf * 16, tv);
                     tm_st16(tPl + hf * 16, pl);
@@ -1226,7 +1245,8 @@ cudaError_t make_map2(CUtensorMap* map, const float* base, int rings_total, int 
 }  // namespace
 
 cudaError_t dense2_prepare_device() {
-    cudaError_t e = cudaFuncSetAttribute(forward_dense2_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)DENSE2_SMEM);
+    cudaError_t e = cudaFuncSetAttribute(forward_dense2_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)DENSE2_SMEM);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(forward_dense2_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)DENSE2_SMEM);
     if (e == cudaSuccess) e = cudaFuncSetAttribute(backward_dq_dense2_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)DQ2_SMEM);
     if (e == cudaSuccess) e = cudaFuncSetAttribute(backward_dkdv_dense2_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)DKDV2_SMEM);
     return e;
@@ -1302,7 +1322,10 @@ cudaError_t launch_forward_dense2(const DevPlan& p, const float* q, const float*
     if (e == cudaSuccess) e = make_map2(&mk, k, N * p.nlat_in, p.nlon_in);
     if (e == cudaSuccess) e = make_map2(&mv, v, N * p.nlat_in, p.nlon_in);
     if (e != cudaSuccess) return e;
-    forward_dense2_kernel<<<(unsigned)blocks, THREADS2, DENSE2_SMEM, stream>>>(p, mq, mk, mv, out, lse, N, LOG2E_2 / sqrtf((float)C), tiles_per_row);
+    if (p.dense_fraction >= 0.999f)   // every window is a whole ring
+        forward_dense2_kernel<true><<<(unsigned)blocks, THREADS2, DENSE2_SMEM, stream>>>(p, mq, mk, mv, out, lse, N, LOG2E_2 / sqrtf((float)C), tiles_per_row);
+    else
+        forward_dense2_kernel<false><<<(unsigned)blocks, THREADS2, DENSE2_SMEM, stream>>>(p, mq, mk, mv, out, lse, N, LOG2E_2 / sqrtf((float)C), tiles_per_row);
     return cudaGetLastError();
 }
 
