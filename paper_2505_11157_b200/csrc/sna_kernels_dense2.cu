@@ -111,6 +111,13 @@ __device__ __forceinline__ void mma_ts(uint32_t d, uint32_t a_tmem, uint64_t b, 
 }
 // byte offset of the 16-byte chunk c4 of row `row` in a K-major tile with 128-byte swizzle
 __device__ __forceinline__ int sw_off(int row, int c4) { return row * 128 + ((c4 ^ (row & 7)) << 4); }
+// Packed fp32 pairs (Blackwell f32x2 arithmetic: one instruction for two lanes of a 64-bit register pair); the element-wise
+// loops are bound by issue slots, so halving their add / multiply / fma instructions pays.
+__device__ __forceinline__ uint64_t pack2(float a, float b) { uint64_t r; asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(a), "f"(b)); return r; }
+__device__ __forceinline__ void unpack2(uint64_t v, float& a, float& b) { asm("mov.b64 {%0, %1}, %2;" : "=f"(a), "=f"(b) : "l"(v)); }
+__device__ __forceinline__ uint64_t fma2(uint64_t a, uint64_t b, uint64_t c) { uint64_t d; asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c)); return d; }
+__device__ __forceinline__ uint64_t mul2(uint64_t a, uint64_t b) { uint64_t d; asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b)); return d; }
+__device__ __forceinline__ uint64_t sub2(uint64_t a, uint64_t b) { uint64_t d; asm("sub.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b)); return d; }
 // BF16 UMMA (K = 16 per instruction) for the two correction terms of a product at once: the 16 k-slots of a step hold
 // [a_lo(8) | a_hi(8)] on the A side against [b_hi(8) ; b_lo(8)] on the B side, so one instruction adds a_lo*b_hi + a_hi*b_lo
 // for 8 contraction indices.  The corrections are ~2^-11 of the product, so BF16's 8 bits leave ~2^-19 relative error:
@@ -707,13 +714,19 @@ backward_dq_dense2_kernel(DevPlan p, const __grid_constant__ CUtensorMap map_k, 
                 // (two instantiations: blocks in which no row of the warp is masked skip the per-element range test)
                 auto elementwise = [&](auto unmasked) {
                     constexpr bool UNMASKED = decltype(unmasked)::value;
+                    const uint64_t scale2 = pack2(scale_log2, scale_log2), nbias2 = pack2(nbias, nbias), D2 = pack2(D, D);
 #pragma unroll
-                    for (int j = 0; j < 32; ++j) {
-                        float pj = ex2f(fmaf(__uint_as_float(sv[j]), scale_log2, nbias));
-                        if (!UNMASKED && (uint32_t)(j - jl) > span) pj = 0.f;
-                        const float ds = pj * (__uint_as_float(tv[j]) - D);
-                        sv[j] = __float_as_uint(ds);                       // dS over S
-                        tv[j] = __float_as_uint(ds - trunc19f(ds));        // dS_lo over T
+                    for (int j = 0; j < 32; j += 2) {
+                        float x0, x1, ds0, ds1, l0, l1;
+                        unpack2(fma2(pack2(__uint_as_float(sv[j]), __uint_as_float(sv[j + 1])), scale2, nbias2), x0, x1);
+                        float p0 = ex2f(x0), p1 = ex2f(x1);
+                        if (!UNMASKED && (uint32_t)(j - jl) > span) p0 = 0.f;
+                        if (!UNMASKED && (uint32_t)(j + 1 - jl) > span) p1 = 0.f;
+                        const uint64_t ds2 = mul2(pack2(p0, p1), sub2(pack2(__uint_as_float(tv[j]), __uint_as_float(tv[j + 1])), D2));
+                        unpack2(ds2, ds0, ds1);
+                        unpack2(sub2(ds2, pack2(trunc19f(ds0), trunc19f(ds1))), l0, l1);
+                        sv[j] = __float_as_uint(ds0); sv[j + 1] = __float_as_uint(ds1);       // dS over S
+                        tv[j] = __float_as_uint(l0); tv[j + 1] = __float_as_uint(l1);         // dS_lo over T
                     }
                 };
                 if (full) elementwise(std::true_type{}); else elementwise(std::false_type{});
