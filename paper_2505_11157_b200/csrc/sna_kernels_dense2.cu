@@ -117,6 +117,7 @@ __device__ __forceinline__ uint64_t pack2(float a, float b) { uint64_t r; asm("m
 __device__ __forceinline__ void unpack2(uint64_t v, float& a, float& b) { asm("mov.b64 {%0, %1}, %2;" : "=f"(a), "=f"(b) : "l"(v)); }
 __device__ __forceinline__ uint64_t fma2(uint64_t a, uint64_t b, uint64_t c) { uint64_t d; asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c)); return d; }
 __device__ __forceinline__ uint64_t mul2(uint64_t a, uint64_t b) { uint64_t d; asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b)); return d; }
+__device__ __forceinline__ uint64_t add2(uint64_t a, uint64_t b) { uint64_t d; asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b)); return d; }
 __device__ __forceinline__ uint64_t sub2(uint64_t a, uint64_t b) { uint64_t d; asm("sub.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b)); return d; }
 // BF16 UMMA (K = 16 per instruction) for the two correction terms of a product at once: the 16 k-slots of a step hold
 // [a_lo(8) | a_hi(8)] on the A side against [b_hi(8) ; b_lo(8)] on the B side, so one instruction adds a_lo*b_hi + a_hi*b_lo
@@ -327,7 +328,10 @@ forward_dense2_kernel(DevPlan p, const __grid_constant__ CUtensorMap map_q, cons
                 tm_ld32_issue(ob, tm + T_O + half * 64 + 32 + lanebits);
                 tm_ld_wait();
 #pragma unroll
-                for (int j = 0; j < C2; ++j) o[j] = fmaf(o[j], corr_prev, __uint_as_float(oa[j]) + __uint_as_float(ob[j]));
+                for (int j = 0; j < C2; j += 2)
+                    unpack2(fma2(pack2(o[j], o[j + 1]), pack2(corr_prev, corr_prev),
+                                 add2(pack2(__uint_as_float(oa[j]), __uint_as_float(oa[j + 1])), pack2(__uint_as_float(ob[j]), __uint_as_float(ob[j + 1])))),
+                            o[j], o[j + 1]);
             }
             if (it < total) {
                 const int b = it & 1, u = it >> 1;
@@ -367,19 +371,25 @@ forward_dense2_kernel(DevPlan p, const __grid_constant__ CUtensorMap map_q, cons
                 m = mx;
                 const float nb = bias - msafe;
                 // pass 2: P over S (its top 19 bits are the hi part) and P_lo = P - trunc19(P) beside it
-                float ps[4] = {0.f, 0.f, 0.f, 0.f};
+                uint64_t ps2[2] = {pack2(0.f, 0.f), pack2(0.f, 0.f)};      // four running sums of P, as two packed pairs
                 auto pass2 = [&](auto unmasked) {
                     constexpr bool UNMASKED = decltype(unmasked)::value;
                     uint32_t bufa[16], bufb[16];
                     auto softmax16 = [&](uint32_t (&x)[16], int c0) {
                         uint32_t lo[16];
+                        const uint64_t scale2 = pack2(scale_log2, scale_log2), nb2 = pack2(nb, nb);
 #pragma unroll
-                        for (int j = 0; j < 16; ++j) {
-                            float pj = ex2f(fmaf(__uint_as_float(x[j]), scale_log2, nb));
-                            if (!UNMASKED && !full && (uint32_t)(c0 + j - jl) > span) pj = 0.f;
-                            ps[j & 3] += pj;
-                            x[j] = __float_as_uint(pj);
-                            lo[j] = __float_as_uint(pj - trunc19f(pj));
+                        for (int j = 0; j < 16; j += 2) {
+                            float x0, x1, l0, l1;
+                            unpack2(fma2(pack2(__uint_as_float(x[j]), __uint_as_float(x[j + 1])), scale2, nb2), x0, x1);
+                            float p0 = ex2f(x0), p1 = ex2f(x1);
+                            if (!UNMASKED && !full && (uint32_t)(c0 + j - jl) > span) p0 = 0.f;
+                            if (!UNMASKED && !full && (uint32_t)(c0 + j + 1 - jl) > span) p1 = 0.f;
+                            const uint64_t p2 = pack2(p0, p1);
+                            ps2[(j >> 1) & 1] = add2(ps2[(j >> 1) & 1], p2);
+                            unpack2(sub2(p2, pack2(trunc19f(p0), trunc19f(p1))), l0, l1);
+                            x[j] = __float_as_uint(p0); x[j + 1] = __float_as_uint(p1);
+                            lo[j] = __float_as_uint(l0); lo[j + 1] = __float_as_uint(l1);
                         }
                         tm_st16(tS + c0, x);
                         tm_st16(tm + T_PLO + half * HC + lanebits + c0, lo);
@@ -396,6 +406,9 @@ forward_dense2_kernel(DevPlan p, const __grid_constant__ CUtensorMap map_q, cons
                     }
                 };
                 if (SPLIT && full) pass2(std::true_type{}); else pass2(std::false_type{});
+                float ps[4];
+                unpack2(ps2[0], ps[0], ps[1]);
+                unpack2(ps2[1], ps[2], ps[3]);
                 l = fmaf(l, corr, (ps[0] + ps[1]) + (ps[2] + ps[3]));
                 asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
                 asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
@@ -744,7 +757,9 @@ backward_dq_dense2_kernel(DevPlan p, const __grid_constant__ CUtensorMap map_k, 
                 tm_ld32_issue(ob, tm + TQ_ACC + grp * 64 + 32 + lanebits);
                 tm_ld_wait();
 #pragma unroll
-                for (int j = 0; j < C2; ++j) acc[j] += __uint_as_float(oa[j]) + __uint_as_float(ob[j]);
+                for (int j = 0; j < C2; j += 2)
+                    unpack2(add2(pack2(acc[j], acc[j + 1]), add2(pack2(__uint_as_float(oa[j]), __uint_as_float(oa[j + 1])),
+                                                                 pack2(__uint_as_float(ob[j]), __uint_as_float(ob[j + 1])))), acc[j], acc[j + 1]);
             }
             if (it < total) {
                 asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
@@ -1024,7 +1039,10 @@ backward_dkdv_dense2_kernel(DevPlan p, const __grid_constant__ CUtensorMap map_q
                 tm_ld32_issue(ob, tm + TK_ACC + 64 + grp * 32 + lanebits);     // dK, this column half
                 tm_ld_wait();
 #pragma unroll
-                for (int j = 0; j < C2; ++j) { gv[j] += __uint_as_float(oa[j]); gk[j] += __uint_as_float(ob[j]); }
+                for (int j = 0; j < C2; j += 2) {
+                    unpack2(add2(pack2(gv[j], gv[j + 1]), pack2(__uint_as_float(oa[j]), __uint_as_float(oa[j + 1]))), gv[j], gv[j + 1]);
+                    unpack2(add2(pack2(gk[j], gk[j + 1]), pack2(__uint_as_float(ob[j]), __uint_as_float(ob[j + 1]))), gk[j], gk[j + 1]);
+                }
             }
             if (it < total) {
                 const int s = it % NSK, b = it & 1;
@@ -1059,16 +1077,24 @@ backward_dkdv_dense2_kernel(DevPlan p, const __grid_constant__ CUtensorMap map_q
                     // (two instantiations: blocks in which no row of the warp is masked skip the per-element range test)
                     auto elementwise = [&](auto unmasked) {
                         constexpr bool UNMASKED = decltype(unmasked)::value;
+                        const uint64_t scale2 = pack2(scale_log2, scale_log2);
 #pragma unroll
-                        for (int j = 0; j < 16; ++j) {
+                        for (int j = 0; j < 16; j += 2) {
                             const int col = hf * 16 + j;
-                            float pj = ex2f(fmaf(__uint_as_float(sv[j]), scale_log2, nlv[j]));
-                            if (!UNMASKED && (uint32_t)(col - jl) > span) pj = 0.f;
-                            const float ds = pj * (__uint_as_float(tv[j]) - Dv[j]);
-                            sv[j] = __float_as_uint(pj);
-                            tv[j] = __float_as_uint(ds);
-                            pl[j] = __float_as_uint(pj - trunc19f(pj));
-                            dl[j] = __float_as_uint(ds - trunc19f(ds));
+                            float x0, x1, ds0, ds1, a0, a1, b0, b1;
+                            unpack2(fma2(pack2(__uint_as_float(sv[j]), __uint_as_float(sv[j + 1])), scale2, pack2(nlv[j], nlv[j + 1])), x0, x1);
+                            float p0 = ex2f(x0), p1 = ex2f(x1);
+                            if (!UNMASKED && (uint32_t)(col - jl) > span) p0 = 0.f;
+                            if (!UNMASKED && (uint32_t)(col + 1 - jl) > span) p1 = 0.f;
+                            const uint64_t p2 = pack2(p0, p1);
+                            const uint64_t ds2 = mul2(p2, sub2(pack2(__uint_as_float(tv[j]), __uint_as_float(tv[j + 1])), pack2(Dv[j], Dv[j + 1])));
+                            unpack2(ds2, ds0, ds1);
+                            unpack2(sub2(p2, pack2(trunc19f(p0), trunc19f(p1))), a0, a1);
+                            unpack2(sub2(ds2, pack2(trunc19f(ds0), trunc19f(ds1))), b0, b1);
+                            sv[j] = __float_as_uint(p0); sv[j + 1] = __float_as_uint(p1);
+                            tv[j] = __float_as_uint(ds0); tv[j + 1] = __float_as_uint(ds1);
+                            pl[j] = __float_as_uint(a0); pl[j + 1] = __float_as_uint(a1);
+                            dl[j] = __float_as_uint(b0); dl[j + 1] = __float_as_uint(b1);
                         }
                     };
                     if (full) elementwise(std::true_type{}); else elementwise(std::false_type{});
