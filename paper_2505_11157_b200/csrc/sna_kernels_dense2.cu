@@ -119,6 +119,20 @@ __device__ __forceinline__ uint64_t fma2(uint64_t a, uint64_t b, uint64_t c) { u
 __device__ __forceinline__ uint64_t mul2(uint64_t a, uint64_t b) { uint64_t d; asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b)); return d; }
 __device__ __forceinline__ uint64_t add2(uint64_t a, uint64_t b) { uint64_t d; asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b)); return d; }
 __device__ __forceinline__ uint64_t sub2(uint64_t a, uint64_t b) { uint64_t d; asm("sub.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b)); return d; }
+// hi = trunc19(x), lo = x - hi for four values, the subtractions as two packed instructions
+__device__ __forceinline__ void split4(const float (&x)[4], float (&hi)[4], float (&lo)[4]) {
+#pragma unroll
+    for (int i = 0; i < 4; ++i) hi[i] = trunc19f(x[i]);
+    unpack2(sub2(pack2(x[0], x[1]), pack2(hi[0], hi[1])), lo[0], lo[1]);
+    unpack2(sub2(pack2(x[2], x[3]), pack2(hi[2], hi[3])), lo[2], lo[3]);
+}
+// x - trunc19(x) for the four components of a float4, as two packed subtractions
+__device__ __forceinline__ float4 lo4p(const float4& x) {
+    float4 r;
+    unpack2(sub2(pack2(x.x, x.y), pack2(trunc19f(x.x), trunc19f(x.y))), r.x, r.y);
+    unpack2(sub2(pack2(x.z, x.w), pack2(trunc19f(x.z), trunc19f(x.w))), r.z, r.w);
+    return r;
+}
 // BF16 UMMA (K = 16 per instruction) for the two correction terms of a product at once: the 16 k-slots of a step hold
 // [a_lo(8) | a_hi(8)] on the A side against [b_hi(8) ; b_lo(8)] on the B side, so one instruction adds a_lo*b_hi + a_hi*b_lo
 // for 8 contraction indices.  The corrections are ~2^-11 of the product, so BF16's 8 bits leave ~2^-19 relative error:
@@ -154,7 +168,9 @@ __device__ __forceinline__ void stack_b16(const unsigned char* raw, unsigned cha
     const float x[8] = {a.x, a.y, a.z, a.w, b.x, b.y, b.z, b.w};
     float hi[8], lo[8];
 #pragma unroll
-    for (int i = 0; i < 8; ++i) { hi[i] = trunc19f(x[i]); lo[i] = x[i] - hi[i]; }
+    for (int i = 0; i < 8; ++i) hi[i] = trunc19f(x[i]);
+#pragma unroll
+    for (int i = 0; i < 8; i += 2) unpack2(sub2(pack2(x[i], x[i + 1]), pack2(hi[i], hi[i + 1])), lo[i], lo[i + 1]);
     *reinterpret_cast<uint4*>(dst + sw_off(row, 2 * grp)) = make_uint4(bf16x2(hi[0], hi[1]), bf16x2(hi[2], hi[3]), bf16x2(hi[4], hi[5]), bf16x2(hi[6], hi[7]));
     *reinterpret_cast<uint4*>(dst + sw_off(row, 2 * grp + 1)) = make_uint4(bf16x2(lo[0], lo[1]), bf16x2(lo[2], lo[3]), bf16x2(lo[4], lo[5]), bf16x2(lo[6], lo[7]));
 }
@@ -527,7 +543,7 @@ forward_dense2_kernel(DevPlan p, const __grid_constant__ CUtensorMap map_q, cons
         for (int j = 0; j < 8; ++j) {
             const int off = (j * 128 + ct) * 16;
             const float4 x = *reinterpret_cast<const float4*>(base + OFF_Q + off);
-            *reinterpret_cast<float4*>(base + OFF_QLO + off) = make_float4(x.x - trunc19f(x.x), x.y - trunc19f(x.y), x.z - trunc19f(x.z), x.w - trunc19f(x.w));
+            *reinterpret_cast<float4*>(base + OFF_QLO + off) = lo4p(x);
         }
         for (int it = 0; it < total && ok; ++it) {
             const int s = it & 1, u = it >> 1;
@@ -538,7 +554,7 @@ forward_dense2_kernel(DevPlan p, const __grid_constant__ CUtensorMap map_q, cons
             for (int j = 0; j < 8; ++j) {
                 const int off = (j * 128 + ct) * 16;
                 const float4 x = *reinterpret_cast<const float4*>(kraw + off);
-                *reinterpret_cast<float4*>(kraw + TILE_B + off) = make_float4(x.x - trunc19f(x.x), x.y - trunc19f(x.y), x.z - trunc19f(x.z), x.w - trunc19f(x.w));
+                *reinterpret_cast<float4*>(kraw + TILE_B + off) = lo4p(x);
             }
             asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
             mb_arrive(s32(&bars[B_KCONV + s]));
@@ -552,14 +568,10 @@ forward_dense2_kernel(DevPlan p, const __grid_constant__ CUtensorMap map_q, cons
             unsigned char* vth = base + OFF_VT + s * 2 * TILE_B + cw * (C2 * 128);
 #pragma unroll
             for (int c8 = 0; c8 < 8; ++c8) {
-                float hi[4], lo[4];
+                float x[4], hi[4], lo[4];
 #pragma unroll
-                for (int i = 0; i < 4; ++i) {
-                    const int col = cw * 32 + c8 * 4 + i;
-                    const float x = *reinterpret_cast<const float*>(vraw + sw_off(col, lane >> 2) + (lane & 3) * 4);
-                    hi[i] = trunc19f(x);
-                    lo[i] = x - hi[i];
-                }
+                for (int i = 0; i < 4; ++i) x[i] = *reinterpret_cast<const float*>(vraw + sw_off(cw * 32 + c8 * 4 + i, lane >> 2) + (lane & 3) * 4);
+                split4(x, hi, lo);
                 *reinterpret_cast<float4*>(vth + sw_off(lane, c8)) = make_float4(hi[0], hi[1], hi[2], hi[3]);
                 *reinterpret_cast<float4*>(vth + TILE_B + sw_off(lane, c8)) = make_float4(lo[0], lo[1], lo[2], lo[3]);
             }
@@ -873,14 +885,10 @@ backward_dq_dense2_kernel(DevPlan p, const __grid_constant__ CUtensorMap map_k, 
                 unsigned char* kth = st + 4 * TILE_Q + (cw >> 1) * (C2 * 128);
 #pragma unroll
                 for (int c8 = 0; c8 < 4; ++c8) {
-                    float hi[4], lo[4];
+                    float x[4], hi[4], lo[4];
 #pragma unroll
-                    for (int i = 0; i < 4; ++i) {
-                        const int col = cw * 16 + c8 * 4 + i;
-                        const float x = *reinterpret_cast<const float*>(st + sw_off(col, lane >> 2) + (lane & 3) * 4);
-                        hi[i] = trunc19f(x);
-                        lo[i] = x - hi[i];
-                    }
+                    for (int i = 0; i < 4; ++i) x[i] = *reinterpret_cast<const float*>(st + sw_off(cw * 16 + c8 * 4 + i, lane >> 2) + (lane & 3) * 4);
+                    split4(x, hi, lo);
                     const int chunk = (cw & 1) * 4 + c8;
                     *reinterpret_cast<float4*>(kth + sw_off(lane, chunk)) = make_float4(hi[0], hi[1], hi[2], hi[3]);
                     *reinterpret_cast<float4*>(kth + TILE_Q + sw_off(lane, chunk)) = make_float4(lo[0], lo[1], lo[2], lo[3]);
@@ -1210,14 +1218,10 @@ backward_dkdv_dense2_kernel(DevPlan p, const __grid_constant__ CUtensorMap map_q
             for (int j = 0; j < BNK * 4 / 128; ++j) stack_b16(raw, lo, (j * 128 + ct) >> 2, ct & 3);
 #pragma unroll
             for (int c8 = 0; c8 < 2; ++c8) {
-                float hi[4], lw[4];
+                float x[4], hi[4], lw[4];
 #pragma unroll
-                for (int i = 0; i < 4; ++i) {
-                    const int col = cw * 8 + c8 * 4 + i;
-                    const float x = *reinterpret_cast<const float*>(raw + sw_off(col, lane >> 2) + (lane & 3) * 4);
-                    hi[i] = trunc19f(x);
-                    lw[i] = x - hi[i];
-                }
+                for (int i = 0; i < 4; ++i) x[i] = *reinterpret_cast<const float*>(raw + sw_off(cw * 8 + c8 * 4 + i, lane >> 2) + (lane & 3) * 4);
+                split4(x, hi, lw);
                 const int chunk = cw * 2 + c8;
                 *reinterpret_cast<float4*>(th + sw_off(lane, chunk)) = make_float4(hi[0], hi[1], hi[2], hi[3]);
                 *reinterpret_cast<float4*>(th + TILE_K + sw_off(lane, chunk)) = make_float4(lw[0], lw[1], lw[2], lw[3]);
