@@ -37,9 +37,9 @@ import numpy as np  # noqa: E402
 # ncu capture on workload c3 (bench.py cannot run ncu itself; the value is reported as `roofline.traffic` for that
 # workload only).
 NCU_DRAM_BYTES_PER_LAUNCH = {
-    ("c3", "forward"): (46562816 + 1140736) + (794043136 + 64422144),
-    ("c3", "backward_dq"): (57897472 + 1610240) + (965255936 + 63726080),
-    ("c3", "backward_dkdv"): (49117952 + 5714432) + (762001152 + 503494912),
+    ("c3", "forward"): (43485952 + 948480) + (794043136 + 64422144),
+    ("c3", "backward_dq"): (54733312 + 1611008) + (965255936 + 63726080),
+    ("c3", "backward_dkdv"): (49035008 + 5539584) + (762001152 + 503494912),
 }
 HBM_GBS_FALLBACK = 6650.0          # used only if MEASURED_PEAKS.json is absent
 L2_BYTES = 126 * 1024 * 1024
