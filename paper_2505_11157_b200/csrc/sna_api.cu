@@ -392,7 +392,7 @@ size_t sna_workspace_bytes(const sna_plan_t* plan, int B, int H, int C) {
 
 int sna_forward_kernel_count(const sna_plan_t* plan, int C, int with_lse) {
     if (plan == nullptr || plan->dev_blob == nullptr || !supported_C(C)) return 0;
-    if (plan->is_global) return 1;
+    if (plan->is_global || sna::dense2_global_supported(plan->dev, C)) return 1;
     return (with_lse && sna::dense2_path_supported(plan->dev, C)) ? 2 : 1;
 }
 
@@ -403,11 +403,12 @@ sna_status_t sna_forward_ex(const sna_plan_t* plan, const float* q, const float*
     if (!q || !k || !v || !out) { set_error("q, k, v and out must not be NULL"); return SNA_ERR_INVALID_ARG; }
     if (!all_aligned(q, k, v, out) || (reinterpret_cast<uintptr_t>(lse) & 3u)) { set_error("device pointers must be 16-byte aligned"); return SNA_ERR_INVALID_ARG; }
     cudaError_t e;
-    if (plan->is_global) {
-        // global attention: the dense kernel alone produces the final out and lse
-        e = (lse != nullptr && sna::dense2_global_supported(plan->dev, C))
-                ? sna::launch_forward_dense2(plan->dev, q, k, v, out, lse, B * H, C, (cudaStream_t)cuda_stream)
-                : sna::launch_forward_generic(plan->dev, q, k, v, out, lse, B * H, C, (cudaStream_t)cuda_stream);
+    if (lse != nullptr && sna::dense2_global_supported(plan->dev, C)) {
+        // every window is a whole ring (a global plan, or a cutoff that reaches every point): the dense kernel alone
+        // produces the final out and lse
+        e = sna::launch_forward_dense2(plan->dev, q, k, v, out, lse, B * H, C, (cudaStream_t)cuda_stream);
+    } else if (plan->is_global) {
+        e = sna::launch_forward_generic(plan->dev, q, k, v, out, lse, B * H, C, (cudaStream_t)cuda_stream);
     } else if (lse != nullptr && sna::dense2_path_supported(plan->dev, C)) {
         // whole-ring and wide windows on the tcgen05 kernel (its partial result travels in out / lse), the rest on the band kernel
         e = sna::launch_forward_dense2(plan->dev, q, k, v, out, lse, B * H, C, (cudaStream_t)cuda_stream);
@@ -436,10 +437,10 @@ sna_status_t sna_backward_dq(const sna_plan_t* plan, const float* q, const float
     cudaError_t e;
     // The dense dq kernel takes the whole-ring and wide windows when they are at least a tenth of the work (measured on the
     // benchmark configurations: -8 % on the dq stage at a 22 % share, -6 % at 13 %).
-    if (plan->is_global) {
-        e = (out != nullptr && out != dq && sna::dense2_global_supported(plan->dev, C))
-                ? sna::launch_backward_dq_dense2(plan->dev, q, k, v, dout, out, lse, dq, D, B * H, C, (cudaStream_t)cuda_stream)
-                : sna::launch_backward_dq_generic(plan->dev, q, k, v, dout, out, lse, dq, D, B * H, C, (cudaStream_t)cuda_stream);
+    if (out != nullptr && out != dq && sna::dense2_global_supported(plan->dev, C)) {
+        e = sna::launch_backward_dq_dense2(plan->dev, q, k, v, dout, out, lse, dq, D, B * H, C, (cudaStream_t)cuda_stream);
+    } else if (plan->is_global) {
+        e = sna::launch_backward_dq_generic(plan->dev, q, k, v, dout, out, lse, dq, D, B * H, C, (cudaStream_t)cuda_stream);
     } else if (out != nullptr && out != dq && plan->dev.dense_fraction >= 0.10f && sna::dense2_path_supported(plan->dev, C)) {
         // whole-ring and wide windows on the tcgen05 kernel (its part of dq is written first), the rest is added by the band kernel
         e = sna::launch_backward_dq_dense2(plan->dev, q, k, v, dout, out, lse, dq, nullptr, B * H, C, (cudaStream_t)cuda_stream);
@@ -461,7 +462,7 @@ sna_status_t sna_backward_dkdv(const sna_plan_t* plan, const float* q, const flo
     if (!q || !k || !v || !dout || !lse || !D || !dk || !dv) { set_error("q, k, v, dout, lse, D, dk and dv must not be NULL"); return SNA_ERR_INVALID_ARG; }
     if (!all_aligned(q, k, v, dout, dk, dv) || ((reinterpret_cast<uintptr_t>(lse) | reinterpret_cast<uintptr_t>(D)) & 3u)) { set_error("device pointers must be 16-byte aligned"); return SNA_ERR_INVALID_ARG; }
     cudaError_t e;
-    if (plan->is_global) {
+    if (plan->is_global || sna::dense2_global_supported(plan->dev, C)) {
         // the dense kernel writes only the rings some window refers to; rings of weight zero get their (zero) gradient here
         const bool dense = sna::dense2_global_supported(plan->dev, C);
         const size_t ring_bytes = (size_t)plan->host.nlon_in * C * sizeof(float), pitch = ring_bytes * plan->host.nlat_in;

@@ -71,7 +71,7 @@ cudaError_t launch_forward_mma(const DevPlan& p, const float* q, const float* k,
 cudaError_t dense2_prepare_device();   // once per device: opt in to the kernels' shared-memory sizes
 bool dense2_path_supported(const DevPlan& p, int C);
 cudaError_t launch_bounded_wait_probe(const DevPlan& p, int polls, cudaStream_t stream);
-bool dense2_global_supported(const DevPlan& p, int C);   // the dense kernels can serve a global plan on their own
+bool dense2_global_supported(const DevPlan& p, int C);   // every window is a whole ring and the dense kernels can do all the work
 cudaError_t launch_forward_dense2(const DevPlan& p, const float* q, const float* k, const float* v, float* out, float* lse,
                                   int N, int C, cudaStream_t stream);
 // The same split for the dq stage: the dense kernel writes its part of dq (out and dq must be different buffers) and,

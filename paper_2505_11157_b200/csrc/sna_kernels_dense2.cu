@@ -69,7 +69,12 @@ constexpr size_t DENSE2_SMEM = OFF_END + 1024;
 constexpr int T_S0 = 0, T_S1 = 128, T_PLO = 256, T_O = 384, T_COLS = 512;   // T_O: four 32-column accumulators, one per P V issuer
 constexpr int PV_ISSUERS = 4;
 
-enum { B_KFULL = 0, B_KCONV = 2, B_KFREE = 4, B_VFULL = 6, B_VRAWFREE = 8, B_VCONV = 10, B_PVDONE = 12 /* [half][stage] */, B_SFULL = 16, B_PREADY = 18 /* [half] */, B_QFULL = 20, B_COUNT = 21 };
+enum { B_KFULL = 0, B_KCONV = 2, B_KFREE = 4, B_VFULL = 6, B_VRAWFREE = 8, B_VCONV = 10, B_PVDONE = 12 /* [half][stage] */, B_SFULL = 16, B_PREADY = 18 /* [half][buffer] */, B_QFULL = 22, B_COUNT = 23 };
+// The "operands ready" barriers that many threads arrive on (PREADY here, DSREADY and READY in the backward kernels) exist
+// once per TMEM buffer: a warp that is a whole block ahead of another warp of its group then arrives on the OTHER buffer's
+// barrier.  With one barrier per group its second arrival would be counted into the phase of the block the slow warp has
+// not finished, and the second GEMM would start on that warp's stale rows (seen as run-to-run differences in 32-row
+// blocks of dk / dv when the dk/dv kernel got its second buffer).
 
 __device__ __forceinline__ uint32_t s32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 __device__ __forceinline__ float ex2f(float x) { float y; asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x)); return y; }
@@ -298,7 +303,8 @@ forward_dense2_kernel(DevPlan p, const __grid_constant__ CUtensorMap map_q, cons
             mb_init(s32(&bars[B_PVDONE + s]), 2);        // column half 0: two issuers
             mb_init(s32(&bars[B_PVDONE + 2 + s]), 2);    // column half 1
             mb_init(s32(&bars[B_SFULL + s]), 1);
-            mb_init(s32(&bars[B_PREADY + s]), 128);      // one per column half (index = half)
+            mb_init(s32(&bars[B_PREADY + s]), 128);      // column half 0, buffer s
+            mb_init(s32(&bars[B_PREADY + 2 + s]), 128);  // column half 1, buffer s
         }
         mb_init(s32(&bars[B_QFULL]), 1);
         fail_s = 0;
@@ -485,7 +491,7 @@ forward_dense2_kernel(DevPlan p, const __grid_constant__ CUtensorMap map_q, cons
                 l = fmaf(l, corr, (ps[0] + ps[1]) + (ps[2] + ps[3]));
                 asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
                 asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
-                mb_arrive(s32(&bars[B_PREADY + half]));
+                mb_arrive(s32(&bars[B_PREADY + 2 * half + b]));
             }
             corr_prev = corr;
         }
@@ -574,7 +580,7 @@ forward_dense2_kernel(DevPlan p, const __grid_constant__ CUtensorMap map_q, cons
             for (int it = 0; it < total && ok; ++it) {
                 const int s = it & 1, u = it >> 1;
                 ok = mb_wait(s32(&bars[B_VCONV + s]), u & 1, ok);
-                ok = mb_wait(s32(&bars[B_PREADY + half]), it & 1, ok) && ok;
+                ok = mb_wait(s32(&bars[B_PREADY + 2 * half + s]), u & 1, ok) && ok;
                 asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
                 const uint32_t tP = tm + (s ? T_S1 : T_S0), tPl = tm + T_PLO;
                 const uint32_t vt = sbase + OFF_VT + s * 2 * TILE_B;
@@ -664,7 +670,7 @@ constexpr int NSQ = 4;                           // shared-memory stages (TMA ru
 constexpr size_t DQ2_SMEM = NSQ * QST + 1024;
 constexpr int TQ_AQ = 0, TQ_AQL = 32, TQ_AY = 64, TQ_AYL = 96, TQ_BUF = 128 /* + 128 b: S | T */, TQ_ACC = 384 /* + 32 part */;
 enum { Q_KFULL = 0, Q_VFULL = 4, Q_KCONV = 8, Q_VCONV = 12, Q_KSFREE = 16, Q_VFREE = 20, Q_KTFREE = 24 /* all [stage] */,
-       Q_STFULL = 28 /* [buffer] */, Q_DSREADY = 30 /* [group] */, Q_G2DONE = 32 /* [group][buffer] */, Q_AREADY = 36, Q_COUNT = 37 };
+       Q_STFULL = 28 /* [buffer] */, Q_DSREADY = 30 /* [group][buffer] */, Q_G2DONE = 34 /* [group][buffer] */, Q_AREADY = 38, Q_COUNT = 39 };
 
 __global__ void __launch_bounds__(THREADS2, 1)
 backward_dq_dense2_kernel(DevPlan p, const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_v,
@@ -703,7 +709,8 @@ backward_dq_dense2_kernel(DevPlan p, const __grid_constant__ CUtensorMap map_k, 
         }
         for (int s = 0; s < 2; ++s) {
             mb_init(s32(&bars[Q_STFULL + s]), 2);
-            mb_init(s32(&bars[Q_DSREADY + s]), 128);
+            mb_init(s32(&bars[Q_DSREADY + s]), 128);          // group 0, buffer s
+            mb_init(s32(&bars[Q_DSREADY + 2 + s]), 128);      // group 1, buffer s
             mb_init(s32(&bars[Q_G2DONE + s]), 2);
             mb_init(s32(&bars[Q_G2DONE + 2 + s]), 2);
         }
@@ -833,10 +840,13 @@ backward_dq_dense2_kernel(DevPlan p, const __grid_constant__ CUtensorMap map_k, 
             if (it < total) {
                 asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
                 asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
-                mb_arrive(s32(&bars[Q_DSREADY + grp]));
+                mb_arrive(s32(&bars[Q_DSREADY + 2 * grp + (it & 1)]));
             }
         }
-        // merge the two column halves of every row through shared memory (the staging tiles are dead by now)
+        // merge the two column halves of every row through shared memory.  The staging tiles are reused for that, so the
+        // OTHER group's second GEMMs, which may still be reading k^T tiles, must have finished too (a thread's last fold
+        // only waited for its own group's).
+        if (total > 0) ok = mb_wait(s32(&bars[Q_G2DONE + 2 * (grp ^ 1) + ((total - 1) & 1)]), ((total - 1) >> 1) & 1, ok) && ok;
         float* xs = reinterpret_cast<float*>(base);
         if (grp == 1) {
 #pragma unroll
@@ -909,7 +919,7 @@ backward_dq_dense2_kernel(DevPlan p, const __grid_constant__ CUtensorMap map_k, 
             for (int it = 0; it < total && ok; ++it) {
                 const int s = it % NSQ, us = it / NSQ, b = it & 1;
                 PROF_WAIT(0, ok = mb_wait(s32(&bars[Q_KCONV + s]), us & 1, ok));
-                PROF_WAIT(1, ok = mb_wait(s32(&bars[Q_DSREADY + grp]), it & 1, ok) && ok);
+                PROF_WAIT(1, ok = mb_wait(s32(&bars[Q_DSREADY + 2 * grp + b]), (it >> 1) & 1, ok) && ok);
                 asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
                 const uint32_t tS = tm + TQ_BUF + 128 * b, tT = tS + BNQ;
                 const uint32_t kt = sbase + s * QST + 4 * TILE_Q;
@@ -993,7 +1003,7 @@ constexpr size_t DKDV2_SMEM = NSK * KST + 1024;
 constexpr int TK_AK = 0, TK_AKL = 32, TK_AV = 64, TK_AVL = 96, TK_BUF = 128 /* + 128 b: S | T | P_lo | dS_lo, 32 columns each */, TK_ACC = 384 /* + 32 part */;
 constexpr int TK_S = 0, TK_T = 32, TK_PLO = 64, TK_DSLO = 96;      // offsets inside a buffer
 enum { K_QFULL = 0, K_YFULL = NSK, K_QCONV = 2 * NSK, K_YCONV = 3 * NSK, K_FREE = 4 * NSK /* all [stage] */, K_STFULL = 5 * NSK /* [buffer] */,
-       K_READY = 5 * NSK + 2 /* [group] */, K_G2DONE = 5 * NSK + 4 /* [group][buffer] */, K_AREADY = 5 * NSK + 8, K_COUNT = 5 * NSK + 9 };
+       K_READY = 5 * NSK + 2 /* [group][buffer] */, K_G2DONE = 5 * NSK + 6 /* [group][buffer] */, K_AREADY = 5 * NSK + 10, K_COUNT = 5 * NSK + 11 };
 
 __global__ void __launch_bounds__(THREADS2, 1)
 backward_dkdv_dense2_kernel(DevPlan p, const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_y,
@@ -1032,7 +1042,8 @@ backward_dkdv_dense2_kernel(DevPlan p, const __grid_constant__ CUtensorMap map_q
         }
         for (int g = 0; g < 2; ++g) {
             mb_init(s32(&bars[K_STFULL + g]), 2);            // buffer g: both first GEMMs
-            mb_init(s32(&bars[K_READY + g]), 128);
+            mb_init(s32(&bars[K_READY + 2 * g]), 128);       // group g, buffer 0
+            mb_init(s32(&bars[K_READY + 2 * g + 1]), 128);   // group g, buffer 1
             mb_init(s32(&bars[K_G2DONE + 2 * g]), 2);        // group g, buffer 0: its dV and dK issuers
             mb_init(s32(&bars[K_G2DONE + 2 * g + 1]), 2);    // group g, buffer 1
         }
@@ -1170,10 +1181,13 @@ backward_dkdv_dense2_kernel(DevPlan p, const __grid_constant__ CUtensorMap map_q
                 }
                 asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
                 asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
-                mb_arrive(s32(&bars[K_READY + grp]));
+                mb_arrive(s32(&bars[K_READY + 2 * grp + b]));
             }
         }
-        // merge the two column halves of every row through shared memory (the staging tiles are dead by now)
+        // merge the two column halves of every row through shared memory.  The staging tiles are reused for that, so the
+        // OTHER group's second GEMMs, which may still be reading q^T / y^T tiles, must have finished too (a thread's last
+        // fold only waited for its own group's).
+        if (total > 0) ok = mb_wait(s32(&bars[K_G2DONE + 2 * (grp ^ 1) + ((total - 1) & 1)]), ((total - 1) >> 1) & 1, ok) && ok;
         float* xs = reinterpret_cast<float*>(base);
         if (grp == 1) {
 #pragma unroll
@@ -1248,7 +1262,7 @@ backward_dkdv_dense2_kernel(DevPlan p, const __grid_constant__ CUtensorMap map_q
                 const int s = it % NSK, us = it / NSK, b = it & 1;
                 const uint32_t tA = tm + TK_BUF + 128 * b + (kind ? TK_T : TK_S), tAl = tm + TK_BUF + 128 * b + (kind ? TK_DSLO : TK_PLO);
                 PROF_WAIT(0, ok = mb_wait(s32(&bars[(kind ? K_QCONV : K_YCONV) + s]), us & 1, ok));
-                PROF_WAIT(1, ok = mb_wait(s32(&bars[K_READY + grp]), it & 1, ok) && ok);
+                PROF_WAIT(1, ok = mb_wait(s32(&bars[K_READY + 2 * grp + b]), (it >> 1) & 1, ok) && ok);
                 asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
                 const uint32_t bt = sbase + s * KST + (kind ? 4 : 6) * TILE_K;          // q^T (dK) or y^T (dV) tiles
 #pragma unroll
@@ -1376,7 +1390,7 @@ bool dense2_path_supported(const DevPlan& p, int C) {
 }
 
 bool dense2_global_supported(const DevPlan& p, int C) {
-    return C == C2 && p.is_global && p.n_dense_rows > 0 && p.n_t_dense_rows > 0 && encode_fn2() != nullptr &&
+    return C == C2 && (p.is_global || p.dense_fraction >= 0.999f) && p.n_dense_rows > 0 && p.n_t_dense_rows > 0 && encode_fn2() != nullptr &&
            (long long)p.nlat_in * p.nlon_in * C < (1LL << 32) && (long long)p.nlat_out * p.nlon_out * C < (1LL << 32);
 }
 

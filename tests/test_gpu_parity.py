@@ -426,6 +426,28 @@ def test_results_are_reproducible_bit_for_bit():
         assert np.array_equal(x, y)
 
 
+@pytest.mark.parametrize("name, runs", [("c2", 12), ("c3", 12), ("c4", 8), ("c5", 12)])
+def test_benchmark_configurations_are_reproducible_bit_for_bit(name, runs):
+    """Every sum is taken in a fixed order, so repeated runs must agree bit for bit at full size too.  This is also the
+    sharpest detector of a race between the roles of the pipelined kernels: a stale operand or an early read changes
+    some 32-row block of some tile in some run (it caught a second arrival counted into the wrong barrier phase and
+    an early reuse of the staging tiles)."""
+    wl = WORKLOADS[name]
+    qd, kd, vd, dd = _dev(*make_inputs(wl))
+    with _plan(wl) as plan:
+        first = None
+        for run in range(runs):
+            out, lse = plan.forward(qd, kd, vd, return_lse=True)
+            dq, dk, dv = plan.backward(qd, kd, vd, dd, out=out, lse=lse)
+            torch.cuda.synchronize()
+            if first is None:
+                first = [t.clone() for t in (out, lse, dq, dk, dv)]
+            else:
+                for tname, a, b in zip(("out", "lse", "dq", "dk", "dv"), (out, lse, dq, dk, dv), first):
+                    assert torch.equal(a, b), (name, run, tname)
+        sna.sna_plan_check(plan.handle)
+
+
 def test_longitude_roll_equivariance_on_gpu():
     wl = SMALL[2]
     q, k, v, dout = make_inputs(wl)
