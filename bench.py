@@ -37,9 +37,9 @@ import numpy as np  # noqa: E402
 # ncu capture on workload c3 (bench.py cannot run ncu itself; the value is reported as `roofline.traffic` for that
 # workload only).
 NCU_DRAM_BYTES_PER_LAUNCH = {
-    ("c3", "forward"): (43485952 + 948480) + (794043136 + 64422144),
-    ("c3", "backward_dq"): (54733312 + 1611008) + (965255936 + 63726080),
-    ("c3", "backward_dkdv"): (49035008 + 5539584) + (762001152 + 503494912),
+    ("c3", "forward"): (44455936 + 725248) + (790744576 + 63745024),
+    ("c3", "backward_dq"): (57742592 + 2146560) + (956322304 + 63501312),
+    ("c3", "backward_dkdv"): (49276928 + 6318592) + (760281856 + 504061184),
 }
 HBM_GBS_FALLBACK = 6650.0          # used only if MEASURED_PEAKS.json is absent
 L2_BYTES = 126 * 1024 * 1024

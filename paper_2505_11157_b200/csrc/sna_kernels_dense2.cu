@@ -74,7 +74,11 @@ enum { B_KFULL = 0, B_KCONV = 2, B_KFREE = 4, B_VFULL = 6, B_VRAWFREE = 8, B_VCO
 // once per TMEM buffer: a warp that is a whole block ahead of another warp of its group then arrives on the OTHER buffer's
 // barrier.  With one barrier per group its second arrival would be counted into the phase of the block the slow warp has
 // not finished, and the second GEMM would start on that warp's stale rows (seen as run-to-run differences in 32-row
-// blocks of dk / dv when the dk/dv kernel got its second buffer).
+// blocks of dk / dv when the dk/dv kernel got its second buffer).  The other barriers with several arrivals are safe
+// as they are: a converter thread arrives on a stage's CONV / RAWFREE barrier again only after the producer has refilled
+// the stage, which waits for the stage's FREE barriers, which the GEMM issuers signal after having waited for the full CONV
+// phase; an issuer commits to a buffer's DONE / STFULL barrier again only for a block whose operands-ready phase needs the
+// element-wise threads to have seen the previous use of that buffer complete.
 
 __device__ __forceinline__ uint32_t s32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 __device__ __forceinline__ float ex2f(float x) { float y; asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x)); return y; }
